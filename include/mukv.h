@@ -1,0 +1,189 @@
+/*
+ * mukv.h -- C ABI of the MuKV compression + retrieval library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel path of MuKV ("Multi-Grained KV Cache
+ * Compression for Long Streaming Video Question-Answering"):
+ *
+ *   mukv_compress_chunk   Sec. 3.3 (Eq. 1-4, top-kappa selection, storing the kept KV
+ *                         slices of all layers with their timestamps) and Eq. 5 of
+ *                         Sec. 3.4 (mean-pooled block representations), applied to one
+ *                         streaming chunk of frames after the LLM prefill.
+ *   mukv_retrieve         Sec. 3.4 (Eq. 6-8): question pooling, cosine scoring against the
+ *                         segment-level and frame-level block keys, top-2k candidates,
+ *                         global-query rerank, final top-k.
+ *   mukv_gather           Sec. 3.5 (Eq. 9): builds R_k, R_v, the contiguous decode context,
+ *                         from the selected blocks.
+ *
+ * Conventions
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  Device pointers
+ *     handed to the library must be 16-byte aligned.
+ *   - Ownership: the caller owns every device buffer (store, workspace, inputs, outputs).
+ *     The library allocates no device memory; a context holds host metadata only.
+ *   - Ordering: all device work is enqueued on the stream given to the call and the call
+ *     returns after enqueueing.  Host-visible counters (frames stored) advance at enqueue
+ *     time; outputs are valid once the stream has reached that point.
+ *   - Errors: every entry point returns a mukv_status.  Argument errors are detected on the
+ *     host before anything is enqueued and leave the store unchanged.  No C++ exception
+ *     crosses this boundary.  mukv_last_error() gives a readable message.
+ *   - Threading: one context is used by one host thread at a time.  mukv_retrieve and
+ *     mukv_gather only read the store.
+ *
+ * Tensor layouts are token-major; element type is mukv_config.dtype (bf16 or fp32):
+ *     Q   [n_frames][P][Hq][D]        last-layer queries of the chunk's visual tokens
+ *     K,V [L][n_frames][P][Hkv][D]    keys / values of every layer
+ * Query head h attends with key head h / (Hq / Hkv) (grouped-query attention).
+ */
+#ifndef MUKV_H_
+#define MUKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mukv_ctx mukv_ctx;          /* opaque, library-owned host object */
+typedef void* mukv_stream;                 /* a cudaStream_t (NULL = legacy default stream) */
+
+typedef enum {
+  MUKV_OK = 0,
+  MUKV_E_INVALID = -1,      /* null pointer, negative count, bad enum */
+  MUKV_E_SHAPE = -2,        /* configuration outside the supported shapes */
+  MUKV_E_DTYPE = -3,
+  MUKV_E_ALIGN = -4,        /* device pointer not 16-byte aligned */
+  MUKV_E_CAPACITY = -5,     /* store / workspace / per-call limit exceeded */
+  MUKV_E_STATE = -6,        /* first_frame does not continue the stream, nothing stored, ... */
+  MUKV_E_CUDA = -7,         /* a CUDA runtime call failed; message in mukv_last_error */
+  MUKV_E_UNSUPPORTED = -8
+} mukv_status;
+
+typedef enum { MUKV_BF16 = 0, MUKV_FP32 = 1 } mukv_dtype;
+
+/* Retrieval variants of Sec. 3.4 / the retrieval-mode ablation:
+ * PARALLEL = stage 1 only (top-k by cosine); HIER = frames only inside the selected
+ * segments; SEMI = the paper's method (stage 1 top-2k, Eq. 8 rerank, top-k). */
+typedef enum { MUKV_RETR_PARALLEL = 0, MUKV_RETR_HIER = 1, MUKV_RETR_SEMI = 2 } mukv_retr_mode;
+
+#define MUKV_MAX_QUESTIONS 128   /* questions per mukv_retrieve / mukv_gather call */
+#define MUKV_MAX_TOPK 256        /* upper bound for k_seg, k_frm (2*k candidates <= 512) */
+#define MUKV_MAX_TOKENS 256      /* upper bound for P (tokens per frame) */
+
+typedef struct {
+  int32_t n_layers;              /* L                                                   */
+  int32_t n_q_heads;             /* Hq, a multiple of n_kv_heads                        */
+  int32_t n_kv_heads;            /* Hkv                                                 */
+  int32_t head_dim;              /* D: 64 or 128                                        */
+  int32_t tokens_per_frame;      /* P <= MUKV_MAX_TOKENS                                */
+  int32_t keep_per_frame;        /* kappa = floor(rho * P), computed by the caller      */
+  int32_t frames_per_segment;    /* frames pooled into one segment-level entry          */
+  int32_t max_frames_per_chunk;  /* upper bound for n_frames of one compress call       */
+  int32_t attn_causal;           /* 0: softmax over the whole frame; 1: keys j <= i     */
+  int32_t keep_low_freq;         /* 0: high frequency scores are kept (paper default)   */
+  float   alpha;                 /* Eq. 4 weight of the attention signal                */
+  float   tie_eps;               /* scores within tie_eps of the k-th count as tied     */
+  int32_t dtype;                 /* mukv_dtype of Q, K, V and of the stored pages       */
+  int32_t reserved;              /* set to 0                                            */
+  int64_t max_frames;            /* capacity of the store, in frames                    */
+} mukv_config;
+
+typedef struct {
+  int64_t frames;                /* frames stored so far                                */
+  int64_t segments;              /* segment entries present (last one may be partial)   */
+  int64_t kept_tokens;           /* frames * kappa                                      */
+  int64_t page_bytes;            /* bytes of one frame's page                           */
+  int64_t store_bytes_used;      /* pages written so far, in bytes                      */
+  int64_t refined_frames;        /* frames whose selection was redone in double         */
+  int64_t refined_questions;     /* reserved (retrieval always scores in double)        */
+  int64_t kernel_launches;       /* kernels launched by this context since creation     */
+  int32_t device_status;         /* 0, or a device-side consistency code                */
+  int32_t reserved;
+} mukv_stats;
+
+/* Bytes the caller must provide for the compressed store / the scratch workspace.
+ * Return 0 if the configuration is invalid. */
+size_t mukv_store_bytes(const mukv_config* cfg);
+size_t mukv_workspace_bytes(const mukv_config* cfg);
+
+/* Creates a context over caller-owned device memory.  d_store and d_workspace must stay
+ * valid until mukv_destroy; both are cleared where needed by stream-ordered memsets on the
+ * legacy default stream followed by a device synchronise (creation is not a hot call).
+ * Errors: INVALID (null), SHAPE/DTYPE (configuration), ALIGN, CAPACITY (buffers too small). */
+mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_bytes,
+                        void* d_workspace, size_t workspace_bytes, mukv_ctx** out);
+void mukv_destroy(mukv_ctx* ctx);
+
+/* Forgets every stored frame (capacity and buffers are kept).  Stream-ordered. */
+mukv_status mukv_reset(mukv_ctx* ctx, mukv_stream stream);
+
+/* Sec. 3.3 + Eq. 5.  Compresses frames first_frame .. first_frame+n_frames-1.
+ *   d_q [n_frames][P][Hq][D], d_k / d_v [L][n_frames][P][Hkv][D]: inputs, read only.
+ *   first_frame must equal the number of frames already stored (timestamps are the
+ *   absolute frame indices); 1 <= n_frames <= max_frames_per_chunk.
+ *   d_kept_out  [n_frames][kappa] int32, ascending kept token ids per frame, or NULL.
+ *   d_scores_out [3][n_frames][P] float: I_att (Eq. 1), I_fft (Eq. 3), fused I (Eq. 4), or NULL.
+ * Per frame the call scores every token, keeps the kappa best (ties within tie_eps go to
+ * the lowest index), copies their K/V rows of all layers into the frame's page, writes the
+ * frame-level entry (float mean of the kept rows per layer, K and V) and refreshes the
+ * entry of every segment the chunk touches (mean over the frames present so far).
+ * Frames whose selection lies too close to a tie boundary for single precision are
+ * re-scored in double precision on the device before they are stored.
+ * Errors: INVALID, ALIGN, STATE (first_frame), CAPACITY (n_frames, store full), CUDA. */
+mukv_status mukv_compress_chunk(mukv_ctx* ctx, const void* d_q, const void* d_k, const void* d_v,
+                                int32_t n_frames, int64_t first_frame,
+                                int32_t* d_kept_out, float* d_scores_out, mukv_stream stream);
+
+/* Sec. 3.4.  Serves nq questions in one batch.
+ *   d_qtok      [sum Nq][Hq][D] last-layer query tokens of all questions, concatenated.
+ *   h_q_offsets [nq+1] token offsets of each question in d_qtok (host, ascending, [0]=0).
+ *   h_t_limit   [nq] or NULL: question i sees frames with id < t_limit[i] and the segments
+ *               whose last stored frame is visible; NULL = everything stored.
+ *   k_seg, k_frm  blocks to select per granularity (<= MUKV_MAX_TOPK); top_n = number of
+ *               segment keys averaged into the global query (0 = k_seg); lambda_frm = Eq. 8
+ *               coherence factor for frames (segments use 0).
+ *   d_seg_idx [nq][k_seg], d_frm_idx [nq][k_frm]: selected ids ascending, unused slots -1.
+ *   d_seg_score / d_frm_score: matching scores (stage-1 cosine for segments, final score
+ *               for frames), or NULL.   d_counts [nq][2]: number of valid (segments, frames).
+ * Errors: INVALID, ALIGN, CAPACITY (nq, k, question length, workspace), STATE (empty store). */
+mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_offsets,
+                          const int64_t* h_t_limit, int32_t nq,
+                          int32_t k_seg, int32_t k_frm, int32_t top_n, float lambda_frm,
+                          int32_t mode,
+                          int32_t* d_seg_idx, int32_t* d_frm_idx,
+                          float* d_seg_score, float* d_frm_score, int32_t* d_counts,
+                          mukv_stream stream);
+
+/* Sec. 3.5.  For question i and layer l the kept K rows of the selected frames (ascending
+ * frame id, ascending token id inside a frame) are concatenated, then the V rows:
+ *   d_decode + i*decode_stride_bytes : [L][2 (K,V)][k_frm*kappa][Hkv][D] in the store dtype.
+ * Only the first counts[i][1]*kappa token slots of each [l][K|V] plane are written.
+ *   d_frm_idx [nq][k_frm], d_counts [nq][2]: as written by mukv_retrieve (device memory).
+ *   d_tok_meta [nq][k_frm*kappa][2] int32 (frame id, token id) per slot, or NULL.
+ * Errors: INVALID, ALIGN, CAPACITY (nq, k_frm, stride too small). */
+mukv_status mukv_gather(mukv_ctx* ctx, const int32_t* d_frm_idx, const int32_t* d_counts,
+                        int32_t nq, int32_t k_frm, void* d_decode, int64_t decode_stride_bytes,
+                        int32_t* d_tok_meta, mukv_stream stream);
+
+/* Device-side views into the store, for inspection and tests (do not write through them).
+ * which: 0 pages (dtype)           [max_frames][L][2][kappa][Hkv][D]
+ *        1 kept ids (int32)        [max_frames][kappa]
+ *        2 frame entries (float)   [max_frames][L][2][C]
+ *        3 segment entries (float) [max_segments][L][2][C]
+ *        4 frame keys (float)      [max_frames][C]
+ *        5 segment keys (float)    [max_segments][C]
+ *        6 frame timestamps (int64)[max_frames]
+ *        7 page table (int64 byte offsets from the store base) [max_frames]
+ * Returns NULL for an unknown region; *bytes (if not NULL) receives the region size. */
+void* mukv_store_region(const mukv_ctx* ctx, int32_t which, size_t* bytes);
+
+/* Reads counters.  Copies a few device words: synchronises the given stream. */
+mukv_status mukv_get_stats(mukv_ctx* ctx, mukv_stats* out, mukv_stream stream);
+
+/* Message of the last failure on this context (valid until the next call on it);
+ * with ctx == NULL, the message of the last failed mukv_create on this thread. */
+const char* mukv_last_error(const mukv_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MUKV_H_ */

@@ -1,0 +1,341 @@
+"""CPU oracle for the MuKV compression + retrieval path (test infrastructure only).
+
+This module is the slow, plain statement of what the CUDA library must compute.
+It is written from the paper's equations (Sec. 3.3 - 3.5), step by step, in
+float64, with numpy only.  It shares no code with the CUDA path and must never
+be imported by the product package: only the tests, the smoke check and the
+benchmark's CPU-baseline leg may use it.
+
+Notation follows the paper: P tokens per frame, D head dimension, H heads,
+L layers, kappa kept tokens per block, C = H*D concatenated feature size,
+k_g retrieved blocks per granularity, lambda_g coherence factor.
+
+Layouts (token-major):
+    Q  [P][Hq][D]      last-layer queries of one frame
+    K  [L][P][Hkv][D]  keys of one frame for all layers (last layer = K[L-1])
+    V  [L][P][Hkv][D]
+Grouped-query attention: query head h attends with key head h // (Hq // Hkv).
+
+Pins: every function here is checked in tests/test_oracle_pins.py against
+library routines, closed forms, invariants or brute force.  The one part that
+has no pin is whether the heuristic keeps the tokens that matter for answer
+accuracy ("parity unpinned": only the paper's accuracy tables speak to that and
+they need its datasets and model weights).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+TIE_EPS = 1e-6
+NORM_FLOOR = 1e-12
+
+
+# --------------------------------------------------------------------------
+# input decoding
+# --------------------------------------------------------------------------
+def as_f64(x: np.ndarray) -> np.ndarray:
+    """Widen an input tensor exactly to float64.
+
+    uint16 arrays hold bfloat16 bit patterns (the upper half of a float32);
+    float32 arrays are taken as they are.
+    """
+    x = np.asarray(x)
+    if x.dtype == np.uint16:
+        return (x.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    if x.dtype in (np.float32, np.float64):
+        return x.astype(np.float64)
+    raise TypeError(f"unsupported input dtype {x.dtype}")
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.3, Eq. 1: attention-based indicator
+# --------------------------------------------------------------------------
+def attention_importance(Q, K_last, causal: bool = False) -> np.ndarray:
+    """I_att[j] = 1/(H*P) * sum_h sum_i A_h[i, j]   (Eq. 1).
+
+    A_h = row-softmax(Q_h K_g^T / sqrt(D)) over the P tokens of the frame,
+    g = h // (Hq/Hkv).  With causal=True query i only sees keys j <= i.
+    """
+    Q = as_f64(Q)
+    K = as_f64(K_last)
+    P, Hq, D = Q.shape
+    Hkv = K.shape[1]
+    G = Hq // Hkv
+    col = np.zeros(P, dtype=np.float64)
+    for h in range(Hq):
+        g = h // G
+        z = (Q[:, h, :] @ K[:, g, :].T) / np.sqrt(float(D))       # [i][j]
+        if causal:
+            z = np.where(np.tril(np.ones((P, P), dtype=bool)), z, -np.inf)
+        m = z.max(axis=1, keepdims=True)
+        e = np.exp(z - m)
+        a = e / e.sum(axis=1, keepdims=True)
+        col += a.sum(axis=0)
+    return col / float(Hq * P)
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.3, Eq. 2-3: frequency-based indicator
+# --------------------------------------------------------------------------
+def dft_matrix(D: int) -> np.ndarray:
+    """W[b, d] = exp(-2*pi*i*b*d/D): the discrete Fourier transform written out."""
+    b = np.arange(D, dtype=np.float64).reshape(D, 1)
+    d = np.arange(D, dtype=np.float64).reshape(1, D)
+    ang = -2.0 * np.pi * np.mod(b * d, float(D)) / float(D)
+    return np.cos(ang) + 1j * np.sin(ang)
+
+
+def frequency_importance(K_last) -> np.ndarray:
+    """I_fft[j] = mean over heads and over the D bins of |DFT_D(k_j,head)|  (Eq. 2-3).
+
+    The transform runs along the feature axis of each token's key vector, per
+    key head; magnitudes of all D complex bins are averaged.
+    """
+    K = as_f64(K_last)
+    P, Hkv, D = K.shape
+    W = dft_matrix(D)
+    Z = K.reshape(P * Hkv, D).astype(np.complex128) @ W.T          # [token*head][bin]
+    mag = np.abs(Z).reshape(P, Hkv, D)
+    return mag.sum(axis=(1, 2)) / float(Hkv * D)
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.3, Eq. 4: dual-signal fusion
+# --------------------------------------------------------------------------
+def minmax(x: np.ndarray) -> np.ndarray:
+    """Min-max normalisation to [0, 1]; a constant vector maps to all zeros."""
+    x = np.asarray(x, dtype=np.float64)
+    lo, hi = x.min(), x.max()
+    if hi == lo:
+        return np.zeros_like(x)
+    return (x - lo) / (hi - lo)
+
+
+def fuse(I_att, I_fft, alpha: float, keep_low_freq: bool = False) -> np.ndarray:
+    """I = alpha * minmax(I_att) + (1 - alpha) * minmax(I_fft)   (Eq. 4)."""
+    a = minmax(I_att)
+    f = minmax(I_fft)
+    if keep_low_freq:
+        f = 1.0 - f
+    return float(alpha) * a + (1.0 - float(alpha)) * f
+
+
+# --------------------------------------------------------------------------
+# top-k selection with the tie band
+# --------------------------------------------------------------------------
+def topk_set(s, k: int, delta: float = TIE_EPS) -> np.ndarray:
+    """Indices of the k highest scores, ascending by index.
+
+    tau is the k-th largest score.  Every score above tau + delta is taken;
+    the scores within delta of tau are treated as tied and the remaining
+    places go to the lowest indices among them.
+    """
+    s = np.asarray(s, dtype=np.float64)
+    n = s.shape[0]
+    k = int(k)
+    if k <= 0 or n == 0:
+        return np.zeros(0, dtype=np.int64)
+    if k >= n:
+        return np.arange(n, dtype=np.int64)
+    tau = np.sort(s)[n - k]
+    sure = np.nonzero(s > tau + delta)[0]
+    band = np.nonzero(np.abs(s - tau) <= delta)[0]
+    need = k - sure.shape[0]
+    out = np.concatenate([sure, band[:need]])
+    return np.sort(out).astype(np.int64)
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.3 "Granularity Adaptive Compression" + Sec. 3.4 Eq. 5: one frame
+# --------------------------------------------------------------------------
+def keep_count(rho: float, n_tokens: int) -> int:
+    """kappa = floor(rho * |block|)."""
+    return int(np.floor(rho * n_tokens + 1e-9))
+
+
+def score_frame(Q, K_last, alpha, causal=False, keep_low_freq=False):
+    """(I_att, I_fft, I) for one frame."""
+    ia = attention_importance(Q, K_last, causal)
+    ifr = frequency_importance(K_last)
+    return ia, ifr, fuse(ia, ifr, alpha, keep_low_freq)
+
+
+def compact_rows(X, kept):
+    """X[L][P][Hkv][D] -> X[L][kappa][Hkv][D] in ascending token order (bytes untouched)."""
+    return np.ascontiguousarray(np.asarray(X)[:, kept, :, :])
+
+
+def pool_rows(Xc):
+    """Sum over the kept tokens of a compacted block: [L][kappa][Hkv][D] -> float64 [L][C]."""
+    X = as_f64(Xc)
+    L, kap, Hkv, D = X.shape
+    return X.sum(axis=1).reshape(L, Hkv * D)
+
+
+class Store:
+    """The compressed cache the oracle builds: one entry per frame, pooled entries per segment."""
+
+    def __init__(self, cfg: dict):
+        self.cfg = dict(cfg)
+        self.kept = []          # per frame: int64 [kappa], ascending
+        self.page_k = []        # per frame: raw-dtype [L][kappa][Hkv][D]
+        self.page_v = []
+        self.sum_k = []         # per frame: float64 [L][C] sums over kept tokens
+        self.sum_v = []
+        self.scores = []        # per frame: (I_att, I_fft, I)
+
+    @property
+    def n_frames(self) -> int:
+        return len(self.kept)
+
+    @property
+    def n_segments(self) -> int:
+        fs = self.cfg["frames_per_segment"]
+        return (self.n_frames + fs - 1) // fs
+
+    # Eq. 5 applied to every layer, K and V: float32 means over the kept tokens
+    def frame_entry(self, t: int):
+        kap = float(self.kept[t].shape[0])
+        return ((self.sum_k[t] / kap).astype(np.float32),
+                (self.sum_v[t] / kap).astype(np.float32))
+
+    def frame_key(self, t: int) -> np.ndarray:
+        """Retrieval key of frame t: mean of the last-layer kept keys, heads concatenated."""
+        return self.frame_entry(t)[0][-1]
+
+    def segment_frames(self, u: int):
+        fs = self.cfg["frames_per_segment"]
+        return range(u * fs, min((u + 1) * fs, self.n_frames))
+
+    def segment_entry(self, u: int):
+        """Mean over all kept tokens of the frames of segment u that are present."""
+        fr = list(self.segment_frames(u))
+        n_tok = float(sum(self.kept[t].shape[0] for t in fr))
+        sk = np.sum([self.sum_k[t] for t in fr], axis=0)
+        sv = np.sum([self.sum_v[t] for t in fr], axis=0)
+        return (sk / n_tok).astype(np.float32), (sv / n_tok).astype(np.float32)
+
+    def segment_key(self, u: int) -> np.ndarray:
+        return self.segment_entry(u)[0][-1]
+
+    def frame_keys(self) -> np.ndarray:
+        return np.stack([self.frame_key(t) for t in range(self.n_frames)])
+
+    def segment_keys(self) -> np.ndarray:
+        return np.stack([self.segment_key(u) for u in range(self.n_segments)])
+
+
+def compress_chunk(store: Store, Q, K, V) -> None:
+    """Append one chunk.  Q[n][P][Hq][D] (last layer), K,V[L][n][P][Hkv][D]."""
+    cfg = store.cfg
+    n = np.asarray(Q).shape[0]
+    for f in range(n):
+        Kf = np.asarray(K)[:, f]
+        Vf = np.asarray(V)[:, f]
+        ia, ifr, I = score_frame(np.asarray(Q)[f], Kf[-1], cfg["alpha"],
+                                 cfg.get("attn_causal", False), cfg.get("keep_low_freq", False))
+        kept = topk_set(I, cfg["keep_per_frame"], cfg.get("tie_eps", TIE_EPS))
+        pk = compact_rows(Kf, kept)
+        pv = compact_rows(Vf, kept)
+        store.kept.append(kept)
+        store.page_k.append(pk)
+        store.page_v.append(pv)
+        store.sum_k.append(pool_rows(pk))
+        store.sum_v.append(pool_rows(pv))
+        store.scores.append((ia, ifr, I))
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.4: semi-hierarchical retrieval
+# --------------------------------------------------------------------------
+def pool_question(Qq, n_kv_heads: int) -> np.ndarray:
+    """q = mean over the question's query tokens (Eq. 6), heads concatenated.
+
+    With grouped-query attention the Hq/Hkv query heads that share a key head
+    are averaged, so that q has the same C = Hkv*D features as the block keys.
+    """
+    X = as_f64(Qq)
+    Nq, Hq, D = X.shape
+    G = Hq // n_kv_heads
+    return X.reshape(Nq, n_kv_heads, G, D).sum(axis=(0, 2)).reshape(n_kv_heads * D) / float(Nq * G)
+
+
+def cosine(q, keys) -> np.ndarray:
+    """cos(q, keys[t]) for every row (Eq. 7); a zero-norm pair scores 0."""
+    q = np.asarray(q, dtype=np.float64)
+    keys = np.asarray(keys, dtype=np.float64)
+    if keys.shape[0] == 0:
+        return np.zeros(0, dtype=np.float64)
+    num = keys @ q
+    den = np.sqrt((keys * keys).sum(axis=1)) * np.sqrt((q * q).sum())
+    return num / np.maximum(den, NORM_FLOOR)
+
+
+MODE_PARALLEL, MODE_HIER, MODE_SEMI = 0, 1, 2
+
+
+def retrieve(store: Store, Qq, k_seg: int, k_frm: int, top_n: int = 0, lam: float = 0.3,
+             mode: int = MODE_SEMI, t_limit=None, delta: float = TIE_EPS):
+    """One question.  Returns dict with ascending seg_idx / frm_idx and their scores.
+
+    Visible frames have id < t_limit; a segment is visible when its last stored
+    frame is.  Stage 1 ranks every visible block by cosine with q and keeps
+    top-2k candidates per granularity; stage 2 (Eq. 8) re-scores the frame
+    candidates with their cosine to the mean of the top-N segment keys.
+    """
+    cfg = store.cfg
+    T = store.n_frames
+    t_limit = T if t_limit is None else min(int(t_limit), T)
+    fs = cfg["frames_per_segment"]
+    n_frm = max(t_limit, 0)
+    n_seg = sum(1 for u in range(store.n_segments) if min((u + 1) * fs, T) <= t_limit)
+
+    q = pool_question(Qq, cfg["n_kv_heads"])
+    key_f = store.frame_keys()[:n_frm].astype(np.float64) if n_frm else np.zeros((0, q.shape[0]))
+    key_s = store.segment_keys()[:n_seg].astype(np.float64) if n_seg else np.zeros((0, q.shape[0]))
+    s_frm = cosine(q, key_f)
+    s_seg = cosine(q, key_s)
+
+    sel_seg = topk_set(s_seg, min(k_seg, n_seg), delta)
+    if mode == MODE_PARALLEL:
+        sel_frm = topk_set(s_frm, min(k_frm, n_frm), delta)
+        final = s_frm[sel_frm]
+    elif mode == MODE_HIER:
+        inside = np.array([t for t in range(n_frm) if (t // fs) in set(sel_seg.tolist())], dtype=np.int64)
+        pick = topk_set(s_frm[inside], min(k_frm, inside.shape[0]), delta)
+        sel_frm = inside[pick]
+        final = s_frm[sel_frm]
+    else:
+        cand = topk_set(s_frm, min(2 * k_frm, n_frm), delta)
+        N = k_seg if top_n <= 0 else top_n
+        top = topk_set(s_seg, min(N, n_seg), delta)
+        if top.shape[0] > 0:
+            g = key_s[top].sum(axis=0) / float(top.shape[0])
+            gamma = cosine(g, key_f[cand])
+        else:
+            gamma = np.zeros(cand.shape[0])
+        s_new = (1.0 - lam) * s_frm[cand] + lam * gamma
+        pick = topk_set(s_new, min(k_frm, cand.shape[0]), delta)
+        sel_frm = cand[pick]
+        final = s_new[pick]
+    return {
+        "q": q, "s_frm": s_frm, "s_seg": s_seg,
+        "seg_idx": sel_seg, "seg_score": s_seg[sel_seg],
+        "frm_idx": sel_frm, "frm_score": final,
+    }
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.5, Eq. 9: the retrieved context R_k, R_v
+# --------------------------------------------------------------------------
+def gather(store: Store, frm_idx):
+    """decode[l][K then V][slot*kappa + r][Hkv][D] for the selected frames in ascending order,
+    and token meta (frame id, token id) per slot."""
+    frm_idx = [int(t) for t in frm_idx]
+    if not frm_idx:
+        return None, np.zeros((0, 2), dtype=np.int32)
+    Rk = np.concatenate([store.page_k[t] for t in frm_idx], axis=1)     # [L][n*kappa][Hkv][D]
+    Rv = np.concatenate([store.page_v[t] for t in frm_idx], axis=1)
+    dec = np.stack([Rk, Rv], axis=1)                                     # [L][2][n*kappa][Hkv][D]
+    meta = np.array([(t, int(j)) for t in frm_idx for j in store.kept[t]], dtype=np.int32)
+    return dec, meta
