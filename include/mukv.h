@@ -15,8 +15,9 @@
  *                         from the selected blocks.
  *
  * Conventions
- *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  Device pointers
- *     handed to the library must be 16-byte aligned.
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  Tensors of the cache
+ *     dtype (Q, K, V, question tokens, decode buffers), the store and the workspace must be
+ *     16-byte aligned; int32 / float index and score arrays need their natural 4-byte alignment.
  *   - Ownership: the caller owns every device buffer (store, workspace, inputs, outputs).
  *     The library allocates no device memory; a context holds host metadata only.
  *   - Ordering: all device work is enqueued on the stream given to the call and the call

@@ -1,0 +1,118 @@
+// Shared device helpers of the MuKV kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "../../include/mukv.h"
+
+namespace mukv {
+
+constexpr int kWarp = 32;
+constexpr unsigned kFull = 0xffffffffu;
+
+// ---------------------------------------------------------------- element access
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+template <typename T> struct ElemTraits;
+template <> struct ElemTraits<__nv_bfloat16> {
+  static constexpr int kPerWord = 2;      // elements in one 32-bit word
+  static constexpr int kPad = 2;          // row padding (elements) that makes the word stride odd
+};
+template <> struct ElemTraits<float> {
+  static constexpr int kPerWord = 1;
+  static constexpr int kPad = 1;
+};
+
+template <typename T> __device__ __forceinline__ float elem_to_float(T x);
+template <> __device__ __forceinline__ float elem_to_float<float>(float x) { return x; }
+template <> __device__ __forceinline__ float elem_to_float<__nv_bfloat16>(__nv_bfloat16 x) {
+  return __bfloat162float(x);
+}
+
+// acc += q.k over the elements packed in one 32-bit word
+template <typename T, typename A> __device__ __forceinline__ A dot_word(uint32_t q, uint32_t k, A acc);
+template <> __device__ __forceinline__ float dot_word<__nv_bfloat16, float>(uint32_t q, uint32_t k, float acc) {
+  acc = fmaf(bf16_lo(q), bf16_lo(k), acc);
+  return fmaf(bf16_hi(q), bf16_hi(k), acc);
+}
+template <> __device__ __forceinline__ double dot_word<__nv_bfloat16, double>(uint32_t q, uint32_t k, double acc) {
+  acc = fma((double)bf16_lo(q), (double)bf16_lo(k), acc);
+  return fma((double)bf16_hi(q), (double)bf16_hi(k), acc);
+}
+template <> __device__ __forceinline__ float dot_word<float, float>(uint32_t q, uint32_t k, float acc) {
+  return fmaf(__uint_as_float(q), __uint_as_float(k), acc);
+}
+template <> __device__ __forceinline__ double dot_word<float, double>(uint32_t q, uint32_t k, double acc) {
+  return fma((double)__uint_as_float(q), (double)__uint_as_float(k), acc);
+}
+
+// ---------------------------------------------------------------- math in the accumulation type
+__device__ __forceinline__ float exp_acc(float x) { return expf(x); }
+__device__ __forceinline__ double exp_acc(double x) { return exp(x); }
+__device__ __forceinline__ float fma_acc(float a, float b, float c) { return fmaf(a, b, c); }
+__device__ __forceinline__ double fma_acc(double a, double b, double c) { return fma(a, b, c); }
+__device__ __forceinline__ float sqrt_acc(float x) { return sqrtf(x); }
+__device__ __forceinline__ double sqrt_acc(double x) { return sqrt(x); }
+template <typename A> __device__ __forceinline__ A neg_inf();
+template <> __device__ __forceinline__ float neg_inf<float>() { return -INFINITY; }
+template <> __device__ __forceinline__ double neg_inf<double>() { return -(double)INFINITY; }
+
+// ---------------------------------------------------------------- warp / block reductions
+template <typename A> __device__ __forceinline__ A warp_sum(A v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+  return v;
+}
+template <typename A> __device__ __forceinline__ A warp_max(A v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    A u = __shfl_xor_sync(kFull, v, o);
+    v = u > v ? u : v;
+  }
+  return v;
+}
+template <typename A> __device__ __forceinline__ A warp_min(A v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    A u = __shfl_xor_sync(kFull, v, o);
+    v = u < v ? u : v;
+  }
+  return v;
+}
+
+// Exclusive prefix count of `flag` over the thread block in thread order, plus the block total.
+// scratch: at least (blockDim.x/32 + 1) ints of shared memory.  Contains two barriers.
+__device__ __forceinline__ int block_excl_count(bool flag, int* scratch, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+  const unsigned b = __ballot_sync(kFull, flag);
+  const int in_warp = __popc(b & ((1u << lane) - 1u));
+  __syncthreads();                       // scratch may still be read from a previous call
+  if (lane == 0) scratch[warp] = __popc(b);
+  __syncthreads();
+  int before = 0, sum = 0;
+  for (int w = 0; w < nwarp; ++w) {
+    const int c = scratch[w];
+    if (w < warp) before += c;
+    sum += c;
+  }
+  total = sum;
+  return before + in_warp;
+}
+
+// 16-byte streaming copies
+__device__ __forceinline__ uint4 ld_stream(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_stream(void* p, const uint4& v) {
+  asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+               : "memory");
+}
+
+}  // namespace mukv

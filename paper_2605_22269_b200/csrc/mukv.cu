@@ -1,0 +1,499 @@
+// Host side of the MuKV library: context, store layout, argument checks, kernel launches.
+// Built for sm_100a only.  No device memory is allocated here: the store and the workspace
+// belong to the caller.
+#include "../../include/mukv.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "common.cuh"
+#include "compact.cuh"
+#include "retrieve.cuh"
+#include "score.cuh"
+
+using namespace mukv;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct StoreLayout {
+  size_t pages, kept, frame_entry, seg_entry, frame_key, seg_key, frame_ts, page_table, frame_ksum, total;
+  size_t page_bytes;
+  long long max_segs;
+};
+
+struct WorkLayout {
+  size_t colsum_f, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, stat_refined;
+  size_t q64, qnorm, s_frm, s_seg, total;
+  size_t zero_begin, zero_end;          // region that must start as zeros
+};
+
+thread_local std::string g_create_error;
+
+}  // namespace
+
+struct mukv_ctx {
+  mukv_config cfg;
+  StoreLayout sl;
+  WorkLayout wl;
+  unsigned char* store;
+  unsigned char* ws;
+  long long frames;
+  long long launches;
+  int C, G, esize, nc;
+  float flag_margin, flat_ratio;
+  std::string err;
+};
+
+namespace {
+
+mukv_status fail(mukv_ctx* ctx, mukv_status st, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (ctx) ctx->err = buf; else g_create_error = buf;
+  return st;
+}
+
+bool is_pow2(long long x) { return x > 0 && (x & (x - 1)) == 0; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+// Returns nullptr if the configuration is supported, else the reason.
+const char* check_config(const mukv_config* c) {
+  if (!c) return "null config";
+  if (c->dtype != MUKV_BF16 && c->dtype != MUKV_FP32) return "dtype must be MUKV_BF16 or MUKV_FP32";
+  if (c->n_layers < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1) return "layer/head counts must be positive";
+  if (c->n_q_heads % c->n_kv_heads != 0) return "n_q_heads must be a multiple of n_kv_heads";
+  if (c->head_dim != 64 && c->head_dim != 128) return "head_dim must be 64 or 128";
+  if (c->tokens_per_frame < 1 || c->tokens_per_frame > MUKV_MAX_TOKENS) return "tokens_per_frame out of range";
+  if (c->keep_per_frame < 1 || c->keep_per_frame > c->tokens_per_frame) return "keep_per_frame out of range";
+  if (c->frames_per_segment < 1) return "frames_per_segment must be positive";
+  if (c->max_frames_per_chunk < 1 || c->max_frames_per_chunk > 4096) return "max_frames_per_chunk out of range";
+  if (c->max_frames < 1) return "max_frames must be positive";
+  if (!(c->alpha >= 0.f && c->alpha <= 1.f)) return "alpha must lie in [0, 1]";
+  if (!(c->tie_eps >= 0.f)) return "tie_eps must be >= 0";
+  const long long esize = c->dtype == MUKV_BF16 ? 2 : 4;
+  const long long row_vec = (long long)c->n_kv_heads * c->head_dim * esize / 16;
+  if (!is_pow2(row_vec) || row_vec > 256) return "Hkv*D*sizeof(element)/16 must be a power of two <= 256";
+  // the scoring kernel keeps one key head of a frame in shared memory
+  const size_t smem = c->dtype == MUKV_BF16
+                          ? score_smem_bytes<__nv_bfloat16, double>(c->tokens_per_frame, c->head_dim)
+                          : score_smem_bytes<float, double>(c->tokens_per_frame, c->head_dim);
+  if (smem > 227 * 1024) return "tokens_per_frame * head_dim too large for shared memory";
+  return nullptr;
+}
+
+StoreLayout store_layout(const mukv_config& c) {
+  StoreLayout s;
+  const size_t esize = c.dtype == MUKV_BF16 ? 2 : 4;
+  const size_t C = (size_t)c.n_kv_heads * c.head_dim;
+  const size_t T = (size_t)c.max_frames;
+  s.max_segs = (c.max_frames + c.frames_per_segment - 1) / c.frames_per_segment;
+  s.page_bytes = (size_t)c.n_layers * 2 * c.keep_per_frame * C * esize;
+  size_t off = 0;
+  s.pages = off;        off = align_up(off + T * s.page_bytes);
+  s.kept = off;         off = align_up(off + T * c.keep_per_frame * sizeof(int));
+  s.frame_entry = off;  off = align_up(off + T * c.n_layers * 2 * C * sizeof(float));
+  s.seg_entry = off;    off = align_up(off + (size_t)s.max_segs * c.n_layers * 2 * C * sizeof(float));
+  s.frame_key = off;    off = align_up(off + T * C * sizeof(float));
+  s.seg_key = off;      off = align_up(off + (size_t)s.max_segs * C * sizeof(float));
+  s.frame_ts = off;     off = align_up(off + T * sizeof(long long));
+  s.page_table = off;   off = align_up(off + T * sizeof(long long));
+  s.frame_ksum = off;   off = align_up(off + T * C * sizeof(double));
+  s.total = off;
+  return s;
+}
+
+WorkLayout work_layout(const mukv_config& c) {
+  WorkLayout w;
+  const size_t F = c.max_frames_per_chunk, P = c.tokens_per_frame;
+  const size_t C = (size_t)c.n_kv_heads * c.head_dim;
+  const size_t max_segs = (c.max_frames + c.frames_per_segment - 1) / c.frames_per_segment;
+  size_t off = 0;
+  w.colsum_f = off;       off = align_up(off + F * c.n_q_heads * P * sizeof(float));
+  w.ifft_f = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(float));
+  w.colsum_d = off;       off = align_up(off + F * c.n_q_heads * P * sizeof(double));
+  w.ifft_d = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(double));
+  w.zero_begin = off;
+  w.frame_counter = off;  off = align_up(off + F * sizeof(int));
+  w.flagged = off;        off = align_up(off + F * sizeof(int));
+  w.n_flagged = off;      off = align_up(off + sizeof(int));
+  w.stat_refined = off;   off = align_up(off + sizeof(long long));
+  w.zero_end = off;
+  w.q64 = off;            off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * C * sizeof(double));
+  w.qnorm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * sizeof(double));
+  w.s_frm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * c.max_frames * sizeof(double));
+  w.s_seg = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * max_segs * sizeof(double));
+  w.total = off;
+  return w;
+}
+
+int pick_nc(int P) { return P <= 64 ? 2 : P <= 128 ? 4 : P <= 224 ? 7 : 8; }
+
+template <typename T, typename A>
+cudaError_t launch_score(const ScoreParams& sp, int nc, dim3 grid, size_t smem, cudaStream_t st) {
+  switch (nc) {
+    case 2: score_kernel<T, A, 2><<<grid, kScoreThreads, smem, st>>>(sp); break;
+    case 4: score_kernel<T, A, 4><<<grid, kScoreThreads, smem, st>>>(sp); break;
+    case 7: score_kernel<T, A, 7><<<grid, kScoreThreads, smem, st>>>(sp); break;
+    default: score_kernel<T, A, 8><<<grid, kScoreThreads, smem, st>>>(sp); break;
+  }
+  return cudaGetLastError();
+}
+
+template <typename T, typename A>
+cudaError_t set_score_attr(int nc, size_t smem) {
+  const void* fn = nullptr;
+  switch (nc) {
+    case 2: fn = (const void*)score_kernel<T, A, 2>; break;
+    case 4: fn = (const void*)score_kernel<T, A, 4>; break;
+    case 7: fn = (const void*)score_kernel<T, A, 7>; break;
+    default: fn = (const void*)score_kernel<T, A, 8>; break;
+  }
+  return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+
+template <typename T>
+mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const void* d_v, int n, long long t0,
+                          int* d_kept_out, float* d_scores_out, cudaStream_t st) {
+  const mukv_config& c = ctx->cfg;
+  const int P = c.tokens_per_frame, L = c.n_layers, C = ctx->C;
+  ScoreParams sp;
+  memset(&sp, 0, sizeof sp);
+  sp.P = P; sp.Hq = c.n_q_heads; sp.Hkv = c.n_kv_heads; sp.D = c.head_dim; sp.G = ctx->G;
+  sp.kappa = c.keep_per_frame; sp.n_frames = n; sp.causal = c.attn_causal; sp.keep_low = c.keep_low_freq;
+  sp.alpha = c.alpha; sp.tie_eps = c.tie_eps; sp.flag_margin = ctx->flag_margin; sp.flat_ratio = ctx->flat_ratio;
+  sp.first_frame = t0;
+  sp.q = d_q;
+  sp.k_last = reinterpret_cast<const T*>(d_k) + (long long)(L - 1) * n * P * C;
+  sp.colsum_part = ctx->ws + ctx->wl.colsum_f;
+  sp.ifft_part = ctx->ws + ctx->wl.ifft_f;
+  sp.frame_counter = reinterpret_cast<int*>(ctx->ws + ctx->wl.frame_counter);
+  sp.flagged = reinterpret_cast<int*>(ctx->ws + ctx->wl.flagged);
+  sp.n_flagged = reinterpret_cast<int*>(ctx->ws + ctx->wl.n_flagged);
+  sp.kept_store = reinterpret_cast<int*>(ctx->store + ctx->sl.kept);
+  sp.kept_out = d_kept_out;
+  sp.scores_out = d_scores_out;
+  sp.frame_ts = reinterpret_cast<long long*>(ctx->store + ctx->sl.frame_ts);
+  sp.page_table = reinterpret_cast<long long*>(ctx->store + ctx->sl.page_table);
+  sp.pages_off = (long long)ctx->sl.pages;
+  sp.page_bytes = (long long)ctx->sl.page_bytes;
+  sp.refine = 0;
+  const dim3 grid(c.n_q_heads, n);
+  cudaError_t e = launch_score<T, float>(sp, ctx->nc, grid, score_smem_bytes<T, float>(P, c.head_dim), st);
+  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "score kernel: %s", cudaGetErrorString(e));
+  // frames too close to a tie boundary: same computation in double (blocks beyond the flagged
+  // count return at once)
+  sp.refine = 1;
+  sp.colsum_part = ctx->ws + ctx->wl.colsum_d;
+  sp.ifft_part = ctx->ws + ctx->wl.ifft_d;
+  e = launch_score<T, double>(sp, ctx->nc, grid, score_smem_bytes<T, double>(P, c.head_dim), st);
+  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "refine kernel: %s", cudaGetErrorString(e));
+
+  CompactParams cp;
+  memset(&cp, 0, sizeof cp);
+  cp.L = L; cp.kappa = c.keep_per_frame; cp.C = C; cp.P = P; cp.n_frames = n; cp.first_frame = t0;
+  cp.k = d_k; cp.v = d_v;
+  cp.kept_store = sp.kept_store;
+  cp.store = ctx->store;
+  cp.page_table = sp.page_table;
+  cp.frame_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.frame_entry);
+  cp.frame_key = reinterpret_cast<float*>(ctx->store + ctx->sl.frame_key);
+  cp.frame_ksum = reinterpret_cast<double*>(ctx->store + ctx->sl.frame_ksum);
+  cp.n_flagged = sp.n_flagged;
+  cp.stat_refined = reinterpret_cast<long long*>(ctx->ws + ctx->wl.stat_refined);
+  compact_kernel<T><<<dim3(L * 2, n), kCompactThreads, 0, st>>>(cp);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "compact kernel: %s", cudaGetErrorString(e));
+
+  SegmentParams gp;
+  gp.L = L; gp.C = C; gp.kappa = c.keep_per_frame; gp.fseg = c.frames_per_segment;
+  gp.first_seg = t0 / c.frames_per_segment;
+  gp.frames_total = t0 + n;
+  gp.frame_entry = cp.frame_entry;
+  gp.frame_ksum = cp.frame_ksum;
+  gp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
+  gp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
+  const long long last_seg = (t0 + n - 1) / c.frames_per_segment;
+  segment_kernel<<<dim3(L * 2, (unsigned)(last_seg - gp.first_seg + 1)), 256, 0, st>>>(gp);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "segment kernel: %s", cudaGetErrorString(e));
+  ctx->launches += 4;
+  ctx->frames = t0 + n;
+  return MUKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t mukv_store_bytes(const mukv_config* cfg) {
+  if (check_config(cfg)) return 0;
+  return store_layout(*cfg).total;
+}
+
+size_t mukv_workspace_bytes(const mukv_config* cfg) {
+  if (check_config(cfg)) return 0;
+  return work_layout(*cfg).total;
+}
+
+mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_bytes, void* d_workspace,
+                        size_t workspace_bytes, mukv_ctx** out) {
+  if (!out) return fail(nullptr, MUKV_E_INVALID, "out is null");
+  *out = nullptr;
+  if (!cfg || !d_store || !d_workspace) return fail(nullptr, MUKV_E_INVALID, "null argument");
+  if (const char* why = check_config(cfg))
+    return fail(nullptr, (cfg->dtype != MUKV_BF16 && cfg->dtype != MUKV_FP32) ? MUKV_E_DTYPE : MUKV_E_SHAPE, "%s", why);
+  if (!aligned16(d_store) || !aligned16(d_workspace))
+    return fail(nullptr, MUKV_E_ALIGN, "store and workspace must be 16-byte aligned");
+  mukv_ctx* ctx = new (std::nothrow) mukv_ctx();
+  if (!ctx) return fail(nullptr, MUKV_E_INVALID, "out of host memory");
+  ctx->cfg = *cfg;
+  ctx->sl = store_layout(*cfg);
+  ctx->wl = work_layout(*cfg);
+  if (store_bytes < ctx->sl.total || workspace_bytes < ctx->wl.total) {
+    const size_t need_s = ctx->sl.total, need_w = ctx->wl.total;
+    delete ctx;
+    return fail(nullptr, MUKV_E_CAPACITY, "store needs %zu bytes (got %zu), workspace needs %zu bytes (got %zu)",
+                need_s, store_bytes, need_w, workspace_bytes);
+  }
+  ctx->store = static_cast<unsigned char*>(d_store);
+  ctx->ws = static_cast<unsigned char*>(d_workspace);
+  ctx->frames = 0;
+  ctx->launches = 0;
+  ctx->C = cfg->n_kv_heads * cfg->head_dim;
+  ctx->G = cfg->n_q_heads / cfg->n_kv_heads;
+  ctx->esize = cfg->dtype == MUKV_BF16 ? 2 : 4;
+  ctx->nc = pick_nc(cfg->tokens_per_frame);
+  ctx->flag_margin = 6e-7f;
+  ctx->flat_ratio = 1e-3f;
+  if (const char* s = getenv("MUKV_FLAG_MARGIN")) ctx->flag_margin = (float)atof(s);
+  if (const char* s = getenv("MUKV_FLAT_RATIO")) ctx->flat_ratio = (float)atof(s);
+  const int P = cfg->tokens_per_frame, D = cfg->head_dim;
+  cudaError_t e;
+  if (cfg->dtype == MUKV_BF16) {
+    e = set_score_attr<__nv_bfloat16, float>(ctx->nc, score_smem_bytes<__nv_bfloat16, float>(P, D));
+    if (e == cudaSuccess) e = set_score_attr<__nv_bfloat16, double>(ctx->nc, score_smem_bytes<__nv_bfloat16, double>(P, D));
+  } else {
+    e = set_score_attr<float, float>(ctx->nc, score_smem_bytes<float, float>(P, D));
+    if (e == cudaSuccess) e = set_score_attr<float, double>(ctx->nc, score_smem_bytes<float, double>(P, D));
+  }
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute((const void*)scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(kScanRows * (ctx->C + 1) * sizeof(float)));
+  if (e == cudaSuccess)
+    e = cudaMemset(ctx->ws + ctx->wl.zero_begin, 0, ctx->wl.zero_end - ctx->wl.zero_begin);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    fail(nullptr, MUKV_E_CUDA, "mukv_create: %s", cudaGetErrorString(e));
+    delete ctx;
+    return MUKV_E_CUDA;
+  }
+  *out = ctx;
+  return MUKV_OK;
+}
+
+void mukv_destroy(mukv_ctx* ctx) { delete ctx; }
+
+mukv_status mukv_reset(mukv_ctx* ctx, mukv_stream stream) {
+  (void)stream;
+  if (!ctx) return MUKV_E_INVALID;
+  ctx->frames = 0;
+  return MUKV_OK;
+}
+
+mukv_status mukv_compress_chunk(mukv_ctx* ctx, const void* d_q, const void* d_k, const void* d_v, int32_t n_frames,
+                                int64_t first_frame, int32_t* d_kept_out, float* d_scores_out,
+                                mukv_stream stream) {
+  if (!ctx) return MUKV_E_INVALID;
+  try {
+    if (!d_q || !d_k || !d_v) return fail(ctx, MUKV_E_INVALID, "null input pointer");
+    if (!aligned16(d_q) || !aligned16(d_k) || !aligned16(d_v) || !aligned4(d_kept_out) || !aligned4(d_scores_out))
+      return fail(ctx, MUKV_E_ALIGN, "d_q, d_k, d_v must be 16-byte aligned, the outputs 4-byte aligned");
+    if (n_frames < 1) return fail(ctx, MUKV_E_INVALID, "n_frames must be >= 1");
+    if (n_frames > ctx->cfg.max_frames_per_chunk)
+      return fail(ctx, MUKV_E_CAPACITY, "n_frames %d exceeds max_frames_per_chunk %d", n_frames,
+                  ctx->cfg.max_frames_per_chunk);
+    if (first_frame != ctx->frames)
+      return fail(ctx, MUKV_E_STATE, "first_frame %lld does not continue the stream (%lld frames stored)",
+                  (long long)first_frame, ctx->frames);
+    if (first_frame + n_frames > ctx->cfg.max_frames)
+      return fail(ctx, MUKV_E_CAPACITY, "store full: %lld + %d frames > max_frames %lld", ctx->frames, n_frames,
+                  (long long)ctx->cfg.max_frames);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->cfg.dtype == MUKV_BF16)
+      return compress_impl<__nv_bfloat16>(ctx, d_q, d_k, d_v, n_frames, first_frame, d_kept_out, d_scores_out, st);
+    return compress_impl<float>(ctx, d_q, d_k, d_v, n_frames, first_frame, d_kept_out, d_scores_out, st);
+  } catch (...) {
+    return fail(ctx, MUKV_E_INVALID, "unexpected exception");
+  }
+}
+
+mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_offsets, const int64_t* h_t_limit,
+                          int32_t nq, int32_t k_seg, int32_t k_frm, int32_t top_n, float lambda_frm, int32_t mode,
+                          int32_t* d_seg_idx, int32_t* d_frm_idx, float* d_seg_score, float* d_frm_score,
+                          int32_t* d_counts, mukv_stream stream) {
+  if (!ctx) return MUKV_E_INVALID;
+  try {
+    if (!d_qtok || !h_q_offsets || !d_seg_idx || !d_frm_idx || !d_counts)
+      return fail(ctx, MUKV_E_INVALID, "null argument");
+    if (!aligned16(d_qtok) || !aligned4(d_seg_idx) || !aligned4(d_frm_idx) || !aligned4(d_seg_score) ||
+        !aligned4(d_frm_score) || !aligned4(d_counts))
+      return fail(ctx, MUKV_E_ALIGN, "d_qtok must be 16-byte aligned, the outputs 4-byte aligned");
+    if (nq < 1) return fail(ctx, MUKV_E_INVALID, "nq must be >= 1");
+    if (nq > MUKV_MAX_QUESTIONS) return fail(ctx, MUKV_E_CAPACITY, "nq %d exceeds %d", nq, MUKV_MAX_QUESTIONS);
+    if (k_seg < 1 || k_frm < 1 || top_n < 0) return fail(ctx, MUKV_E_INVALID, "k_seg, k_frm must be >= 1, top_n >= 0");
+    if (k_seg > MUKV_MAX_TOPK || k_frm > MUKV_MAX_TOPK || top_n > MUKV_MAX_TOPK)
+      return fail(ctx, MUKV_E_CAPACITY, "k_seg / k_frm / top_n exceed %d", MUKV_MAX_TOPK);
+    if (mode != MUKV_RETR_PARALLEL && mode != MUKV_RETR_HIER && mode != MUKV_RETR_SEMI)
+      return fail(ctx, MUKV_E_INVALID, "unknown retrieval mode %d", mode);
+    if (!(lambda_frm >= 0.f && lambda_frm <= 1.f)) return fail(ctx, MUKV_E_INVALID, "lambda_frm must lie in [0, 1]");
+    if (ctx->frames < 1) return fail(ctx, MUKV_E_STATE, "the store is empty");
+    QMeta meta;
+    if (h_q_offsets[0] != 0) return fail(ctx, MUKV_E_INVALID, "q_offsets[0] must be 0");
+    for (int i = 0; i < nq; ++i) {
+      if (h_q_offsets[i + 1] <= h_q_offsets[i])
+        return fail(ctx, MUKV_E_INVALID, "question %d has no tokens (offsets must ascend)", i);
+      if (h_t_limit && h_t_limit[i] < 0) return fail(ctx, MUKV_E_INVALID, "t_limit[%d] is negative", i);
+    }
+    for (int i = 0; i <= nq; ++i) meta.off[i] = h_q_offsets[i];
+    for (int i = 0; i < nq; ++i) meta.t_limit[i] = h_t_limit ? (long long)h_t_limit[i] : ctx->frames;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const mukv_config& c = ctx->cfg;
+    const int C = ctx->C;
+    double* q64 = reinterpret_cast<double*>(ctx->ws + ctx->wl.q64);
+    double* qnorm = reinterpret_cast<double*>(ctx->ws + ctx->wl.qnorm);
+    double* s_frm = reinterpret_cast<double*>(ctx->ws + ctx->wl.s_frm);
+    double* s_seg = reinterpret_cast<double*>(ctx->ws + ctx->wl.s_seg);
+    const float* frame_key = reinterpret_cast<const float*>(ctx->store + ctx->sl.frame_key);
+    const float* seg_key = reinterpret_cast<const float*>(ctx->store + ctx->sl.seg_key);
+    const long long n_frm = ctx->frames;
+    const long long n_seg = (n_frm + c.frames_per_segment - 1) / c.frames_per_segment;
+    if (c.dtype == MUKV_BF16)
+      qpool_kernel<__nv_bfloat16><<<nq, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(d_qtok), meta,
+                                                     c.n_q_heads, c.n_kv_heads, c.head_dim, q64, qnorm);
+    else
+      qpool_kernel<float><<<nq, 256, 0, st>>>(reinterpret_cast<const float*>(d_qtok), meta, c.n_q_heads,
+                                             c.n_kv_heads, c.head_dim, q64, qnorm);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "qpool kernel: %s", cudaGetErrorString(e));
+    const long long rows = n_frm + n_seg;
+    const unsigned blocks = (unsigned)((rows + kScanRows - 1) / kScanRows);
+    scan_kernel<<<blocks, 256, kScanRows * (C + 1) * sizeof(float), st>>>(frame_key, seg_key, n_frm, n_seg, C, nq, q64,
+                                                                         qnorm, s_frm, s_seg, c.max_frames,
+                                                                         ctx->sl.max_segs);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "scan kernel: %s", cudaGetErrorString(e));
+    RankParams rp;
+    memset(&rp, 0, sizeof rp);
+    rp.nq = nq; rp.C = C; rp.fseg = c.frames_per_segment;
+    rp.k_seg = k_seg; rp.k_frm = k_frm; rp.top_n = top_n; rp.mode = mode;
+    rp.lambda = (double)lambda_frm; rp.delta = (double)c.tie_eps;
+    rp.n_frm = n_frm; rp.n_seg = n_seg;
+    rp.s_frm = s_frm; rp.s_seg = s_seg; rp.frm_stride = c.max_frames; rp.seg_stride = ctx->sl.max_segs;
+    rp.frame_key = frame_key; rp.seg_key = seg_key;
+    rp.seg_idx = d_seg_idx; rp.frm_idx = d_frm_idx; rp.seg_score = d_seg_score; rp.frm_score = d_frm_score;
+    rp.counts = d_counts;
+    rank_kernel<<<nq, kRankThreads, C * sizeof(double), st>>>(rp, meta);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "rank kernel: %s", cudaGetErrorString(e));
+    ctx->launches += 3;
+    return MUKV_OK;
+  } catch (...) {
+    return fail(ctx, MUKV_E_INVALID, "unexpected exception");
+  }
+}
+
+mukv_status mukv_gather(mukv_ctx* ctx, const int32_t* d_frm_idx, const int32_t* d_counts, int32_t nq, int32_t k_frm,
+                        void* d_decode, int64_t decode_stride_bytes, int32_t* d_tok_meta, mukv_stream stream) {
+  if (!ctx) return MUKV_E_INVALID;
+  try {
+    if (!d_frm_idx || !d_counts || !d_decode) return fail(ctx, MUKV_E_INVALID, "null argument");
+    if (!aligned4(d_frm_idx) || !aligned4(d_counts) || !aligned16(d_decode) || !aligned4(d_tok_meta))
+      return fail(ctx, MUKV_E_ALIGN, "d_decode must be 16-byte aligned, index arrays 4-byte aligned");
+    if (nq < 1 || k_frm < 1) return fail(ctx, MUKV_E_INVALID, "nq and k_frm must be >= 1");
+    if (nq > MUKV_MAX_QUESTIONS || k_frm > MUKV_MAX_TOPK)
+      return fail(ctx, MUKV_E_CAPACITY, "nq or k_frm too large");
+    const mukv_config& c = ctx->cfg;
+    const long long run = (long long)c.keep_per_frame * ctx->C * ctx->esize;
+    const long long need = (long long)c.n_layers * 2 * k_frm * run;
+    if (decode_stride_bytes < need)
+      return fail(ctx, MUKV_E_CAPACITY, "decode_stride_bytes %lld < %lld needed per question",
+                  (long long)decode_stride_bytes, need);
+    if (decode_stride_bytes % 16 != 0) return fail(ctx, MUKV_E_ALIGN, "decode_stride_bytes must be a multiple of 16");
+    GatherParams gp;
+    gp.nq = nq; gp.k_frm = k_frm; gp.L = c.n_layers; gp.kappa = c.keep_per_frame;
+    gp.run_bytes = run;
+    gp.frm_idx = d_frm_idx; gp.counts = d_counts;
+    gp.store = ctx->store;
+    gp.page_table = reinterpret_cast<const long long*>(ctx->store + ctx->sl.page_table);
+    gp.kept_store = reinterpret_cast<const int*>(ctx->store + ctx->sl.kept);
+    gp.decode = static_cast<unsigned char*>(d_decode);
+    gp.decode_stride = decode_stride_bytes;
+    gp.tok_meta = d_tok_meta;
+    const long long units = (long long)nq * c.n_layers * 2 * k_frm;
+    const unsigned blocks = (unsigned)(units < 148 * 8 ? units : 148 * 8);
+    gather_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(gp);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "gather kernel: %s", cudaGetErrorString(e));
+    ctx->launches += 1;
+    return MUKV_OK;
+  } catch (...) {
+    return fail(ctx, MUKV_E_INVALID, "unexpected exception");
+  }
+}
+
+void* mukv_store_region(const mukv_ctx* ctx, int32_t which, size_t* bytes) {
+  if (!ctx) return nullptr;
+  const mukv_config& c = ctx->cfg;
+  const StoreLayout& s = ctx->sl;
+  const size_t T = (size_t)c.max_frames, C = (size_t)ctx->C;
+  size_t off = 0, sz = 0;
+  switch (which) {
+    case 0: off = s.pages; sz = T * s.page_bytes; break;
+    case 1: off = s.kept; sz = T * c.keep_per_frame * sizeof(int); break;
+    case 2: off = s.frame_entry; sz = T * c.n_layers * 2 * C * sizeof(float); break;
+    case 3: off = s.seg_entry; sz = (size_t)s.max_segs * c.n_layers * 2 * C * sizeof(float); break;
+    case 4: off = s.frame_key; sz = T * C * sizeof(float); break;
+    case 5: off = s.seg_key; sz = (size_t)s.max_segs * C * sizeof(float); break;
+    case 6: off = s.frame_ts; sz = T * sizeof(long long); break;
+    case 7: off = s.page_table; sz = T * sizeof(long long); break;
+    default: return nullptr;
+  }
+  if (bytes) *bytes = sz;
+  return ctx->store + off;
+}
+
+mukv_status mukv_get_stats(mukv_ctx* ctx, mukv_stats* out, mukv_stream stream) {
+  if (!ctx || !out) return MUKV_E_INVALID;
+  memset(out, 0, sizeof *out);
+  long long refined = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(&refined, ctx->ws + ctx->wl.stat_refined, sizeof refined, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "mukv_get_stats: %s", cudaGetErrorString(e));
+  const mukv_config& c = ctx->cfg;
+  out->frames = ctx->frames;
+  out->segments = (ctx->frames + c.frames_per_segment - 1) / c.frames_per_segment;
+  out->kept_tokens = ctx->frames * c.keep_per_frame;
+  out->page_bytes = (long long)ctx->sl.page_bytes;
+  out->store_bytes_used = ctx->frames * (long long)ctx->sl.page_bytes;
+  out->refined_frames = refined;
+  out->kernel_launches = ctx->launches;
+  return MUKV_OK;
+}
+
+const char* mukv_last_error(const mukv_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,401 @@
+// Semi-hierarchical retrieval (Sec. 3.4, Eq. 6-8) and the gather of the retrieved context
+// (Sec. 3.5, Eq. 9).
+//
+// All ranking arithmetic is double precision: the work is a few hundred MFLOP per batch of
+// questions, tiny next to the gather, and it makes the selected indices independent of
+// summation order.  Kernels:
+//   qpool_kernel    Eq. 6   one block per question
+//   scan_kernel     Eq. 7   cosine of every question with every frame key and segment key
+//   rank_kernel     stage-1 candidates, Eq. 8 rerank, final top-k; one block per question
+//   gather_kernel   Eq. 9   copies the selected pages into the per-question decode buffers
+#pragma once
+#include "common.cuh"
+
+namespace mukv {
+
+struct QMeta {
+  int off[MUKV_MAX_QUESTIONS + 1];
+  long long t_limit[MUKV_MAX_QUESTIONS];
+};
+
+// ------------------------------------------------------------------------------ Eq. 6
+template <typename T>
+__global__ void __launch_bounds__(256) qpool_kernel(const T* __restrict__ qtok, const QMeta meta, int Hq, int Hkv,
+                                                    int D, double* __restrict__ q64, double* __restrict__ qnorm) {
+  __shared__ double s_part[8];
+  const int qi = blockIdx.x;
+  const int C = Hkv * D, G = Hq / Hkv;
+  const int n0 = meta.off[qi], n1 = meta.off[qi + 1];
+  double sq = 0.0;
+  for (int col = threadIdx.x; col < C; col += blockDim.x) {
+    const int g = col / D, d = col % D;
+    double t = 0.0;
+    for (int n = n0; n < n1; ++n) {
+      const T* row = qtok + ((long long)n * Hq + (long long)g * G) * D + d;
+      for (int j = 0; j < G; ++j) t += (double)elem_to_float<T>(row[(long long)j * D]);
+    }
+    t = t / (double)((long long)(n1 - n0) * G);
+    q64[(long long)qi * C + col] = t;
+    sq += t * t;
+  }
+  sq = warp_sum(sq);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = sq;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += s_part[w];
+    qnorm[qi] = sqrt(t);
+  }
+}
+
+// ------------------------------------------------------------------------------ Eq. 7
+// Rows 0..n_frm-1 are frame keys, rows n_frm..n_frm+n_seg-1 segment keys.  A block stages
+// kScanRows rows in shared memory; thread (warp w, lane r) owns row r and the questions
+// w, w+8, ...: the row value is converted once and reused for kScanQ questions.
+constexpr int kScanRows = 32;
+constexpr int kScanQ = 4;
+
+__global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ frame_key,
+                                                   const float* __restrict__ seg_key, long long n_frm,
+                                                   long long n_seg, int C, int nq, const double* __restrict__ q64,
+                                                   const double* __restrict__ qnorm, double* __restrict__ s_frm,
+                                                   double* __restrict__ s_seg, long long frm_stride,
+                                                   long long seg_stride) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* rows = reinterpret_cast<float*>(smem_raw);                 // [kScanRows][C+1]
+  const int CS = C + 1;
+  const long long row0 = (long long)blockIdx.x * kScanRows;
+  const long long n_rows = n_frm + n_seg;
+  for (int v = threadIdx.x; v < kScanRows * C; v += blockDim.x) {
+    const int r = v / C, c = v % C;
+    const long long row = row0 + r;
+    float x = 0.f;
+    if (row < n_frm) x = frame_key[row * C + c];
+    else if (row < n_rows) x = seg_key[(row - n_frm) * C + c];
+    rows[r * CS + c] = x;
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long row = row0 + lane;
+  const float* mine = rows + lane * CS;
+  double kk = 0.0;
+  for (int c = 0; c < C; ++c) {
+    const double x = (double)mine[c];
+    kk = fma(x, x, kk);
+  }
+  const double knorm = sqrt(kk);
+  for (int qb = warp * kScanQ; qb < nq; qb += 8 * kScanQ) {
+    double acc[kScanQ];
+#pragma unroll
+    for (int i = 0; i < kScanQ; ++i) acc[i] = 0.0;
+    for (int c = 0; c < C; ++c) {
+      const double x = (double)mine[c];
+#pragma unroll
+      for (int i = 0; i < kScanQ; ++i) {
+        const int qi = min(qb + i, nq - 1);
+        acc[i] = fma(x, __ldg(q64 + (long long)qi * C + c), acc[i]);
+      }
+    }
+    if (row < n_rows) {
+#pragma unroll
+      for (int i = 0; i < kScanQ; ++i) {
+        const int qi = qb + i;
+        if (qi < nq) {
+          double den = knorm * qnorm[qi];
+          den = den > 1e-12 ? den : 1e-12;
+          const double s = acc[i] / den;
+          if (row < n_frm) s_frm[(long long)qi * frm_stride + row] = s;
+          else s_seg[(long long)qi * seg_stride + (row - n_frm)] = s;
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------ ranking
+__device__ __forceinline__ unsigned long long order_key(double x) {
+  const unsigned long long b = (unsigned long long)__double_as_longlong(x);
+  return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
+}
+__device__ __forceinline__ double order_key_inv(unsigned long long k) {
+  const unsigned long long b = (k >> 63) ? (k & 0x7fffffffffffffffull) : ~k;
+  return __longlong_as_double((long long)b);
+}
+
+struct RankScratch {
+  unsigned int hist[256];
+  int scan[40];
+  unsigned long long prefix;
+  int remaining;
+};
+
+// Indices of the k highest scores among i in [0,n) with member(i) true, ascending by index, with
+// the tie band: tau = k-th largest; scores above tau+delta are taken; those within delta of tau
+// share the remaining places by lowest index.  Run by the whole block; returns the count
+// (= min(k, number of members)).  score(i) must be cheap and pure.
+template <typename ScoreFn, typename MemberFn>
+__device__ int block_topk_set(ScoreFn score, MemberFn member, int n, int k, double delta, int* out_idx,
+                              double* out_score, RankScratch* sc) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  // how many members are there at all
+  int local = 0;
+  for (int i = tid; i < n; i += nt) local += member(i) ? 1 : 0;
+  __syncthreads();
+  if (tid == 0) sc->remaining = 0;
+  __syncthreads();
+  local = warp_sum(local);
+  if ((tid & 31) == 0 && local) atomicAdd(&sc->remaining, local);
+  __syncthreads();
+  const int n_mem = sc->remaining;
+  __syncthreads();
+  if (k > n_mem) k = n_mem;
+  if (k <= 0) return 0;
+  double tau;
+  if (k == n_mem) {
+    tau = -1.0e300;     // everything is taken; handled below by the "all" flag
+  } else {
+    // radix select of the k-th largest order key, 8 bits per pass from the top
+    if (tid == 0) { sc->prefix = 0ull; sc->remaining = k; }
+    for (int pass = 0; pass < 8; ++pass) {
+      const int shift = 56 - 8 * pass;
+      for (int b = tid; b < 256; b += nt) sc->hist[b] = 0u;
+      __syncthreads();
+      const unsigned long long prefix = sc->prefix;
+      const unsigned long long himask = pass == 0 ? 0ull : (~0ull << (shift + 8));
+      for (int i = tid; i < n; i += nt) {
+        if (!member(i)) continue;
+        const unsigned long long key = order_key(score(i));
+        if ((key & himask) == prefix) atomicAdd(&sc->hist[(unsigned)(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int rem = sc->remaining;
+        int b = 255;
+        for (; b > 0; --b) {
+          const int c = (int)sc->hist[b];
+          if (rem <= c) break;
+          rem -= c;
+        }
+        sc->prefix = prefix | ((unsigned long long)b << shift);
+        sc->remaining = rem;
+      }
+      __syncthreads();
+    }
+    tau = order_key_inv(sc->prefix);
+  }
+  const bool all = (k == n_mem);
+  // count the sure ones
+  int cnt = 0;
+  for (int i = tid; i < n; i += nt)
+    if (member(i) && !all && score(i) > tau + delta) ++cnt;
+  __syncthreads();
+  if (tid == 0) sc->remaining = 0;
+  __syncthreads();
+  cnt = warp_sum(cnt);
+  if ((tid & 31) == 0 && cnt) atomicAdd(&sc->remaining, cnt);
+  __syncthreads();
+  const int need = k - sc->remaining;
+  __syncthreads();
+  // ordered emission
+  int band_before = 0, out_before = 0;
+  for (int base = 0; base < n; base += nt) {
+    const int i = base + tid;
+    bool sure = false, band = false;
+    double s = 0.0;
+    if (i < n && member(i)) {
+      s = score(i);
+      if (all) sure = true;
+      else {
+        sure = s > tau + delta;
+        band = !sure && s >= tau - delta;
+      }
+    }
+    int n_band, n_out;
+    const int br = band_before + block_excl_count(band, sc->scan, n_band);
+    const bool keep = sure || (band && br < need);
+    const int pos = out_before + block_excl_count(keep, sc->scan, n_out);
+    if (keep) {
+      out_idx[pos] = i;
+      if (out_score) out_score[pos] = s;
+    }
+    band_before += n_band;
+    out_before += n_out;
+  }
+  __syncthreads();
+  return k;
+}
+
+struct RankParams {
+  int nq, C, fseg;
+  int k_seg, k_frm, top_n, mode;
+  double lambda, delta;
+  long long n_frm, n_seg;                 // stored
+  const double* s_frm;                    // [nq][frm_stride]
+  const double* s_seg;
+  long long frm_stride, seg_stride;
+  const float* frame_key;
+  const float* seg_key;
+  int* seg_idx; int* frm_idx; float* seg_score; float* frm_score; int* counts;
+};
+
+constexpr int kRankThreads = 512;
+constexpr int kMaxCand = 2 * MUKV_MAX_TOPK;
+
+__global__ void __launch_bounds__(kRankThreads) rank_kernel(const RankParams p, const QMeta meta) {
+  __shared__ RankScratch sc;
+  __shared__ int s_sel_seg[MUKV_MAX_TOPK];
+  __shared__ double s_sel_seg_score[MUKV_MAX_TOPK];
+  __shared__ int s_top[MUKV_MAX_TOPK];
+  __shared__ int s_cand[kMaxCand];
+  __shared__ double s_cand_score[kMaxCand];
+  __shared__ double s_new[kMaxCand];
+  __shared__ int s_pick[MUKV_MAX_TOPK];
+  __shared__ double s_pick_score[MUKV_MAX_TOPK];
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* gq = reinterpret_cast<double*>(smem_raw);               // [C] global query
+  __shared__ double s_gn;
+
+  const int qi = blockIdx.x, tid = threadIdx.x;
+  const int C = p.C;
+  long long tl = meta.t_limit[qi];
+  if (tl > p.n_frm) tl = p.n_frm;
+  if (tl < 0) tl = 0;
+  const int n_frm = (int)tl;
+  // segment u is visible when its last stored frame is: min((u+1)*fseg, n_stored) <= t_limit
+  int n_seg = (int)(tl / p.fseg);
+  if (tl == p.n_frm && (p.n_frm % p.fseg) != 0) n_seg += 1;
+  if (n_seg > p.n_seg) n_seg = (int)p.n_seg;
+  const double* sf = p.s_frm + (long long)qi * p.frm_stride;
+  const double* ss = p.s_seg + (long long)qi * p.seg_stride;
+  auto seg_score = [&](int i) { return ss[i]; };
+  auto frm_score = [&](int i) { return sf[i]; };
+  auto always = [](int) { return true; };
+
+  // ---- segments: lambda = 0, final = stage-1 top-k
+  const int c_seg = block_topk_set(seg_score, always, n_seg, p.k_seg, p.delta, s_sel_seg, s_sel_seg_score, &sc);
+  for (int i = tid; i < p.k_seg; i += kRankThreads) {
+    p.seg_idx[(long long)qi * p.k_seg + i] = i < c_seg ? s_sel_seg[i] : -1;
+    if (p.seg_score) p.seg_score[(long long)qi * p.k_seg + i] = i < c_seg ? (float)s_sel_seg_score[i] : 0.f;
+  }
+  __syncthreads();
+
+  int c_frm = 0;
+  if (p.mode == MUKV_RETR_PARALLEL) {
+    c_frm = block_topk_set(frm_score, always, n_frm, p.k_frm, p.delta, s_pick, s_pick_score, &sc);
+  } else if (p.mode == MUKV_RETR_HIER) {
+    const int fseg = p.fseg;
+    auto inside = [&](int t) {
+      const int u = t / fseg;
+      for (int i = 0; i < c_seg; ++i)
+        if (s_sel_seg[i] == u) return true;
+      return false;
+    };
+    c_frm = block_topk_set(frm_score, inside, n_frm, p.k_frm, p.delta, s_pick, s_pick_score, &sc);
+  } else {
+    // stage 1: top-2k frame candidates
+    const int n_cand = block_topk_set(frm_score, always, n_frm, 2 * p.k_frm, p.delta, s_cand, s_cand_score, &sc);
+    // global query = mean of the top-N segment keys
+    const int N = p.top_n > 0 ? p.top_n : p.k_seg;
+    const int n_top = block_topk_set(seg_score, always, n_seg, N, p.delta, s_top, (double*)nullptr, &sc);
+    double part = 0.0;
+    for (int c = tid; c < C; c += kRankThreads) {
+      double t = 0.0;
+      for (int i = 0; i < n_top; ++i) t += (double)p.seg_key[(long long)s_top[i] * C + c];
+      t = n_top > 0 ? t / (double)n_top : 0.0;
+      gq[c] = t;
+      part += t * t;
+    }
+    if (tid == 0) s_gn = 0.0;
+    __syncthreads();
+    part = warp_sum(part);
+    if ((tid & 31) == 0) atomicAdd(&s_gn, part);
+    __syncthreads();
+    const double gnorm = sqrt(s_gn);
+    // Eq. 8 for every candidate: one warp per candidate
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int ci = warp; ci < n_cand; ci += kRankThreads / 32) {
+      const float* kr = p.frame_key + (long long)s_cand[ci] * C;
+      double dot = 0.0, kk = 0.0;
+      for (int c = lane; c < C; c += 32) {
+        const double x = (double)kr[c];
+        dot = fma(x, gq[c], dot);
+        kk = fma(x, x, kk);
+      }
+      dot = warp_sum(dot);
+      kk = warp_sum(kk);
+      if (lane == 0) {
+        double gamma = 0.0;
+        if (n_top > 0) {
+          double den = sqrt(kk) * gnorm;
+          den = den > 1e-12 ? den : 1e-12;
+          gamma = dot / den;
+        }
+        s_new[ci] = (1.0 - p.lambda) * s_cand_score[ci] + p.lambda * gamma;
+      }
+    }
+    __syncthreads();
+    auto new_score = [&](int i) { return s_new[i]; };
+    c_frm = block_topk_set(new_score, always, n_cand, p.k_frm, p.delta, s_pick, s_pick_score, &sc);
+    // s_pick holds positions in the candidate list (ascending position = ascending frame id)
+    for (int i = tid; i < c_frm; i += kRankThreads) s_pick[i] = s_cand[s_pick[i]];
+    __syncthreads();
+  }
+  for (int i = tid; i < p.k_frm; i += kRankThreads) {
+    p.frm_idx[(long long)qi * p.k_frm + i] = i < c_frm ? s_pick[i] : -1;
+    if (p.frm_score) p.frm_score[(long long)qi * p.k_frm + i] = i < c_frm ? (float)s_pick_score[i] : 0.f;
+  }
+  if (tid == 0) {
+    p.counts[2 * qi] = c_seg;
+    p.counts[2 * qi + 1] = c_frm;
+  }
+}
+
+// ------------------------------------------------------------------------------ Eq. 9
+struct GatherParams {
+  int nq, k_frm, L, kappa;
+  long long run_bytes;                     // kappa * C * sizeof(T): one (frame, layer, K|V) run
+  const int* frm_idx; const int* counts;
+  const unsigned char* store; const long long* page_table; const int* kept_store;
+  unsigned char* decode; long long decode_stride;
+  int* tok_meta;
+};
+
+// unit = (question, plane = l*2+kv, slot): one contiguous run of the page goes to one contiguous
+// run of the decode buffer.
+__global__ void __launch_bounds__(256) gather_kernel(const GatherParams p) {
+  const long long planes = (long long)p.L * 2;
+  const long long n_units = (long long)p.nq * planes * p.k_frm;
+  for (long long u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const int slot = (int)(u % p.k_frm);
+    const long long r = u / p.k_frm;
+    const int plane = (int)(r % planes);
+    const int qi = (int)(r / planes);
+    if (slot >= p.counts[2 * qi + 1]) continue;
+    const int f = p.frm_idx[(long long)qi * p.k_frm + slot];
+    const unsigned char* src = p.store + p.page_table[f] + (long long)plane * p.run_bytes;
+    unsigned char* dst = p.decode + (long long)qi * p.decode_stride +
+                         ((long long)plane * p.k_frm + slot) * p.run_bytes;
+    const long long nvec = p.run_bytes >> 4;
+    long long v = threadIdx.x;
+    for (; v + 3 * 256 < nvec; v += 4 * 256) {
+      uint4 x0 = ld_stream(src + (v << 4));
+      uint4 x1 = ld_stream(src + ((v + 256) << 4));
+      uint4 x2 = ld_stream(src + ((v + 512) << 4));
+      uint4 x3 = ld_stream(src + ((v + 768) << 4));
+      st_stream(dst + (v << 4), x0);
+      st_stream(dst + ((v + 256) << 4), x1);
+      st_stream(dst + ((v + 512) << 4), x2);
+      st_stream(dst + ((v + 768) << 4), x3);
+    }
+    for (; v < nvec; v += 256) st_stream(dst + (v << 4), ld_stream(src + (v << 4)));
+    if (plane == 0 && p.tok_meta) {
+      for (int t = threadIdx.x; t < p.kappa; t += 256) {
+        int* m = p.tok_meta + (((long long)qi * p.k_frm + slot) * p.kappa + t) * 2;
+        m[0] = f;
+        m[1] = p.kept_store[(long long)f * p.kappa + t];
+      }
+    }
+  }
+}
+
+}  // namespace mukv

@@ -1,0 +1,341 @@
+// Per-frame token scoring and selection (Sec. 3.3, Eq. 1-4 and the top-kappa rule).
+//
+// score_kernel<T, A, NC>: one thread block per (query head h, frame f).
+//   * Eq. 1: S = Q_h K_g^T / sqrt(D) over the frame's P tokens, row softmax, column sums.
+//     Lanes own key columns (j = lane + 32c), a warp walks the query rows four at a time, so
+//     the column sums stay in registers and only the row maximum / row sum cross lanes.
+//     The attention matrix is never written anywhere.
+//   * Eq. 2-3: the G query-head blocks that share key head g split that head's tokens and
+//     transform each key vector along the feature axis; sum of the D bin magnitudes per token.
+//   * The block that finishes a frame last (arrival counter, nobody waits) reduces the
+//     per-head partials in a fixed order, applies Eq. 4 and selects the kappa tokens.
+// T is the input element type, A the arithmetic type: float for the normal path, double for
+// the frames whose selection is too close to a tie boundary to trust single precision.
+#pragma once
+#include "common.cuh"
+
+namespace mukv {
+
+constexpr int kScoreThreads = 256;
+constexpr int kScoreWarps = kScoreThreads / 32;
+constexpr int kRowsPerStep = 4;
+
+struct ScoreParams {
+  int P, Hq, Hkv, D, G, kappa;
+  int n_frames;                 // frames in this chunk
+  int causal, keep_low;
+  float alpha, tie_eps, flag_margin, flat_ratio;
+  long long first_frame;
+  // inputs
+  const void* q;                // [n][P][Hq][D]
+  const void* k_last;           // [n][P][Hkv][D]  (last layer of K)
+  // scratch
+  void* colsum_part;            // A [F][Hq][P]
+  void* ifft_part;              // A [F][Hkv][P]
+  int* frame_counter;           // [F], zero between launches
+  int* flagged;                 // [F] frame slots needing the double pass
+  int* n_flagged;               // count (written by the float pass, read by the double pass)
+  // outputs
+  int* kept_store;              // [max_frames][kappa]
+  int* kept_out;                // [n][kappa] or null
+  float* scores_out;            // [3][n][P] or null
+  long long* frame_ts;          // [max_frames]
+  long long* page_table;        // [max_frames]
+  long long pages_off, page_bytes;
+  int refine;                   // 1: frames come from the flagged list, no further flagging
+};
+
+template <typename T>
+__host__ __device__ constexpr int score_row_stride(int D) { return D + ElemTraits<T>::kPad; }
+
+template <typename T, typename A>
+__host__ inline size_t score_smem_bytes(int P, int D) {
+  size_t ks = (size_t)P * score_row_stride<T>(D) * sizeof(T);
+  size_t qs = (size_t)kScoreWarps * kRowsPerStep * D * sizeof(T);
+  size_t tw = (size_t)D * 2 * sizeof(A);
+  size_t red = (size_t)kScoreWarps * 256 * sizeof(A);
+  size_t sel = (size_t)256 * sizeof(double) + 64 * sizeof(double) + 64 * sizeof(int);
+  return ((ks + 15) / 16) * 16 + qs + tw + red + sel + 64;
+}
+
+// Eq. 4 and the top-kappa rule for one frame, run by the whole block (blockDim.x >= P).
+// att_raw / fft_raw are this thread's token's I_att and I_fft; s_sc, s_int, s_misc are shared scratch.
+// The arithmetic here is always double: it is a few hundred operations per frame and keeps
+// the normalisation from adding rounding noise of its own to the scores.
+__device__ inline void select_frame(const ScoreParams& p, int f, double att_raw, double fft_raw, double* s_sc,
+                                    int* s_int, double* s_misc) {
+  typedef double A;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int P = p.P;
+  const bool valid = tid < P;
+  const A big = (A)3.0e38;
+  // ---- min / max of both signals over the frame
+  A v[4] = {valid ? att_raw : big, valid ? att_raw : -big, valid ? fft_raw : big, valid ? fft_raw : -big};
+  v[0] = warp_min(v[0]); v[1] = warp_max(v[1]); v[2] = warp_min(v[2]); v[3] = warp_max(v[3]);
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s_misc[warp * 4 + i] = v[i];
+  }
+  __syncthreads();
+  A amin = big, amax = -big, fmin_ = big, fmax_ = -big;
+  for (int w = 0; w < kScoreWarps; ++w) {
+    amin = s_misc[w * 4 + 0] < amin ? s_misc[w * 4 + 0] : amin;
+    amax = s_misc[w * 4 + 1] > amax ? s_misc[w * 4 + 1] : amax;
+    fmin_ = s_misc[w * 4 + 2] < fmin_ ? s_misc[w * 4 + 2] : fmin_;
+    fmax_ = s_misc[w * 4 + 3] > fmax_ ? s_misc[w * 4 + 3] : fmax_;
+  }
+  __syncthreads();
+  // ---- Eq. 4
+  A an = (amax == amin) ? (A)0 : (att_raw - amin) / (amax - amin);
+  A fn = (fmax_ == fmin_) ? (A)0 : (fft_raw - fmin_) / (fmax_ - fmin_);
+  if (p.keep_low) fn = (A)1 - fn;
+  const A alpha = (A)p.alpha;
+  const A s = alpha * an + ((A)1 - alpha) * fn;
+  if (valid) s_sc[tid] = s;
+  __syncthreads();
+  // ---- tau = kappa-th largest score (rank counting; P <= 256)
+  const int kappa = p.kappa;
+  if (valid) {
+    int gt = 0, ge = 0;
+    for (int i = 0; i < P; ++i) {
+      const A o = s_sc[i];
+      gt += (o > s);
+      ge += (o >= s);
+    }
+    if (gt < kappa && kappa <= ge) s_misc[0] = s;      // every writer holds the same value
+  }
+  __syncthreads();
+  const A tau = s_misc[0];
+  const A delta = (A)p.tie_eps;
+  const bool sure = valid && (s > tau + delta);
+  const bool band = valid && !sure && (s >= tau - delta);
+  int n_sure, n_dummy;
+  block_excl_count(sure, s_int, n_sure);
+  const int band_rank = block_excl_count(band, s_int, n_dummy);
+  const bool keep = sure || (band && band_rank < kappa - n_sure);
+  int n_keep;
+  const int pos = block_excl_count(keep, s_int, n_keep);
+  const long long f_abs = p.first_frame + f;
+  if (keep) {
+    p.kept_store[f_abs * kappa + pos] = tid;
+    if (p.kept_out) p.kept_out[(long long)f * kappa + pos] = tid;
+  }
+  if (p.scores_out && valid) {
+    const long long np = (long long)p.n_frames * P;
+    p.scores_out[0 * np + (long long)f * P + tid] = (float)att_raw;
+    p.scores_out[1 * np + (long long)f * P + tid] = (float)fft_raw;
+    p.scores_out[2 * np + (long long)f * P + tid] = (float)s;
+  }
+  if (tid == 0) {
+    p.frame_ts[f_abs] = f_abs;
+    p.page_table[f_abs] = p.pages_off + f_abs * p.page_bytes;
+  }
+  // ---- does single precision decide this frame safely?
+  if (!p.refine) {
+    const A m = (A)p.flag_margin;
+    const A da = s - (tau + delta), db = s - (tau - delta);
+    bool risky = valid && ((da <= m && da >= -m) || (db <= m && db >= -m));
+    // a nearly flat signal amplifies rounding noise through the min-max division
+    if (tid == 0) {
+      const A fr = (A)p.flat_ratio;
+      const A aabs = amax > -amin ? amax : -amin, fabs_ = fmax_ > -fmin_ ? fmax_ : -fmin_;
+      if (amax != amin && (amax - amin) < fr * aabs && p.alpha != 0.f) risky = true;
+      if (fmax_ != fmin_ && (fmax_ - fmin_) < fr * fabs_ && p.alpha != 1.f) risky = true;
+    }
+    int n_risky;
+    block_excl_count(risky, s_int, n_risky);
+    if (tid == 0 && n_risky > 0) {
+      const int slot = atomicAdd(p.n_flagged, 1);
+      p.flagged[slot] = f;
+    }
+  }
+}
+
+template <typename T, typename A, int NC>
+__global__ void __launch_bounds__(kScoreThreads) score_kernel(const ScoreParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int h = blockIdx.x;
+  int f = blockIdx.y;
+  if (p.refine) {
+    if ((int)blockIdx.y >= *p.n_flagged) return;
+    f = p.flagged[blockIdx.y];
+  }
+  const int P = p.P, D = p.D, Hq = p.Hq, Hkv = p.Hkv, G = p.G;
+  const int g = h / G;
+  constexpr int EPW = ElemTraits<T>::kPerWord;
+  const int DS = score_row_stride<T>(D);
+  const int WS = DS / EPW;                         // words per padded K row
+  const int DW = D / EPW;                          // words per vector
+
+  // ---- shared memory carve-up
+  size_t off = 0;
+  T* Ks = reinterpret_cast<T*>(smem_raw);
+  off = (((size_t)P * DS * sizeof(T)) + 15) / 16 * 16;
+  T* Qs = reinterpret_cast<T*>(smem_raw + off);
+  off += (size_t)kScoreWarps * kRowsPerStep * D * sizeof(T);
+  A* tw = reinterpret_cast<A*>(smem_raw + off);
+  off += (size_t)D * 2 * sizeof(A);
+  A* red = reinterpret_cast<A*>(smem_raw + off);
+  off += (size_t)kScoreWarps * 256 * sizeof(A);
+  double* s_sc = reinterpret_cast<double*>(smem_raw + off);
+  off += (size_t)256 * sizeof(double);
+  double* s_misc = reinterpret_cast<double*>(smem_raw + off);
+  off += 64 * sizeof(double);
+  int* s_int = reinterpret_cast<int*>(smem_raw + off);
+
+  // ---- stage K_g of this frame (rows padded so that 32 consecutive rows hit 32 banks)
+  const T* Kg = reinterpret_cast<const T*>(p.k_last) + ((long long)f * P * Hkv + g) * D;
+  {
+    constexpr int VE = 16 / sizeof(T);             // elements per 16-byte vector
+    const int vec_per_row = D / VE;
+    for (int v = tid; v < P * vec_per_row; v += kScoreThreads) {
+      const int j = v / vec_per_row, c = v % vec_per_row;
+      const uint4 x = *reinterpret_cast<const uint4*>(Kg + (long long)j * Hkv * D + c * VE);
+      uint32_t* dst = reinterpret_cast<uint32_t*>(Ks + (size_t)j * DS + c * VE);
+      dst[0] = x.x; dst[1] = x.y; dst[2] = x.z; dst[3] = x.w;
+    }
+    for (int d = tid; d < D; d += kScoreThreads) {
+      double sn, cs;
+      sincospi(2.0 * (double)d / (double)D, &sn, &cs);
+      tw[2 * d] = (A)cs;
+      tw[2 * d + 1] = (A)sn;
+    }
+  }
+  __syncthreads();
+
+  // ---- Eq. 1: column sums of the row softmax
+  const uint32_t* Kw = reinterpret_cast<const uint32_t*>(Ks);
+  uint32_t* Qw = reinterpret_cast<uint32_t*>(Qs) + (size_t)warp * kRowsPerStep * DW;
+  const T* Qh = reinterpret_cast<const T*>(p.q) + ((long long)f * P * Hq + h) * D;
+  // 1/sqrt(D) as a two-term constant, so that single precision scales the logits without a
+  // systematic relative error shared by every element
+  const double scale_d = 1.0 / sqrt((double)D);
+  const A scale = (A)scale_d;
+  const A scale_lo = (A)(scale_d - (double)scale);
+  A csum[NC];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) csum[c] = (A)0;
+  int jrow[NC];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) jrow[c] = min(lane + 32 * c, P - 1) * WS;
+
+  const int n_steps = (P + kRowsPerStep - 1) / kRowsPerStep;
+  for (int rb = warp; rb < n_steps; rb += kScoreWarps) {
+    __syncwarp();
+#pragma unroll
+    for (int r = 0; r < kRowsPerStep; ++r) {
+      const int i = rb * kRowsPerStep + r;
+      const uint32_t* src = reinterpret_cast<const uint32_t*>(Qh + (long long)min(i, P - 1) * Hq * D);
+      for (int w = lane; w < DW; w += 32) Qw[r * DW + w] = (i < P) ? __ldg(src + w) : 0u;
+    }
+    __syncwarp();
+    A acc[kRowsPerStep][NC];
+#pragma unroll
+    for (int r = 0; r < kRowsPerStep; ++r)
+#pragma unroll
+      for (int c = 0; c < NC; ++c) acc[r][c] = (A)0;
+#pragma unroll 2
+    for (int w = 0; w < DW; ++w) {
+      uint32_t qw[kRowsPerStep];
+#pragma unroll
+      for (int r = 0; r < kRowsPerStep; ++r) qw[r] = Qw[r * DW + w];
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const uint32_t kw = Kw[jrow[c] + w];
+#pragma unroll
+        for (int r = 0; r < kRowsPerStep; ++r) acc[r][c] = dot_word<T, A>(qw[r], kw, acc[r][c]);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < kRowsPerStep; ++r) {
+      const int i = rb * kRowsPerStep + r;
+      A z[NC];
+      A m = neg_inf<A>();
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const int j = lane + 32 * c;
+        const bool ok = (j < P) && (!p.causal || j <= i);
+        z[c] = ok ? fma_acc(acc[r][c], scale, acc[r][c] * scale_lo) : neg_inf<A>();
+        m = z[c] > m ? z[c] : m;
+      }
+      m = warp_max(m);
+      A l = (A)0;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        z[c] = (z[c] == neg_inf<A>()) ? (A)0 : exp_acc(z[c] - m);
+        l += z[c];
+      }
+      l = warp_sum(l);
+      const A inv = (i < P) ? (A)1 / l : (A)0;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) csum[c] += z[c] * inv;
+    }
+  }
+  // cross-warp reduction in a fixed order
+#pragma unroll
+  for (int c = 0; c < NC; ++c) red[warp * 256 + lane + 32 * c] = csum[c];
+  __syncthreads();
+  if (tid < P) {
+    A t = (A)0;
+    for (int w = 0; w < kScoreWarps; ++w) t += red[w * 256 + tid];
+    reinterpret_cast<A*>(p.colsum_part)[((long long)f * Hq + h) * P + tid] = t;
+  }
+
+  // ---- Eq. 2-3: sum over the D bins of |DFT(k_j)| for this block's share of head g's tokens
+  {
+    const int hg = h % G;
+    const int half = D / 2;
+    for (int j = hg + warp * G; j < P; j += kScoreWarps * G) {
+      const T* kr = Ks + (size_t)j * DS;
+      A total = (A)0;
+      // bins 1 .. D/2-1 (twice, by conjugate symmetry) and bin 0
+      for (int b = lane; b < half; b += 32) {
+        A re = (A)0, im = (A)0;
+        for (int d = 0; d < D; ++d) {
+          const A x = (A)elem_to_float<T>(kr[d]);
+          const int m = (b * d) & (D - 1);
+          re += x * tw[2 * m];
+          im -= x * tw[2 * m + 1];
+        }
+        const A mag = sqrt_acc(re * re + im * im);
+        total += (b == 0) ? mag : (A)2 * mag;
+      }
+      // bin D/2: alternating sum
+      A alt = (A)0;
+      for (int d = lane; d < D; d += 32) {
+        const A x = (A)elem_to_float<T>(kr[d]);
+        alt += (d & 1) ? -x : x;
+      }
+      total = warp_sum(total);
+      alt = warp_sum(alt);
+      if (lane == 0)
+        reinterpret_cast<A*>(p.ifft_part)[((long long)f * Hkv + g) * P + j] = total + (alt < (A)0 ? -alt : alt);
+    }
+  }
+
+  // ---- last block of the frame finishes Eq. 1 / Eq. 3 and selects
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int old = atomicAdd(p.frame_counter + f, 1);
+    s_int[63] = (old == Hq - 1);
+    if (old == Hq - 1) p.frame_counter[f] = 0;      // ready for the next launch
+  }
+  __syncthreads();
+  if (!s_int[63]) return;
+  __threadfence();
+  double att = 0.0, fft = 0.0;
+  if (tid < P) {
+    const A* cp = reinterpret_cast<const A*>(p.colsum_part) + (long long)f * Hq * P + tid;
+    for (int hh = 0; hh < Hq; ++hh) att += (double)__ldcg(cp + (long long)hh * P);
+    att = att / (double)((long long)Hq * P);
+    const A* fp = reinterpret_cast<const A*>(p.ifft_part) + (long long)f * Hkv * P + tid;
+    for (int gg = 0; gg < Hkv; ++gg) fft += (double)__ldcg(fp + (long long)gg * P);
+    fft = fft / (double)((long long)Hkv * D);
+  }
+  __syncthreads();
+  select_frame(p, f, att, fft, s_sc, s_int, s_misc);
+}
+
+}  // namespace mukv

@@ -68,17 +68,21 @@ def normal_table() -> np.ndarray:
     return _TABLE
 
 
-def normals(key: int, count: int) -> np.ndarray:
-    """float32 N(0,1) values for element indices 0..count-1 of stream ``key``.
+def normals(key: int, count: int, start: int = 0) -> np.ndarray:
+    """float32 N(0,1) values for element indices start..start+count-1 of stream ``key``.
 
     Element e uses 16 bits of hash word e >> 2 (four elements per 64-bit word).
     """
-    e = np.arange(count, dtype=np.uint64)
+    if count <= 0:
+        return np.zeros(0, dtype=np.float32)
+    w0, w1 = start >> 2, (start + count + 3) >> 2
+    words = np.arange(w0, w1, dtype=np.uint64)
     with np.errstate(over="ignore"):
-        w = np.uint64(key) + ((e >> np.uint64(2)) + np.uint64(1)) * np.uint64(GOLD)
-    h = _mix64_np(w)
-    idx = (h >> ((e & np.uint64(3)) * np.uint64(16))) & np.uint64(0xFFFF)
-    return normal_table()[idx.astype(np.int64)]
+        h = _mix64_np(np.uint64(key) + (words + np.uint64(1)) * np.uint64(GOLD))
+    shifts = np.array([0, 16, 32, 48], dtype=np.uint64)
+    idx = ((h[:, None] >> shifts[None, :]) & np.uint64(0xFFFF)).reshape(-1).astype(np.int64)
+    lo = start - (w0 << 2)
+    return normal_table()[idx[lo:lo + count]]
 
 
 def to_bf16_bits(x: np.ndarray) -> np.ndarray:
@@ -156,17 +160,20 @@ class StreamSpec:
         L, H, D = self.n_layers, self.n_kv_heads, self.head_dim
         return normals(stream_key(self.seed, TAG_MU, int(c)), L * H * D).reshape(L, H, D)
 
-    def frame_kv(self, t: int):
-        """K, V of absolute frame t: [L][P][Hkv][D] each."""
+    def frame_kv(self, t: int, last_layer_only: bool = False):
+        """K, V of absolute frame t: [L][P][Hkv][D] each ([1][P][Hkv][D] with last_layer_only)."""
         L, H, D, P = self.n_layers, self.n_kv_heads, self.head_dim, self.tokens_per_frame
-        cnt = L * P * H * D
-        scale = self.out_scale()[:, None, :, :]
-        k = normals(stream_key(self.seed, TAG_K, t), cnt).reshape(L, P, H, D) * scale
-        v = normals(stream_key(self.seed, TAG_V, t), cnt).reshape(L, P, H, D) * scale
+        l0 = L - 1 if last_layer_only else 0
+        n_l = L - l0
+        start, cnt = l0 * P * H * D, n_l * P * H * D
+        scale = self.out_scale()[l0:, None, :, :]
+        k = normals(stream_key(self.seed, TAG_K, t), cnt, start).reshape(n_l, P, H, D) * scale
+        v = normals(stream_key(self.seed, TAG_V, t), cnt, start).reshape(n_l, P, H, D) * scale
         if self.has_scenes:
             c = int(self.scene_of_frame()[t])
-            mu = self.scene_mean(c) * np.float32(self.scene_sigma)
-            nu = normals(stream_key(self.seed, TAG_NU, t), L * H * D).reshape(L, H, D) * np.float32(self.frame_sigma)
+            mu = self.scene_mean(c)[l0:] * np.float32(self.scene_sigma)
+            nu = normals(stream_key(self.seed, TAG_NU, t), n_l * H * D, l0 * H * D).reshape(n_l, H, D) \
+                * np.float32(self.frame_sigma)
             k = (k + mu[:, None, :, :]) + nu[:, None, :, :]
         return self._finish(k), self._finish(v)
 
@@ -175,11 +182,11 @@ class StreamSpec:
         P, Hq, D = self.tokens_per_frame, self.n_q_heads, self.head_dim
         return self._finish(normals(stream_key(self.seed, TAG_Q, t), P * Hq * D).reshape(P, Hq, D))
 
-    def chunk(self, t0: int, n: int):
+    def chunk(self, t0: int, n: int, last_layer_only: bool = False):
         """Q[n][P][Hq][D], K[L][n][P][Hkv][D], V[L][n][P][Hkv][D] for frames t0..t0+n-1."""
         qs, ks, vs = [], [], []
         for t in range(t0, t0 + n):
-            k, v = self.frame_kv(t)
+            k, v = self.frame_kv(t, last_layer_only)
             qs.append(self.frame_q(t))
             ks.append(k)
             vs.append(v)

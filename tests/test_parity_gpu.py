@@ -1,0 +1,190 @@
+"""CUDA path vs CPU oracle, through the C ABI, on the same seeded inputs.
+
+Bar: kept-token / segment / frame indices and gathered bytes bit-exact; scores and pooled
+entries within 1e-3 relative + 1e-5 absolute.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mukv_oracle as O
+from paper_2605_22269_b200 import binding as B
+from paper_2605_22269_b200.synth.cpu import StreamSpec, workload
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def full_compress_check(run: H.GpuRun, chunk=None):
+    """Whole (small) stream: every frame, every layer, segment entries, keys, timestamps."""
+    run.compress(chunk)
+    spec, cfg = run.spec, run.cfg
+    T = run.n_frames
+    st = H.oracle_stream(spec, H.oracle_cfg(cfg), range(T), last_only=False, workers=1)
+    H.check_frames_against_oracle(run, st, range(T), full_layers=True)
+    seg = run.ctx.region(3).cpu().numpy()
+    fkey = run.ctx.region(4).cpu().numpy()
+    skey = run.ctx.region(5).cpu().numpy()
+    for t in range(T):
+        assert fkey[t].tobytes() == st.frame_key(t).tobytes(), f"frame key {t} not bit-exact"
+    assert st.n_segments == (T + cfg.frames_per_segment - 1) // cfg.frames_per_segment
+    for u in range(st.n_segments):
+        sk, sv = st.segment_entry(u)
+        H.close(seg[u][:, 0], sk, f"segment entry K {u}")
+        H.close(seg[u][:, 1], sv, f"segment entry V {u}")
+        assert skey[u].tobytes() == st.segment_key(u).tobytes(), f"segment key {u} not bit-exact"
+    ts = run.ctx.region(6).cpu().numpy()[:T]
+    assert ts.tolist() == list(range(T))
+    stats = run.ctx.mukv_get_stats()
+    assert stats.frames == T and stats.segments == st.n_segments and stats.kept_tokens == T * cfg.keep_per_frame
+    return st
+
+
+def retrieval_check(run: H.GpuRun, st: O.Store, qtok, offs, k_seg, k_frm, lam, mode, t_limit=None, top_n=0):
+    nq = len(offs) - 1
+    ret = run.retrieve(qtok, offs, k_seg, k_frm, top_n, lam, mode, t_limit)
+    dec, meta = run.gather(ret, k_frm)
+    seg_idx, frm_idx = ret["seg_idx"].cpu().numpy(), ret["frm_idx"].cpu().numpy()
+    seg_sc, frm_sc = ret["seg_score"].cpu().numpy(), ret["frm_score"].cpu().numpy()
+    counts = ret["counts"].cpu().numpy()
+    kap = run.cfg.keep_per_frame
+    dec_np = H.to_numpy_bits(dec)
+    meta_np = meta.cpu().numpy()
+    for i in range(nq):
+        r = O.retrieve(st, qtok[offs[i]:offs[i + 1]], k_seg, k_frm, top_n, lam, mode,
+                       None if t_limit is None else int(t_limit[i]))
+        ns, nf = len(r["seg_idx"]), len(r["frm_idx"])
+        assert counts[i].tolist() == [ns, nf], f"question {i}: counts {counts[i]} vs {(ns, nf)}"
+        assert seg_idx[i, :ns].tolist() == r["seg_idx"].tolist(), f"question {i}: segments differ"
+        assert frm_idx[i, :nf].tolist() == r["frm_idx"].tolist(), f"question {i}: frames differ"
+        assert np.all(seg_idx[i, ns:] == -1) and np.all(frm_idx[i, nf:] == -1)
+        H.close(seg_sc[i, :ns], r["seg_score"], f"question {i} segment scores")
+        H.close(frm_sc[i, :nf], r["frm_score"], f"question {i} frame scores")
+        if st.cfg["n_layers"] == run.cfg.n_layers and nf > 0:
+            ref_dec, ref_meta = O.gather(st, r["frm_idx"])
+            assert dec_np[i][:, :, :nf * kap].tobytes() == ref_dec.tobytes(), f"question {i}: gathered bytes differ"
+            assert meta_np[i, :nf * kap].tolist() == ref_meta.tolist()
+    return ret
+
+
+def questions(run, n_q=None, q_len=None):
+    wl = run.wl
+    n_q = n_q or wl["n_questions"]
+    lo, hi = q_len or wl["q_len"]
+    return run.spec.questions(n_q, lo, hi)
+
+
+# ------------------------------------------------------------------------------- config 1
+def test_tiny_fp32_full_parity():
+    run = H.GpuRun("tiny")
+    st = full_compress_check(run)
+    qtok, offs, _ = questions(run)
+    wl = run.wl
+    for mode in (B.RETR_SEMI, B.RETR_PARALLEL, B.RETR_HIER):
+        retrieval_check(run, st, qtok, offs, wl["k_seg"], wl["k_frm"], wl["lam"], mode)
+
+
+def test_tiny_chunking_and_partial_segment():
+    # 7 frames in chunks of 3 with segments of 4: segments straddle chunks, the last one is partial
+    wl = dict(workload("tiny"))
+    run = H.GpuRun(wl, n_frames=7)
+    st = full_compress_check(run, chunk=3)
+    qtok, offs, _ = run.spec.questions(3, 1, 9)
+    retrieval_check(run, st, qtok, offs, 2, 3, 0.3, B.RETR_SEMI)
+    retrieval_check(run, st, qtok, offs, 2, 3, 0.3, B.RETR_SEMI, t_limit=np.array([5, 4, 7]))
+    retrieval_check(run, st, qtok, offs, 50, 50, 0.5, B.RETR_SEMI)          # k larger than what exists
+
+
+@pytest.mark.parametrize("over", [dict(attn_causal=1), dict(keep_low_freq=1), dict(alpha=0.0), dict(alpha=1.0),
+                                  dict(alpha=0.5), dict(keep_per_frame=1), dict(keep_per_frame=64)])
+def test_tiny_variants(over):
+    run = H.GpuRun("tiny", **over)
+    full_compress_check(run)
+
+
+def test_odd_shapes_bf16():
+    # P not a multiple of 32 or 4, GQA with G = 3, D = 64, ragged chunks
+    spec = StreamSpec(seed=11, n_layers=3, n_q_heads=6, n_kv_heads=2, head_dim=64, tokens_per_frame=77,
+                      bf16=True, n_outlier=2, n_frames=11, scene_sigma=1.0, frame_sigma=0.5, scene_min=3, scene_max=5)
+    wl = dict(spec=spec, keep=19, fseg=4, chunk=5, alpha=0.7, n_questions=4, q_len=(1, 7), k_seg=2, k_frm=3, lam=0.3)
+    run = H.GpuRun(wl)
+    st = full_compress_check(run)
+    qtok, offs, _ = questions(run)
+    for mode in (B.RETR_SEMI, B.RETR_PARALLEL, B.RETR_HIER):
+        retrieval_check(run, st, qtok, offs, 2, 3, 0.3, mode)
+
+
+def test_degenerate_inputs():
+    # constant keys and zero queries: both signals flat, every score 0, lowest indices kept
+    run = H.GpuRun("tiny")
+    c = run.cfg
+    P, L = c.tokens_per_frame, c.n_layers
+    q = torch.zeros((2, P, c.n_q_heads, c.head_dim), device="cuda:0")
+    k = torch.full((L, 2, P, c.n_kv_heads, c.head_dim), 0.5, device="cuda:0")
+    v = torch.ones_like(k)
+    kept = torch.zeros((2, c.keep_per_frame), dtype=torch.int32, device="cuda:0")
+    run.ctx.mukv_compress_chunk(q, k, v, 2, 0, kept, None)
+    torch.cuda.synchronize()
+    assert kept.cpu().numpy().tolist() == [list(range(c.keep_per_frame))] * 2
+    st = O.Store(H.oracle_cfg(c))
+    O.compress_chunk(st, q.cpu().numpy(), k.cpu().numpy(), v.cpu().numpy())
+    assert st.kept[0].tolist() == list(range(c.keep_per_frame))
+    assert torch.all(run.ctx.region(2)[0, :, 0] == 0.5) and torch.all(run.ctx.region(2)[1, :, 1] == 1.0)
+
+
+# ------------------------------------------------------------------------------- config 2
+def test_chunk7b_full_parity():
+    run = H.GpuRun("chunk7b")
+    st = full_compress_check(run)
+    worst = np.abs(run.scores[2] - np.stack([s[2] for s in st.scores])).max()
+    print(f"chunk7b: max |fused score - oracle| = {worst:.3e}; refined frames = "
+          f"{run.ctx.mukv_get_stats().refined_frames}")
+    qtok, offs, _ = questions(run)
+    wl = run.wl
+    retrieval_check(run, st, qtok, offs, wl["k_seg"], wl["k_frm"], wl["lam"], B.RETR_SEMI)
+
+
+def test_chunk7b_causal():
+    run = H.GpuRun("chunk7b", n_frames=4, attn_causal=1)
+    full_compress_check(run)
+
+
+# ------------------------------------------------------------------------------- config 3
+def test_stream_1h():
+    run = H.GpuRun("stream_1h").compress()
+    spec, cfg = run.spec, run.cfg
+    T = run.n_frames
+    assert T == 1800 and run.ctx.mukv_get_stats().segments == 113
+    # every frame: kept ids and scores (oracle on the last layer, which is all that scoring reads)
+    st = H.oracle_stream(spec, H.oracle_cfg(cfg), range(T), last_only=True)
+    worst = H.check_frames_against_oracle(run, st, range(T), full_layers=False)
+    print(f"stream_1h: max |fused score - oracle| = {worst:.3e}; refined = {run.ctx.mukv_get_stats().refined_frames}")
+    fkey = run.ctx.region(4).cpu().numpy()[:T]
+    assert fkey.tobytes() == st.frame_keys().tobytes()
+    skey = run.ctx.region(5).cpu().numpy()[:113]
+    assert skey.tobytes() == st.segment_keys().tobytes()
+    # sampled frames: all layers (pages, frame entries)
+    sample = [0, 1, 15, 16, 799, 1234, 1792, 1799]
+    st_full = H.oracle_stream(spec, H.oracle_cfg(cfg), sample, last_only=False, workers=1)
+    for i, t in enumerate(sample):
+        assert st_full.kept[i].tolist() == st.kept[t].tolist()
+    H.check_frames_against_oracle(run, st_full, sample, full_layers=True)
+    # the last segment is partial (8 frames)
+    seg = run.ctx.region(3)[112].cpu().numpy()
+    last = H.oracle_stream(spec, H.oracle_cfg(cfg), range(1792, 1800), last_only=False, workers=1)
+    sk = np.sum(last.sum_k, axis=0) / (8.0 * cfg.keep_per_frame)
+    H.close(seg[:, 0], sk.astype(np.float32), "partial segment entry")
+    # retrieval
+    qtok, offs, _ = questions(run)
+    wl = run.wl
+    ret = retrieval_check(run, st, qtok, offs, wl["k_seg"], wl["k_frm"], wl["lam"], B.RETR_SEMI)
+    retrieval_check(run, st, qtok, offs, wl["k_seg"], wl["k_frm"], wl["lam"], B.RETR_SEMI,
+                    t_limit=np.array([900, 1, 17, 1799, 1800, 16, 450, 1000]))
+    # gathered bytes of the first question against an all-layer oracle of its frames
+    frm = ret["frm_idx"].cpu().numpy()[0]
+    stq = H.oracle_stream(spec, H.oracle_cfg(cfg), frm.tolist(), last_only=False, workers=1)
+    ref_dec, ref_meta = O.gather(stq, range(len(frm)))
+    dec, meta = run.gather(ret, wl["k_frm"])
+    assert H.to_numpy_bits(dec)[0].tobytes() == ref_dec.tobytes()
+    assert meta.cpu().numpy()[0][:, 1].tolist() == ref_meta[:, 1].tolist()
+    assert meta.cpu().numpy()[0][:, 0].tolist() == np.repeat(frm, cfg.keep_per_frame).tolist()
