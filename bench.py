@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the MuKV compression + retrieval path on B200.
+
+A step is one pass of the whole path over the three-hour stream workload: 675 calls of
+mukv_compress_chunk (16 frames each, 10,800 frames) into an empty store, then one batched
+mukv_retrieve + mukv_gather for 64 questions.  The raw K/V of a chunk cannot all be resident
+(136 GB), so each chunk is generated on the device right before its call; the generator and an
+L2 flush run between the timed calls and are excluded: the step time is the sum of the
+CUDA-event intervals around the library calls.
+
+Prints ONE JSON line (rank 0).  `python bench.py --impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compressed_frames_per_s"
+UNIT = "frames/s"
+WORKLOAD = "stream_3h"
+
+
+def load_peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), source="measured")
+    return dict(hbm_gbs=6650.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=5)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+def algorithmic_bytes(cfg, k_frm: int) -> dict:
+    """Bytes the method has to move, per unit ('Rooflines')."""
+    es = 2 if cfg.dtype == 0 else 4
+    C = cfg.n_kv_heads * cfg.head_dim
+    P, L, kap = cfg.tokens_per_frame, cfg.n_layers, cfg.keep_per_frame
+    q = P * cfg.n_q_heads * cfg.head_dim * es
+    klast = P * C * es
+    kept = L * 2 * kap * C * es
+    pooled = L * 2 * C * 4
+    small = kap * 4 + C * 4 + C * 8 + 16
+    score = q + klast + P * 4 * (cfg.n_q_heads + cfg.n_kv_heads)           # inputs + partial sums
+    compact = 2 * kept + pooled + small
+    seg = pooled / cfg.frames_per_segment * 2
+    frame = q + klast + 2 * kept + pooled + pooled / cfg.frames_per_segment + small
+    gather_q = 2 * k_frm * kept
+    return dict(per_frame=frame, score_per_frame=score, compact_per_frame=compact, segment_per_frame=seg,
+                gather_per_question=gather_q, index_row=C * 4)
+
+
+def oracle_sample(n_frames: int, n_questions: int):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload.  Returns
+    (frames/s, retrievals/s, threads, description)."""
+    from threadpoolctl import threadpool_info
+    from oracle import mukv_oracle as O
+    from paper_2605_22269_b200.synth.cpu import workload
+    wl = workload(WORKLOAD)
+    spec = wl["spec"]
+    ocfg = dict(n_layers=spec.n_layers, n_q_heads=spec.n_q_heads, n_kv_heads=spec.n_kv_heads,
+                head_dim=spec.head_dim, tokens_per_frame=spec.tokens_per_frame, keep_per_frame=wl["keep"],
+                frames_per_segment=wl["fseg"], alpha=wl["alpha"])
+    q, k, v = spec.chunk(0, n_frames)                       # inputs generated outside the timed part
+    st = O.Store(ocfg)
+    t0 = time.perf_counter()
+    O.compress_chunk(st, q, k, v)
+    t_c = time.perf_counter() - t0
+    qtok, offs, _ = spec.questions(n_questions, *wl["q_len"])
+    t0 = time.perf_counter()
+    for i in range(n_questions):
+        r = O.retrieve(st, qtok[offs[i]:offs[i + 1]], wl["k_seg"], wl["k_frm"], 0, wl["lam"], O.MODE_SEMI)
+        O.gather(st, r["frm_idx"])
+    t_r = time.perf_counter() - t0
+    threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    desc = (f"first {n_frames} frames of the {WORKLOAD} stream compressed (all 28 layers), then {n_questions} "
+            f"questions retrieved+gathered from that {n_frames}-frame store; numpy float64")
+    return n_frames / t_c, n_questions / t_r, threads, desc
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for i in range(args.warmup + args.steps):
+        fps, rps, threads, desc = oracle_sample(args.oracle_frames, 4)
+        if i >= args.warmup:
+            vals.append((fps, rps))
+    fps = statistics.mean(v[0] for v in vals)
+    rps = statistics.mean(v[1] for v in vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * args.oracle_frames / fps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "step": desc},
+        "retrievals_per_s": rps,
+        "cpu_baseline": {"value": fps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": fps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--frames", type=int, default=0, help="shorten the stream (debugging / profiling only)")
+    ap.add_argument("--oracle-frames", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    from paper_2605_22269_b200 import binding as B
+    from paper_2605_22269_b200 import build as BUILD
+    from paper_2605_22269_b200 import dist as D
+    from paper_2605_22269_b200.synth.cpu import workload
+    from paper_2605_22269_b200.synth.gpu import GpuStream
+
+    BUILD.build()
+    rank, world, local = D.init_from_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    wl = workload(WORKLOAD)
+    spec = wl["spec"]
+    spec.seed = spec.seed + 1000 * rank                      # every replica compresses its own stream
+    T = args.frames or spec.n_frames
+    chunk = wl["chunk"]
+    cfg = B.make_config(n_layers=spec.n_layers, n_q_heads=spec.n_q_heads, n_kv_heads=spec.n_kv_heads,
+                        head_dim=spec.head_dim, tokens_per_frame=spec.tokens_per_frame, keep_per_frame=wl["keep"],
+                        frames_per_segment=wl["fseg"], max_frames_per_chunk=chunk, max_frames=T, alpha=wl["alpha"])
+    ctx = B.MukvContext(cfg, dev)
+    gs = GpuStream(spec, dev)
+    bufs = {n: gs.alloc(n) for n in {chunk, T % chunk} if n}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    nq, k_seg, k_frm, lam = wl["n_questions"], wl["k_seg"], wl["k_frm"], wl["lam"]
+    qtok_np, offs, _ = spec.questions(nq, *wl["q_len"])
+    qtok = torch.from_numpy(qtok_np).view(torch.int16).to(dev).view(torch.bfloat16)
+    stride = ctx.decode_stride_bytes(k_frm)
+    n_sets = 2
+    decode = [torch.empty((nq, stride), dtype=torch.uint8, device=dev) for _ in range(n_sets)]
+    seg_idx = torch.empty((nq, k_seg), dtype=torch.int32, device=dev)
+    frm_idx = torch.empty((nq, k_frm), dtype=torch.int32, device=dev)
+    seg_sc = torch.empty((nq, k_seg), dtype=torch.float32, device=dev)
+    frm_sc = torch.empty((nq, k_frm), dtype=torch.float32, device=dev)
+    counts = torch.empty((nq, 2), dtype=torch.int32, device=dev)
+    kept = torch.empty((chunk, cfg.keep_per_frame), dtype=torch.int32, device=dev)
+    n_calls = (T + chunk - 1) // chunk
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_calls + 2)]
+    step_no = [0]
+
+    def one_step():
+        """Returns (compress ms, retrieve ms, gather ms) of this step, device time."""
+        ctx.mukv_reset()
+        for i, t0 in enumerate(range(0, T, chunk)):
+            n = min(chunk, T - t0)
+            q, k, v = bufs[n]
+            gs.fill(t0, n, q, k, v)
+            flush.zero_()
+            ev[i][0].record()
+            ctx.mukv_compress_chunk(q, k, v, n, t0, kept[:n], None)
+            ev[i][1].record()
+        flush.zero_()
+        ev[n_calls][0].record()
+        ctx.mukv_retrieve(qtok, offs, None, k_seg, k_frm, 0, lam, B.RETR_SEMI, seg_idx, frm_idx, seg_sc, frm_sc,
+                          counts)
+        ev[n_calls][1].record()
+        ev[n_calls + 1][0].record()
+        ctx.mukv_gather(frm_idx, counts, nq, k_frm, decode[step_no[0] % n_sets], stride, None)
+        ev[n_calls + 1][1].record()
+        step_no[0] += 1
+        torch.cuda.synchronize()
+        c_ms = sum(ev[i][0].elapsed_time(ev[i][1]) for i in range(n_calls))
+        return c_ms, ev[n_calls][0].elapsed_time(ev[n_calls][1]), ev[n_calls + 1][0].elapsed_time(ev[n_calls + 1][1])
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    launches0 = ctx.mukv_get_stats().kernel_launches
+    sampler = ClockSampler(local)
+    sampler.start()
+    D.barrier()
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    times = [one_step() for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    D.barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.stop()
+    stats = ctx.mukv_get_stats()
+    launches = stats.kernel_launches - launches0
+    c_ms = sum(t[0] for t in times)
+    r_ms = sum(t[1] for t in times)
+    g_ms = sum(t[2] for t in times)
+    fps = D.throughput(c_ms, T * args.steps, dev)
+    rps = D.throughput(r_ms + g_ms, nq * args.steps, dev)
+    step_ms, _ = D.combine((c_ms + r_ms + g_ms) / args.steps, 0, dev)
+
+    # ---- per-kernel durations, measured live with events around every launch (one extra step)
+    ctx.mukv_profile_enable(True)
+    one_step()
+    prof = ctx.mukv_profile_read()
+    ctx.mukv_profile_enable(False)
+    peaks = load_peaks()
+    ab = algorithmic_bytes(cfg, k_frm)
+    frames_per_launch = T / n_calls
+    kernels = {}
+    bytes_per_launch = {"score": ab["score_per_frame"] * frames_per_launch,
+                        "compact": ab["compact_per_frame"] * frames_per_launch,
+                        "segment": ab["segment_per_frame"] * frames_per_launch,
+                        "gather": ab["gather_per_question"] * nq,
+                        "scan": ab["index_row"] * (T + (T + wl["fseg"] - 1) // wl["fseg"])}
+    total_ms = sum(v[0] for v in prof.values()) or 1.0
+    for kname, (ms, n) in prof.items():
+        if n == 0:
+            continue
+        d = dict(launches=int(n), avg_us=1e3 * ms / n, share=ms / total_ms)
+        if kname in bytes_per_launch:
+            d["algorithmic_bytes"] = bytes_per_launch[kname]
+            d["achieved_gbs"] = bytes_per_launch[kname] / (ms / n * 1e-3) / 1e9
+            d["frac_of_hbm_peak"] = d["achieved_gbs"] / peaks["hbm_gbs"]
+        kernels[kname] = d
+    compress_kinds = [k for k in ("score", "refine", "compact", "segment") if k in kernels]
+    dom = max(compress_kinds, key=lambda k: kernels[k]["share"])
+    if dom == "score":
+        # Eq. 1 on CUDA cores: 2*Hq*P^2*D flop per frame against the fp32 FMA rate
+        flop = 2.0 * cfg.n_q_heads * cfg.tokens_per_frame ** 2 * cfg.head_dim * frames_per_launch
+        peak_tf = 148 * 128 * 2 * (clocks["sm_mhz"] or 1500.0) * 1e6 / 1e12
+        ach = flop / (kernels["score"]["avg_us"] * 1e-6) / 1e12
+        roofline = dict(kernel="score_kernel", bound="alu", achieved=ach, peak=peak_tf, unit="TFLOP/s",
+                        frac=ach / peak_tf, traffic=None,
+                        peak_source="148 SMs x 128 fp32 FMA lanes x 2 flop x sampled SM clock")
+    else:
+        roofline = dict(kernel=dom + "_kernel", bound="hbm", achieved=kernels[dom]["achieved_gbs"],
+                        peak=peaks["hbm_gbs"], unit="GB/s", frac=kernels[dom]["frac_of_hbm_peak"], traffic=None,
+                        peak_source=peaks["source"] + " copy bandwidth")
+    path_gbs = ab["per_frame"] * fps / world / 1e9
+    retr_gbs = (ab["gather_per_question"] + ab["index_row"] * T / nq) * rps / world / 1e9
+
+    # ---- end to end: host buffers, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        n = chunk
+        q, k, v = bufs[n]
+        hq, hk, hv = (torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for x in (q, k, v))
+        gs.fill(0, n, q, k, v)
+        hq.copy_(q); hk.copy_(k); hv.copy_(v)
+        hkept = torch.empty(kept.shape, dtype=kept.dtype, pin_memory=True)
+        n_e2e = min(16, n_calls)
+        ctx.mukv_reset()
+        torch.cuda.synchronize()
+        D.barrier()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            q.copy_(hq, non_blocking=True); k.copy_(hk, non_blocking=True); v.copy_(hv, non_blocking=True)
+            ctx.mukv_compress_chunk(q, k, v, n, i * n, kept, None)
+            hkept.copy_(kept, non_blocking=True)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        e2e_fps = D.throughput(dt * 1e3, n_e2e * n, dev)
+        e2e = {"value": e2e_fps, "unit": UNIT,
+               "h2d_bytes_per_step": int(sum(x.numel() * x.element_size() for x in (hq, hk, hv))),
+               "d2h_bytes_per_step": int(hkept.numel() * 4),
+               "note": f"{n_e2e} chunks: pinned-host Q/K/V copied in, compressed, kept ids copied out; a step here "
+                       f"is one chunk of {n} frames"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        o_fps, o_rps, threads, desc = oracle_sample(args.oracle_frames, 4)
+        cpu = {"value": o_fps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
+               "retrievals_per_s": o_rps}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "frames": T, "chunk_frames": chunk, "questions": nq, "k_seg": k_seg,
+                       "k_frm": k_frm, "parallelism": f"{world} independent replica(s)",
+                       "timing": "sum of CUDA-event intervals around the library calls; the chunk generator and "
+                                 "a 256 MiB L2 flush run between calls and are excluded",
+                       "l2": "flushed by a 256 MiB memset before every timed call"},
+            "retrievals_per_s": rps,
+            "retrieve_ms": r_ms / args.steps, "gather_ms": g_ms / args.steps, "compress_ms": c_ms / args.steps,
+            "wall_s_per_step_with_generation": wall / args.steps,
+            "path_algorithmic_gbs": {"compress": path_gbs, "compress_frac_of_peak": path_gbs / peaks["hbm_gbs"],
+                                     "retrieve_gather": retr_gbs,
+                                     "retrieve_gather_frac_of_peak": retr_gbs / peaks["hbm_gbs"],
+                                     "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"]},
+            "roofline": roofline, "kernels": kernels,
+            "refined_frames": int(stats.refined_frames),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -180,6 +180,16 @@ void* mukv_store_region(const mukv_ctx* ctx, int32_t which, size_t* bytes);
 /* Reads counters.  Copies a few device words: synchronises the given stream. */
 mukv_status mukv_get_stats(mukv_ctx* ctx, mukv_stats* out, mukv_stream stream);
 
+/* Optional per-kernel timing for benchmarks.  While enabled, every kernel launch of this
+ * context is bracketed by a pair of CUDA events on the call's stream (host objects; no device
+ * memory).  mukv_profile_read waits for the recorded events, adds up the elapsed milliseconds
+ * and the launch counts per kernel kind since the last read, and forgets them.
+ * Kinds: 0 score, 1 refine (double-precision score), 2 compact+pool, 3 segment pool,
+ *        4 question pool, 5 index scan, 6 rank, 7 gather. */
+#define MUKV_PROF_KINDS 8
+mukv_status mukv_profile_enable(mukv_ctx* ctx, int32_t on);
+mukv_status mukv_profile_read(mukv_ctx* ctx, double* ms, int64_t* launches);
+
 /* Message of the last failure on this context (valid until the next call on it);
  * with ctx == NULL, the message of the last failed mukv_create on this thread. */
 const char* mukv_last_error(const mukv_ctx* ctx);

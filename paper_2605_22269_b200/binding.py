@@ -24,7 +24,8 @@ STATUS_NAMES = {0: "MUKV_OK", -1: "MUKV_E_INVALID", -2: "MUKV_E_SHAPE", -3: "MUK
 
 EXPORTS = ["mukv_store_bytes", "mukv_workspace_bytes", "mukv_create", "mukv_destroy", "mukv_reset",
            "mukv_compress_chunk", "mukv_retrieve", "mukv_gather", "mukv_store_region", "mukv_get_stats",
-           "mukv_last_error"]
+           "mukv_last_error", "mukv_profile_enable", "mukv_profile_read"]
+PROF_KINDS = ["score", "refine", "compact", "segment", "qpool", "scan", "rank", "gather"]
 
 
 class MukvError(RuntimeError):
@@ -84,6 +85,10 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.mukv_store_region.argtypes = [vp, i32, C.POINTER(C.c_size_t)]
     lib.mukv_get_stats.restype = i32
     lib.mukv_get_stats.argtypes = [vp, C.POINTER(MukvStats), vp]
+    lib.mukv_profile_enable.restype = i32
+    lib.mukv_profile_enable.argtypes = [vp, i32]
+    lib.mukv_profile_read.restype = i32
+    lib.mukv_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.mukv_last_error.restype = C.c_char_p
     lib.mukv_last_error.argtypes = [vp]
     if path == _build.lib_path("libmukv.so"):
@@ -176,6 +181,16 @@ class MukvContext:
         s = MukvStats()
         self._check(self.lib.mukv_get_stats(self.handle, C.byref(s), _stream(stream)))
         return s
+
+    def mukv_profile_enable(self, on: bool):
+        self._check(self.lib.mukv_profile_enable(self.handle, 1 if on else 0))
+
+    def mukv_profile_read(self) -> dict:
+        """{kind: (milliseconds, launches)} since the last read."""
+        ms = (C.c_double * len(PROF_KINDS))()
+        n = (C.c_int64 * len(PROF_KINDS))()
+        self._check(self.lib.mukv_profile_read(self.handle, ms, n))
+        return {k: (ms[i], n[i]) for i, k in enumerate(PROF_KINDS)}
 
     # ---- views into the store (tests, inspection) ---------------------------------------------
     def region(self, which: int) -> torch.Tensor:

@@ -11,6 +11,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <vector>
 
 #include "common.cuh"
 #include "compact.cuh"
@@ -51,6 +52,10 @@ struct mukv_ctx {
   int C, G, esize, nc;
   float flag_margin, flat_ratio;
   std::string err;
+  // optional per-kernel timing (host objects only)
+  bool prof_on = false;
+  std::vector<cudaEvent_t> prof_ev;      // pairs: start, stop
+  std::vector<int> prof_kind;            // kind of each used pair
 };
 
 namespace {
@@ -64,6 +69,28 @@ mukv_status fail(mukv_ctx* ctx, mukv_status st, const char* fmt, ...) {
   if (ctx) ctx->err = buf; else g_create_error = buf;
   return st;
 }
+
+// Brackets one kernel launch with a pair of events when profiling is on.
+struct ProfScope {
+  mukv_ctx* c;
+  cudaStream_t st;
+  cudaEvent_t stop = nullptr;
+  ProfScope(mukv_ctx* ctx, int kind, cudaStream_t s) : c(ctx), st(s) {
+    if (!c->prof_on) return;
+    const size_t used = c->prof_kind.size();
+    while (c->prof_ev.size() < 2 * (used + 1)) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      c->prof_ev.push_back(e);
+    }
+    c->prof_kind.push_back(kind);
+    cudaEventRecord(c->prof_ev[2 * used], st);
+    stop = c->prof_ev[2 * used + 1];
+  }
+  ~ProfScope() {
+    if (stop) cudaEventRecord(stop, st);
+  }
+};
 
 bool is_pow2(long long x) { return x > 0 && (x & (x - 1)) == 0; }
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -191,14 +218,21 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   sp.page_bytes = (long long)ctx->sl.page_bytes;
   sp.refine = 0;
   const dim3 grid(c.n_q_heads, n);
-  cudaError_t e = launch_score<T, float>(sp, ctx->nc, grid, score_smem_bytes<T, float>(P, c.head_dim), st);
+  cudaError_t e;
+  {
+    ProfScope ps(ctx, 0, st);
+    e = launch_score<T, float>(sp, ctx->nc, grid, score_smem_bytes<T, float>(P, c.head_dim), st);
+  }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "score kernel: %s", cudaGetErrorString(e));
   // frames too close to a tie boundary: same computation in double (blocks beyond the flagged
   // count return at once)
   sp.refine = 1;
   sp.colsum_part = ctx->ws + ctx->wl.colsum_d;
   sp.ifft_part = ctx->ws + ctx->wl.ifft_d;
-  e = launch_score<T, double>(sp, ctx->nc, grid, score_smem_bytes<T, double>(P, c.head_dim), st);
+  {
+    ProfScope ps(ctx, 1, st);
+    e = launch_score<T, double>(sp, ctx->nc, grid, score_smem_bytes<T, double>(P, c.head_dim), st);
+  }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "refine kernel: %s", cudaGetErrorString(e));
 
   CompactParams cp;
@@ -213,7 +247,10 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   cp.frame_ksum = reinterpret_cast<double*>(ctx->store + ctx->sl.frame_ksum);
   cp.n_flagged = sp.n_flagged;
   cp.stat_refined = reinterpret_cast<long long*>(ctx->ws + ctx->wl.stat_refined);
-  compact_kernel<T><<<dim3(L * 2, n), kCompactThreads, 0, st>>>(cp);
+  {
+    ProfScope ps(ctx, 2, st);
+    compact_kernel<T><<<dim3(L * 2, n), kCompactThreads, 0, st>>>(cp);
+  }
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "compact kernel: %s", cudaGetErrorString(e));
 
@@ -226,7 +263,10 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   gp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
   gp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
   const long long last_seg = (t0 + n - 1) / c.frames_per_segment;
-  segment_kernel<<<dim3(L * 2, (unsigned)(last_seg - gp.first_seg + 1)), 256, 0, st>>>(gp);
+  {
+    ProfScope ps(ctx, 3, st);
+    segment_kernel<<<dim3(L * 2, (unsigned)(last_seg - gp.first_seg + 1)), 256, 0, st>>>(gp);
+  }
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "segment kernel: %s", cudaGetErrorString(e));
   ctx->launches += 4;
@@ -304,7 +344,33 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
   return MUKV_OK;
 }
 
-void mukv_destroy(mukv_ctx* ctx) { delete ctx; }
+void mukv_destroy(mukv_ctx* ctx) {
+  if (!ctx) return;
+  for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
+  delete ctx;
+}
+
+mukv_status mukv_profile_enable(mukv_ctx* ctx, int32_t on) {
+  if (!ctx) return MUKV_E_INVALID;
+  ctx->prof_on = on != 0;
+  ctx->prof_kind.clear();
+  return MUKV_OK;
+}
+
+mukv_status mukv_profile_read(mukv_ctx* ctx, double* ms, int64_t* launches) {
+  if (!ctx || !ms || !launches) return MUKV_E_INVALID;
+  for (int i = 0; i < MUKV_PROF_KINDS; ++i) { ms[i] = 0.0; launches[i] = 0; }
+  for (size_t i = 0; i < ctx->prof_kind.size(); ++i) {
+    float t = 0.f;
+    cudaError_t e = cudaEventSynchronize(ctx->prof_ev[2 * i + 1]);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&t, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]);
+    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "mukv_profile_read: %s", cudaGetErrorString(e));
+    ms[ctx->prof_kind[i]] += (double)t;
+    launches[ctx->prof_kind[i]] += 1;
+  }
+  ctx->prof_kind.clear();
+  return MUKV_OK;
+}
 
 mukv_status mukv_reset(mukv_ctx* ctx, mukv_stream stream) {
   (void)stream;
@@ -380,19 +446,25 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
     const float* seg_key = reinterpret_cast<const float*>(ctx->store + ctx->sl.seg_key);
     const long long n_frm = ctx->frames;
     const long long n_seg = (n_frm + c.frames_per_segment - 1) / c.frames_per_segment;
-    if (c.dtype == MUKV_BF16)
-      qpool_kernel<__nv_bfloat16><<<nq, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(d_qtok), meta,
-                                                     c.n_q_heads, c.n_kv_heads, c.head_dim, q64, qnorm);
-    else
-      qpool_kernel<float><<<nq, 256, 0, st>>>(reinterpret_cast<const float*>(d_qtok), meta, c.n_q_heads,
-                                             c.n_kv_heads, c.head_dim, q64, qnorm);
+    {
+      ProfScope ps(ctx, 4, st);
+      if (c.dtype == MUKV_BF16)
+        qpool_kernel<__nv_bfloat16><<<nq, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(d_qtok), meta,
+                                                       c.n_q_heads, c.n_kv_heads, c.head_dim, q64, qnorm);
+      else
+        qpool_kernel<float><<<nq, 256, 0, st>>>(reinterpret_cast<const float*>(d_qtok), meta, c.n_q_heads,
+                                               c.n_kv_heads, c.head_dim, q64, qnorm);
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "qpool kernel: %s", cudaGetErrorString(e));
     const long long rows = n_frm + n_seg;
     const unsigned blocks = (unsigned)((rows + kScanRows - 1) / kScanRows);
-    scan_kernel<<<blocks, 256, kScanRows * (C + 1) * sizeof(float), st>>>(frame_key, seg_key, n_frm, n_seg, C, nq, q64,
-                                                                         qnorm, s_frm, s_seg, c.max_frames,
-                                                                         ctx->sl.max_segs);
+    {
+      ProfScope ps(ctx, 5, st);
+      scan_kernel<<<blocks, 256, kScanRows * (C + 1) * sizeof(float), st>>>(frame_key, seg_key, n_frm, n_seg, C, nq,
+                                                                           q64, qnorm, s_frm, s_seg, c.max_frames,
+                                                                           ctx->sl.max_segs);
+    }
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "scan kernel: %s", cudaGetErrorString(e));
     RankParams rp;
@@ -405,7 +477,10 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
     rp.frame_key = frame_key; rp.seg_key = seg_key;
     rp.seg_idx = d_seg_idx; rp.frm_idx = d_frm_idx; rp.seg_score = d_seg_score; rp.frm_score = d_frm_score;
     rp.counts = d_counts;
-    rank_kernel<<<nq, kRankThreads, C * sizeof(double), st>>>(rp, meta);
+    {
+      ProfScope ps(ctx, 6, st);
+      rank_kernel<<<nq, kRankThreads, C * sizeof(double), st>>>(rp, meta);
+    }
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "rank kernel: %s", cudaGetErrorString(e));
     ctx->launches += 3;
@@ -444,7 +519,10 @@ mukv_status mukv_gather(mukv_ctx* ctx, const int32_t* d_frm_idx, const int32_t* 
     gp.tok_meta = d_tok_meta;
     const long long units = (long long)nq * c.n_layers * 2 * k_frm;
     const unsigned blocks = (unsigned)(units < 148 * 8 ? units : 148 * 8);
-    gather_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(gp);
+    {
+      ProfScope ps(ctx, 7, static_cast<cudaStream_t>(stream));
+      gather_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(gp);
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "gather kernel: %s", cudaGetErrorString(e));
     ctx->launches += 1;
