@@ -3,8 +3,10 @@
 // belong to the caller.
 #include "../../include/mukv.h"
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <cstdlib>
@@ -17,6 +19,7 @@
 #include "compact.cuh"
 #include "retrieve.cuh"
 #include "score.cuh"
+#include "score_tc.cuh"
 
 using namespace mukv;
 
@@ -32,9 +35,16 @@ struct StoreLayout {
 };
 
 struct WorkLayout {
-  size_t colsum_f, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, stat_refined;
-  size_t q64, qnorm, s_frm, s_seg, total;
+  size_t colsum_f, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, stat_refined, dev_status;
+  size_t q64, qnorm, s_frm, s_seg, wtab, total;
   size_t zero_begin, zero_end;          // region that must start as zeros
+};
+
+// Tiling of the tensor-core scoring kernel (bf16 inputs only).
+struct TcShape {
+  bool ok;
+  int tpt, tiles, npad, n_mt, tmem_cols;
+  size_t smem;
 };
 
 thread_local std::string g_create_error;
@@ -51,6 +61,8 @@ struct mukv_ctx {
   long long launches;
   int C, G, esize, nc;
   float flag_margin, flat_ratio;
+  TcShape tcs;                           // tcs.ok: the chunk is scored on the tensor cores
+  CUtensorMap wmap;                      // DFT matrix terms [3*D][D] bf16
   std::string err;
   // optional per-kernel timing (host objects only)
   bool prof_on = false;
@@ -142,13 +154,33 @@ StoreLayout store_layout(const mukv_config& c) {
   return s;
 }
 
+TcShape tc_shape(const mukv_config& c) {
+  TcShape t;
+  memset(&t, 0, sizeof t);
+  const int G = c.n_q_heads / c.n_kv_heads;
+  if (c.dtype != MUKV_BF16 || G > 128) return t;
+  t.tpt = 128 / G;
+  t.tiles = (c.tokens_per_frame + t.tpt - 1) / t.tpt;
+  t.npad = (c.tokens_per_frame + 15) / 16 * 16;
+  t.n_mt = (c.tokens_per_frame + 127) / 128;
+  int need = t.npad > c.head_dim ? t.npad : c.head_dim;
+  t.tmem_cols = 32;
+  while (t.tmem_cols < need) t.tmem_cols *= 2;
+  t.smem = score_tc_smem_bytes(c.tokens_per_frame, c.head_dim);
+  t.ok = t.smem <= 227 * 1024;
+  return t;
+}
+
 WorkLayout work_layout(const mukv_config& c) {
   WorkLayout w;
   const size_t F = c.max_frames_per_chunk, P = c.tokens_per_frame;
   const size_t C = (size_t)c.n_kv_heads * c.head_dim;
   const size_t max_segs = (c.max_frames + c.frames_per_segment - 1) / c.frames_per_segment;
   size_t off = 0;
-  w.colsum_f = off;       off = align_up(off + F * c.n_q_heads * P * sizeof(float));
+  const TcShape ts = tc_shape(c);
+  const size_t parts = ts.ok && (size_t)c.n_kv_heads * ts.tiles > (size_t)c.n_q_heads
+                           ? (size_t)c.n_kv_heads * ts.tiles : (size_t)c.n_q_heads;
+  w.colsum_f = off;       off = align_up(off + F * parts * P * sizeof(float));
   w.ifft_f = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(float));
   w.colsum_d = off;       off = align_up(off + F * c.n_q_heads * P * sizeof(double));
   w.ifft_d = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(double));
@@ -157,11 +189,13 @@ WorkLayout work_layout(const mukv_config& c) {
   w.flagged = off;        off = align_up(off + F * sizeof(int));
   w.n_flagged = off;      off = align_up(off + sizeof(int));
   w.stat_refined = off;   off = align_up(off + sizeof(long long));
+  w.dev_status = off;     off = align_up(off + sizeof(int));
   w.zero_end = off;
   w.q64 = off;            off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * C * sizeof(double));
   w.qnorm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * sizeof(double));
   w.s_frm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * c.max_frames * sizeof(double));
   w.s_seg = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * max_segs * sizeof(double));
+  w.wtab = off;           off = align_up(off + (ts.ok ? (size_t)3 * c.head_dim * c.head_dim * 2 : 0));
   w.total = off;
   return w;
 }
@@ -189,6 +223,113 @@ cudaError_t set_score_attr(int nc, size_t smem) {
     default: fn = (const void*)score_kernel<T, A, 8>; break;
   }
   return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+
+// ---------------------------------------------------------------- TMA descriptors
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// bf16 tensor [rows][mid][D] (D contiguous) seen as a rank-3 map; the box is box_rows x box_mid x 64
+// channels, written to shared memory with the 128-byte swizzle.  Out-of-range rows read as zero.
+bool encode_map3(CUtensorMap* m, const void* base, int D, int mid, long long rows, int box_mid, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)mid, (cuuint64_t)rows};
+  const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)mid * D * 2};
+  const cuuint32_t box[3] = {64u, (cuuint32_t)box_mid, (cuuint32_t)box_rows};
+  const cuuint32_t estr[3] = {1u, 1u, 1u};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool encode_map2(CUtensorMap* m, const void* base, int cols, long long rows, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1u, 1u};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+uint16_t bf16_rne(float x) {
+  uint32_t b;
+  memcpy(&b, &x, 4);
+  b += 0x7FFFu + ((b >> 16) & 1u);
+  return (uint16_t)(b >> 16);
+}
+float bf16_val(uint16_t h) {
+  const uint32_t b = (uint32_t)h << 16;
+  float x;
+  memcpy(&x, &b, 4);
+  return x;
+}
+
+// The D-point DFT as a matrix, rows = output column n, columns = input channel d (the layout of
+// a K-major B operand): n <= D/2 holds cos(2 pi n d / D), n > D/2 holds -sin(2 pi (n - D/2) d / D).
+// Each entry is split into three bf16 terms, hi + mid + lo, stored as [3][D][D].
+std::vector<uint16_t> dft_terms(int D) {
+  std::vector<uint16_t> w((size_t)3 * D * D);
+  const double pi = 3.14159265358979323846;
+  for (int n = 0; n < D; ++n)
+    for (int d = 0; d < D; ++d) {
+      const int b = n <= D / 2 ? n : n - D / 2;
+      const int m = (int)(((long long)b * d) % D);
+      const double ang = 2.0 * pi * (double)m / (double)D;
+      const double x = n <= D / 2 ? std::cos(ang) : -std::sin(ang);
+      const uint16_t hi = bf16_rne((float)x);
+      const double r1 = x - (double)bf16_val(hi);
+      const uint16_t mid = bf16_rne((float)r1);
+      const double r2 = r1 - (double)bf16_val(mid);
+      const uint16_t lo = bf16_rne((float)r2);
+      w[((size_t)0 * D + n) * D + d] = hi;
+      w[((size_t)1 * D + n) * D + d] = mid;
+      w[((size_t)2 * D + n) * D + d] = lo;
+    }
+  return w;
+}
+
+// Scores a bf16 chunk on the tensor cores (Eq. 1-4 and the selection).
+cudaError_t launch_score_tc(mukv_ctx* ctx, const ScoreParams& sp, const void* d_q, const void* k_last, int n,
+                            cudaStream_t st, const char** why) {
+  const mukv_config& c = ctx->cfg;
+  const TcShape& t = ctx->tcs;
+  const int P = c.tokens_per_frame, D = c.head_dim;
+  CUtensorMap qmap, kmap, kmap_dft;
+  const long long rows = (long long)n * P;
+  if (!encode_map3(&qmap, d_q, D, c.n_q_heads, rows, ctx->G, t.tpt) ||
+      !encode_map3(&kmap, k_last, D, c.n_kv_heads, rows, 1, t.npad) ||
+      !encode_map3(&kmap_dft, k_last, D, c.n_kv_heads, rows, 1, 128)) {
+    *why = "cuTensorMapEncodeTiled failed";
+    return cudaErrorInvalidValue;
+  }
+  ScoreTcParams tp;
+  memset(&tp, 0, sizeof tp);
+  tp.sp = sp;
+  tp.tiles = t.tiles; tp.tpt = t.tpt; tp.npad = t.npad; tp.n_mt = t.n_mt; tp.tmem_cols = t.tmem_cols;
+  tp.op_bytes = score_tc_op_bytes(P, D);
+  tp.exp2_scale = (float)(1.4426950408889634 / std::sqrt((double)D));
+  tp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
+  const dim3 grid(t.n_mt + t.tiles, c.n_kv_heads, n);
+  score_tc_kernel<<<grid, kTcThreads, t.smem, st>>>(tp, qmap, kmap, kmap_dft, ctx->wmap);
+  *why = "score_tc kernel";
+  return cudaGetLastError();
 }
 
 template <typename T>
@@ -219,11 +360,15 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   sp.refine = 0;
   const dim3 grid(c.n_q_heads, n);
   cudaError_t e;
+  const char* what = "score kernel";
   {
     ProfScope ps(ctx, 0, st);
-    e = launch_score<T, float>(sp, ctx->nc, grid, score_smem_bytes<T, float>(P, c.head_dim), st);
+    if (ctx->tcs.ok)
+      e = launch_score_tc(ctx, sp, d_q, sp.k_last, n, st, &what);
+    else
+      e = launch_score<T, float>(sp, ctx->nc, grid, score_smem_bytes<T, float>(P, c.head_dim), st);
   }
-  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "score kernel: %s", cudaGetErrorString(e));
+  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "%s: %s", what, cudaGetErrorString(e));
   // frames too close to a tie boundary: same computation in double (blocks beyond the flagged
   // count return at once)
   sp.refine = 1;
@@ -316,7 +461,9 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
   ctx->G = cfg->n_q_heads / cfg->n_kv_heads;
   ctx->esize = cfg->dtype == MUKV_BF16 ? 2 : 4;
   ctx->nc = pick_nc(cfg->tokens_per_frame);
-  ctx->flag_margin = 6e-7f;
+  ctx->tcs = tc_shape(*cfg);
+  if (const char* s = getenv("MUKV_SCORE_FMA")) if (atoi(s) != 0) ctx->tcs.ok = false;
+  ctx->flag_margin = 3e-6f;
   ctx->flat_ratio = 1e-3f;
   if (const char* s = getenv("MUKV_FLAG_MARGIN")) ctx->flag_margin = (float)atof(s);
   if (const char* s = getenv("MUKV_FLAT_RATIO")) ctx->flat_ratio = (float)atof(s);
@@ -332,6 +479,14 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute((const void*)scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(kScanRows * (ctx->C + 1) * sizeof(float)));
+  if (e == cudaSuccess && ctx->tcs.ok) {
+    const std::vector<uint16_t> w = dft_terms(D);
+    e = cudaMemcpy(ctx->ws + ctx->wl.wtab, w.data(), w.size() * 2, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !encode_map2(&ctx->wmap, ctx->ws + ctx->wl.wtab, D, 3LL * D, D)) e = cudaErrorInvalidValue;
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute((const void*)score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)ctx->tcs.smem);
+  }
   if (e == cudaSuccess)
     e = cudaMemset(ctx->ws + ctx->wl.zero_begin, 0, ctx->wl.zero_end - ctx->wl.zero_begin);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -557,8 +712,11 @@ mukv_status mukv_get_stats(mukv_ctx* ctx, mukv_stats* out, mukv_stream stream) {
   if (!ctx || !out) return MUKV_E_INVALID;
   memset(out, 0, sizeof *out);
   long long refined = 0;
+  int dev_status = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemcpyAsync(&refined, ctx->ws + ctx->wl.stat_refined, sizeof refined, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(&dev_status, ctx->ws + ctx->wl.dev_status, sizeof dev_status, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "mukv_get_stats: %s", cudaGetErrorString(e));
   const mukv_config& c = ctx->cfg;
@@ -569,6 +727,7 @@ mukv_status mukv_get_stats(mukv_ctx* ctx, mukv_stats* out, mukv_stream stream) {
   out->store_bytes_used = ctx->frames * (long long)ctx->sl.page_bytes;
   out->refined_frames = refined;
   out->kernel_launches = ctx->launches;
+  out->device_status = dev_status;
   return MUKV_OK;
 }
 

@@ -58,19 +58,34 @@ __host__ inline size_t score_smem_bytes(int P, int D) {
   return ((ks + 15) / 16) * 16 + qs + tw + red + sel + 64;
 }
 
-// Eq. 4 and the top-kappa rule for one frame, run by the whole block (blockDim.x >= P).
-// att_raw / fft_raw are this thread's token's I_att and I_fft; s_sc, s_int, s_misc are shared scratch.
+// Eq. 4 and the top-kappa rule for one frame, run by the whole block.  Thread tid owns the tokens
+// tid + k*blockDim.x, k < TOK (TOK*blockDim.x >= P); att_raw / fft_raw are their I_att and I_fft;
+// s_sc (P doubles), s_int (one int per warp + 1), s_misc (4 doubles per warp) are shared scratch.
 // The arithmetic here is always double: it is a few hundred operations per frame and keeps
 // the normalisation from adding rounding noise of its own to the scores.
-__device__ inline void select_frame(const ScoreParams& p, int f, double att_raw, double fft_raw, double* s_sc,
-                                    int* s_int, double* s_misc) {
+template <int TOK>
+__device__ inline void select_frame(const ScoreParams& p, int f, const double (&att_raw)[TOK],
+                                    const double (&fft_raw)[TOK], double* s_sc, int* s_int, double* s_misc) {
   typedef double A;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nt = blockDim.x, nwarp = nt >> 5;
   const int P = p.P;
-  const bool valid = tid < P;
   const A big = (A)3.0e38;
+  int tok[TOK];
+  bool valid[TOK];
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) { tok[k] = tid + k * nt; valid[k] = tok[k] < P; }
   // ---- min / max of both signals over the frame
-  A v[4] = {valid ? att_raw : big, valid ? att_raw : -big, valid ? fft_raw : big, valid ? fft_raw : -big};
+  A v[4] = {big, -big, big, -big};
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    if (valid[k]) {
+      v[0] = att_raw[k] < v[0] ? att_raw[k] : v[0];
+      v[1] = att_raw[k] > v[1] ? att_raw[k] : v[1];
+      v[2] = fft_raw[k] < v[2] ? fft_raw[k] : v[2];
+      v[3] = fft_raw[k] > v[3] ? fft_raw[k] : v[3];
+    }
+  }
   v[0] = warp_min(v[0]); v[1] = warp_max(v[1]); v[2] = warp_min(v[2]); v[3] = warp_max(v[3]);
   if (lane == 0) {
 #pragma unroll
@@ -78,7 +93,7 @@ __device__ inline void select_frame(const ScoreParams& p, int f, double att_raw,
   }
   __syncthreads();
   A amin = big, amax = -big, fmin_ = big, fmax_ = -big;
-  for (int w = 0; w < kScoreWarps; ++w) {
+  for (int w = 0; w < nwarp; ++w) {
     amin = s_misc[w * 4 + 0] < amin ? s_misc[w * 4 + 0] : amin;
     amax = s_misc[w * 4 + 1] > amax ? s_misc[w * 4 + 1] : amax;
     fmin_ = s_misc[w * 4 + 2] < fmin_ ? s_misc[w * 4 + 2] : fmin_;
@@ -86,67 +101,108 @@ __device__ inline void select_frame(const ScoreParams& p, int f, double att_raw,
   }
   __syncthreads();
   // ---- Eq. 4
-  A an = (amax == amin) ? (A)0 : (att_raw - amin) / (amax - amin);
-  A fn = (fmax_ == fmin_) ? (A)0 : (fft_raw - fmin_) / (fmax_ - fmin_);
-  if (p.keep_low) fn = (A)1 - fn;
   const A alpha = (A)p.alpha;
-  const A s = alpha * an + ((A)1 - alpha) * fn;
-  if (valid) s_sc[tid] = s;
+  A s[TOK];
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    A an = (amax == amin) ? (A)0 : (att_raw[k] - amin) / (amax - amin);
+    A fn = (fmax_ == fmin_) ? (A)0 : (fft_raw[k] - fmin_) / (fmax_ - fmin_);
+    if (p.keep_low) fn = (A)1 - fn;
+    s[k] = alpha * an + ((A)1 - alpha) * fn;
+    if (valid[k]) s_sc[tok[k]] = s[k];
+  }
   __syncthreads();
   // ---- tau = kappa-th largest score (rank counting; P <= 256)
   const int kappa = p.kappa;
-  if (valid) {
-    int gt = 0, ge = 0;
-    for (int i = 0; i < P; ++i) {
-      const A o = s_sc[i];
-      gt += (o > s);
-      ge += (o >= s);
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    if (valid[k]) {
+      int gt = 0, ge = 0;
+      for (int i = 0; i < P; ++i) {
+        const A o = s_sc[i];
+        gt += (o > s[k]);
+        ge += (o >= s[k]);
+      }
+      if (gt < kappa && kappa <= ge) s_misc[0] = s[k];      // every writer holds the same value
     }
-    if (gt < kappa && kappa <= ge) s_misc[0] = s;      // every writer holds the same value
   }
   __syncthreads();
   const A tau = s_misc[0];
   const A delta = (A)p.tie_eps;
-  const bool sure = valid && (s > tau + delta);
-  const bool band = valid && !sure && (s >= tau - delta);
-  int n_sure, n_dummy;
-  block_excl_count(sure, s_int, n_sure);
-  const int band_rank = block_excl_count(band, s_int, n_dummy);
-  const bool keep = sure || (band && band_rank < kappa - n_sure);
-  int n_keep;
-  const int pos = block_excl_count(keep, s_int, n_keep);
-  const long long f_abs = p.first_frame + f;
-  if (keep) {
-    p.kept_store[f_abs * kappa + pos] = tid;
-    if (p.kept_out) p.kept_out[(long long)f * kappa + pos] = tid;
+  bool sure[TOK], band[TOK], keep[TOK];
+  int n_sure = 0;
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    sure[k] = valid[k] && (s[k] > tau + delta);
+    band[k] = valid[k] && !sure[k] && (s[k] >= tau - delta);
+    int t;
+    block_excl_count(sure[k], s_int, t);
+    n_sure += t;
   }
-  if (p.scores_out && valid) {
-    const long long np = (long long)p.n_frames * P;
-    p.scores_out[0 * np + (long long)f * P + tid] = (float)att_raw;
-    p.scores_out[1 * np + (long long)f * P + tid] = (float)fft_raw;
-    p.scores_out[2 * np + (long long)f * P + tid] = (float)s;
+  int band_before = 0;
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    int t;
+    const int band_rank = band_before + block_excl_count(band[k], s_int, t);
+    band_before += t;
+    keep[k] = sure[k] || (band[k] && band_rank < kappa - n_sure);
+  }
+  const long long f_abs = p.first_frame + f;
+  int out_before = 0;
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    int t;
+    const int pos = out_before + block_excl_count(keep[k], s_int, t);
+    out_before += t;
+    if (keep[k]) {
+      p.kept_store[f_abs * kappa + pos] = tok[k];
+      if (p.kept_out) p.kept_out[(long long)f * kappa + pos] = tok[k];
+    }
+    if (p.scores_out && valid[k]) {
+      const long long np = (long long)p.n_frames * P;
+      p.scores_out[0 * np + (long long)f * P + tok[k]] = (float)att_raw[k];
+      p.scores_out[1 * np + (long long)f * P + tok[k]] = (float)fft_raw[k];
+      p.scores_out[2 * np + (long long)f * P + tok[k]] = (float)s[k];
+    }
   }
   if (tid == 0) {
     p.frame_ts[f_abs] = f_abs;
     p.page_table[f_abs] = p.pages_off + f_abs * p.page_bytes;
   }
   // ---- does single precision decide this frame safely?
+  // With a = lowest kept score and b = highest dropped score, the kept set is the same for every
+  // perturbation of the scores below flag_margin / 2 as long as a - b > tie_eps + flag_margin: no
+  // dropped token can then enter the tie band of the kappa-th score.  Anything closer is redone
+  // in double precision.
   if (!p.refine) {
-    const A m = (A)p.flag_margin;
-    const A da = s - (tau + delta), db = s - (tau - delta);
-    bool risky = valid && ((da <= m && da >= -m) || (db <= m && db >= -m));
-    // a nearly flat signal amplifies rounding noise through the min-max division
+    A a = big, b = -big;
+#pragma unroll
+    for (int k = 0; k < TOK; ++k) {
+      if (valid[k]) {
+        if (keep[k]) a = s[k] < a ? s[k] : a;
+        else b = s[k] > b ? s[k] : b;
+      }
+    }
+    a = warp_min(a);
+    b = warp_max(b);
+    __syncthreads();
+    if (lane == 0) { s_misc[warp * 4] = a; s_misc[warp * 4 + 1] = b; }
+    __syncthreads();
     if (tid == 0) {
+      for (int w = 1; w < nwarp; ++w) {
+        a = s_misc[w * 4] < a ? s_misc[w * 4] : a;
+        b = s_misc[w * 4 + 1] > b ? s_misc[w * 4 + 1] : b;
+      }
+      bool risky = (kappa < P) && (a - b <= delta + (A)p.flag_margin);
+      // a nearly flat signal amplifies rounding noise through the min-max division
       const A fr = (A)p.flat_ratio;
       const A aabs = amax > -amin ? amax : -amin, fabs_ = fmax_ > -fmin_ ? fmax_ : -fmin_;
       if (amax != amin && (amax - amin) < fr * aabs && p.alpha != 0.f) risky = true;
       if (fmax_ != fmin_ && (fmax_ - fmin_) < fr * fabs_ && p.alpha != 1.f) risky = true;
-    }
-    int n_risky;
-    block_excl_count(risky, s_int, n_risky);
-    if (tid == 0 && n_risky > 0) {
-      const int slot = atomicAdd(p.n_flagged, 1);
-      p.flagged[slot] = f;
+      if (risky) {
+        const int slot = atomicAdd(p.n_flagged, 1);
+        p.flagged[slot] = f;
+      }
     }
   }
 }
@@ -325,17 +381,17 @@ __global__ void __launch_bounds__(kScoreThreads) score_kernel(const ScoreParams 
   __syncthreads();
   if (!s_int[63]) return;
   __threadfence();
-  double att = 0.0, fft = 0.0;
+  double att[1] = {0.0}, fft[1] = {0.0};
   if (tid < P) {
     const A* cp = reinterpret_cast<const A*>(p.colsum_part) + (long long)f * Hq * P + tid;
-    for (int hh = 0; hh < Hq; ++hh) att += (double)__ldcg(cp + (long long)hh * P);
-    att = att / (double)((long long)Hq * P);
+    for (int hh = 0; hh < Hq; ++hh) att[0] += (double)__ldcg(cp + (long long)hh * P);
+    att[0] = att[0] / (double)((long long)Hq * P);
     const A* fp = reinterpret_cast<const A*>(p.ifft_part) + (long long)f * Hkv * P + tid;
-    for (int gg = 0; gg < Hkv; ++gg) fft += (double)__ldcg(fp + (long long)gg * P);
-    fft = fft / (double)((long long)Hkv * D);
+    for (int gg = 0; gg < Hkv; ++gg) fft[0] += (double)__ldcg(fp + (long long)gg * P);
+    fft[0] = fft[0] / (double)((long long)Hkv * D);
   }
   __syncthreads();
-  select_frame(p, f, att, fft, s_sc, s_int, s_misc);
+  select_frame<1>(p, f, att, fft, s_sc, s_int, s_misc);
 }
 
 }  // namespace mukv

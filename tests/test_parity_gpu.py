@@ -149,6 +149,28 @@ def test_chunk7b_causal():
     full_compress_check(run)
 
 
+def test_chunk7b_cuda_core_scoring(monkeypatch):
+    # bf16 inputs scored by the plain multiply-add kernel (the one fp32 inputs always use)
+    monkeypatch.setenv("MUKV_SCORE_FMA", "1")
+    run = H.GpuRun("chunk7b", n_frames=3)
+    full_compress_check(run)
+
+
+@pytest.mark.parametrize("shape", [dict(n_q_heads=8, n_kv_heads=8, head_dim=64, tokens_per_frame=130, keep=33),
+                                   dict(n_q_heads=16, n_kv_heads=2, head_dim=128, tokens_per_frame=256, keep=64),
+                                   dict(n_q_heads=12, n_kv_heads=4, head_dim=64, tokens_per_frame=16, keep=5)])
+def test_tensor_core_tilings(shape):
+    # G = 1, 8, 3; P below, at and above one 128-row tile; both head sizes
+    keep = shape.pop("keep")
+    spec = StreamSpec(seed=21, n_layers=2, bf16=True, n_outlier=2, n_frames=5, scene_sigma=1.0, frame_sigma=0.5,
+                      scene_min=2, scene_max=3, **shape)
+    wl = dict(spec=spec, keep=keep, fseg=2, chunk=3, alpha=0.7, n_questions=2, q_len=(2, 5), k_seg=1, k_frm=2,
+              lam=0.3)
+    run = H.GpuRun(wl)
+    full_compress_check(run)
+    assert run.ctx.mukv_get_stats().device_status == 0
+
+
 # ------------------------------------------------------------------------------- config 3
 def test_stream_1h():
     run = H.GpuRun("stream_1h").compress()
