@@ -290,12 +290,22 @@ def main():
             d["achieved_gbs"] = bytes_per_launch[kname] / (ms / n * 1e-3) / 1e9
             d["frac_of_hbm_peak"] = d["achieved_gbs"] / peaks["hbm_gbs"]
         kernels[kname] = d
-    compress_kinds = [k for k in ("score", "refine", "compact", "segment") if k in kernels]
+    compress_kinds = [k for k in ("score", "compact", "segment") if k in kernels]
     dom = max(compress_kinds, key=lambda k: kernels[k]["share"])
-    if dom == "score":
-        # Eq. 1 on CUDA cores: 2*Hq*P^2*D flop per frame against the fp32 FMA rate
+    sm_hz = (clocks["sm_mhz"] or 1500.0) * 1e6
+    if dom == "score" and cfg.dtype == 0:
+        # Eq. 1 on the tensor cores: the softmax epilogue evaluates one exponential per attention
+        # logit on the SM's 16-lane special-function unit, the scarcest unit this kernel uses
+        n_exp = float(cfg.n_q_heads) * cfg.tokens_per_frame ** 2 * frames_per_launch
+        peak = 148 * 16 * sm_hz / 1e9
+        ach = n_exp / (kernels["score"]["avg_us"] * 1e-6) / 1e9
+        roofline = dict(kernel="score_tc_kernel", bound="alu", achieved=ach, peak=peak, unit="Gexp/s",
+                        frac=ach / peak, traffic=None,
+                        peak_source="148 SMs x 16 ex2/clk x sampled SM clock")
+    elif dom == "score":
+        # Eq. 1 on CUDA cores (fp32 inputs): 2*Hq*P^2*D flop per frame against the fp32 FMA rate
         flop = 2.0 * cfg.n_q_heads * cfg.tokens_per_frame ** 2 * cfg.head_dim * frames_per_launch
-        peak_tf = 148 * 128 * 2 * (clocks["sm_mhz"] or 1500.0) * 1e6 / 1e12
+        peak_tf = 148 * 128 * 2 * sm_hz / 1e12
         ach = flop / (kernels["score"]["avg_us"] * 1e-6) / 1e12
         roofline = dict(kernel="score_kernel", bound="alu", achieved=ach, peak=peak_tf, unit="TFLOP/s",
                         frac=ach / peak_tf, traffic=None,
