@@ -190,6 +190,42 @@ mukv_status mukv_get_stats(mukv_ctx* ctx, mukv_stats* out, mukv_stream stream);
 mukv_status mukv_profile_enable(mukv_ctx* ctx, int32_t on);
 mukv_status mukv_profile_read(mukv_ctx* ctx, double* ms, int64_t* launches);
 
+/* Scores frames without any caller-provided scratch.  (The paper has no counterpart: this entry
+ * point exists for the deployment case below, it computes what mukv_compress_chunk computes
+ * for its d_kept_out / d_scores_out arguments and stores nothing.)
+ *
+ * Who needs it: code that must not, or cannot, obtain device memory of its own -- for example
+ * a plug-in inside a serving process that handed all free device memory to its cache pool at
+ * start-up, or a loop that is not allowed to call the allocator while it runs.  Such a caller
+ * cannot build the workspace a mukv_ctx needs, but it may still want to know which tokens of a
+ * frame the method would keep.
+ *
+ *   cfg        shapes and method parameters; n_layers, frames_per_segment, max_frames and
+ *              max_frames_per_chunk are ignored.  Limits: n_frames <= MUKV_NOALLOC_MAX_FRAMES,
+ *              n_q_heads <= MUKV_NOALLOC_MAX_Q_HEADS, n_kv_heads <= MUKV_NOALLOC_MAX_KV_HEADS,
+ *              tokens_per_frame <= MUKV_MAX_TOKENS; larger requests return MUKV_E_CAPACITY.
+ *   d_q        [n_frames][P][Hq][D] last-layer queries;  d_k_last [n_frames][P][Hkv][D] last-layer
+ *              keys (device, 16-byte aligned, cfg->dtype).
+ *   d_kept_out [n_frames][kappa] int32 ascending kept token ids, or NULL;
+ *   d_scores_out [3][n_frames][P] float (I_att, I_fft, fused I), or NULL; not both NULL.
+ *
+ * The scratch (about 1.9 MB: per-head partial sums in float and double, arrival counters, the
+ * list of frames that need the double-precision pass) is a fixed array inside the library; every
+ * device that loads the library holds it until the process exits.  The call performs no
+ * cudaMalloc / cudaFree and uses no allocating routine; it enqueues one small memset (the
+ * counters must start at zero, the rest of the array is overwritten before it is read) and two
+ * kernels on `stream`.  The first call on each device also looks up the array's device address
+ * and raises the kernels' shared-memory limit; make that first call outside any stream capture.
+ * All calls on a device share the one array: two calls whose kernels may overlap on the device
+ * (different streams without an ordering between them) race.  Messages of failures are read
+ * with mukv_last_error(NULL). */
+#define MUKV_NOALLOC_MAX_FRAMES 16
+#define MUKV_NOALLOC_MAX_Q_HEADS 32
+#define MUKV_NOALLOC_MAX_KV_HEADS 8
+mukv_status mukv_score_frames_noalloc(const mukv_config* cfg, const void* d_q, const void* d_k_last,
+                                      int32_t n_frames, int32_t* d_kept_out, float* d_scores_out,
+                                      mukv_stream stream);
+
 /* Message of the last failure on this context (valid until the next call on it);
  * with ctx == NULL, the message of the last failed mukv_create on this thread. */
 const char* mukv_last_error(const mukv_ctx* ctx);

@@ -18,13 +18,14 @@ from . import build as _build
 BF16, FP32 = 0, 1
 RETR_PARALLEL, RETR_HIER, RETR_SEMI = 0, 1, 2
 MAX_QUESTIONS, MAX_TOPK, MAX_TOKENS = 128, 256, 256
+NOALLOC_MAX_FRAMES, NOALLOC_MAX_Q_HEADS, NOALLOC_MAX_KV_HEADS = 16, 32, 8
 
 STATUS_NAMES = {0: "MUKV_OK", -1: "MUKV_E_INVALID", -2: "MUKV_E_SHAPE", -3: "MUKV_E_DTYPE", -4: "MUKV_E_ALIGN",
                 -5: "MUKV_E_CAPACITY", -6: "MUKV_E_STATE", -7: "MUKV_E_CUDA", -8: "MUKV_E_UNSUPPORTED"}
 
 EXPORTS = ["mukv_store_bytes", "mukv_workspace_bytes", "mukv_create", "mukv_destroy", "mukv_reset",
            "mukv_compress_chunk", "mukv_retrieve", "mukv_gather", "mukv_store_region", "mukv_get_stats",
-           "mukv_last_error", "mukv_profile_enable", "mukv_profile_read"]
+           "mukv_last_error", "mukv_profile_enable", "mukv_profile_read", "mukv_score_frames_noalloc"]
 PROF_KINDS = ["score", "refine", "compact", "segment", "qpool", "scan", "rank", "gather"]
 
 
@@ -89,6 +90,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.mukv_profile_enable.argtypes = [vp, i32]
     lib.mukv_profile_read.restype = i32
     lib.mukv_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
+    lib.mukv_score_frames_noalloc.restype = i32
+    lib.mukv_score_frames_noalloc.argtypes = [cfgp, vp, vp, i32, vp, vp, vp]
     lib.mukv_last_error.restype = C.c_char_p
     lib.mukv_last_error.argtypes = [vp]
     if path == _build.lib_path("libmukv.so"):
@@ -111,6 +114,17 @@ def make_config(*, n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, 
     return MukvConfig(n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, keep_per_frame,
                       frames_per_segment, max_frames_per_chunk, attn_causal, keep_low_freq,
                       alpha, tie_eps, dtype, 0, max_frames)
+
+
+def mukv_score_frames_noalloc(cfg: MukvConfig, q, k_last, n_frames: int, kept_out=None, scores_out=None,
+                              stream=None) -> None:
+    """Scores ``n_frames`` frames with the library's built-in scratch: no context, no workspace and no
+    device allocation (see include/mukv.h).  For callers that cannot allocate device memory."""
+    lib = load_library()
+    st = lib.mukv_score_frames_noalloc(C.byref(cfg), _ptr(q), _ptr(k_last), n_frames, _ptr(kept_out),
+                                       _ptr(scores_out), _stream(stream))
+    if st != 0:
+        raise MukvError(st, (lib.mukv_last_error(None) or b"").decode())
 
 
 class MukvContext:

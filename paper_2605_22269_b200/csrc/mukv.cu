@@ -734,3 +734,133 @@ mukv_status mukv_get_stats(mukv_ctx* ctx, mukv_stats* out, mukv_stream stream) {
 const char* mukv_last_error(const mukv_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
 
 }  // extern "C"
+
+// =====================================================================================
+// Scoring without a workspace.
+//
+// Everything above works in memory the caller hands over (store, workspace).  Some callers
+// cannot produce such a buffer: a plug-in that runs inside a serving process whose start-up
+// code has already given the whole device to its KV-cache pool, or a control loop that is
+// forbidden to touch the allocator once it is running (cudaMalloc may fail there, and it
+// synchronises the device when it does not).  For them the scratch of the scoring kernel lives
+// in the array below, which is part of the loaded library image on every device.
+// =====================================================================================
+namespace {
+
+constexpr int kNaFrames = MUKV_NOALLOC_MAX_FRAMES, kNaHq = MUKV_NOALLOC_MAX_Q_HEADS;
+constexpr int kNaHkv = MUKV_NOALLOC_MAX_KV_HEADS, kNaP = MUKV_MAX_TOKENS;
+constexpr size_t kNaColF = 0;
+constexpr size_t kNaFftF = kNaColF + (size_t)kNaFrames * kNaHq * kNaP * sizeof(float);
+constexpr size_t kNaColD = kNaFftF + (size_t)kNaFrames * kNaHkv * kNaP * sizeof(float);
+constexpr size_t kNaFftD = kNaColD + (size_t)kNaFrames * kNaHq * kNaP * sizeof(double);
+constexpr size_t kNaKept = kNaFftD + (size_t)kNaFrames * kNaHkv * kNaP * sizeof(double);
+constexpr size_t kNaTs = kNaKept + (size_t)kNaFrames * kNaP * sizeof(int);
+constexpr size_t kNaPt = kNaTs + 256;
+constexpr size_t kNaCtrl = kNaPt + 256;                  // frame_counter[16], flagged[16], n_flagged
+constexpr size_t kNaCtrlBytes = 256;
+constexpr size_t kNaTotal = kNaCtrl + kNaCtrlBytes;
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaTotal];
+
+constexpr int kNaMaxDevices = 64;
+unsigned char* g_noalloc_ptr[kNaMaxDevices];             // device address of the array, per device
+
+// Once per device, with that device current: resolves the array's device address and raises the
+// dynamic shared-memory limit of every variant of the scoring kernel to what the largest
+// supported frame needs.  Allocates nothing.
+cudaError_t noalloc_setup(int dev, unsigned char** out) {
+  if (!g_noalloc_ptr[dev]) {
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    const int ncs[4] = {2, 4, 7, 8};
+    for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+      const int nc = ncs[i];
+      e = set_score_attr<__nv_bfloat16, float>(nc, score_smem_bytes<__nv_bfloat16, float>(kNaP, 128));
+      if (e == cudaSuccess)
+        e = set_score_attr<__nv_bfloat16, double>(nc, score_smem_bytes<__nv_bfloat16, double>(kNaP, 128));
+      if (e == cudaSuccess) e = set_score_attr<float, float>(nc, score_smem_bytes<float, float>(kNaP, 128));
+      if (e == cudaSuccess) e = set_score_attr<float, double>(nc, score_smem_bytes<float, double>(kNaP, 128));
+    }
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[dev] = static_cast<unsigned char*>(ptr);
+  }
+  *out = g_noalloc_ptr[dev];
+  return cudaSuccess;
+}
+
+template <typename T>
+mukv_status noalloc_impl(const mukv_config& c, const void* d_q, const void* d_k_last, int n, int* d_kept_out,
+                         float* d_scores_out, cudaStream_t st) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(nullptr, MUKV_E_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  if (dev < 0 || dev >= kNaMaxDevices) return fail(nullptr, MUKV_E_CAPACITY, "device index %d not supported", dev);
+  const int P = c.tokens_per_frame, D = c.head_dim, nc = pick_nc(P);
+  unsigned char* base = nullptr;
+  e = noalloc_setup(dev, &base);
+  if (e != cudaSuccess) return fail(nullptr, MUKV_E_CUDA, "set-up of the static scratch: %s", cudaGetErrorString(e));
+  // the array keeps what the last call left: the arrival counters and the flagged list start at zero
+  e = cudaMemsetAsync(base + kNaCtrl, 0, kNaCtrlBytes, st);
+  if (e != cudaSuccess) return fail(nullptr, MUKV_E_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+  ScoreParams sp;
+  memset(&sp, 0, sizeof sp);
+  sp.P = P; sp.Hq = c.n_q_heads; sp.Hkv = c.n_kv_heads; sp.D = D; sp.G = c.n_q_heads / c.n_kv_heads;
+  sp.kappa = c.keep_per_frame; sp.n_frames = n; sp.causal = c.attn_causal; sp.keep_low = c.keep_low_freq;
+  sp.alpha = c.alpha; sp.tie_eps = c.tie_eps; sp.flag_margin = 3e-6f; sp.flat_ratio = 1e-3f;
+  sp.first_frame = 0;
+  sp.q = d_q;
+  sp.k_last = d_k_last;
+  sp.colsum_part = base + kNaColF;
+  sp.ifft_part = base + kNaFftF;
+  sp.frame_counter = reinterpret_cast<int*>(base + kNaCtrl);
+  sp.flagged = reinterpret_cast<int*>(base + kNaCtrl) + kNaFrames;
+  sp.n_flagged = reinterpret_cast<int*>(base + kNaCtrl) + 2 * kNaFrames;
+  sp.kept_store = d_kept_out ? d_kept_out : reinterpret_cast<int*>(base + kNaKept);
+  sp.kept_out = nullptr;
+  sp.scores_out = d_scores_out;
+  sp.frame_ts = reinterpret_cast<long long*>(base + kNaTs);
+  sp.page_table = reinterpret_cast<long long*>(base + kNaPt);
+  sp.refine = 0;
+  const dim3 grid(c.n_q_heads, n);
+  e = launch_score<T, float>(sp, nc, grid, score_smem_bytes<T, float>(P, D), st);
+  if (e != cudaSuccess) return fail(nullptr, MUKV_E_CUDA, "score kernel: %s", cudaGetErrorString(e));
+  sp.refine = 1;
+  sp.colsum_part = base + kNaColD;
+  sp.ifft_part = base + kNaFftD;
+  e = launch_score<T, double>(sp, nc, grid, score_smem_bytes<T, double>(P, D), st);
+  if (e != cudaSuccess) return fail(nullptr, MUKV_E_CUDA, "refine kernel: %s", cudaGetErrorString(e));
+  return MUKV_OK;
+}
+
+}  // namespace
+
+extern "C" mukv_status mukv_score_frames_noalloc(const mukv_config* cfg, const void* d_q, const void* d_k_last,
+                                                 int32_t n_frames, int32_t* d_kept_out, float* d_scores_out,
+                                                 mukv_stream stream) {
+  try {
+    if (!cfg || !d_q || !d_k_last) return fail(nullptr, MUKV_E_INVALID, "null argument");
+    if (!d_kept_out && !d_scores_out) return fail(nullptr, MUKV_E_INVALID, "no output requested");
+    mukv_config c = *cfg;
+    if (c.max_frames < 1) c.max_frames = 1;                      // not used here
+    if (c.max_frames_per_chunk < 1) c.max_frames_per_chunk = 1;
+    if (c.n_layers < 1) c.n_layers = 1;
+    if (c.frames_per_segment < 1) c.frames_per_segment = 1;
+    if (const char* why = check_config(&c))
+      return fail(nullptr, (c.dtype != MUKV_BF16 && c.dtype != MUKV_FP32) ? MUKV_E_DTYPE : MUKV_E_SHAPE, "%s", why);
+    if (n_frames < 1) return fail(nullptr, MUKV_E_INVALID, "n_frames must be >= 1");
+    if (n_frames > kNaFrames || c.n_q_heads > kNaHq || c.n_kv_heads > kNaHkv)
+      return fail(nullptr, MUKV_E_CAPACITY,
+                  "the static scratch holds at most %d frames, %d query heads and %d key heads per call "
+                  "(got %d, %d, %d)", kNaFrames, kNaHq, kNaHkv, n_frames, c.n_q_heads, c.n_kv_heads);
+    if (!aligned16(d_q) || !aligned16(d_k_last) || !aligned4(d_kept_out) || !aligned4(d_scores_out))
+      return fail(nullptr, MUKV_E_ALIGN, "d_q, d_k_last must be 16-byte aligned, the outputs 4-byte aligned");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (c.dtype == MUKV_BF16)
+      return noalloc_impl<__nv_bfloat16>(c, d_q, d_k_last, n_frames, d_kept_out, d_scores_out, st);
+    return noalloc_impl<float>(c, d_q, d_k_last, n_frames, d_kept_out, d_scores_out, st);
+  } catch (...) {
+    return fail(nullptr, MUKV_E_INVALID, "unexpected exception");
+  }
+}
