@@ -83,15 +83,30 @@ template <typename A> __device__ __forceinline__ A warp_min(A v) {
   return v;
 }
 
-// Exclusive prefix count of `flag` over the thread block in thread order, plus the block total.
-// scratch: at least (blockDim.x/32 + 1) ints of shared memory.  Contains two barriers.
-__device__ __forceinline__ int block_excl_count(bool flag, int* scratch, int& total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+// A set of threads that synchronise together: the whole block, or a fixed sub-range of its
+// threads on a named barrier (warp-specialised kernels, where other warps never join).
+struct BlockGroup {
+  __device__ __forceinline__ static int tid() { return threadIdx.x; }
+  __device__ __forceinline__ static int size() { return blockDim.x; }
+  __device__ __forceinline__ static void sync() { __syncthreads(); }
+};
+template <int ID, int NT, int OFF> struct NamedGroup {
+  __device__ __forceinline__ static int tid() { return (int)threadIdx.x - OFF; }
+  __device__ __forceinline__ static int size() { return NT; }
+  __device__ __forceinline__ static void sync() { asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(NT) : "memory"); }
+};
+
+// Exclusive prefix count of `flag` over the group in thread order, plus the group total.
+// scratch: at least (size/32 + 1) ints of shared memory.  Contains two barriers.
+template <class Grp>
+__device__ __forceinline__ int group_excl_count(bool flag, int* scratch, int& total) {
+  const int t = Grp::tid();
+  const int lane = t & 31, warp = t >> 5, nwarp = (Grp::size() + 31) >> 5;
   const unsigned b = __ballot_sync(kFull, flag);
   const int in_warp = __popc(b & ((1u << lane) - 1u));
-  __syncthreads();                       // scratch may still be read from a previous call
+  Grp::sync();                           // scratch may still be read from a previous call
   if (lane == 0) scratch[warp] = __popc(b);
-  __syncthreads();
+  Grp::sync();
   int before = 0, sum = 0;
   for (int w = 0; w < nwarp; ++w) {
     const int c = scratch[w];
@@ -100,6 +115,9 @@ __device__ __forceinline__ int block_excl_count(bool flag, int* scratch, int& to
   }
   total = sum;
   return before + in_warp;
+}
+__device__ __forceinline__ int block_excl_count(bool flag, int* scratch, int& total) {
+  return group_excl_count<BlockGroup>(flag, scratch, total);
 }
 
 // 16-byte streaming copies

@@ -19,6 +19,7 @@
 #include "compact.cuh"
 #include "retrieve.cuh"
 #include "score.cuh"
+#include "score_ps.cuh"
 #include "score_tc.cuh"
 
 using namespace mukv;
@@ -35,16 +36,17 @@ struct StoreLayout {
 };
 
 struct WorkLayout {
-  size_t colsum_f, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, stat_refined, dev_status;
+  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, stat_refined, dev_status;
   size_t q64, qnorm, s_frm, s_seg, wtab, total;
   size_t zero_begin, zero_end;          // region that must start as zeros
 };
 
 // Tiling of the tensor-core scoring kernel (bf16 inputs only).
 struct TcShape {
-  bool ok;
+  bool ok;                 // bf16 chunk scored on the tensor cores
+  bool persistent;         // by the persistent kernel (its operand buffers fit in shared memory)
   int tpt, tiles, npad, n_mt, tmem_cols;
-  size_t smem;
+  size_t smem, smem_ps;
 };
 
 thread_local std::string g_create_error;
@@ -62,6 +64,7 @@ struct mukv_ctx {
   int C, G, esize, nc;
   float flag_margin, flat_ratio;
   TcShape tcs;                           // tcs.ok: the chunk is scored on the tensor cores
+  int n_sms;
   CUtensorMap wmap;                      // DFT matrix terms [3*D][D] bf16
   std::string err;
   // optional per-kernel timing (host objects only)
@@ -167,7 +170,9 @@ TcShape tc_shape(const mukv_config& c) {
   t.tmem_cols = 32;
   while (t.tmem_cols < need) t.tmem_cols *= 2;
   t.smem = score_tc_smem_bytes(c.tokens_per_frame, c.head_dim);
+  t.smem_ps = score_ps_smem_bytes(c.tokens_per_frame, c.head_dim);
   t.ok = t.smem <= 227 * 1024;
+  t.persistent = t.ok && t.smem_ps <= 227 * 1024;
   return t;
 }
 
@@ -181,6 +186,7 @@ WorkLayout work_layout(const mukv_config& c) {
   const size_t parts = ts.ok && (size_t)c.n_kv_heads * ts.tiles > (size_t)c.n_q_heads
                            ? (size_t)c.n_kv_heads * ts.tiles : (size_t)c.n_q_heads;
   w.colsum_f = off;       off = align_up(off + F * parts * P * sizeof(float));
+  w.colsum_p = off;       off = align_up(off + (ts.persistent ? (kPsMaxBlocks + F) * P * sizeof(float) : 0));
   w.ifft_f = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(float));
   w.colsum_d = off;       off = align_up(off + F * c.n_q_heads * P * sizeof(double));
   w.ifft_d = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(double));
@@ -318,6 +324,21 @@ cudaError_t launch_score_tc(mukv_ctx* ctx, const ScoreParams& sp, const void* d_
       !encode_map3(&kmap_dft, k_last, D, c.n_kv_heads, rows, 1, 128)) {
     *why = "cuTensorMapEncodeTiled failed";
     return cudaErrorInvalidValue;
+  }
+  if (t.persistent) {
+    ScorePsParams pp;
+    memset(&pp, 0, sizeof pp);
+    pp.sp = sp;
+    pp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
+    pp.tiles = t.tiles; pp.tpt = t.tpt; pp.npad = t.npad; pp.n_mt = t.n_mt;
+    pp.n_items = n * c.n_kv_heads * (t.n_mt + t.tiles);
+    pp.exp2_scale = (float)(1.4426950408889634 / std::sqrt((double)D));
+    pp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
+    int blocks = ctx->n_sms < kPsMaxBlocks ? ctx->n_sms : kPsMaxBlocks;
+    if (blocks > pp.n_items) blocks = pp.n_items;
+    score_ps_kernel<<<blocks, kPsThreads, t.smem_ps, st>>>(pp, qmap, kmap, ctx->wmap);
+    *why = "score_ps kernel";
+    return cudaGetLastError();
   }
   ScoreTcParams tp;
   memset(&tp, 0, sizeof tp);
@@ -462,7 +483,9 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
   ctx->esize = cfg->dtype == MUKV_BF16 ? 2 : 4;
   ctx->nc = pick_nc(cfg->tokens_per_frame);
   ctx->tcs = tc_shape(*cfg);
-  if (const char* s = getenv("MUKV_SCORE_FMA")) if (atoi(s) != 0) ctx->tcs.ok = false;
+  if (const char* s = getenv("MUKV_SCORE_FMA")) if (atoi(s) != 0) ctx->tcs.ok = ctx->tcs.persistent = false;
+  if (const char* s = getenv("MUKV_SCORE_TILE_BLOCKS")) if (atoi(s) != 0) ctx->tcs.persistent = false;
+  ctx->n_sms = 1;
   ctx->flag_margin = 3e-6f;
   ctx->flat_ratio = 1e-3f;
   if (const char* s = getenv("MUKV_FLAG_MARGIN")) ctx->flag_margin = (float)atof(s);
@@ -486,6 +509,12 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute((const void*)score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)ctx->tcs.smem);
+    if (e == cudaSuccess && ctx->tcs.persistent)
+      e = cudaFuncSetAttribute((const void*)score_ps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)ctx->tcs.smem_ps);
+    int dev = 0;
+    if (e == cudaSuccess) e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, dev);
   }
   if (e == cudaSuccess)
     e = cudaMemset(ctx->ws + ctx->wl.zero_begin, 0, ctx->wl.zero_end - ctx->wl.zero_begin);

@@ -58,17 +58,17 @@ __host__ inline size_t score_smem_bytes(int P, int D) {
   return ((ks + 15) / 16) * 16 + qs + tw + red + sel + 64;
 }
 
-// Eq. 4 and the top-kappa rule for one frame, run by the whole block.  Thread tid owns the tokens
-// tid + k*blockDim.x, k < TOK (TOK*blockDim.x >= P); att_raw / fft_raw are their I_att and I_fft;
+// Eq. 4 and the top-kappa rule for one frame, run by all threads of the group Grp.  Thread tid owns
+// the tokens tid + k*size, k < TOK (TOK*size >= P); att_raw / fft_raw are their I_att and I_fft;
 // s_sc (P doubles), s_int (one int per warp + 1), s_misc (4 doubles per warp) are shared scratch.
 // The arithmetic here is always double: it is a few hundred operations per frame and keeps
 // the normalisation from adding rounding noise of its own to the scores.
-template <int TOK>
+template <int TOK, class Grp = BlockGroup>
 __device__ inline void select_frame(const ScoreParams& p, int f, const double (&att_raw)[TOK],
                                     const double (&fft_raw)[TOK], double* s_sc, int* s_int, double* s_misc) {
   typedef double A;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int nt = blockDim.x, nwarp = nt >> 5;
+  const int tid = Grp::tid(), lane = tid & 31, warp = tid >> 5;
+  const int nt = Grp::size(), nwarp = nt >> 5;
   const int P = p.P;
   const A big = (A)3.0e38;
   int tok[TOK];
@@ -91,7 +91,7 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
 #pragma unroll
     for (int i = 0; i < 4; ++i) s_misc[warp * 4 + i] = v[i];
   }
-  __syncthreads();
+  Grp::sync();
   A amin = big, amax = -big, fmin_ = big, fmax_ = -big;
   for (int w = 0; w < nwarp; ++w) {
     amin = s_misc[w * 4 + 0] < amin ? s_misc[w * 4 + 0] : amin;
@@ -99,7 +99,7 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
     fmin_ = s_misc[w * 4 + 2] < fmin_ ? s_misc[w * 4 + 2] : fmin_;
     fmax_ = s_misc[w * 4 + 3] > fmax_ ? s_misc[w * 4 + 3] : fmax_;
   }
-  __syncthreads();
+  Grp::sync();
   // ---- Eq. 4
   const A alpha = (A)p.alpha;
   A s[TOK];
@@ -111,7 +111,7 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
     s[k] = alpha * an + ((A)1 - alpha) * fn;
     if (valid[k]) s_sc[tok[k]] = s[k];
   }
-  __syncthreads();
+  Grp::sync();
   // ---- tau = kappa-th largest score (rank counting; P <= 256)
   const int kappa = p.kappa;
 #pragma unroll
@@ -126,7 +126,7 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
       if (gt < kappa && kappa <= ge) s_misc[0] = s[k];      // every writer holds the same value
     }
   }
-  __syncthreads();
+  Grp::sync();
   const A tau = s_misc[0];
   const A delta = (A)p.tie_eps;
   bool sure[TOK], band[TOK], keep[TOK];
@@ -136,14 +136,14 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
     sure[k] = valid[k] && (s[k] > tau + delta);
     band[k] = valid[k] && !sure[k] && (s[k] >= tau - delta);
     int t;
-    block_excl_count(sure[k], s_int, t);
+    group_excl_count<Grp>(sure[k], s_int, t);
     n_sure += t;
   }
   int band_before = 0;
 #pragma unroll
   for (int k = 0; k < TOK; ++k) {
     int t;
-    const int band_rank = band_before + block_excl_count(band[k], s_int, t);
+    const int band_rank = band_before + group_excl_count<Grp>(band[k], s_int, t);
     band_before += t;
     keep[k] = sure[k] || (band[k] && band_rank < kappa - n_sure);
   }
@@ -152,7 +152,7 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
 #pragma unroll
   for (int k = 0; k < TOK; ++k) {
     int t;
-    const int pos = out_before + block_excl_count(keep[k], s_int, t);
+    const int pos = out_before + group_excl_count<Grp>(keep[k], s_int, t);
     out_before += t;
     if (keep[k]) {
       p.kept_store[f_abs * kappa + pos] = tok[k];
@@ -185,9 +185,9 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
     }
     a = warp_min(a);
     b = warp_max(b);
-    __syncthreads();
+    Grp::sync();
     if (lane == 0) { s_misc[warp * 4] = a; s_misc[warp * 4 + 1] = b; }
-    __syncthreads();
+    Grp::sync();
     if (tid == 0) {
       for (int w = 1; w < nwarp; ++w) {
         a = s_misc[w * 4] < a ? s_misc[w * 4] : a;

@@ -1,0 +1,461 @@
+// Persistent, warp-specialised tensor-core scoring of a bf16 chunk (Sec. 3.3, Eq. 1-4).
+//
+// score_ps_kernel: one block of 320 threads per SM.  The chunk is a list of items, ordered by
+// (frame, key head): first the DFT row tiles of that head's keys (Eq. 2-3), then the attention
+// row tiles (Eq. 1; the G query heads of the group are flattened with the tokens into rows, as
+// in score_tc_kernel).  Each block takes a contiguous share of the list.
+//
+//   warp 0      TMA producer: the three bf16 terms of the DFT matrix once, the key tile K_g of a
+//               (frame, head) when the head changes, a Q row tile per attention item (2 stages).
+//   warp 1      issues tcgen05.mma into one of two 256-column accumulators in tensor memory and
+//               commits to the barriers that free the operand buffers.
+//   warps 2-9   epilogue.  Two warps share each 32-lane quarter of the accumulator and split its
+//               columns.  Attention item: row maximum, exp and row sum (both exchanged between the
+//               two warps through shared memory), then acc[column] += e / sum in registers.  The
+//               32 rows of a warp are added only when the block leaves a frame (shuffle butterfly),
+//               so the per-tile cost is one fused multiply-add per logit.  DFT item: magnitudes of
+//               the D bins of each key vector, summed.
+//
+// Per frame, every block that worked on it stores its column sums in a slot of its own; the
+// block that arrives last (counter, nobody waits) adds the slots in a fixed order, applies
+// Eq. 4 and selects the kappa tokens.  All mbarrier waits are bounded; a wait that runs out
+// makes the role record a code in the status word and leave its loop.
+#pragma once
+#include "common.cuh"
+#include "score.cuh"
+#include "score_tc.cuh"
+#include "tc.cuh"
+
+namespace mukv {
+
+constexpr int kPsThreads = 320;
+constexpr int kPsEpiThreads = 256;
+constexpr int kPsEpiOff = 64;              // first epilogue thread
+constexpr int kPsMiscBytes = 8192;
+constexpr int kPsMaxBlocks = 256;          // bound on the grid (slots of partial sums)
+typedef NamedGroup<5, kPsEpiThreads, kPsEpiOff> PsEpiGroup;
+
+struct ScorePsParams {
+  ScoreParams sp;            // colsum_part: float [grid + n_frames][P] slots, ifft_part: float [F][Hkv][P]
+  int tiles, tpt, npad, n_mt;
+  int n_items;               // n_frames * Hkv * (n_mt + tiles)
+  float exp2_scale;          // log2(e) / sqrt(D)
+  int* status;
+};
+
+__host__ inline size_t score_ps_smem_bytes(int P, int D) {
+  const size_t KB = D / 64, npad = (P + 15) / 16 * 16;
+  return KB * npad * 128 + 2 * KB * 128 * 128 + 3 * KB * (size_t)D * 128 + kPsMiscBytes + 1024;
+}
+
+// owner of item i when n items are split into contiguous shares [c*n/nb, (c+1)*n/nb)
+__device__ __forceinline__ int ps_owner(long long i, long long n, long long nb) {
+  return (int)(((i + 1) * nb - 1) / n);
+}
+
+__device__ __forceinline__ float ps_chunk_max(const uint32_t (&r)[16], int col0, int P, bool causal, int i_tok) {
+  float m0 = -INFINITY, m1 = -INFINITY;
+  if (!causal && col0 + 16 <= P) {
+#pragma unroll
+    for (int k = 0; k < 16; k += 4) {
+      m0 = fmaxf(m0, fmaxf(__uint_as_float(r[k]), __uint_as_float(r[k + 1])));
+      m1 = fmaxf(m1, fmaxf(__uint_as_float(r[k + 2]), __uint_as_float(r[k + 3])));
+    }
+  } else {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const int j = col0 + k;
+      const bool ok = (j < P) && (!causal || j <= i_tok);
+      m0 = ok ? fmaxf(m0, __uint_as_float(r[k])) : m0;
+    }
+  }
+  return fmaxf(m0, m1);
+}
+
+// r <- exp2(r * c - mc) (0 where masked); returns the sum
+__device__ __forceinline__ float ps_chunk_exp(uint32_t (&r)[16], float c, float mc, int col0, int P, bool causal,
+                                              int i_tok) {
+  float l0 = 0.f, l1 = 0.f;
+  if (!causal && col0 + 16 <= P) {
+#pragma unroll
+    for (int k = 0; k < 16; k += 2) {
+      const float e0 = ex2_approx(fmaf(__uint_as_float(r[k]), c, -mc));
+      const float e1 = ex2_approx(fmaf(__uint_as_float(r[k + 1]), c, -mc));
+      l0 += e0;
+      l1 += e1;
+      r[k] = __float_as_uint(e0);
+      r[k + 1] = __float_as_uint(e1);
+    }
+  } else {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const int j = col0 + k;
+      const bool ok = (j < P) && (!causal || j <= i_tok);
+      const float e = ok ? ex2_approx(fmaf(__uint_as_float(r[k]), c, -mc)) : 0.f;
+      l0 += e;
+      r[k] = __float_as_uint(e);
+    }
+  }
+  return l0 + l1;
+}
+
+// Eq. 4 and the selection for frame f, run by the epilogue warps of the block that finished the
+// frame last.  Kept out of line so that the tile loop's register allocation is not disturbed.
+__device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c_first, int c_last, double* s_sc,
+                                             int* s_int, double* s_misc) {
+  const int et = PsEpiGroup::tid();
+  const int P = sp.P, Hkv = sp.Hkv;
+  double att[1] = {0.0}, fft[1] = {0.0};
+  if (et < P) {
+    const float* cp = reinterpret_cast<const float*>(sp.colsum_part) + et;
+    for (int cc = c_first; cc <= c_last; ++cc) att[0] += (double)__ldcg(cp + (long long)(cc + f) * P);
+    att[0] = att[0] / (double)((long long)sp.Hq * P);
+    const float* fp = reinterpret_cast<const float*>(sp.ifft_part) + (long long)f * Hkv * P + et;
+    for (int gg = 0; gg < Hkv; ++gg) fft[0] += (double)__ldcg(fp + (long long)gg * P);
+    fft[0] = fft[0] / (double)((long long)Hkv * sp.D);
+  }
+  PsEpiGroup::sync();
+  select_frame<1, PsEpiGroup>(sp, f, att, fft, s_sc, s_int, s_misc);
+}
+
+__global__ void __maxnreg__(200) score_ps_kernel(const ScorePsParams p,
+                                                                 const __grid_constant__ CUtensorMap qmap,
+                                                                 const __grid_constant__ CUtensorMap kmap,
+                                                                 const __grid_constant__ CUtensorMap wmap) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = tc::smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* sm = smem_raw + (base - raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const ScoreParams& sp = p.sp;
+  const int P = sp.P, D = sp.D, G = sp.G, Hkv = sp.Hkv, KB = D >> 6;
+  const int ipu = p.n_mt + p.tiles;                      // items per (frame, key head)
+  const int ipf = Hkv * ipu;                             // items per frame
+  const int n_cta = gridDim.x, cta = blockIdx.x;
+  const int i0 = (int)((long long)cta * p.n_items / n_cta);
+  const int i1 = (int)((long long)(cta + 1) * p.n_items / n_cta);
+  const int rows_q = p.tpt * G;
+
+  const uint32_t k_kb = (uint32_t)p.npad * 128u, q_kb = 128u * 128u, w_kb = (uint32_t)D * 128u;
+  const uint32_t sK = base;
+  const uint32_t sQ = sK + (uint32_t)KB * k_kb;
+  const uint32_t sW = sQ + 2u * KB * q_kb;
+  const uint32_t misc_off = (uint32_t)KB * k_kb + 2u * KB * q_kb + 3u * KB * w_kb;
+  float* s_col = reinterpret_cast<float*>(sm + misc_off);                     // [4][256]
+  float* s_mx = reinterpret_cast<float*>(sm + misc_off + 4096);               // [2][128]
+  float* s_sum = s_mx + 256;                                                  // [2][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + misc_off + 6144);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + misc_off + 6144 + 96);
+  int* s_flag = reinterpret_cast<int*>(sm + misc_off + 6144 + 100);
+  const uint32_t b0 = tc::smem_u32(bars);
+  const uint32_t bar_w = b0, bar_kf = b0 + 8, bar_ke = b0 + 16;
+  // stage / buffer s of: Q full, Q empty, accumulator full, accumulator empty
+#define PS_BAR_QF(s) (b0 + 24u + 8u * (uint32_t)(s))
+#define PS_BAR_QE(s) (b0 + 40u + 8u * (uint32_t)(s))
+#define PS_BAR_AF(s) (b0 + 56u + 8u * (uint32_t)(s))
+#define PS_BAR_AE(s) (b0 + 72u + 8u * (uint32_t)(s))
+
+  if (tid == 0) {
+    tc::mbar_init(bar_w, 1);
+    tc::mbar_init(bar_kf, 1);
+    tc::mbar_init(bar_ke, 1);
+    for (int s = 0; s < 2; ++s) {
+      tc::mbar_init(PS_BAR_QF(s), 1);
+      tc::mbar_init(PS_BAR_QE(s), 1);
+      tc::mbar_init(PS_BAR_AF(s), 1);
+      tc::mbar_init(PS_BAR_AE(s), 8);                    // one arrival per epilogue warp
+    }
+    tc::fence_mbar_init();
+    tc::prefetch_tmap(&qmap);
+    tc::prefetch_tmap(&kmap);
+    tc::prefetch_tmap(&wmap);
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tc::tmem_alloc(tc::smem_u32(tmem_slot), 512u);
+  }
+  // rows of the Q stages that the TMA box never writes must not hold stale bits
+  {
+    const int pad_rows = 128 - rows_q;
+    uint4* q4 = reinterpret_cast<uint4*>(sm + (size_t)KB * k_kb);
+    for (int i = tid; i < 2 * KB * pad_rows * 8; i += kPsThreads) {
+      const int blk = i / (pad_rows * 8), rem = i % (pad_rows * 8);
+      q4[(size_t)blk * (q_kb / 16) + (size_t)rows_q * 8 + rem] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+  tc::fence_proxy_async_smem();
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ================================================================== TMA producer
+    if (lane == 0) {
+      bool ok = true;
+      tc::mbar_expect_tx(bar_w, 3u * KB * w_kb);
+      for (int t = 0; t < 3; ++t)
+        for (int kb = 0; kb < KB; ++kb)
+          tc::tma_load_2d(sW + (uint32_t)(t * KB + kb) * w_kb, &wmap, kb * 64, t * D, bar_w);
+      int nk = 0, nq = 0, last_unit = -1;
+      for (int i = i0; i < i1; ++i) {
+        const int unit = i / ipu, x = i % ipu;
+        const int f = unit / Hkv, g = unit % Hkv;
+        if (unit != last_unit) {
+          ok = tc::mbar_wait(bar_ke, (uint32_t)((nk & 1) ^ 1));
+          if (!ok) break;
+          tc::mbar_expect_tx(bar_kf, (uint32_t)KB * k_kb);
+          for (int kb = 0; kb < KB; ++kb) tc::tma_load_3d(sK + kb * k_kb, &kmap, kb * 64, g, f * P, bar_kf);
+          ++nk;
+          last_unit = unit;
+        }
+        if (x >= p.n_mt) {
+          const int s = nq & 1;
+          ok = tc::mbar_wait(PS_BAR_QE(s), (uint32_t)(((nq >> 1) & 1) ^ 1));
+          if (!ok) break;
+          tc::mbar_expect_tx(PS_BAR_QF(s), (uint32_t)KB * (uint32_t)rows_q * 128u);
+          for (int kb = 0; kb < KB; ++kb)
+            tc::tma_load_3d(sQ + (uint32_t)(s * KB + kb) * q_kb, &qmap, kb * 64, g * G,
+                            f * P + (x - p.n_mt) * p.tpt, PS_BAR_QF(s));
+          ++nq;
+        }
+      }
+      if (!ok) atomicCAS(p.status, 0, 3);
+      // copies of this thread still in flight land before the block goes away
+      tc::mbar_wait(bar_w, 0);
+      if (nk) tc::mbar_wait(bar_kf, (uint32_t)((nk - 1) & 1));
+      for (int s = 0; s < 2; ++s) {
+        const int cnt = (nq + 1 - s) >> 1;
+        if (cnt) tc::mbar_wait(PS_BAR_QF(s), (uint32_t)((cnt - 1) & 1));
+      }
+    }
+  } else if (warp == 1) {
+    // ================================================================== MMA issuer
+    if (lane == 0) {
+      bool ok = tc::mbar_wait(bar_w, 0);
+      tc::tc_fence_after_sync();
+      const uint32_t idesc_att = tc::idesc_bf16_f32(128, p.npad), idesc_dft = tc::idesc_bf16_f32(128, D);
+      int nk = 0, nq = 0, it = 0, last_unit = -1;
+      for (int i = i0; i < i1 && ok; ++i, ++it) {
+        const int unit = i / ipu, x = i % ipu;
+        if (unit != last_unit) {
+          ok = tc::mbar_wait(bar_kf, (uint32_t)(nk & 1));
+          if (!ok) break;
+          ++nk;
+          last_unit = unit;
+        }
+        const int b = it & 1;
+        ok = tc::mbar_wait(PS_BAR_AE(b), (uint32_t)(((it >> 1) & 1) ^ 1));
+        if (!ok) break;
+        tc::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem + (uint32_t)b * 256u;
+        if (x < p.n_mt) {
+          // smallest term first: lo, mid, hi
+          uint32_t accum = 0;
+          for (int t = 2; t >= 0; --t)
+            for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                tc::mma_bf16_ss(d_tmem, tc::smem_desc_sw128(sK + kb * k_kb + (uint32_t)x * q_kb + k * 32),
+                                tc::smem_desc_sw128(sW + (uint32_t)(t * KB + kb) * w_kb + k * 32), idesc_dft, accum);
+                accum = 1;
+              }
+        } else {
+          const int s = nq & 1;
+          ok = tc::mbar_wait(PS_BAR_QF(s), (uint32_t)((nq >> 1) & 1));
+          if (!ok) break;
+          tc::tc_fence_after_sync();
+          for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              tc::mma_bf16_ss(d_tmem, tc::smem_desc_sw128(sQ + (uint32_t)(s * KB + kb) * q_kb + k * 32),
+                              tc::smem_desc_sw128(sK + kb * k_kb + k * 32), idesc_att, (kb | k) != 0);
+          tc::mma_commit(PS_BAR_QE(s));
+          ++nq;
+        }
+        tc::mma_commit(PS_BAR_AF(b));
+        if (i + 1 == i1 || (i + 1) / ipu != unit) tc::mma_commit(bar_ke);
+      }
+      if (!ok) atomicCAS(p.status, 0, 4);
+    }
+  } else {
+    // ================================================================== epilogue
+    const int et = tid - kPsEpiOff, ew = et >> 5;
+    const int q = warp & 3, h = ew >> 2;                 // TMEM lane quarter, column half
+    const int row = q * 32 + lane;
+    const uint32_t tlane = (uint32_t)(q * 32) << 16;
+    const int nch16 = p.npad >> 4, nch0 = (nch16 + 1) >> 1;
+    const int my_c0 = h ? nch0 : 0, my_nch = h ? nch16 - nch0 : nch0;
+    const bool causal = sp.causal != 0;
+    const float c = p.exp2_scale;
+    float acc[128];
+#pragma unroll
+    for (int k = 0; k < 128; ++k) acc[k] = 0.f;
+    bool ok = true;
+    int it = 0;
+    for (int i = i0; i < i1; ++i, ++it) {
+      const int unit = i / ipu, x = i % ipu;
+      const int f = unit / Hkv, g = unit % Hkv;
+      const int b = it & 1;
+      const bool done = tc::mbar_wait(PS_BAR_AF(b), (uint32_t)((it >> 1) & 1));
+      ok = tc::named_sync_and(5, kPsEpiThreads, done);
+      if (!ok) break;
+      tc::tc_fence_after_sync();
+      const uint32_t tb = tmem + (uint32_t)b * 256u + tlane;
+      if (x < p.n_mt) {
+        // ---- Eq. 2-3: this thread's half of the bins of its token
+        const int H2 = D >> 1, bins = H2 >> 1, bin0 = h * bins;
+        float tot = 0.f;
+#pragma unroll 1
+        for (int cc = 0; cc < bins; cc += 16) {
+          uint32_t re[16], im[16];
+          tc::tmem_ld16(tb + bin0 + cc, re);
+          tc::tmem_ld16(tb + H2 + bin0 + cc, im);
+          tc::tmem_wait_ld16x2(re, im);
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            const float a = __uint_as_float(re[k]), bb = __uint_as_float(im[k]);
+            const float mag = sqrtf(fmaf(a, a, bb * bb));
+            // bins 0 and D/2 are real: their two values sit in the re/im slots of "bin 0"
+            tot += (bin0 + cc + k == 0) ? fabsf(a) + fabsf(bb) : 2.f * mag;
+          }
+        }
+        s_sum[h * 128 + row] = tot;
+        tc::named_sync(1 + q, 64);
+        const int token = x * 128 + row;
+        if (h == 0 && token < P)
+          reinterpret_cast<float*>(sp.ifft_part)[((long long)f * Hkv + g) * P + token] = s_sum[row] + s_sum[128 + row];
+      } else {
+        // ---- Eq. 1
+        const int tile = x - p.n_mt;
+        const int i_tok = tile * p.tpt + row / G;
+        const bool valid = (row < rows_q) && (i_tok < P);
+        // pass A: row maximum
+        float m = -INFINITY;
+#pragma unroll 1
+        for (int ch = 0; ch < my_nch; ch += 2) {
+          uint32_t r0[16], r1[16];
+          const int col = (my_c0 + ch) * 16;
+          tc::tmem_ld16(tb + col, r0);
+          if (ch + 1 < my_nch) {
+            tc::tmem_ld16(tb + col + 16, r1);
+            tc::tmem_wait_ld16x2(r0, r1);
+            m = fmaxf(m, fmaxf(ps_chunk_max(r0, col, P, causal, i_tok), ps_chunk_max(r1, col + 16, P, causal, i_tok)));
+          } else {
+            tc::tmem_wait_ld16(r0);
+            m = fmaxf(m, ps_chunk_max(r0, col, P, causal, i_tok));
+          }
+        }
+        s_mx[h * 128 + row] = m;
+        tc::named_sync(1 + q, 64);
+        m = fmaxf(s_mx[row], s_mx[128 + row]);
+        // pass B: e = exp(z - max) back into tensor memory, row sum
+        const float mc = m * c;
+        float l = 0.f;
+#pragma unroll 1
+        for (int ch = 0; ch < my_nch; ch += 2) {
+          uint32_t r0[16], r1[16];
+          const int col = (my_c0 + ch) * 16;
+          tc::tmem_ld16(tb + col, r0);
+          if (ch + 1 < my_nch) {
+            tc::tmem_ld16(tb + col + 16, r1);
+            tc::tmem_wait_ld16x2(r0, r1);
+            l += ps_chunk_exp(r0, c, mc, col, P, causal, i_tok);
+            l += ps_chunk_exp(r1, c, mc, col + 16, P, causal, i_tok);
+            tc::tmem_st16(tb + col, r0);
+            tc::tmem_st16(tb + col + 16, r1);
+          } else {
+            tc::tmem_wait_ld16(r0);
+            l += ps_chunk_exp(r0, c, mc, col, P, causal, i_tok);
+            tc::tmem_st16(tb + col, r0);
+          }
+        }
+        tc::tmem_wait_st();
+        s_sum[h * 128 + row] = l;
+        tc::named_sync(1 + q, 64);
+        l = s_sum[row] + s_sum[128 + row];
+        const float inv = valid ? 1.f / l : 0.f;
+        const bool all_valid = __all_sync(kFull, valid);
+        // pass C: acc[column] += e / sum
+#pragma unroll
+        for (int pp = 0; pp < 4; ++pp) {
+          const int n_in = my_nch - 2 * pp;
+          if (n_in > 0) {
+            uint32_t r0[16], r1[16];
+            const int col = (my_c0 + 2 * pp) * 16;
+            tc::tmem_ld16(tb + col, r0);
+            if (n_in >= 2) {
+              tc::tmem_ld16(tb + col + 16, r1);
+              tc::tmem_wait_ld16x2(r0, r1);
+            } else {
+              tc::tmem_wait_ld16(r0);
+#pragma unroll
+              for (int k = 0; k < 16; ++k) r1[k] = 0u;
+            }
+            if (!all_valid && !valid) {
+#pragma unroll
+              for (int k = 0; k < 16; ++k) { r0[k] = 0u; r1[k] = 0u; }
+            }
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+              acc[pp * 32 + k] = fmaf(__uint_as_float(r0[k]), inv, acc[pp * 32 + k]);
+              acc[pp * 32 + 16 + k] = fmaf(__uint_as_float(r1[k]), inv, acc[pp * 32 + 16 + k]);
+            }
+          }
+        }
+      }
+      // the accumulator may be overwritten
+      tc::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(PS_BAR_AE(b));
+
+      if (i + 1 == i1 || (i + 1) / ipf != f) {
+        // ---- leaving frame f: publish this block's column sums, the last block selects
+#pragma unroll
+        for (int pp = 0; pp < 4; ++pp) {
+          float v[32];
+#pragma unroll
+          for (int k = 0; k < 32; ++k) { v[k] = acc[pp * 32 + k]; acc[pp * 32 + k] = 0.f; }
+          const float s = warp_column_sums(v, lane);
+          if (2 * pp + (lane >> 4) < my_nch) s_col[q * 256 + (my_c0 + 2 * pp) * 16 + lane] = s;
+        }
+        PsEpiGroup::sync();
+        float* slot = reinterpret_cast<float*>(sp.colsum_part) + (long long)(cta + f) * P;
+        for (int t = et; t < P; t += kPsEpiThreads)
+          slot[t] = (s_col[t] + s_col[256 + t]) + (s_col[512 + t] + s_col[768 + t]);
+        __threadfence();
+        PsEpiGroup::sync();
+        const int c_first = ps_owner((long long)f * ipf, p.n_items, n_cta);
+        const int c_last = ps_owner((long long)(f + 1) * ipf - 1, p.n_items, n_cta);
+        if (et == 0) {
+          const int n_slots = c_last - c_first + 1;
+          const int old = atomicAdd(sp.frame_counter + f, 1);
+          s_flag[0] = (old == n_slots - 1);
+          if (old == n_slots - 1) sp.frame_counter[f] = 0;          // ready for the next launch
+        }
+        PsEpiGroup::sync();
+        if (s_flag[0]) {
+          __threadfence();
+          ps_finish_frame(sp, f, c_first, c_last, reinterpret_cast<double*>(s_col),
+                          reinterpret_cast<int*>(sm + misc_off + 2560),
+                          reinterpret_cast<double*>(sm + misc_off + 2048));
+        }
+        PsEpiGroup::sync();
+      }
+    }
+    if (!ok && et == 0) atomicCAS(p.status, 0, 5);
+  }
+#undef PS_BAR_QF
+#undef PS_BAR_QE
+#undef PS_BAR_AF
+#undef PS_BAR_AE
+
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc::tmem_dealloc(tmem, 512u);
+  }
+}
+
+}  // namespace mukv

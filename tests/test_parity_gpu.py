@@ -149,6 +149,14 @@ def test_chunk7b_causal():
     full_compress_check(run)
 
 
+def test_chunk7b_tile_block_scoring(monkeypatch):
+    # the one-tile-per-block tensor-core kernel (used when the persistent kernel's buffers do not fit)
+    monkeypatch.setenv("MUKV_SCORE_TILE_BLOCKS", "1")
+    run = H.GpuRun("chunk7b", n_frames=5)
+    full_compress_check(run)
+    assert run.ctx.mukv_get_stats().device_status == 0
+
+
 def test_chunk7b_cuda_core_scoring(monkeypatch):
     # bf16 inputs scored by the plain multiply-add kernel (the one fp32 inputs always use)
     monkeypatch.setenv("MUKV_SCORE_FMA", "1")
