@@ -6,7 +6,8 @@
 // token order, to the frame's page; the same registers feed the mean over the kept rows.
 // The last-layer key plane is summed in double: its mean is the retrieval key (Eq. 5) that
 // later ranks blocks, so it is kept free of accumulation-order noise.
-// segment_kernel: mean over the frames of a segment that are present.
+// The block that finishes a (layer, K|V) plane of the chunk last (arrival counter, nobody waits)
+// refreshes that plane of every segment entry the chunk touches: mean over the frames present.
 #pragma once
 #include "common.cuh"
 
@@ -28,6 +29,11 @@ struct CompactParams {
   double* frame_ksum;             // [max_frames][C]  exact sums of the last-layer kept keys
   int* n_flagged;                 // reset here for the next chunk
   long long* stat_refined;        // device counter
+  // segment entries (Eq. 5 at segment level)
+  int fseg;                       // frames per segment
+  int* plane_counter;             // [L*2] arrivals per plane, zero between launches
+  float* seg_entry;               // [max_segs][L][2][C]
+  float* seg_key;                 // [max_segs][C]
 };
 
 // NV = 16-byte vectors per row; the block covers 256/NV rows per pass.
@@ -117,40 +123,40 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
       fe[col] = t / (float)kappa;
     }
   }
-}
 
-struct SegmentParams {
-  int L, C, kappa, fseg;
-  long long first_seg;            // first segment touched by the chunk
-  long long frames_total;         // frames stored after this chunk
-  const float* frame_entry;       // [max_frames][L][2][C]
-  const double* frame_ksum;       // [max_frames][C]
-  float* seg_entry;               // [max_segs][L][2][C]
-  float* seg_key;                 // [max_segs][C]
-};
-
-// one block per (plane, touched segment)
-__global__ void __launch_bounds__(256) segment_kernel(const SegmentParams p) {
-  const int plane = blockIdx.x, l = plane >> 1, kv = plane & 1;
-  const long long u = p.first_seg + blockIdx.y;
-  const long long t0 = u * p.fseg;
-  long long t1 = t0 + p.fseg;
-  if (t1 > p.frames_total) t1 = p.frames_total;
-  const int nf = (int)(t1 - t0);
-  const bool exact = (l == p.L - 1) && (kv == 0);
-  for (int col = threadIdx.x; col < p.C; col += blockDim.x) {
-    float m;
-    if (exact) {
-      double t = 0.0;
-      for (long long f = t0; f < t1; ++f) t += p.frame_ksum[f * p.C + col];
-      m = (float)(t / ((double)nf * (double)p.kappa));
-      p.seg_key[u * p.C + col] = m;
-    } else {
-      float t = 0.f;
-      for (long long f = t0; f < t1; ++f) t += p.frame_entry[((f * p.L + l) * 2 + kv) * p.C + col];
-      m = t / (float)nf;
+  // ---- segment entries of this plane, by the block that completes the plane
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int old = atomicAdd(p.plane_counter + plane, 1);
+    s_last = (old == p.n_frames - 1);
+    if (s_last) p.plane_counter[plane] = 0;            // ready for the next launch
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const long long frames_total = p.first_frame + p.n_frames;
+  const long long first_seg = p.first_frame / p.fseg, last_seg = (frames_total - 1) / p.fseg;
+  for (long long u = first_seg; u <= last_seg; ++u) {
+    const long long t0 = u * p.fseg;
+    long long t1 = t0 + p.fseg;
+    if (t1 > frames_total) t1 = frames_total;
+    const int nf = (int)(t1 - t0);
+    for (int col = tid; col < C; col += kCompactThreads) {
+      float m;
+      if (exact) {
+        double t = 0.0;
+        for (long long ff = t0; ff < t1; ++ff) t += __ldcg(p.frame_ksum + ff * C + col);
+        m = (float)(t / ((double)nf * (double)kappa));
+        p.seg_key[u * C + col] = m;
+      } else {
+        float t = 0.f;
+        for (long long ff = t0; ff < t1; ++ff) t += __ldcg(p.frame_entry + ((ff * p.L + l) * 2 + kv) * C + col);
+        m = t / (float)nf;
+      }
+      p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = m;
     }
-    p.seg_entry[((u * p.L + l) * 2 + kv) * p.C + col] = m;
   }
 }
 

@@ -36,7 +36,7 @@ struct StoreLayout {
 };
 
 struct WorkLayout {
-  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, stat_refined, dev_status;
+  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, stat_refined, dev_status, plane_counter;
   size_t q64, qnorm, s_frm, s_seg, wtab, total;
   size_t zero_begin, zero_end;          // region that must start as zeros
 };
@@ -196,6 +196,7 @@ WorkLayout work_layout(const mukv_config& c) {
   w.n_flagged = off;      off = align_up(off + sizeof(int));
   w.stat_refined = off;   off = align_up(off + sizeof(long long));
   w.dev_status = off;     off = align_up(off + sizeof(int));
+  w.plane_counter = off;  off = align_up(off + (size_t)c.n_layers * 2 * sizeof(int));
   w.zero_end = off;
   w.q64 = off;            off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * C * sizeof(double));
   w.qnorm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * sizeof(double));
@@ -413,6 +414,10 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   cp.frame_ksum = reinterpret_cast<double*>(ctx->store + ctx->sl.frame_ksum);
   cp.n_flagged = sp.n_flagged;
   cp.stat_refined = reinterpret_cast<long long*>(ctx->ws + ctx->wl.stat_refined);
+  cp.fseg = c.frames_per_segment;
+  cp.plane_counter = reinterpret_cast<int*>(ctx->ws + ctx->wl.plane_counter);
+  cp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
+  cp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
   {
     ProfScope ps(ctx, 2, st);
     compact_kernel<T><<<dim3(L * 2, n), kCompactThreads, 0, st>>>(cp);
@@ -420,22 +425,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "compact kernel: %s", cudaGetErrorString(e));
 
-  SegmentParams gp;
-  gp.L = L; gp.C = C; gp.kappa = c.keep_per_frame; gp.fseg = c.frames_per_segment;
-  gp.first_seg = t0 / c.frames_per_segment;
-  gp.frames_total = t0 + n;
-  gp.frame_entry = cp.frame_entry;
-  gp.frame_ksum = cp.frame_ksum;
-  gp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
-  gp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
-  const long long last_seg = (t0 + n - 1) / c.frames_per_segment;
-  {
-    ProfScope ps(ctx, 3, st);
-    segment_kernel<<<dim3(L * 2, (unsigned)(last_seg - gp.first_seg + 1)), 256, 0, st>>>(gp);
-  }
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "segment kernel: %s", cudaGetErrorString(e));
-  ctx->launches += 4;
+  ctx->launches += 3;
   ctx->frames = t0 + n;
   return MUKV_OK;
 }

@@ -118,7 +118,7 @@ __device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c
   select_frame<1, PsEpiGroup>(sp, f, att, fft, s_sc, s_int, s_misc);
 }
 
-__global__ void __maxnreg__(192) score_ps_kernel(const ScorePsParams p,
+__global__ void __maxnreg__(184) score_ps_kernel(const ScorePsParams p,
                                                                  const __grid_constant__ CUtensorMap qmap,
                                                                  const __grid_constant__ CUtensorMap kmap,
                                                                  const __grid_constant__ CUtensorMap wmap) {
