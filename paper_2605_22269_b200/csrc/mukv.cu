@@ -490,8 +490,7 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
     if (e == cudaSuccess) e = set_score_attr<float, double>(ctx->nc, score_smem_bytes<float, double>(P, D));
   }
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute((const void*)scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)(kScanRows * (ctx->C + 1) * sizeof(float)));
+    e = cudaFuncSetAttribute((const void*)rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRankStageBytes);
   if (e == cudaSuccess && ctx->tcs.ok) {
     const std::vector<uint16_t> w = dft_terms(D);
     e = cudaMemcpy(ctx->ws + ctx->wl.wtab, w.data(), w.size() * 2, cudaMemcpyHostToDevice);
@@ -623,10 +622,10 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
     {
       ProfScope ps(ctx, 4, st);
       if (c.dtype == MUKV_BF16)
-        qpool_kernel<__nv_bfloat16><<<nq, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(d_qtok), meta,
+        qpool_kernel<__nv_bfloat16><<<nq, kPoolThreads, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(d_qtok), meta,
                                                        c.n_q_heads, c.n_kv_heads, c.head_dim, q64, qnorm);
       else
-        qpool_kernel<float><<<nq, 256, 0, st>>>(reinterpret_cast<const float*>(d_qtok), meta, c.n_q_heads,
+        qpool_kernel<float><<<nq, kPoolThreads, 0, st>>>(reinterpret_cast<const float*>(d_qtok), meta, c.n_q_heads,
                                                c.n_kv_heads, c.head_dim, q64, qnorm);
     }
     cudaError_t e = cudaGetLastError();
@@ -635,7 +634,7 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
     const unsigned blocks = (unsigned)((rows + kScanRows - 1) / kScanRows);
     {
       ProfScope ps(ctx, 5, st);
-      scan_kernel<<<blocks, 256, kScanRows * (C + 1) * sizeof(float), st>>>(frame_key, seg_key, n_frm, n_seg, C, nq,
+      scan_kernel<<<blocks, 256, 0, st>>>(frame_key, seg_key, n_frm, n_seg, C, nq,
                                                                            q64, qnorm, s_frm, s_seg, c.max_frames,
                                                                            ctx->sl.max_segs);
     }
@@ -653,7 +652,11 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
     rp.counts = d_counts;
     {
       ProfScope ps(ctx, 6, st);
-      rank_kernel<<<nq, kRankThreads, C * sizeof(double), st>>>(rp, meta);
+      size_t rank_smem = (size_t)C * sizeof(double);
+      const size_t staged = rank_smem + (size_t)(n_frm + n_seg) * sizeof(double);
+      rp.stage = staged <= (size_t)kRankStageBytes ? 1 : 0;
+      if (rp.stage) rank_smem = staged;
+      rank_kernel<<<nq, kRankThreads, rank_smem, st>>>(rp, meta);
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "rank kernel: %s", cudaGetErrorString(e));

@@ -5,7 +5,8 @@
 // questions, tiny next to the gather, and it makes the selected indices independent of
 // summation order.  Kernels:
 //   qpool_kernel    Eq. 6   one block per question
-//   scan_kernel     Eq. 7   cosine of every question with every frame key and segment key
+//   scan_kernel     Eq. 7   cosine of every question with every frame key and segment key (a skinny
+//                           double-precision product, tiled through shared memory)
 //   rank_kernel     stage-1 candidates, Eq. 8 rerank, final top-k; one block per question
 //   gather_kernel   Eq. 9   copies the selected pages into the per-question decode buffers
 #pragma once
@@ -19,23 +20,45 @@ struct QMeta {
 };
 
 // ------------------------------------------------------------------------------ Eq. 6
+// One block per question.  The question's tokens are dealt to kPoolSlices groups of threads so that
+// many loads are in flight; the slices are added in a fixed order.  The pooled query is written
+// transposed, q64t[c][question] (row stride MUKV_MAX_QUESTIONS), the layout scan_kernel stages.
+constexpr int kPoolThreads = 1024;
+constexpr int kPoolSmemDoubles = 5632;
+
 template <typename T>
-__global__ void __launch_bounds__(256) qpool_kernel(const T* __restrict__ qtok, const QMeta meta, int Hq, int Hkv,
-                                                    int D, double* __restrict__ q64, double* __restrict__ qnorm) {
-  __shared__ double s_part[8];
+__global__ void __launch_bounds__(kPoolThreads) qpool_kernel(const T* __restrict__ qtok, const QMeta meta, int Hq,
+                                                             int Hkv, int D, double* __restrict__ q64t,
+                                                             double* __restrict__ qnorm) {
+  __shared__ double s_acc[kPoolSmemDoubles];
+  __shared__ double s_part[kPoolThreads / 32];
   const int qi = blockIdx.x;
   const int C = Hkv * D, G = Hq / Hkv;
   const int n0 = meta.off[qi], n1 = meta.off[qi + 1];
-  double sq = 0.0;
-  for (int col = threadIdx.x; col < C; col += blockDim.x) {
+  int nsl = kPoolSmemDoubles / C;
+  nsl = nsl > 4 ? 4 : (nsl < 1 ? 1 : nsl);
+  for (int idx = threadIdx.x; idx < nsl * C; idx += kPoolThreads) {
+    const int sl = idx / C, col = idx % C;
     const int g = col / D, d = col % D;
-    double t = 0.0;
-    for (int n = n0; n < n1; ++n) {
+    double t0 = 0.0, t1 = 0.0;
+    for (int n = n0 + sl; n < n1; n += nsl) {
       const T* row = qtok + ((long long)n * Hq + (long long)g * G) * D + d;
-      for (int j = 0; j < G; ++j) t += (double)elem_to_float<T>(row[(long long)j * D]);
+      int j = 0;
+      for (; j + 1 < G; j += 2) {
+        t0 += (double)elem_to_float<T>(row[(long long)j * D]);
+        t1 += (double)elem_to_float<T>(row[(long long)(j + 1) * D]);
+      }
+      if (j < G) t0 += (double)elem_to_float<T>(row[(long long)j * D]);
     }
+    s_acc[idx] = t0 + t1;
+  }
+  __syncthreads();
+  double sq = 0.0;
+  for (int col = threadIdx.x; col < C; col += kPoolThreads) {
+    double t = 0.0;
+    for (int sl = 0; sl < nsl; ++sl) t += s_acc[sl * C + col];
     t = t / (double)((long long)(n1 - n0) * G);
-    q64[(long long)qi * C + col] = t;
+    q64t[(long long)col * MUKV_MAX_QUESTIONS + qi] = t;
     sq += t * t;
   }
   sq = warp_sum(sq);
@@ -43,70 +66,92 @@ __global__ void __launch_bounds__(256) qpool_kernel(const T* __restrict__ qtok, 
   __syncthreads();
   if (threadIdx.x == 0) {
     double t = 0.0;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += s_part[w];
+    for (int w = 0; w < kPoolThreads / 32; ++w) t += s_part[w];
     qnorm[qi] = sqrt(t);
   }
 }
 
 // ------------------------------------------------------------------------------ Eq. 7
-// Rows 0..n_frm-1 are frame keys, rows n_frm..n_frm+n_seg-1 segment keys.  A block stages
-// kScanRows rows in shared memory; thread (warp w, lane r) owns row r and the questions
-// w, w+8, ...: the row value is converted once and reused for kScanQ questions.
+// Rows 0..n_frm-1 are frame keys, rows n_frm..n_frm+n_seg-1 segment keys.  A block owns
+// kScanRows rows and walks the feature axis in chunks of kScanCC: the rows' chunk (float) and the
+// chunk of up to kScanQB pooled queries (double) are staged in shared memory, thread
+// (row pair, question quad) keeps a 2 x 4 tile of double dot products.
 constexpr int kScanRows = 32;
-constexpr int kScanQ = 4;
+constexpr int kScanCC = 64;
+constexpr int kScanQB = 64;
 
 __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ frame_key,
                                                    const float* __restrict__ seg_key, long long n_frm,
-                                                   long long n_seg, int C, int nq, const double* __restrict__ q64,
+                                                   long long n_seg, int C, int nq, const double* __restrict__ q64t,
                                                    const double* __restrict__ qnorm, double* __restrict__ s_frm,
                                                    double* __restrict__ s_seg, long long frm_stride,
                                                    long long seg_stride) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* rows = reinterpret_cast<float*>(smem_raw);                 // [kScanRows][C+1]
-  const int CS = C + 1;
+  __shared__ float rows[kScanRows][kScanCC + 1];
+  __shared__ __align__(16) double qs[kScanCC][kScanQB];
+  __shared__ double s_knorm[kScanRows];
+  const int tid = threadIdx.x;
   const long long row0 = (long long)blockIdx.x * kScanRows;
   const long long n_rows = n_frm + n_seg;
-  for (int v = threadIdx.x; v < kScanRows * C; v += blockDim.x) {
-    const int r = v / C, c = v % C;
-    const long long row = row0 + r;
-    float x = 0.f;
-    if (row < n_frm) x = frame_key[row * C + c];
-    else if (row < n_rows) x = seg_key[(row - n_frm) * C + c];
-    rows[r * CS + c] = x;
-  }
-  __syncthreads();
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const long long row = row0 + lane;
-  const float* mine = rows + lane * CS;
-  double kk = 0.0;
-  for (int c = 0; c < C; ++c) {
-    const double x = (double)mine[c];
-    kk = fma(x, x, kk);
-  }
-  const double knorm = sqrt(kk);
-  for (int qb = warp * kScanQ; qb < nq; qb += 8 * kScanQ) {
-    double acc[kScanQ];
+  const int lr = tid >> 3, lc = (tid & 7) * 8;               // staging: row, first column of 8
+  const long long my_row = row0 + lr;
+  const float* src = my_row < n_frm ? frame_key + my_row * C
+                                    : (my_row < n_rows ? seg_key + (my_row - n_frm) * C : nullptr);
+  const int rp = tid >> 4, qd = tid & 15;                    // compute: rows rp, rp+16; questions 4qd..4qd+3
+  for (int qb = 0; qb < nq; qb += kScanQB) {
+    double acc[2][4];
 #pragma unroll
-    for (int i = 0; i < kScanQ; ++i) acc[i] = 0.0;
-    for (int c = 0; c < C; ++c) {
-      const double x = (double)mine[c];
+    for (int i = 0; i < 2; ++i)
 #pragma unroll
-      for (int i = 0; i < kScanQ; ++i) {
-        const int qi = min(qb + i, nq - 1);
-        acc[i] = fma(x, __ldg(q64 + (long long)qi * C + c), acc[i]);
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+    double kk = 0.0;
+    for (int c0 = 0; c0 < C; c0 += kScanCC) {
+      __syncthreads();                                       // the previous chunk has been consumed
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int cc = lc + i;
+        const float x = (src && c0 + cc < C) ? src[c0 + cc] : 0.f;
+        rows[lr][cc] = x;
+        kk = fma((double)x, (double)x, kk);
+      }
+      for (int idx = tid; idx < kScanCC * kScanQB; idx += 256) {
+        const int cc = idx / kScanQB, qq = idx % kScanQB;
+        qs[cc][qq] = (c0 + cc < C && qb + qq < nq) ? q64t[(long long)(c0 + cc) * MUKV_MAX_QUESTIONS + qb + qq] : 0.0;
+      }
+      __syncthreads();
+#pragma unroll 8
+      for (int cc = 0; cc < kScanCC; ++cc) {
+        const double a0 = (double)rows[rp][cc], a1 = (double)rows[rp + 16][cc];
+        const double2 q01 = *reinterpret_cast<const double2*>(&qs[cc][4 * qd]);
+        const double2 q23 = *reinterpret_cast<const double2*>(&qs[cc][4 * qd + 2]);
+        acc[0][0] = fma(a0, q01.x, acc[0][0]); acc[0][1] = fma(a0, q01.y, acc[0][1]);
+        acc[0][2] = fma(a0, q23.x, acc[0][2]); acc[0][3] = fma(a0, q23.y, acc[0][3]);
+        acc[1][0] = fma(a1, q01.x, acc[1][0]); acc[1][1] = fma(a1, q01.y, acc[1][1]);
+        acc[1][2] = fma(a1, q23.x, acc[1][2]); acc[1][3] = fma(a1, q23.y, acc[1][3]);
       }
     }
-    if (row < n_rows) {
+    if (qb == 0) {
+      // the 8 staging threads of a row hold the parts of its squared norm
+      kk += __shfl_xor_sync(kFull, kk, 1);
+      kk += __shfl_xor_sync(kFull, kk, 2);
+      kk += __shfl_xor_sync(kFull, kk, 4);
+      if ((tid & 7) == 0) s_knorm[lr] = sqrt(kk);
+    }
+    __syncthreads();
 #pragma unroll
-      for (int i = 0; i < kScanQ; ++i) {
-        const int qi = qb + i;
-        if (qi < nq) {
-          double den = knorm * qnorm[qi];
-          den = den > 1e-12 ? den : 1e-12;
-          const double s = acc[i] / den;
-          if (row < n_frm) s_frm[(long long)qi * frm_stride + row] = s;
-          else s_seg[(long long)qi * seg_stride + (row - n_frm)] = s;
-        }
+    for (int i = 0; i < 2; ++i) {
+      const int r = rp + 16 * i;
+      const long long row = row0 + r;
+      if (row >= n_rows) continue;
+      const double knorm = s_knorm[r];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int qi = qb + 4 * qd + j;
+        if (qi >= nq) continue;
+        double den = knorm * qnorm[qi];
+        den = den > 1e-12 ? den : 1e-12;
+        const double sc = acc[i][j] / den;
+        if (row < n_frm) s_frm[(long long)qi * frm_stride + row] = sc;
+        else s_seg[(long long)qi * seg_stride + (row - n_frm)] = sc;
       }
     }
   }
@@ -236,9 +281,11 @@ struct RankParams {
   const float* frame_key;
   const float* seg_key;
   int* seg_idx; int* frm_idx; float* seg_score; float* frm_score; int* counts;
+  int stage;                              // 1: the question's scores are copied to shared memory first
 };
 
 constexpr int kRankThreads = 512;
+constexpr int kRankStageBytes = 192 * 1024;       // dynamic shared memory the kernel may be given
 constexpr int kMaxCand = 2 * MUKV_MAX_TOPK;
 
 __global__ void __launch_bounds__(kRankThreads) rank_kernel(const RankParams p, const QMeta meta) {
@@ -267,6 +314,16 @@ __global__ void __launch_bounds__(kRankThreads) rank_kernel(const RankParams p, 
   if (n_seg > p.n_seg) n_seg = (int)p.n_seg;
   const double* sf = p.s_frm + (long long)qi * p.frm_stride;
   const double* ss = p.s_seg + (long long)qi * p.seg_stride;
+  if (p.stage) {
+    // every selection below scans the scores several times: do that out of shared memory
+    double* st_f = gq + C;
+    double* st_s = st_f + n_frm;
+    for (int i = tid; i < n_frm; i += kRankThreads) st_f[i] = sf[i];
+    for (int i = tid; i < n_seg; i += kRankThreads) st_s[i] = ss[i];
+    __syncthreads();
+    sf = st_f;
+    ss = st_s;
+  }
   auto seg_score = [&](int i) { return ss[i]; };
   auto frm_score = [&](int i) { return sf[i]; };
   auto always = [](int) { return true; };
