@@ -172,7 +172,7 @@ TcShape tc_shape(const mukv_config& c) {
   t.smem = score_tc_smem_bytes(c.tokens_per_frame, c.head_dim);
   t.smem_ps = score_ps_smem_bytes(c.tokens_per_frame, c.head_dim);
   t.ok = t.smem <= 227 * 1024;
-  t.persistent = t.ok && t.smem_ps <= 227 * 1024;
+  t.persistent = t.ok && t.smem_ps <= 227 * 1024 && t.npad <= 2 * kPsAccCols;
   return t;
 }
 

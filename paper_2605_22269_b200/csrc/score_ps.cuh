@@ -33,6 +33,9 @@ constexpr int kPsEpiThreads = 256;
 constexpr int kPsEpiOff = 64;              // first epilogue thread
 constexpr int kPsMiscBytes = 8192;
 constexpr int kPsMaxBlocks = 256;          // bound on the grid (slots of partial sums)
+constexpr int kPsAccCols = 112;            // accumulator columns per epilogue thread: P <= 2 * 112
+// Ten warps put three on one scheduler, whose 16 K registers then allow 168 per thread: the column
+// accumulators, two 16-column chunks in flight and the addressing have to fit in that.
 typedef NamedGroup<5, kPsEpiThreads, kPsEpiOff> PsEpiGroup;
 
 struct ScorePsParams {
@@ -118,7 +121,7 @@ __device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c
   select_frame<1, PsEpiGroup>(sp, f, att, fft, s_sc, s_int, s_misc);
 }
 
-__global__ void __maxnreg__(184) score_ps_kernel(const ScorePsParams p,
+__global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
                                                                  const __grid_constant__ CUtensorMap qmap,
                                                                  const __grid_constant__ CUtensorMap kmap,
                                                                  const __grid_constant__ CUtensorMap wmap) {
@@ -288,9 +291,9 @@ __global__ void __maxnreg__(184) score_ps_kernel(const ScorePsParams p,
     const int my_c0 = h ? nch0 : 0, my_nch = h ? nch16 - nch0 : nch0;
     const bool causal = sp.causal != 0;
     const float c = p.exp2_scale;
-    float acc[128];
+    float acc[kPsAccCols];                               // column sums of this thread's row, over tiles
 #pragma unroll
-    for (int k = 0; k < 128; ++k) acc[k] = 0.f;
+    for (int k = 0; k < kPsAccCols; ++k) acc[k] = 0.f;
     bool ok = true;
     int it = 0;
     for (int i = i0; i < i1; ++i, ++it) {
@@ -378,29 +381,17 @@ __global__ void __maxnreg__(184) score_ps_kernel(const ScorePsParams p,
         const bool all_valid = __all_sync(kFull, valid);
         // pass C: acc[column] += e / sum
 #pragma unroll
-        for (int pp = 0; pp < 4; ++pp) {
-          const int n_in = my_nch - 2 * pp;
-          if (n_in > 0) {
-            uint32_t r0[16], r1[16];
-            const int col = (my_c0 + 2 * pp) * 16;
-            tc::tmem_ld16(tb + col, r0);
-            if (n_in >= 2) {
-              tc::tmem_ld16(tb + col + 16, r1);
-              tc::tmem_wait_ld16x2(r0, r1);
-            } else {
-              tc::tmem_wait_ld16(r0);
-#pragma unroll
-              for (int k = 0; k < 16; ++k) r1[k] = 0u;
-            }
+        for (int ch = 0; ch < kPsAccCols / 16; ++ch) {
+          if (ch < my_nch) {
+            uint32_t r0[16];
+            tc::tmem_ld16(tb + (my_c0 + ch) * 16, r0);
+            tc::tmem_wait_ld16(r0);
             if (!all_valid && !valid) {
 #pragma unroll
-              for (int k = 0; k < 16; ++k) { r0[k] = 0u; r1[k] = 0u; }
+              for (int k = 0; k < 16; ++k) r0[k] = 0u;
             }
 #pragma unroll
-            for (int k = 0; k < 16; ++k) {
-              acc[pp * 32 + k] = fmaf(__uint_as_float(r0[k]), inv, acc[pp * 32 + k]);
-              acc[pp * 32 + 16 + k] = fmaf(__uint_as_float(r1[k]), inv, acc[pp * 32 + 16 + k]);
-            }
+            for (int k = 0; k < 16; ++k) acc[ch * 16 + k] = fmaf(__uint_as_float(r0[k]), inv, acc[ch * 16 + k]);
           }
         }
       }
@@ -412,10 +403,13 @@ __global__ void __maxnreg__(184) score_ps_kernel(const ScorePsParams p,
       if (i + 1 == i1 || (i + 1) / ipf != f) {
         // ---- leaving frame f: publish this block's column sums, the last block selects
 #pragma unroll
-        for (int pp = 0; pp < 4; ++pp) {
+        for (int pp = 0; pp < (kPsAccCols + 31) / 32; ++pp) {
           float v[32];
 #pragma unroll
-          for (int k = 0; k < 32; ++k) { v[k] = acc[pp * 32 + k]; acc[pp * 32 + k] = 0.f; }
+          for (int k = 0; k < 32; ++k) {
+            if (pp * 32 + k < kPsAccCols) { v[k] = acc[pp * 32 + k]; acc[pp * 32 + k] = 0.f; }
+            else v[k] = 0.f;
+          }
           const float s = warp_column_sums(v, lane);
           if (2 * pp + (lane >> 4) < my_nch) s_col[q * 256 + (my_c0 + 2 * pp) * 16 + lane] = s;
         }
