@@ -145,14 +145,28 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
     const int nf = (int)(t1 - t0);
     for (int col = tid; col < C; col += kCompactThreads) {
       float m;
+      // eight loads in flight at a time, added in frame order
       if (exact) {
         double t = 0.0;
-        for (long long ff = t0; ff < t1; ++ff) t += __ldcg(p.frame_ksum + ff * C + col);
+        for (long long ff = t0; ff < t1; ff += 8) {
+          double x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[i] = ff + i < t1 ? __ldcg(p.frame_ksum + (ff + i) * C + col) : 0.0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) t += x[i];
+        }
         m = (float)(t / ((double)nf * (double)kappa));
         p.seg_key[u * C + col] = m;
       } else {
         float t = 0.f;
-        for (long long ff = t0; ff < t1; ++ff) t += __ldcg(p.frame_entry + ((ff * p.L + l) * 2 + kv) * C + col);
+        for (long long ff = t0; ff < t1; ff += 8) {
+          float x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            x[i] = ff + i < t1 ? __ldcg(p.frame_entry + (((ff + i) * p.L + l) * 2 + kv) * C + col) : 0.f;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) t += x[i];
+        }
         m = t / (float)nf;
       }
       p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = m;

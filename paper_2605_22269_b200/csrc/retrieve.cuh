@@ -213,16 +213,29 @@ __device__ int block_topk_set(ScoreFn score, MemberFn member, int n, int k, doub
         if ((key & himask) == prefix) atomicAdd(&sc->hist[(unsigned)(key >> shift) & 255u], 1u);
       }
       __syncthreads();
-      if (tid == 0) {
-        int rem = sc->remaining;
-        int b = 255;
-        for (; b > 0; --b) {
-          const int c = (int)sc->hist[b];
-          if (rem <= c) break;
-          rem -= c;
+      if (tid < 32) {
+        // warp 0 finds the bin that holds the remaining-th largest key: lane l owns bins 8l .. 8l+7
+        int c[8], T = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { c[i] = (int)sc->hist[8 * tid + i]; T += c[i]; }
+        int incl = T;                                   // keys in this lane's bins and all higher ones
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_down_sync(kFull, incl, o);
+          if (tid + o < 32) incl += v;
         }
-        sc->prefix = prefix | ((unsigned long long)b << shift);
-        sc->remaining = rem;
+        const int above = incl - T;
+        const int rem = sc->remaining;
+        __syncwarp();
+        if (above < rem && rem <= above + T) {          // true for exactly one lane
+          int r = rem - above, b = 7;
+          for (; b > 0; --b) {
+            if (r <= c[b]) break;
+            r -= c[b];
+          }
+          sc->prefix = prefix | ((unsigned long long)(8 * tid + b) << shift);
+          sc->remaining = r;
+        }
       }
       __syncthreads();
     }
