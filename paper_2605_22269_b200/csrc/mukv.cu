@@ -45,7 +45,7 @@ struct WorkLayout {
 struct TcShape {
   bool ok;                 // bf16 chunk scored on the tensor cores
   bool persistent;         // by the persistent kernel (its operand buffers fit in shared memory)
-  int tpt, tiles, npad, n_mt, tmem_cols;
+  int tpt, tiles, npad, n_mt, tmem_cols, ps_stages;
   size_t smem, smem_ps;
 };
 
@@ -170,9 +170,10 @@ TcShape tc_shape(const mukv_config& c) {
   t.tmem_cols = 32;
   while (t.tmem_cols < need) t.tmem_cols *= 2;
   t.smem = score_tc_smem_bytes(c.tokens_per_frame, c.head_dim);
-  t.smem_ps = score_ps_smem_bytes(c.tokens_per_frame, c.head_dim);
+  t.ps_stages = score_ps_stages(c.tokens_per_frame, c.head_dim, 227 * 1024);
+  t.smem_ps = score_ps_smem_bytes(c.tokens_per_frame, c.head_dim, t.ps_stages < 2 ? 2 : t.ps_stages);
   t.ok = t.smem <= 227 * 1024;
-  t.persistent = t.ok && t.smem_ps <= 227 * 1024 && t.npad <= 2 * kPsAccCols;
+  t.persistent = t.ok && t.ps_stages >= 2 && t.npad <= 2 * kPsAccCols;
   return t;
 }
 
@@ -331,7 +332,7 @@ cudaError_t launch_score_tc(mukv_ctx* ctx, const ScoreParams& sp, const void* d_
     memset(&pp, 0, sizeof pp);
     pp.sp = sp;
     pp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
-    pp.tiles = t.tiles; pp.tpt = t.tpt; pp.npad = t.npad; pp.n_mt = t.n_mt;
+    pp.tiles = t.tiles; pp.tpt = t.tpt; pp.npad = t.npad; pp.n_mt = t.n_mt; pp.n_stages = t.ps_stages;
     pp.n_items = n * c.n_kv_heads * (t.n_mt + t.tiles);
     pp.exp2_scale = (float)(1.4426950408889634 / std::sqrt((double)D));
     pp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);

@@ -5,16 +5,20 @@
 // row tiles (Eq. 1; the G query heads of the group are flattened with the tokens into rows, as
 // in score_tc_kernel).  Each block takes a contiguous share of the list.
 //
-//   warp 0      TMA producer: the three bf16 terms of the DFT matrix once, the key tile K_g of a
-//               (frame, head) when the head changes, a Q row tile per attention item (2 stages).
+//   warp 0      TMA producer.  The key tile K_g of a (frame, head) goes to one of two buffers when
+//               the head changes; everything else streams through a ring of 32 KB operand stages:
+//               one Q row tile per attention item, the three bf16 terms of the DFT matrix (read
+//               from L2) per DFT item.
 //   warp 1      issues tcgen05.mma into one of two 256-column accumulators in tensor memory and
-//               commits to the barriers that free the operand buffers.
+//               commits to the barriers that free the stages and the key buffers.
 //   warps 2-9   epilogue.  Two warps share each 32-lane quarter of the accumulator and split its
-//               columns.  Attention item: row maximum, exp and row sum (both exchanged between the
-//               two warps through shared memory), then acc[column] += e / sum in registers.  The
-//               32 rows of a warp are added only when the block leaves a frame (shuffle butterfly),
-//               so the per-tile cost is one fused multiply-add per logit.  DFT item: magnitudes of
-//               the D bins of each key vector, summed.
+//               columns.  Attention item: one sweep takes a running row maximum, writes
+//               exp(z - running max) back into tensor memory and keeps the row sum (rescaled when
+//               the maximum grows); the two warps of a row exchange (max, sum) through shared
+//               memory; a second sweep adds e * 2^(ref - max) / sum to per-column accumulators in
+//               registers.  The 32 rows of a warp are added only when the block leaves a frame
+//               (shuffle butterfly), so the per-tile cost is one fused multiply-add per logit.
+//               DFT item: magnitudes of the D bins of each key vector, summed.
 //
 // Per frame, every block that worked on it stores its column sums in a slot of its own; the
 // block that arrives last (counter, nobody waits) adds the slots in a fixed order, applies
@@ -41,14 +45,22 @@ typedef NamedGroup<5, kPsEpiThreads, kPsEpiOff> PsEpiGroup;
 struct ScorePsParams {
   ScoreParams sp;            // colsum_part: float [grid + n_frames][P] slots, ifft_part: float [F][Hkv][P]
   int tiles, tpt, npad, n_mt;
+  int n_stages;              // operand stages in the ring (2 .. kPsMaxStages)
   int n_items;               // n_frames * Hkv * (n_mt + tiles)
   float exp2_scale;          // log2(e) / sqrt(D)
   int* status;
 };
 
-__host__ inline size_t score_ps_smem_bytes(int P, int D) {
+constexpr int kPsMaxStages = 6;
+// two key buffers + n_stages operand stages + scratch (+ slack to align the tiles to 1024 bytes)
+__host__ inline size_t score_ps_smem_bytes(int P, int D, int n_stages) {
   const size_t KB = D / 64, npad = (P + 15) / 16 * 16;
-  return KB * npad * 128 + 2 * KB * 128 * 128 + 3 * KB * (size_t)D * 128 + kPsMiscBytes + 1024;
+  return 2 * KB * npad * 128 + (size_t)n_stages * KB * 128 * 128 + kPsMiscBytes + 1024;
+}
+__host__ inline int score_ps_stages(int P, int D, size_t limit) {
+  int n = kPsMaxStages;
+  while (n >= 2 && score_ps_smem_bytes(P, D, n) > limit) --n;
+  return n;                  // < 2: the kernel does not fit
 }
 
 // owner of item i when n items are split into contiguous shares [c*n/nb, (c+1)*n/nb)
@@ -122,9 +134,9 @@ __device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c
 }
 
 __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
-                                                                 const __grid_constant__ CUtensorMap qmap,
-                                                                 const __grid_constant__ CUtensorMap kmap,
-                                                                 const __grid_constant__ CUtensorMap wmap) {
+                                                 const __grid_constant__ CUtensorMap qmap,
+                                                 const __grid_constant__ CUtensorMap kmap,
+                                                 const __grid_constant__ CUtensorMap wmap) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = tc::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -132,6 +144,7 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const ScoreParams& sp = p.sp;
   const int P = sp.P, D = sp.D, G = sp.G, Hkv = sp.Hkv, KB = D >> 6;
+  const int NS = p.n_stages;
   const int ipu = p.n_mt + p.tiles;                      // items per (frame, key head)
   const int ipf = Hkv * ipu;                             // items per frame
   const int n_cta = gridDim.x, cta = blockIdx.x;
@@ -139,34 +152,36 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
   const int i1 = (int)((long long)(cta + 1) * p.n_items / n_cta);
   const int rows_q = p.tpt * G;
 
-  const uint32_t k_kb = (uint32_t)p.npad * 128u, q_kb = 128u * 128u, w_kb = (uint32_t)D * 128u;
-  const uint32_t sK = base;
-  const uint32_t sQ = sK + (uint32_t)KB * k_kb;
-  const uint32_t sW = sQ + 2u * KB * q_kb;
-  const uint32_t misc_off = (uint32_t)KB * k_kb + 2u * KB * q_kb + 3u * KB * w_kb;
+  const uint32_t k_kb = (uint32_t)p.npad * 128u, st_kb = 128u * 128u;
+  const uint32_t k_buf = (uint32_t)KB * k_kb, st_buf = (uint32_t)KB * st_kb;
+  const uint32_t sK = base;                              // two key buffers
+  const uint32_t sS = sK + 2u * k_buf;                   // NS operand stages
+  const uint32_t misc_off = 2u * k_buf + (uint32_t)NS * st_buf;
   float* s_col = reinterpret_cast<float*>(sm + misc_off);                     // [4][256]
   float* s_mx = reinterpret_cast<float*>(sm + misc_off + 4096);               // [2][128]
   float* s_sum = s_mx + 256;                                                  // [2][128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + misc_off + 6144);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + misc_off + 6144 + 96);
-  int* s_flag = reinterpret_cast<int*>(sm + misc_off + 6144 + 100);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + misc_off + 6144 + 192);
+  int* s_flag = reinterpret_cast<int*>(sm + misc_off + 6144 + 196);
   const uint32_t b0 = tc::smem_u32(bars);
-  const uint32_t bar_w = b0, bar_kf = b0 + 8, bar_ke = b0 + 16;
-  // stage / buffer s of: Q full, Q empty, accumulator full, accumulator empty
-#define PS_BAR_QF(s) (b0 + 24u + 8u * (uint32_t)(s))
-#define PS_BAR_QE(s) (b0 + 40u + 8u * (uint32_t)(s))
-#define PS_BAR_AF(s) (b0 + 56u + 8u * (uint32_t)(s))
-#define PS_BAR_AE(s) (b0 + 72u + 8u * (uint32_t)(s))
+  // key buffer full / empty, accumulator full / empty (2 each), stage full / empty (kPsMaxStages each)
+#define PS_BAR_KF(s) (b0 + 8u * (uint32_t)(s))
+#define PS_BAR_KE(s) (b0 + 16u + 8u * (uint32_t)(s))
+#define PS_BAR_AF(s) (b0 + 32u + 8u * (uint32_t)(s))
+#define PS_BAR_AE(s) (b0 + 48u + 8u * (uint32_t)(s))
+#define PS_BAR_SF(s) (b0 + 64u + 8u * (uint32_t)(s))
+#define PS_BAR_SE(s) (b0 + 64u + 8u * (uint32_t)kPsMaxStages + 8u * (uint32_t)(s))
 
   if (tid == 0) {
-    tc::mbar_init(bar_w, 1);
-    tc::mbar_init(bar_kf, 1);
-    tc::mbar_init(bar_ke, 1);
     for (int s = 0; s < 2; ++s) {
-      tc::mbar_init(PS_BAR_QF(s), 1);
-      tc::mbar_init(PS_BAR_QE(s), 1);
+      tc::mbar_init(PS_BAR_KF(s), 1);
+      tc::mbar_init(PS_BAR_KE(s), 1);
       tc::mbar_init(PS_BAR_AF(s), 1);
       tc::mbar_init(PS_BAR_AE(s), 8);                    // one arrival per epilogue warp
+    }
+    for (int s = 0; s < kPsMaxStages; ++s) {
+      tc::mbar_init(PS_BAR_SF(s), 1);
+      tc::mbar_init(PS_BAR_SE(s), 1);
     }
     tc::fence_mbar_init();
     tc::prefetch_tmap(&qmap);
@@ -177,13 +192,15 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
     __syncwarp();
     tc::tmem_alloc(tc::smem_u32(tmem_slot), 512u);
   }
-  // rows of the Q stages that the TMA box never writes must not hold stale bits
+  // Rows of a stage that a Q box never writes (rows_q .. 127) are read by the MMA as rows of the
+  // tile; they only produce rows of the product that are never used, but they must be finite.
+  // A DFT term fills all D rows of a stage it uses, so a stage may hold old matrix rows there: finite too.
   {
     const int pad_rows = 128 - rows_q;
-    uint4* q4 = reinterpret_cast<uint4*>(sm + (size_t)KB * k_kb);
-    for (int i = tid; i < 2 * KB * pad_rows * 8; i += kPsThreads) {
+    uint4* s4 = reinterpret_cast<uint4*>(sm + 2u * k_buf);
+    for (int i = tid; i < NS * KB * pad_rows * 8; i += kPsThreads) {
       const int blk = i / (pad_rows * 8), rem = i % (pad_rows * 8);
-      q4[(size_t)blk * (q_kb / 16) + (size_t)rows_q * 8 + rem] = make_uint4(0u, 0u, 0u, 0u);
+      s4[(size_t)blk * (st_kb / 16) + (size_t)rows_q * 8 + rem] = make_uint4(0u, 0u, 0u, 0u);
     }
   }
   tc::fence_proxy_async_smem();
@@ -196,53 +213,59 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
     // ================================================================== TMA producer
     if (lane == 0) {
       bool ok = true;
-      tc::mbar_expect_tx(bar_w, 3u * KB * w_kb);
-      for (int t = 0; t < 3; ++t)
-        for (int kb = 0; kb < KB; ++kb)
-          tc::tma_load_2d(sW + (uint32_t)(t * KB + kb) * w_kb, &wmap, kb * 64, t * D, bar_w);
-      int nk = 0, nq = 0, last_unit = -1;
-      for (int i = i0; i < i1; ++i) {
+      int nk = 0, ns = 0, last_unit = -1;
+      for (int i = i0; i < i1 && ok; ++i) {
         const int unit = i / ipu, x = i % ipu;
         const int f = unit / Hkv, g = unit % Hkv;
         if (unit != last_unit) {
-          ok = tc::mbar_wait(bar_ke, (uint32_t)((nk & 1) ^ 1));
+          const int kb_i = nk & 1;
+          ok = tc::mbar_wait(PS_BAR_KE(kb_i), (uint32_t)(((nk >> 1) & 1) ^ 1));
           if (!ok) break;
-          tc::mbar_expect_tx(bar_kf, (uint32_t)KB * k_kb);
-          for (int kb = 0; kb < KB; ++kb) tc::tma_load_3d(sK + kb * k_kb, &kmap, kb * 64, g, f * P, bar_kf);
+          tc::mbar_expect_tx(PS_BAR_KF(kb_i), k_buf);
+          for (int kb = 0; kb < KB; ++kb)
+            tc::tma_load_3d(sK + (uint32_t)kb_i * k_buf + kb * k_kb, &kmap, kb * 64, g, f * P, PS_BAR_KF(kb_i));
           ++nk;
           last_unit = unit;
         }
-        if (x >= p.n_mt) {
-          const int s = nq & 1;
-          ok = tc::mbar_wait(PS_BAR_QE(s), (uint32_t)(((nq >> 1) & 1) ^ 1));
+        const int n_ld = x < p.n_mt ? 3 : 1;             // DFT item: the three matrix terms, smallest first
+        for (int t = 0; t < n_ld && ok; ++t) {
+          const int s = ns % NS;
+          ok = tc::mbar_wait(PS_BAR_SE(s), (uint32_t)(((ns / NS) & 1) ^ 1));
           if (!ok) break;
-          tc::mbar_expect_tx(PS_BAR_QF(s), (uint32_t)KB * (uint32_t)rows_q * 128u);
-          for (int kb = 0; kb < KB; ++kb)
-            tc::tma_load_3d(sQ + (uint32_t)(s * KB + kb) * q_kb, &qmap, kb * 64, g * G,
-                            f * P + (x - p.n_mt) * p.tpt, PS_BAR_QF(s));
-          ++nq;
+          const uint32_t dst = sS + (uint32_t)s * st_buf;
+          if (x < p.n_mt) {
+            tc::mbar_expect_tx(PS_BAR_SF(s), (uint32_t)KB * (uint32_t)D * 128u);
+            for (int kb = 0; kb < KB; ++kb) tc::tma_load_2d(dst + kb * st_kb, &wmap, kb * 64, (2 - t) * D, PS_BAR_SF(s));
+          } else {
+            tc::mbar_expect_tx(PS_BAR_SF(s), (uint32_t)KB * (uint32_t)rows_q * 128u);
+            for (int kb = 0; kb < KB; ++kb)
+              tc::tma_load_3d(dst + kb * st_kb, &qmap, kb * 64, g * G, f * P + (x - p.n_mt) * p.tpt, PS_BAR_SF(s));
+          }
+          ++ns;
         }
       }
       if (!ok) atomicCAS(p.status, 0, 3);
       // copies of this thread still in flight land before the block goes away
-      tc::mbar_wait(bar_w, 0);
-      if (nk) tc::mbar_wait(bar_kf, (uint32_t)((nk - 1) & 1));
       for (int s = 0; s < 2; ++s) {
-        const int cnt = (nq + 1 - s) >> 1;
-        if (cnt) tc::mbar_wait(PS_BAR_QF(s), (uint32_t)((cnt - 1) & 1));
+        const int cnt = (nk + 1 - s) >> 1;
+        if (cnt) tc::mbar_wait(PS_BAR_KF(s), (uint32_t)((cnt - 1) & 1));
+      }
+      for (int s = 0; s < NS; ++s) {
+        const int cnt = (ns + NS - 1 - s) / NS;
+        if (cnt) tc::mbar_wait(PS_BAR_SF(s), (uint32_t)((cnt - 1) & 1));
       }
     }
   } else if (warp == 1) {
     // ================================================================== MMA issuer
     if (lane == 0) {
-      bool ok = tc::mbar_wait(bar_w, 0);
-      tc::tc_fence_after_sync();
+      bool ok = true;
       const uint32_t idesc_att = tc::idesc_bf16_f32(128, p.npad), idesc_dft = tc::idesc_bf16_f32(128, D);
-      int nk = 0, nq = 0, it = 0, last_unit = -1;
+      int nk = 0, ns = 0, it = 0, last_unit = -1, kb_i = 0;
       for (int i = i0; i < i1 && ok; ++i, ++it) {
         const int unit = i / ipu, x = i % ipu;
         if (unit != last_unit) {
-          ok = tc::mbar_wait(bar_kf, (uint32_t)(nk & 1));
+          kb_i = nk & 1;
+          ok = tc::mbar_wait(PS_BAR_KF(kb_i), (uint32_t)((nk >> 1) & 1));
           if (!ok) break;
           ++nk;
           last_unit = unit;
@@ -252,32 +275,34 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
         if (!ok) break;
         tc::tc_fence_after_sync();
         const uint32_t d_tmem = tmem + (uint32_t)b * 256u;
-        if (x < p.n_mt) {
-          // smallest term first: lo, mid, hi
-          uint32_t accum = 0;
-          for (int t = 2; t >= 0; --t)
-            for (int kb = 0; kb < KB; ++kb)
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                tc::mma_bf16_ss(d_tmem, tc::smem_desc_sw128(sK + kb * k_kb + (uint32_t)x * q_kb + k * 32),
-                                tc::smem_desc_sw128(sW + (uint32_t)(t * KB + kb) * w_kb + k * 32), idesc_dft, accum);
-                accum = 1;
-              }
-        } else {
-          const int s = nq & 1;
-          ok = tc::mbar_wait(PS_BAR_QF(s), (uint32_t)((nq >> 1) & 1));
+        const uint32_t kbase = sK + (uint32_t)kb_i * k_buf;
+        const int n_ld = x < p.n_mt ? 3 : 1;
+        for (int t = 0; t < n_ld && ok; ++t) {
+          const int s = ns % NS;
+          ok = tc::mbar_wait(PS_BAR_SF(s), (uint32_t)((ns / NS) & 1));
           if (!ok) break;
           tc::tc_fence_after_sync();
-          for (int kb = 0; kb < KB; ++kb)
+          const uint32_t sbase = sS + (uint32_t)s * st_buf;
+          if (x < p.n_mt) {
+            // rows x*128 .. of the key tile times one term of the DFT matrix
+            for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              tc::mma_bf16_ss(d_tmem, tc::smem_desc_sw128(sQ + (uint32_t)(s * KB + kb) * q_kb + k * 32),
-                              tc::smem_desc_sw128(sK + kb * k_kb + k * 32), idesc_att, (kb | k) != 0);
-          tc::mma_commit(PS_BAR_QE(s));
-          ++nq;
+              for (int k = 0; k < 4; ++k)
+                tc::mma_bf16_ss(d_tmem, tc::smem_desc_sw128(kbase + kb * k_kb + (uint32_t)x * st_kb + k * 32),
+                                tc::smem_desc_sw128(sbase + kb * st_kb + k * 32), idesc_dft, (t | kb | k) != 0);
+          } else {
+            for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                tc::mma_bf16_ss(d_tmem, tc::smem_desc_sw128(sbase + kb * st_kb + k * 32),
+                                tc::smem_desc_sw128(kbase + kb * k_kb + k * 32), idesc_att, (kb | k) != 0);
+          }
+          tc::mma_commit(PS_BAR_SE(s));
+          ++ns;
         }
+        if (!ok) break;
         tc::mma_commit(PS_BAR_AF(b));
-        if (i + 1 == i1 || (i + 1) / ipu != unit) tc::mma_commit(bar_ke);
+        if (i + 1 == i1 || (i + 1) / ipu != unit) tc::mma_commit(PS_BAR_KE(kb_i));
       }
       if (!ok) atomicCAS(p.status, 0, 4);
     }
@@ -291,6 +316,7 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
     const int my_c0 = h ? nch0 : 0, my_nch = h ? nch16 - nch0 : nch0;
     const bool causal = sp.causal != 0;
     const float c = p.exp2_scale;
+    constexpr int kMaxCh = kPsAccCols / 16;
     float acc[kPsAccCols];                               // column sums of this thread's row, over tiles
 #pragma unroll
     for (int k = 0; k < kPsAccCols; ++k) acc[k] = 0.f;
@@ -333,65 +359,53 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
         const int tile = x - p.n_mt;
         const int i_tok = tile * p.tpt + row / G;
         const bool valid = (row < rows_q) && (i_tok < P);
-        // pass A: row maximum
-        float m = -INFINITY;
-#pragma unroll 1
-        for (int ch = 0; ch < my_nch; ch += 2) {
-          uint32_t r0[16], r1[16];
-          const int col = (my_c0 + ch) * 16;
-          tc::tmem_ld16(tb + col, r0);
-          if (ch + 1 < my_nch) {
-            tc::tmem_ld16(tb + col + 16, r1);
-            tc::tmem_wait_ld16x2(r0, r1);
-            m = fmaxf(m, fmaxf(ps_chunk_max(r0, col, P, causal, i_tok), ps_chunk_max(r1, col + 16, P, causal, i_tok)));
+        // sweep 1: running maximum, e = exp(z - running max) back into tensor memory, row sum.
+        // The load of chunk ch+1 is issued before chunk ch is worked on.
+        float mref[kMaxCh];
+        float m_run = -INFINITY, l = 0.f;
+        uint32_t ra[16], rb[16];
+        tc::tmem_ld16(tb + my_c0 * 16, ra);
+#pragma unroll
+        for (int ch = 0; ch < kMaxCh; ++ch) {
+          uint32_t(&cur)[16] = (ch & 1) ? rb : ra;
+          uint32_t(&nxt)[16] = (ch & 1) ? ra : rb;
+          if (ch < my_nch) {
+            const int col = (my_c0 + ch) * 16;
+            tc::tmem_wait_ld16(cur);
+            if (ch + 1 < my_nch) tc::tmem_ld16(tb + col + 16, nxt);
+            const float m_new = fmaxf(m_run, ps_chunk_max(cur, col, P, causal, i_tok));
+            const float resc = (m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * c);
+            l = l * resc + ps_chunk_exp(cur, c, m_new * c, col, P, causal, i_tok);
+            tc::tmem_st16(tb + col, cur);
+            mref[ch] = m_new;
+            m_run = m_new;
           } else {
-            tc::tmem_wait_ld16(r0);
-            m = fmaxf(m, ps_chunk_max(r0, col, P, causal, i_tok));
-          }
-        }
-        s_mx[h * 128 + row] = m;
-        tc::named_sync(1 + q, 64);
-        m = fmaxf(s_mx[row], s_mx[128 + row]);
-        // pass B: e = exp(z - max) back into tensor memory, row sum
-        const float mc = m * c;
-        float l = 0.f;
-#pragma unroll 1
-        for (int ch = 0; ch < my_nch; ch += 2) {
-          uint32_t r0[16], r1[16];
-          const int col = (my_c0 + ch) * 16;
-          tc::tmem_ld16(tb + col, r0);
-          if (ch + 1 < my_nch) {
-            tc::tmem_ld16(tb + col + 16, r1);
-            tc::tmem_wait_ld16x2(r0, r1);
-            l += ps_chunk_exp(r0, c, mc, col, P, causal, i_tok);
-            l += ps_chunk_exp(r1, c, mc, col + 16, P, causal, i_tok);
-            tc::tmem_st16(tb + col, r0);
-            tc::tmem_st16(tb + col + 16, r1);
-          } else {
-            tc::tmem_wait_ld16(r0);
-            l += ps_chunk_exp(r0, c, mc, col, P, causal, i_tok);
-            tc::tmem_st16(tb + col, r0);
+            mref[ch] = -INFINITY;
           }
         }
         tc::tmem_wait_st();
+        s_mx[h * 128 + row] = m_run;
         s_sum[h * 128 + row] = l;
         tc::named_sync(1 + q, 64);
-        l = s_sum[row] + s_sum[128 + row];
-        const float inv = valid ? 1.f / l : 0.f;
-        const bool all_valid = __all_sync(kFull, valid);
-        // pass C: acc[column] += e / sum
+        const float m0 = s_mx[row], m1 = s_mx[128 + row];
+        const float m = fmaxf(m0, m1);
+        const float lsum = s_sum[row] * ex2_approx((m0 - m) * c) + s_sum[128 + row] * ex2_approx((m1 - m) * c);
+        const float inv = valid ? 1.f / lsum : 0.f;
+        // sweep 2: acc[column] += e * 2^(ref - max) / sum
+        tc::tmem_ld16(tb + my_c0 * 16, ra);
 #pragma unroll
-        for (int ch = 0; ch < kPsAccCols / 16; ++ch) {
+        for (int ch = 0; ch < kMaxCh; ++ch) {
+          uint32_t(&cur)[16] = (ch & 1) ? rb : ra;
+          uint32_t(&nxt)[16] = (ch & 1) ? ra : rb;
           if (ch < my_nch) {
-            uint32_t r0[16];
-            tc::tmem_ld16(tb + (my_c0 + ch) * 16, r0);
-            tc::tmem_wait_ld16(r0);
-            if (!all_valid && !valid) {
+            const int col = (my_c0 + ch) * 16;
+            tc::tmem_wait_ld16(cur);
+            if (ch + 1 < my_nch) tc::tmem_ld16(tb + col + 16, nxt);
+            // rows outside the frame contribute nothing, whatever bits they hold
+            const float w = valid ? ex2_approx((mref[ch] - m) * c) * inv : 0.f;
 #pragma unroll
-              for (int k = 0; k < 16; ++k) r0[k] = 0u;
-            }
-#pragma unroll
-            for (int k = 0; k < 16; ++k) acc[ch * 16 + k] = fmaf(__uint_as_float(r0[k]), inv, acc[ch * 16 + k]);
+            for (int k = 0; k < 16; ++k)
+              acc[ch * 16 + k] = valid ? fmaf(__uint_as_float(cur[k]), w, acc[ch * 16 + k]) : acc[ch * 16 + k];
           }
         }
       }
@@ -439,10 +453,12 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
     }
     if (!ok && et == 0) atomicCAS(p.status, 0, 5);
   }
-#undef PS_BAR_QF
-#undef PS_BAR_QE
+#undef PS_BAR_KF
+#undef PS_BAR_KE
 #undef PS_BAR_AF
 #undef PS_BAR_AE
+#undef PS_BAR_SF
+#undef PS_BAR_SE
 
   tc::tc_fence_before_sync();
   __syncthreads();
