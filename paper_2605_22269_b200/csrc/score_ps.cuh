@@ -1,6 +1,6 @@
 // Persistent, warp-specialised tensor-core scoring of a bf16 chunk (Sec. 3.3, Eq. 1-4).
 //
-// score_ps_kernel: one block of 320 threads per SM.  The chunk is a list of items, ordered by
+// score_ps_kernel: one block of 384 threads per SM.  The chunk is a list of items, ordered by
 // (frame, key head): first the DFT row tiles of that head's keys (Eq. 2-3), then the attention
 // row tiles (Eq. 1; the G query heads of the group are flattened with the tokens into rows, as
 // in score_tc_kernel).  Each block takes a contiguous share of the list.
@@ -11,7 +11,7 @@
 //               from L2) per DFT item.
 //   warp 1      issues tcgen05.mma into one of two 256-column accumulators in tensor memory and
 //               commits to the barriers that free the stages and the key buffers.
-//   warps 2-9   epilogue.  Two warps share each 32-lane quarter of the accumulator and split its
+//   warps 4-11  epilogue (warps 2-3 only hand their registers over).  Two warps share each 32-lane quarter of the accumulator and split its
 //               columns.  Attention item: one sweep takes a running row maximum, writes
 //               exp(z - running max) back into tensor memory and keeps the row sum (rescaled when
 //               the maximum grows); the two warps of a row exchange (max, sum) through shared
@@ -32,14 +32,17 @@
 
 namespace mukv {
 
-constexpr int kPsThreads = 320;
+constexpr int kPsThreads = 384;           // warpgroup 0: control, warpgroups 1-2: epilogue
 constexpr int kPsEpiThreads = 256;
-constexpr int kPsEpiOff = 64;              // first epilogue thread
+constexpr int kPsEpiOff = 128;             // first epilogue thread
 constexpr int kPsMiscBytes = 8192;
 constexpr int kPsMaxBlocks = 256;          // bound on the grid (slots of partial sums)
 constexpr int kPsAccCols = 112;            // accumulator columns per epilogue thread: P <= 2 * 112
-// Ten warps put three on one scheduler, whose 16 K registers then allow 168 per thread: the column
-// accumulators, two 16-column chunks in flight and the addressing have to fit in that.
+// Twelve warps put three on each scheduler, whose 16 K registers allow 168 per thread at launch.
+// The control warpgroup then gives registers back (setmaxnreg) and the epilogue warpgroups take
+// them: 4*32*40 + 8*32*232 = 64,512 registers.
+constexpr int kPsCtrlRegs = 40;
+constexpr int kPsEpiRegs = 232;
 typedef NamedGroup<5, kPsEpiThreads, kPsEpiOff> PsEpiGroup;
 
 struct ScorePsParams {
@@ -209,6 +212,9 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
   tc::tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
 
+  if (warp < 4) {
+    // the control warpgroup (warps 2 and 3 have no other job) hands its registers over
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kPsCtrlRegs));
   if (warp == 0) {
     // ================================================================== TMA producer
     if (lane == 0) {
@@ -306,8 +312,10 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
       }
       if (!ok) atomicCAS(p.status, 0, 4);
     }
+  }
   } else {
     // ================================================================== epilogue
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kPsEpiRegs));
     const int et = tid - kPsEpiOff, ew = et >> 5;
     const int q = warp & 3, h = ew >> 2;                 // TMEM lane quarter, column half
     const int row = q * 32 + lane;
