@@ -35,7 +35,7 @@ namespace mukv {
 constexpr int kPsThreads = 384;           // warpgroup 0: control, warpgroups 1-2: epilogue
 constexpr int kPsEpiThreads = 256;
 constexpr int kPsEpiOff = 128;             // first epilogue thread
-constexpr int kPsMiscBytes = 8192;
+constexpr int kPsMiscBytes = 16384;
 constexpr int kPsMaxBlocks = 256;          // bound on the grid (slots of partial sums)
 constexpr int kPsAccCols = 112;            // accumulator columns per epilogue thread: P <= 2 * 112
 // Twelve warps put three on each scheduler, whose 16 K registers allow 168 per thread at launch.
@@ -166,6 +166,7 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + misc_off + 6144);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + misc_off + 6144 + 192);
   int* s_flag = reinterpret_cast<int*>(sm + misc_off + 6144 + 196);
+  float* s_mref = reinterpret_cast<float*>(sm + misc_off + 8192);             // [8 chunks][256 threads]
   const uint32_t b0 = tc::smem_u32(bars);
   // key buffer full / empty, accumulator full / empty (2 each), stage full / empty (kPsMaxStages each)
 #define PS_BAR_KF(s) (b0 + 8u * (uint32_t)(s))
@@ -368,27 +369,33 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
         const int i_tok = tile * p.tpt + row / G;
         const bool valid = (row < rows_q) && (i_tok < P);
         // sweep 1: running maximum, e = exp(z - running max) back into tensor memory, row sum.
-        // The load of chunk ch+1 is issued before chunk ch is worked on.
-        float mref[kMaxCh];
+        // Two chunks per trip, the load of the next chunk in flight while one is worked on.  The
+        // loop is kept rolled: eight warps walking a long unrolled body starve on instruction fetch.
         float m_run = -INFINITY, l = 0.f;
         uint32_t ra[16], rb[16];
         tc::tmem_ld16(tb + my_c0 * 16, ra);
-#pragma unroll
-        for (int ch = 0; ch < kMaxCh; ++ch) {
-          uint32_t(&cur)[16] = (ch & 1) ? rb : ra;
-          uint32_t(&nxt)[16] = (ch & 1) ? ra : rb;
-          if (ch < my_nch) {
-            const int col = (my_c0 + ch) * 16;
-            tc::tmem_wait_ld16(cur);
-            if (ch + 1 < my_nch) tc::tmem_ld16(tb + col + 16, nxt);
-            const float m_new = fmaxf(m_run, ps_chunk_max(cur, col, P, causal, i_tok));
+#pragma unroll 1
+        for (int ch = 0; ch < my_nch; ch += 2) {
+          const int col = (my_c0 + ch) * 16;
+          tc::tmem_wait_ld16(ra);
+          if (ch + 1 < my_nch) tc::tmem_ld16(tb + col + 16, rb);
+          {
+            const float m_new = fmaxf(m_run, ps_chunk_max(ra, col, P, causal, i_tok));
             const float resc = (m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * c);
-            l = l * resc + ps_chunk_exp(cur, c, m_new * c, col, P, causal, i_tok);
-            tc::tmem_st16(tb + col, cur);
-            mref[ch] = m_new;
+            l = l * resc + ps_chunk_exp(ra, c, m_new * c, col, P, causal, i_tok);
+            tc::tmem_st16(tb + col, ra);
+            s_mref[ch * kPsEpiThreads + et] = m_new;
             m_run = m_new;
-          } else {
-            mref[ch] = -INFINITY;
+          }
+          if (ch + 1 < my_nch) {
+            tc::tmem_wait_ld16(rb);
+            if (ch + 2 < my_nch) tc::tmem_ld16(tb + col + 32, ra);
+            const float m_new = fmaxf(m_run, ps_chunk_max(rb, col + 16, P, causal, i_tok));
+            const float resc = (m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * c);
+            l = l * resc + ps_chunk_exp(rb, c, m_new * c, col + 16, P, causal, i_tok);
+            tc::tmem_st16(tb + col + 16, rb);
+            s_mref[(ch + 1) * kPsEpiThreads + et] = m_new;
+            m_run = m_new;
           }
         }
         tc::tmem_wait_st();
@@ -410,7 +417,7 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
             tc::tmem_wait_ld16(cur);
             if (ch + 1 < my_nch) tc::tmem_ld16(tb + col + 16, nxt);
             // rows outside the frame contribute nothing, whatever bits they hold
-            const float w = valid ? ex2_approx((mref[ch] - m) * c) * inv : 0.f;
+            const float w = valid ? ex2_approx((s_mref[ch * kPsEpiThreads + et] - m) * c) * inv : 0.f;
 #pragma unroll
             for (int k = 0; k < 16; ++k)
               acc[ch * 16 + k] = valid ? fmaf(__uint_as_float(cur[k]), w, acc[ch * 16 + k]) : acc[ch * 16 + k];
