@@ -173,7 +173,7 @@ TcShape tc_shape(const mukv_config& c) {
   t.ps_stages = score_ps_stages(c.tokens_per_frame, c.head_dim, 227 * 1024);
   t.smem_ps = score_ps_smem_bytes(c.tokens_per_frame, c.head_dim, t.ps_stages < 2 ? 2 : t.ps_stages);
   t.ok = t.smem <= 227 * 1024;
-  t.persistent = t.ok && t.ps_stages >= 2 && t.npad <= 2 * kPsAccCols;
+  t.persistent = t.ok && t.ps_stages >= 2 && t.npad <= kPsSplit * kPsAccCols;
   return t;
 }
 

@@ -1,6 +1,6 @@
 // Persistent, warp-specialised tensor-core scoring of a bf16 chunk (Sec. 3.3, Eq. 1-4).
 //
-// score_ps_kernel: one block of 384 threads per SM.  The chunk is a list of items, ordered by
+// score_ps_kernel: one block of 640 threads per SM.  The chunk is a list of items, ordered by
 // (frame, key head): first the DFT row tiles of that head's keys (Eq. 2-3), then the attention
 // row tiles (Eq. 1; the G query heads of the group are flattened with the tokens into rows, as
 // in score_tc_kernel).  Each block takes a contiguous share of the list.
@@ -11,10 +11,10 @@
 //               from L2) per DFT item.
 //   warp 1      issues tcgen05.mma into one of two 256-column accumulators in tensor memory and
 //               commits to the barriers that free the stages and the key buffers.
-//   warps 4-11  epilogue (warps 2-3 only hand their registers over).  Two warps share each 32-lane quarter of the accumulator and split its
+//   warps 4-19  epilogue (warps 2-3 only hand their registers over).  Four warps share each 32-lane quarter of the accumulator and split its
 //               columns.  Attention item: one sweep takes a running row maximum, writes
 //               exp(z - running max) back into tensor memory and keeps the row sum (rescaled when
-//               the maximum grows); the two warps of a row exchange (max, sum) through shared
+//               the maximum grows); the warps of a row exchange (max, sum) through shared
 //               memory; a second sweep adds e * 2^(ref - max) / sum to per-column accumulators in
 //               registers.  The 32 rows of a warp are added only when the block leaves a frame
 //               (shuffle butterfly), so the per-tile cost is one fused multiply-add per logit.
@@ -32,17 +32,18 @@
 
 namespace mukv {
 
-constexpr int kPsThreads = 384;           // warpgroup 0: control, warpgroups 1-2: epilogue
-constexpr int kPsEpiThreads = 256;
+constexpr int kPsThreads = 640;           // warpgroup 0: control, warpgroups 1-4: epilogue
+constexpr int kPsEpiThreads = 512;
+constexpr int kPsSplit = 4;                // warps that share a row (32-lane quarter), each a column range
 constexpr int kPsEpiOff = 128;             // first epilogue thread
-constexpr int kPsMiscBytes = 16384;
+constexpr int kPsMiscBytes = 20480;
 constexpr int kPsMaxBlocks = 256;          // bound on the grid (slots of partial sums)
-constexpr int kPsAccCols = 112;            // accumulator columns per epilogue thread: P <= 2 * 112
-// Twelve warps put three on each scheduler, whose 16 K registers allow 168 per thread at launch.
+constexpr int kPsAccCols = 64;             // accumulator columns per epilogue thread: P <= 4 * 64
+// Twenty warps put five on each scheduler, whose 16 K registers allow 96 per thread at launch.
 // The control warpgroup then gives registers back (setmaxnreg) and the epilogue warpgroups take
-// them: 4*32*40 + 8*32*232 = 64,512 registers.
+// them: 4*32*40 + 16*32*112 = 62,464 registers.
 constexpr int kPsCtrlRegs = 40;
-constexpr int kPsEpiRegs = 232;
+constexpr int kPsEpiRegs = 112;
 typedef NamedGroup<5, kPsEpiThreads, kPsEpiOff> PsEpiGroup;
 
 struct ScorePsParams {
@@ -136,7 +137,7 @@ __device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c
   select_frame<1, PsEpiGroup>(sp, f, att, fft, s_sc, s_int, s_misc);
 }
 
-__global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
+__global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
                                                  const __grid_constant__ CUtensorMap qmap,
                                                  const __grid_constant__ CUtensorMap kmap,
                                                  const __grid_constant__ CUtensorMap wmap) {
@@ -161,12 +162,12 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
   const uint32_t sS = sK + 2u * k_buf;                   // NS operand stages
   const uint32_t misc_off = 2u * k_buf + (uint32_t)NS * st_buf;
   float* s_col = reinterpret_cast<float*>(sm + misc_off);                     // [4][256]
-  float* s_mx = reinterpret_cast<float*>(sm + misc_off + 4096);               // [2][128]
-  float* s_sum = s_mx + 256;                                                  // [2][128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + misc_off + 6144);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + misc_off + 6144 + 192);
-  int* s_flag = reinterpret_cast<int*>(sm + misc_off + 6144 + 196);
-  float* s_mref = reinterpret_cast<float*>(sm + misc_off + 8192);             // [8 chunks][256 threads]
+  float* s_mx = reinterpret_cast<float*>(sm + misc_off + 4096);               // [kPsSplit][128]
+  float* s_sum = s_mx + kPsSplit * 128;                                       // [kPsSplit][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + misc_off + 8192);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + misc_off + 8192 + 192);
+  int* s_flag = reinterpret_cast<int*>(sm + misc_off + 8192 + 196);
+  float* s_mref = reinterpret_cast<float*>(sm + misc_off + 10240);            // [4 chunks][512 threads]
   const uint32_t b0 = tc::smem_u32(bars);
   // key buffer full / empty, accumulator full / empty (2 each), stage full / empty (kPsMaxStages each)
 #define PS_BAR_KF(s) (b0 + 8u * (uint32_t)(s))
@@ -181,7 +182,7 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
       tc::mbar_init(PS_BAR_KF(s), 1);
       tc::mbar_init(PS_BAR_KE(s), 1);
       tc::mbar_init(PS_BAR_AF(s), 1);
-      tc::mbar_init(PS_BAR_AE(s), 8);                    // one arrival per epilogue warp
+      tc::mbar_init(PS_BAR_AE(s), kPsEpiThreads / 32);   // one arrival per epilogue warp
     }
     for (int s = 0; s < kPsMaxStages; ++s) {
       tc::mbar_init(PS_BAR_SF(s), 1);
@@ -318,11 +319,11 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
     // ================================================================== epilogue
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kPsEpiRegs));
     const int et = tid - kPsEpiOff, ew = et >> 5;
-    const int q = warp & 3, h = ew >> 2;                 // TMEM lane quarter, column half
+    const int q = warp & 3, h = ew >> 2;                 // TMEM lane quarter, column range
     const int row = q * 32 + lane;
     const uint32_t tlane = (uint32_t)(q * 32) << 16;
-    const int nch16 = p.npad >> 4, nch0 = (nch16 + 1) >> 1;
-    const int my_c0 = h ? nch0 : 0, my_nch = h ? nch16 - nch0 : nch0;
+    const int nch16 = p.npad >> 4, ch_base = nch16 / kPsSplit, ch_rem = nch16 % kPsSplit;
+    const int my_c0 = h * ch_base + (h < ch_rem ? h : ch_rem), my_nch = ch_base + (h < ch_rem ? 1 : 0);
     const bool causal = sp.causal != 0;
     const float c = p.exp2_scale;
     constexpr int kMaxCh = kPsAccCols / 16;
@@ -342,85 +343,80 @@ __global__ void __maxnreg__(168) score_ps_kernel(const ScorePsParams p,
       const uint32_t tb = tmem + (uint32_t)b * 256u + tlane;
       if (x < p.n_mt) {
         // ---- Eq. 2-3: this thread's half of the bins of its token
-        const int H2 = D >> 1, bins = H2 >> 1, bin0 = h * bins;
+        const int H2 = D >> 1;
+        const int bins = H2 / kPsSplit >= 16 ? H2 / kPsSplit : 16;   // per warp of the row, a multiple of 16
+        const int bin0 = h * bins;
         float tot = 0.f;
+        if (bin0 < H2) {
 #pragma unroll 1
-        for (int cc = 0; cc < bins; cc += 16) {
-          uint32_t re[16], im[16];
-          tc::tmem_ld16(tb + bin0 + cc, re);
-          tc::tmem_ld16(tb + H2 + bin0 + cc, im);
-          tc::tmem_wait_ld16x2(re, im);
+          for (int cc = 0; cc < bins; cc += 16) {
+            uint32_t re[16], im[16];
+            tc::tmem_ld16(tb + bin0 + cc, re);
+            tc::tmem_ld16(tb + H2 + bin0 + cc, im);
+            tc::tmem_wait_ld16x2(re, im);
 #pragma unroll
-          for (int k = 0; k < 16; ++k) {
-            const float a = __uint_as_float(re[k]), bb = __uint_as_float(im[k]);
-            const float mag = sqrtf(fmaf(a, a, bb * bb));
-            // bins 0 and D/2 are real: their two values sit in the re/im slots of "bin 0"
-            tot += (bin0 + cc + k == 0) ? fabsf(a) + fabsf(bb) : 2.f * mag;
+            for (int k = 0; k < 16; ++k) {
+              const float a = __uint_as_float(re[k]), bb = __uint_as_float(im[k]);
+              const float mag = sqrtf(fmaf(a, a, bb * bb));
+              // bins 0 and D/2 are real: their two values sit in the re/im slots of "bin 0"
+              tot += (bin0 + cc + k == 0) ? fabsf(a) + fabsf(bb) : 2.f * mag;
+            }
           }
         }
         s_sum[h * 128 + row] = tot;
-        tc::named_sync(1 + q, 64);
+        tc::named_sync(1 + q, 32 * kPsSplit);
         const int token = x * 128 + row;
-        if (h == 0 && token < P)
-          reinterpret_cast<float*>(sp.ifft_part)[((long long)f * Hkv + g) * P + token] = s_sum[row] + s_sum[128 + row];
+        if (h == 0 && token < P) {
+          float t4 = 0.f;
+#pragma unroll
+          for (int hh = 0; hh < kPsSplit; ++hh) t4 += s_sum[hh * 128 + row];
+          reinterpret_cast<float*>(sp.ifft_part)[((long long)f * Hkv + g) * P + token] = t4;
+        }
       } else {
         // ---- Eq. 1
         const int tile = x - p.n_mt;
         const int i_tok = tile * p.tpt + row / G;
         const bool valid = (row < rows_q) && (i_tok < P);
         // sweep 1: running maximum, e = exp(z - running max) back into tensor memory, row sum.
-        // Two chunks per trip, the load of the next chunk in flight while one is worked on.  The
-        // loop is kept rolled: eight warps walking a long unrolled body starve on instruction fetch.
+        // One 16-column chunk per trip; the other warps of the scheduler cover the load latency.
+        // The loop is kept rolled: many warps walking a long unrolled body starve on instruction fetch.
         float m_run = -INFINITY, l = 0.f;
-        uint32_t ra[16], rb[16];
-        tc::tmem_ld16(tb + my_c0 * 16, ra);
 #pragma unroll 1
-        for (int ch = 0; ch < my_nch; ch += 2) {
+        for (int ch = 0; ch < my_nch; ++ch) {
           const int col = (my_c0 + ch) * 16;
+          uint32_t ra[16];
+          tc::tmem_ld16(tb + col, ra);
           tc::tmem_wait_ld16(ra);
-          if (ch + 1 < my_nch) tc::tmem_ld16(tb + col + 16, rb);
-          {
-            const float m_new = fmaxf(m_run, ps_chunk_max(ra, col, P, causal, i_tok));
-            const float resc = (m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * c);
-            l = l * resc + ps_chunk_exp(ra, c, m_new * c, col, P, causal, i_tok);
-            tc::tmem_st16(tb + col, ra);
-            s_mref[ch * kPsEpiThreads + et] = m_new;
-            m_run = m_new;
-          }
-          if (ch + 1 < my_nch) {
-            tc::tmem_wait_ld16(rb);
-            if (ch + 2 < my_nch) tc::tmem_ld16(tb + col + 32, ra);
-            const float m_new = fmaxf(m_run, ps_chunk_max(rb, col + 16, P, causal, i_tok));
-            const float resc = (m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * c);
-            l = l * resc + ps_chunk_exp(rb, c, m_new * c, col + 16, P, causal, i_tok);
-            tc::tmem_st16(tb + col + 16, rb);
-            s_mref[(ch + 1) * kPsEpiThreads + et] = m_new;
-            m_run = m_new;
-          }
+          const float m_new = fmaxf(m_run, ps_chunk_max(ra, col, P, causal, i_tok));
+          const float resc = (m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * c);
+          l = l * resc + ps_chunk_exp(ra, c, m_new * c, col, P, causal, i_tok);
+          tc::tmem_st16(tb + col, ra);
+          s_mref[ch * kPsEpiThreads + et] = m_new;
+          m_run = m_new;
         }
         tc::tmem_wait_st();
         s_mx[h * 128 + row] = m_run;
         s_sum[h * 128 + row] = l;
-        tc::named_sync(1 + q, 64);
-        const float m0 = s_mx[row], m1 = s_mx[128 + row];
-        const float m = fmaxf(m0, m1);
-        const float lsum = s_sum[row] * ex2_approx((m0 - m) * c) + s_sum[128 + row] * ex2_approx((m1 - m) * c);
+        tc::named_sync(1 + q, 32 * kPsSplit);
+        float m = s_mx[row];
+#pragma unroll
+        for (int hh = 1; hh < kPsSplit; ++hh) m = fmaxf(m, s_mx[hh * 128 + row]);
+        float lsum = 0.f;
+#pragma unroll
+        for (int hh = 0; hh < kPsSplit; ++hh) lsum += s_sum[hh * 128 + row] * ex2_approx((s_mx[hh * 128 + row] - m) * c);
         const float inv = valid ? 1.f / lsum : 0.f;
         // sweep 2: acc[column] += e * 2^(ref - max) / sum
-        tc::tmem_ld16(tb + my_c0 * 16, ra);
 #pragma unroll
         for (int ch = 0; ch < kMaxCh; ++ch) {
-          uint32_t(&cur)[16] = (ch & 1) ? rb : ra;
-          uint32_t(&nxt)[16] = (ch & 1) ? ra : rb;
           if (ch < my_nch) {
-            const int col = (my_c0 + ch) * 16;
-            tc::tmem_wait_ld16(cur);
-            if (ch + 1 < my_nch) tc::tmem_ld16(tb + col + 16, nxt);
+            uint32_t ra[16];
+            tc::tmem_ld16(tb + (my_c0 + ch) * 16, ra);
             // rows outside the frame contribute nothing, whatever bits they hold
             const float w = valid ? ex2_approx((s_mref[ch * kPsEpiThreads + et] - m) * c) * inv : 0.f;
+            tc::tmem_wait_ld16(ra);
 #pragma unroll
             for (int k = 0; k < 16; ++k)
-              acc[ch * 16 + k] = valid ? fmaf(__uint_as_float(cur[k]), w, acc[ch * 16 + k]) : acc[ch * 16 + k];
+              acc[ch * 16 + k] = valid ? fmaf(__uint_as_float(ra[k]), w, acc[ch * 16 + k]) : acc[ch * 16 + k];
           }
         }
       }
