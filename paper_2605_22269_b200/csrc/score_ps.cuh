@@ -40,10 +40,12 @@ constexpr int kPsMiscBytes = 20480;
 constexpr int kPsMaxBlocks = 256;          // bound on the grid (slots of partial sums)
 constexpr int kPsAccCols = 64;             // accumulator columns per epilogue thread: P <= 4 * 64
 // Twenty warps put five on each scheduler, whose 16 K registers allow 96 per thread at launch.
-// The control warpgroup then gives registers back (setmaxnreg) and the epilogue warpgroups take
-// them: 4*32*40 + 16*32*112 = 62,464 registers.
-constexpr int kPsCtrlRegs = 40;
+// The control warpgroup then gives registers back (setmaxnreg.dec) and the four epilogue warpgroups
+// take them.  The hand-over has to balance: what the control warpgroup releases, 128 * (96 - 32),
+// is all the epilogue warpgroups can claim, 512 * (112 - 96); a larger claim would block forever.
+constexpr int kPsCtrlRegs = 32;
 constexpr int kPsEpiRegs = 112;
+static_assert(128 * (96 - kPsCtrlRegs) >= 512 * (kPsEpiRegs - 96), "register hand-over does not balance");
 typedef NamedGroup<5, kPsEpiThreads, kPsEpiOff> PsEpiGroup;
 
 struct ScorePsParams {

@@ -1,7 +1,7 @@
 // Thin wrappers over the sm_100a instructions the tensor-core kernels use: mbarriers, TMA tile
 // loads, tensor memory (TMEM) allocation and access, tcgen05.mma and its descriptors.
-// Every wait is bounded: after kSpinLimit unsuccessful polls it gives up and reports false, so
-// a kernel can record an error code and leave instead of hanging.
+// Every wait is bounded: after kWaitLimitNs of polling it gives up and reports false, so a kernel
+// can record an error code and leave instead of hanging.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -10,7 +10,7 @@
 namespace mukv {
 namespace tc {
 
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr unsigned long long kWaitLimitNs = 1500000000ull;     // 1.5 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -37,13 +37,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// true once the phase with the given parity has completed; false if it never did within the limit
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// true once the phase with the given parity has completed; false if it has not after kWaitLimitNs
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (it > 256) __nanosleep(64);
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    for (int it = 0; it < 32; ++it) {
+      if (mbar_try_wait(bar, parity)) return true;
+    }
+    if (global_ns() - t0 > kWaitLimitNs) return false;
+    __nanosleep(64);
   }
-  return false;
 }
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
