@@ -121,22 +121,134 @@ __device__ __forceinline__ float ps_chunk_exp(uint32_t (&r)[16], float c, float 
 }
 
 // Eq. 4 and the selection for frame f, run by the epilogue warps of the block that finished the
-// frame last.  Kept out of line so that the tile loop's register allocation is not disturbed.
+// frame last.  Same rule as select_frame (score.cuh), written for this kernel's 512 threads and
+// P <= 256 with few barriers, because it sits on the critical path at the end of the launch:
+// fused scores lie in [0, 1], so their bit patterns order like the values and the rank counting
+// runs on integer compares, two threads per token.  Kept out of line so that the tile loop's
+// register allocation is not disturbed.
 __device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c_first, int c_last, double* s_sc,
-                                             int* s_int, double* s_misc) {
-  const int et = PsEpiGroup::tid();
-  const int P = sp.P, Hkv = sp.Hkv;
-  double att[1] = {0.0}, fft[1] = {0.0};
-  if (et < P) {
+                                             int* s_int, double* s_misc, int* s_cnt) {
+  const int et = PsEpiGroup::tid(), lane = et & 31, warp = et >> 5;
+  const int P = sp.P, Hkv = sp.Hkv, kappa = sp.kappa;
+  const bool valid = et < P;
+  const double big = 3.0e38;
+  double att = 0.0, fft = 0.0;
+  if (valid) {
+    // the blocks' column sums, eight loads in flight at a time, added in block order
     const float* cp = reinterpret_cast<const float*>(sp.colsum_part) + et;
-    for (int cc = c_first; cc <= c_last; ++cc) att[0] += (double)__ldcg(cp + (long long)(cc + f) * P);
-    att[0] = att[0] / (double)((long long)sp.Hq * P);
+    for (int cc = c_first; cc <= c_last; cc += 8) {
+      float x[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) x[i] = cc + i <= c_last ? __ldcg(cp + (long long)(cc + i + f) * P) : 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) att += (double)x[i];
+    }
+    att = att / (double)((long long)sp.Hq * P);
     const float* fp = reinterpret_cast<const float*>(sp.ifft_part) + (long long)f * Hkv * P + et;
-    for (int gg = 0; gg < Hkv; ++gg) fft[0] += (double)__ldcg(fp + (long long)gg * P);
-    fft[0] = fft[0] / (double)((long long)Hkv * sp.D);
+    for (int gg = 0; gg < Hkv; ++gg) fft += (double)__ldcg(fp + (long long)gg * P);
+    fft = fft / (double)((long long)Hkv * sp.D);
+  }
+  // ---- min / max of both signals over the frame (the tokens live in the first eight warps)
+  if (warp < 8) {
+    double v0 = warp_min(valid ? att : big), v1 = warp_max(valid ? att : -big);
+    double v2 = warp_min(valid ? fft : big), v3 = warp_max(valid ? fft : -big);
+    if (lane == 0) { s_misc[warp * 4] = v0; s_misc[warp * 4 + 1] = v1; s_misc[warp * 4 + 2] = v2; s_misc[warp * 4 + 3] = v3; }
   }
   PsEpiGroup::sync();
-  select_frame<1, PsEpiGroup>(sp, f, att, fft, s_sc, s_int, s_misc);
+  double amin = big, amax = -big, fmin_ = big, fmax_ = -big;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) {
+    amin = s_misc[w * 4 + 0] < amin ? s_misc[w * 4 + 0] : amin;
+    amax = s_misc[w * 4 + 1] > amax ? s_misc[w * 4 + 1] : amax;
+    fmin_ = s_misc[w * 4 + 2] < fmin_ ? s_misc[w * 4 + 2] : fmin_;
+    fmax_ = s_misc[w * 4 + 3] > fmax_ ? s_misc[w * 4 + 3] : fmax_;
+  }
+  // ---- Eq. 4
+  const double an = (amax == amin) ? 0.0 : (att - amin) / (amax - amin);
+  double fn = (fmax_ == fmin_) ? 0.0 : (fft - fmin_) / (fmax_ - fmin_);
+  if (sp.keep_low) fn = 1.0 - fn;
+  const double alpha = (double)sp.alpha;
+  const double s = alpha * an + (1.0 - alpha) * fn;
+  if (valid) s_sc[et] = s;
+  PsEpiGroup::sync();
+  // ---- tau = kappa-th largest score: rank counting, each token's scan split over two threads
+  {
+    const int t = et & 255, half = et >> 8;
+    const int mid = (P + 1) >> 1;
+    const int j0 = half ? mid : 0, j1 = half ? P : mid;
+    int gt = 0, ge = 0;
+    if (t < P) {
+      const long long key = __double_as_longlong(s_sc[t]);
+      for (int j = j0; j < j1; ++j) {
+        const long long o = __double_as_longlong(s_sc[j]);
+        gt += (o > key);
+        ge += (o >= key);
+      }
+    }
+    s_cnt[half * 256 + t] = gt | (ge << 16);
+  }
+  PsEpiGroup::sync();
+  if (valid) {
+    const int c0 = s_cnt[et], c1 = s_cnt[256 + et];
+    const int gt = (c0 & 0xffff) + (c1 & 0xffff), ge = (c0 >> 16) + (c1 >> 16);
+    if (gt < kappa && kappa <= ge) s_misc[32] = s;          // every writer holds the same value
+  }
+  PsEpiGroup::sync();
+  const double tau = s_misc[32];
+  const double delta = (double)sp.tie_eps;
+  const bool sure = valid && (s > tau + delta);
+  const bool band = valid && !sure && (s >= tau - delta);
+  const unsigned lt = (1u << lane) - 1u;
+  const unsigned b_sure = __ballot_sync(kFull, sure), b_band = __ballot_sync(kFull, band);
+  if (lane == 0 && warp < 8) { s_int[warp] = __popc(b_sure); s_int[8 + warp] = __popc(b_band); }
+  PsEpiGroup::sync();
+  int n_sure = 0, band_rank = __popc(b_band & lt);
+#pragma unroll
+  for (int w = 0; w < 8; ++w) {
+    n_sure += s_int[w];
+    if (w < warp) band_rank += s_int[8 + w];
+  }
+  const bool keep = sure || (band && band_rank < kappa - n_sure);
+  const unsigned b_keep = __ballot_sync(kFull, keep);
+  if (lane == 0 && warp < 8) s_int[16 + warp] = __popc(b_keep);
+  // lowest kept and highest dropped score, for the safety test below
+  if (warp < 8) {
+    const double a = warp_min(keep ? s : big), b = warp_max((valid && !keep) ? s : -big);
+    if (lane == 0) { s_misc[40 + warp * 2] = a; s_misc[41 + warp * 2] = b; }
+  }
+  PsEpiGroup::sync();
+  const long long f_abs = sp.first_frame + f;
+  if (keep) {
+    int pos = __popc(b_keep & lt);
+    for (int w = 0; w < warp; ++w) pos += s_int[16 + w];
+    sp.kept_store[f_abs * kappa + pos] = et;
+    if (sp.kept_out) sp.kept_out[(long long)f * kappa + pos] = et;
+  }
+  if (sp.scores_out && valid) {
+    const long long np = (long long)sp.n_frames * P;
+    sp.scores_out[0 * np + (long long)f * P + et] = (float)att;
+    sp.scores_out[1 * np + (long long)f * P + et] = (float)fft;
+    sp.scores_out[2 * np + (long long)f * P + et] = (float)s;
+  }
+  if (et == 0) {
+    sp.frame_ts[f_abs] = f_abs;
+    sp.page_table[f_abs] = sp.pages_off + f_abs * sp.page_bytes;
+    // does single precision decide this frame safely?  (see select_frame)
+    double a = big, b = -big;
+    for (int w = 0; w < 8; ++w) {
+      a = s_misc[40 + w * 2] < a ? s_misc[40 + w * 2] : a;
+      b = s_misc[41 + w * 2] > b ? s_misc[41 + w * 2] : b;
+    }
+    bool risky = (kappa < P) && (a - b <= delta + (double)sp.flag_margin);
+    const double fr = (double)sp.flat_ratio;
+    const double aabs = amax > -amin ? amax : -amin, fabs_ = fmax_ > -fmin_ ? fmax_ : -fmin_;
+    if (amax != amin && (amax - amin) < fr * aabs && sp.alpha != 0.f) risky = true;
+    if (fmax_ != fmin_ && (fmax_ - fmin_) < fr * fabs_ && sp.alpha != 1.f) risky = true;
+    if (risky) {
+      const int slot = atomicAdd(sp.n_flagged, 1);
+      sp.flagged[slot] = f;
+    }
+  }
 }
 
 __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
@@ -458,8 +570,8 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
         if (s_flag[0]) {
           __threadfence();
           ps_finish_frame(sp, f, c_first, c_last, reinterpret_cast<double*>(s_col),
-                          reinterpret_cast<int*>(sm + misc_off + 2560),
-                          reinterpret_cast<double*>(sm + misc_off + 2048));
+                          reinterpret_cast<int*>(sm + misc_off + 3072),
+                          reinterpret_cast<double*>(sm + misc_off + 2048), reinterpret_cast<int*>(s_mref));
         }
         PsEpiGroup::sync();
       }
