@@ -121,68 +121,78 @@ __device__ __forceinline__ float ps_chunk_exp(uint32_t (&r)[16], float c, float 
 }
 
 // Eq. 4 and the selection for frame f, run by the epilogue warps of the block that finished the
-// frame last.  Same rule as select_frame (score.cuh), written for this kernel's 512 threads and
-// P <= 256 with few barriers, because it sits on the critical path at the end of the launch:
-// fused scores lie in [0, 1], so their bit patterns order like the values and the rank counting
-// runs on integer compares, two threads per token.  Kept out of line so that the tile loop's
-// register allocation is not disturbed.
-__device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c_first, int c_last, double* s_sc,
-                                             int* s_int, double* s_misc, int* s_cnt) {
+// frame last.  It sits on the critical path at the end of the launch, so it is written for speed:
+// the partial sums are added in double and in block order, everything after that is single
+// precision (double-precision arithmetic is slow on this part), few barriers, and the rank counting
+// runs on the scores' bit patterns (scores lie in [0, 1], so the patterns order like the values),
+// two threads per token.  Single precision adds about 1e-7 to the score error, which the safety
+// test below covers: a frame whose lowest kept and highest dropped score are closer than
+// tie_eps + flag_margin is left to the double-precision pass (score_kernel<T, double> with
+// select_frame), which applies the same rule.  Kept out of line so that the tile loop's register
+// allocation is not disturbed.
+__device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c_first, int c_last, float* s_sc,
+                                             int* s_int, float* s_misc, int* s_cnt) {
   const int et = PsEpiGroup::tid(), lane = et & 31, warp = et >> 5;
   const int P = sp.P, Hkv = sp.Hkv, kappa = sp.kappa;
   const bool valid = et < P;
-  const double big = 3.0e38;
-  double att = 0.0, fft = 0.0;
+  const float big = 3.0e38f;
+  float att = 0.f, fft = 0.f;
   if (valid) {
-    // the blocks' column sums, eight loads in flight at a time, added in block order
+    // the blocks' column sums, sixteen loads in flight at a time, added in block order
     const float* cp = reinterpret_cast<const float*>(sp.colsum_part) + et;
-    for (int cc = c_first; cc <= c_last; cc += 8) {
-      float x[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) x[i] = cc + i <= c_last ? __ldcg(cp + (long long)(cc + i + f) * P) : 0.f;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) att += (double)x[i];
-    }
-    att = att / (double)((long long)sp.Hq * P);
     const float* fp = reinterpret_cast<const float*>(sp.ifft_part) + (long long)f * Hkv * P + et;
-    for (int gg = 0; gg < Hkv; ++gg) fft += (double)__ldcg(fp + (long long)gg * P);
-    fft = fft / (double)((long long)Hkv * sp.D);
+    double a64 = 0.0, f64 = 0.0;
+    float y[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) y[i] = i < Hkv ? __ldcg(fp + (long long)i * P) : 0.f;
+    for (int cc = c_first; cc <= c_last; cc += 16) {
+      float x[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) x[i] = cc + i <= c_last ? __ldcg(cp + (long long)(cc + i + f) * P) : 0.f;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) a64 += (double)x[i];
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f64 += (double)y[i];
+    for (int gg = 8; gg < Hkv; ++gg) f64 += (double)__ldcg(fp + (long long)gg * P);
+    att = (float)a64 * (1.f / (float)((long long)sp.Hq * P));
+    fft = (float)f64 * (1.f / (float)((long long)Hkv * sp.D));
   }
   // ---- min / max of both signals over the frame (the tokens live in the first eight warps)
   if (warp < 8) {
-    double v0 = warp_min(valid ? att : big), v1 = warp_max(valid ? att : -big);
-    double v2 = warp_min(valid ? fft : big), v3 = warp_max(valid ? fft : -big);
+    const float v0 = warp_min(valid ? att : big), v1 = warp_max(valid ? att : -big);
+    const float v2 = warp_min(valid ? fft : big), v3 = warp_max(valid ? fft : -big);
     if (lane == 0) { s_misc[warp * 4] = v0; s_misc[warp * 4 + 1] = v1; s_misc[warp * 4 + 2] = v2; s_misc[warp * 4 + 3] = v3; }
   }
   PsEpiGroup::sync();
-  double amin = big, amax = -big, fmin_ = big, fmax_ = -big;
+  float amin = big, amax = -big, fmin_ = big, fmax_ = -big;
 #pragma unroll
   for (int w = 0; w < 8; ++w) {
-    amin = s_misc[w * 4 + 0] < amin ? s_misc[w * 4 + 0] : amin;
-    amax = s_misc[w * 4 + 1] > amax ? s_misc[w * 4 + 1] : amax;
-    fmin_ = s_misc[w * 4 + 2] < fmin_ ? s_misc[w * 4 + 2] : fmin_;
-    fmax_ = s_misc[w * 4 + 3] > fmax_ ? s_misc[w * 4 + 3] : fmax_;
+    amin = fminf(amin, s_misc[w * 4 + 0]);
+    amax = fmaxf(amax, s_misc[w * 4 + 1]);
+    fmin_ = fminf(fmin_, s_misc[w * 4 + 2]);
+    fmax_ = fmaxf(fmax_, s_misc[w * 4 + 3]);
   }
   // ---- Eq. 4
-  const double an = (amax == amin) ? 0.0 : (att - amin) / (amax - amin);
-  double fn = (fmax_ == fmin_) ? 0.0 : (fft - fmin_) / (fmax_ - fmin_);
-  if (sp.keep_low) fn = 1.0 - fn;
-  const double alpha = (double)sp.alpha;
-  const double s = alpha * an + (1.0 - alpha) * fn;
-  if (valid) s_sc[et] = s;
+  const float an = (amax == amin) ? 0.f : (att - amin) / (amax - amin);
+  float fn = (fmax_ == fmin_) ? 0.f : (fft - fmin_) / (fmax_ - fmin_);
+  if (sp.keep_low) fn = 1.f - fn;
+  const float s = sp.alpha * an + (1.f - sp.alpha) * fn;
+  if (et < 256) s_sc[et] = valid ? s : -1.f;                 // slots past P hold -1: below every score
   PsEpiGroup::sync();
   // ---- tau = kappa-th largest score: rank counting, each token's scan split over two threads
   {
     const int t = et & 255, half = et >> 8;
-    const int mid = (P + 1) >> 1;
-    const int j0 = half ? mid : 0, j1 = half ? P : mid;
+    const int n4 = (P + 3) >> 2, mid = (n4 + 1) >> 1;
+    const int j0 = half ? mid : 0, j1 = half ? n4 : mid;
     int gt = 0, ge = 0;
     if (t < P) {
-      const long long key = __double_as_longlong(s_sc[t]);
+      const int key = __float_as_int(s_sc[t]);
+      const int4* v = reinterpret_cast<const int4*>(s_sc);
       for (int j = j0; j < j1; ++j) {
-        const long long o = __double_as_longlong(s_sc[j]);
-        gt += (o > key);
-        ge += (o >= key);
+        const int4 o = v[j];
+        gt += (o.x > key) + (o.y > key) + (o.z > key) + (o.w > key);
+        ge += (o.x >= key) + (o.y >= key) + (o.z >= key) + (o.w >= key);
       }
     }
     s_cnt[half * 256 + t] = gt | (ge << 16);
@@ -194,8 +204,8 @@ __device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c
     if (gt < kappa && kappa <= ge) s_misc[32] = s;          // every writer holds the same value
   }
   PsEpiGroup::sync();
-  const double tau = s_misc[32];
-  const double delta = (double)sp.tie_eps;
+  const float tau = s_misc[32];
+  const float delta = sp.tie_eps;
   const bool sure = valid && (s > tau + delta);
   const bool band = valid && !sure && (s >= tau - delta);
   const unsigned lt = (1u << lane) - 1u;
@@ -213,7 +223,7 @@ __device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c
   if (lane == 0 && warp < 8) s_int[16 + warp] = __popc(b_keep);
   // lowest kept and highest dropped score, for the safety test below
   if (warp < 8) {
-    const double a = warp_min(keep ? s : big), b = warp_max((valid && !keep) ? s : -big);
+    const float a = warp_min(keep ? s : big), b = warp_max((valid && !keep) ? s : -big);
     if (lane == 0) { s_misc[40 + warp * 2] = a; s_misc[41 + warp * 2] = b; }
   }
   PsEpiGroup::sync();
@@ -226,24 +236,23 @@ __device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c
   }
   if (sp.scores_out && valid) {
     const long long np = (long long)sp.n_frames * P;
-    sp.scores_out[0 * np + (long long)f * P + et] = (float)att;
-    sp.scores_out[1 * np + (long long)f * P + et] = (float)fft;
-    sp.scores_out[2 * np + (long long)f * P + et] = (float)s;
+    sp.scores_out[0 * np + (long long)f * P + et] = att;
+    sp.scores_out[1 * np + (long long)f * P + et] = fft;
+    sp.scores_out[2 * np + (long long)f * P + et] = s;
   }
   if (et == 0) {
     sp.frame_ts[f_abs] = f_abs;
     sp.page_table[f_abs] = sp.pages_off + f_abs * sp.page_bytes;
     // does single precision decide this frame safely?  (see select_frame)
-    double a = big, b = -big;
+    float a = big, b = -big;
     for (int w = 0; w < 8; ++w) {
-      a = s_misc[40 + w * 2] < a ? s_misc[40 + w * 2] : a;
-      b = s_misc[41 + w * 2] > b ? s_misc[41 + w * 2] : b;
+      a = fminf(a, s_misc[40 + w * 2]);
+      b = fmaxf(b, s_misc[41 + w * 2]);
     }
-    bool risky = (kappa < P) && (a - b <= delta + (double)sp.flag_margin);
-    const double fr = (double)sp.flat_ratio;
-    const double aabs = amax > -amin ? amax : -amin, fabs_ = fmax_ > -fmin_ ? fmax_ : -fmin_;
-    if (amax != amin && (amax - amin) < fr * aabs && sp.alpha != 0.f) risky = true;
-    if (fmax_ != fmin_ && (fmax_ - fmin_) < fr * fabs_ && sp.alpha != 1.f) risky = true;
+    bool risky = (kappa < P) && (a - b <= delta + sp.flag_margin);
+    const float aabs = fmaxf(amax, -amin), fabs_ = fmaxf(fmax_, -fmin_);
+    if (amax != amin && (amax - amin) < sp.flat_ratio * aabs && sp.alpha != 0.f) risky = true;
+    if (fmax_ != fmin_ && (fmax_ - fmin_) < sp.flat_ratio * fabs_ && sp.alpha != 1.f) risky = true;
     if (risky) {
       const int slot = atomicAdd(sp.n_flagged, 1);
       sp.flagged[slot] = f;
@@ -569,9 +578,8 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
         PsEpiGroup::sync();
         if (s_flag[0]) {
           __threadfence();
-          ps_finish_frame(sp, f, c_first, c_last, reinterpret_cast<double*>(s_col),
-                          reinterpret_cast<int*>(sm + misc_off + 3072),
-                          reinterpret_cast<double*>(sm + misc_off + 2048), reinterpret_cast<int*>(s_mref));
+          ps_finish_frame(sp, f, c_first, c_last, s_col, reinterpret_cast<int*>(sm + misc_off + 3072),
+                          reinterpret_cast<float*>(sm + misc_off + 2048), reinterpret_cast<int*>(s_mref));
         }
         PsEpiGroup::sync();
       }
