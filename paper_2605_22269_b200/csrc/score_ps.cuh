@@ -291,6 +291,9 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + misc_off + 8192 + 192);
   int* s_flag = reinterpret_cast<int*>(sm + misc_off + 8192 + 196);
   float* s_mref = reinterpret_cast<float*>(sm + misc_off + 10240);            // [4 chunks][512 threads]
+  // the selection routine is a real call: it reads the parameters from this copy, so that the
+  // kernel's own parameter block never has its address taken (which would move it to local memory)
+  ScoreParams* s_sp = reinterpret_cast<ScoreParams*>(sm + misc_off + 3328);
   const uint32_t b0 = tc::smem_u32(bars);
   // key buffer full / empty, accumulator full / empty (2 each), stage full / empty (kPsMaxStages each)
 #define PS_BAR_KF(s) (b0 + 8u * (uint32_t)(s))
@@ -312,6 +315,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
       tc::mbar_init(PS_BAR_SE(s), 1);
     }
     tc::fence_mbar_init();
+    *s_sp = p.sp;
     tc::prefetch_tmap(&qmap);
     tc::prefetch_tmap(&kmap);
     tc::prefetch_tmap(&wmap);
@@ -578,7 +582,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
         PsEpiGroup::sync();
         if (s_flag[0]) {
           __threadfence();
-          ps_finish_frame(sp, f, c_first, c_last, s_col, reinterpret_cast<int*>(sm + misc_off + 3072),
+          ps_finish_frame(*s_sp, f, c_first, c_last, s_col, reinterpret_cast<int*>(sm + misc_off + 3072),
                           reinterpret_cast<float*>(sm + misc_off + 2048), reinterpret_cast<int*>(s_mref));
         }
         PsEpiGroup::sync();
