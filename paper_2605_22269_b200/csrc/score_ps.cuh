@@ -293,7 +293,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
   float* s_mref = reinterpret_cast<float*>(sm + misc_off + 10240);            // [4 chunks][512 threads]
   // the selection routine is a real call: it reads the parameters from this copy, so that the
   // kernel's own parameter block never has its address taken (which would move it to local memory)
-  ScoreParams* s_sp = reinterpret_cast<ScoreParams*>(sm + misc_off + 3328);
+  ScoreParams* s_sp = reinterpret_cast<ScoreParams*>(sm + misc_off + 8704);
   const uint32_t b0 = tc::smem_u32(bars);
   // key buffer full / empty, accumulator full / empty (2 each), stage full / empty (kPsMaxStages each)
 #define PS_BAR_KF(s) (b0 + 8u * (uint32_t)(s))
