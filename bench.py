@@ -25,6 +25,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one score_ps_kernel launch on a 16-frame chunk of this
+# workload (ncu capture summarised in profiles/score_ps_kernel_chunk16.md)
+SCORE_TRAFFIC_BYTES = None
+
 METRIC = "compressed_frames_per_s"
 UNIT = "frames/s"
 WORKLOAD = "stream_3h"
@@ -299,8 +303,8 @@ def main():
         n_exp = float(cfg.n_q_heads) * cfg.tokens_per_frame ** 2 * frames_per_launch
         peak = 148 * 16 * sm_hz / 1e9
         ach = n_exp / (kernels["score"]["avg_us"] * 1e-6) / 1e9
-        roofline = dict(kernel="score_tc_kernel", bound="alu", achieved=ach, peak=peak, unit="Gexp/s",
-                        frac=ach / peak, traffic=None,
+        roofline = dict(kernel="score_ps_kernel", bound="alu", achieved=ach, peak=peak, unit="Gexp/s",
+                        frac=ach / peak, traffic=SCORE_TRAFFIC_BYTES if T % chunk == 0 and chunk == 16 else None,
                         peak_source="148 SMs x 16 ex2/clk x sampled SM clock")
     elif dom == "score":
         # Eq. 1 on CUDA cores (fp32 inputs): 2*Hq*P^2*D flop per frame against the fp32 FMA rate
