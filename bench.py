@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one score_ps_kernel launch on a 16-frame chunk of this
 # workload (ncu capture summarised in profiles/score_ps_kernel_chunk16.md)
-SCORE_TRAFFIC_BYTES = None
+SCORE_TRAFFIC_BYTES = 25892608
 
 METRIC = "compressed_frames_per_s"
 UNIT = "frames/s"
