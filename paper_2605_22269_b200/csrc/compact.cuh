@@ -10,6 +10,7 @@
 // refreshes that plane of every segment entry the chunk touches: mean over the frames present.
 #pragma once
 #include "common.cuh"
+#include "tc.cuh"
 
 namespace mukv {
 
@@ -35,6 +36,50 @@ struct CompactParams {
   float* seg_entry;               // [max_segs][L][2][C]
   float* seg_key;                 // [max_segs][C]
 };
+
+// Segment entries (Eq. 5 at segment level) of one (layer, K|V) plane for every segment the chunk
+// touches: mean over the frames present.  Run by one whole block.
+__device__ inline void compact_segment_plane(const CompactParams& p, int l, int kv) {
+  const int tid = threadIdx.x;
+  const int C = p.C, kappa = p.kappa;
+  const bool exact = (l == p.L - 1) && (kv == 0);
+  const long long frames_total = p.first_frame + p.n_frames;
+  const long long first_seg = p.first_frame / p.fseg, last_seg = (frames_total - 1) / p.fseg;
+  for (long long u = first_seg; u <= last_seg; ++u) {
+    const long long t0 = u * p.fseg;
+    long long t1 = t0 + p.fseg;
+    if (t1 > frames_total) t1 = frames_total;
+    const int nf = (int)(t1 - t0);
+    for (int col = tid; col < C; col += kCompactThreads) {
+      float m;
+      // eight loads in flight at a time, added in frame order
+      if (exact) {
+        double t = 0.0;
+        for (long long ff = t0; ff < t1; ff += 8) {
+          double x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[i] = ff + i < t1 ? __ldcg(p.frame_ksum + (ff + i) * C + col) : 0.0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) t += x[i];
+        }
+        m = (float)(t / ((double)nf * (double)kappa));
+        p.seg_key[u * C + col] = m;
+      } else {
+        float t = 0.f;
+        for (long long ff = t0; ff < t1; ff += 8) {
+          float x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            x[i] = ff + i < t1 ? __ldcg(p.frame_entry + (((ff + i) * p.L + l) * 2 + kv) * C + col) : 0.f;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) t += x[i];
+        }
+        m = t / (float)nf;
+      }
+      p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = m;
+    }
+  }
+}
 
 // NV = 16-byte vectors per row; the block covers 256/NV rows per pass.
 template <typename T>
@@ -136,42 +181,135 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  const long long frames_total = p.first_frame + p.n_frames;
-  const long long first_seg = p.first_frame / p.fseg, last_seg = (frames_total - 1) / p.fseg;
-  for (long long u = first_seg; u <= last_seg; ++u) {
-    const long long t0 = u * p.fseg;
-    long long t1 = t0 + p.fseg;
-    if (t1 > frames_total) t1 = frames_total;
-    const int nf = (int)(t1 - t0);
-    for (int col = tid; col < C; col += kCompactThreads) {
-      float m;
-      // eight loads in flight at a time, added in frame order
-      if (exact) {
-        double t = 0.0;
-        for (long long ff = t0; ff < t1; ff += 8) {
-          double x[8];
+  compact_segment_plane(p, l, kv);
+}
+
+// compact_bulk_kernel<T>: the same work with the copy done by the bulk-copy engine.  One block per
+// (layer, K|V, frame): the kappa kept rows are fetched with one bulk copy each into shared memory
+// (all in flight at once), leave as ONE contiguous bulk store into the frame's page, and are summed
+// for the pooled entry out of shared memory meanwhile.  Used when the plane fits in shared memory.
+constexpr int kCompactScratchBytes = 16384;      // cross-group partial sums (float or double)
+constexpr int kCompactTailBytes = 2048;          // kept ids, barrier
+
+__host__ inline size_t compact_bulk_smem_bytes(int kappa, int C, int esize) {
+  return ((size_t)kappa * C * esize + 127) / 128 * 128 + kCompactScratchBytes + kCompactTailBytes + 128;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kCompactThreads) compact_bulk_kernel(const CompactParams p, int* status) {
+  constexpr int VE = 16 / sizeof(T);
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = tc::smem_u32(smem_raw);
+  const uint32_t base = (raw + 127u) & ~127u;
+  unsigned char* sm = smem_raw + (base - raw);
+  const int tid = threadIdx.x;
+  const int plane = blockIdx.x;                 // l*2 + kv
+  const int l = plane >> 1, kv = plane & 1;
+  const int f = blockIdx.y;
+  const long long f_abs = p.first_frame + f;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
+    *p.stat_refined += *p.n_flagged;
+    *p.n_flagged = 0;
+  }
+  const int kappa = p.kappa, C = p.C;
+  const uint32_t row_bytes = (uint32_t)C * sizeof(T);
+  const uint32_t rows_bytes = ((uint32_t)kappa * row_bytes + 127u) / 128u * 128u;
+  unsigned char* s_rows = sm;
+  unsigned char* s_scratch = sm + rows_bytes;
+  int* s_kept = reinterpret_cast<int*>(sm + rows_bytes + kCompactScratchBytes);
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(sm + rows_bytes + kCompactScratchBytes + 1024);
+  const uint32_t bar = tc::smem_u32(s_bar);
+  for (int r = tid; r < kappa; r += kCompactThreads) s_kept[r] = p.kept_store[f_abs * kappa + r];
+  if (tid == 0) {
+    tc::mbar_init(bar, 1);
+    tc::fence_mbar_init();
+    tc::mbar_expect_tx(bar, (uint32_t)kappa * row_bytes);
+  }
+  __syncthreads();
+  const unsigned char* src_base =
+      reinterpret_cast<const unsigned char*>(kv ? p.v : p.k) + ((long long)l * p.n_frames + f) * p.P * (long long)row_bytes;
+  for (int r = tid; r < kappa; r += kCompactThreads)
+    tc::bulk_load(base + (uint32_t)r * row_bytes, src_base + (long long)s_kept[r] * row_bytes, row_bytes, bar);
+  const bool landed = tc::mbar_wait(bar, 0) || tc::mbar_wait(bar, 0);
+  const int bad = __syncthreads_or(landed ? 0 : 1);
+  unsigned char* page = p.store + p.page_table[f_abs];
+  if (bad) {
+    if (tid == 0) atomicCAS(status, 0, 6);
+  } else if (tid == 0) {
+    tc::bulk_store(page + (long long)plane * kappa * row_bytes, base, (uint32_t)kappa * row_bytes);
+  }
+  // ---- pooled entry out of shared memory: thread = (row group, 16-byte column)
+  const int NV = C / VE;                        // vectors per row (power of two, <= 256)
+  const int rows_per_pass = kCompactThreads / NV;
+  const int c = tid % NV, r0 = tid / NV;
+  const bool exact = (l == p.L - 1) && (kv == 0);
+  float acc[VE];
+  double acc64[VE];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) x[i] = ff + i < t1 ? __ldcg(p.frame_ksum + (ff + i) * C + col) : 0.0;
+  for (int e = 0; e < VE; ++e) { acc[e] = 0.f; acc64[e] = 0.0; }
+  if (!bad) {
+    for (int r = r0; r < kappa; r += rows_per_pass) {
+      const uint4 x = *reinterpret_cast<const uint4*>(s_rows + (size_t)r * row_bytes + (size_t)c * 16);
+      const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+      float e[VE];
+      if constexpr (sizeof(T) == 2) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) t += x[i];
-        }
-        m = (float)(t / ((double)nf * (double)kappa));
-        p.seg_key[u * C + col] = m;
+        for (int i = 0; i < 4; ++i) { e[(2 * i) % VE] = bf16_lo(w[i]); e[(2 * i + 1) % VE] = bf16_hi(w[i]); }
       } else {
-        float t = 0.f;
-        for (long long ff = t0; ff < t1; ff += 8) {
-          float x[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            x[i] = ff + i < t1 ? __ldcg(p.frame_entry + (((ff + i) * p.L + l) * 2 + kv) * C + col) : 0.f;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) t += x[i];
-        }
-        m = t / (float)nf;
+        for (int i = 0; i < 4; ++i) e[i % VE] = __uint_as_float(w[i]);
       }
-      p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = m;
+      if (exact) {
+#pragma unroll
+        for (int i = 0; i < VE; ++i) acc64[i] += (double)e[i];
+      } else {
+#pragma unroll
+        for (int i = 0; i < VE; ++i) acc[i] += e[i];
+      }
     }
   }
+  // reduce the row groups (fixed order) and write the mean
+  float* s_red = reinterpret_cast<float*>(s_scratch);
+  double* s_red64 = reinterpret_cast<double*>(s_scratch);
+  if (exact) {
+#pragma unroll
+    for (int i = 0; i < VE; ++i) s_red64[tid * VE + i] = acc64[i];
+  } else {
+#pragma unroll
+    for (int i = 0; i < VE; ++i) s_red[tid * VE + i] = acc[i];
+  }
+  __syncthreads();
+  float* fe = p.frame_entry + ((f_abs * p.L + l) * 2 + kv) * C;
+  for (int col = tid; col < C; col += kCompactThreads) {
+    const int cv = col / VE, ce = col % VE;
+    if (exact) {
+      double t = 0.0;
+      for (int g = 0; g < rows_per_pass; ++g) t += s_red64[(g * NV + cv) * VE + ce];
+      p.frame_ksum[f_abs * C + col] = t;
+      const float m = (float)(t / (double)kappa);
+      fe[col] = m;
+      p.frame_key[f_abs * C + col] = m;
+    } else {
+      float t = 0.f;
+      for (int g = 0; g < rows_per_pass; ++g) t += s_red[(g * NV + cv) * VE + ce];
+      fe[col] = t / (float)kappa;
+    }
+  }
+  if (tid == 0 && !bad) tc::bulk_store_wait_read();      // shared memory stays valid until the store has read it
+
+  // ---- segment entries of this plane, by the block that completes the plane
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int old = atomicAdd(p.plane_counter + plane, 1);
+    s_last = (old == p.n_frames - 1);
+    if (s_last) p.plane_counter[plane] = 0;            // ready for the next launch
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  compact_segment_plane(p, l, kv);
 }
 
 }  // namespace mukv
