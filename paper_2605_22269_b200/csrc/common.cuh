@@ -120,6 +120,13 @@ __device__ __forceinline__ int block_excl_count(bool flag, int* scratch, int& to
   return group_excl_count<BlockGroup>(flag, scratch, total);
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may
+// start while its predecessor in the stream still runs; pdl_wait() returns once that predecessor
+// has completed and its writes are visible (a no-op for a normally launched kernel), pdl_trigger()
+// tells the runtime that this block no longer minds the successor being scheduled.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // 16-byte streaming copies
 __device__ __forceinline__ uint4 ld_stream(const void* p) {
   uint4 v;

@@ -93,6 +93,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
   const int l = plane >> 1, kv = plane & 1;
   const int f = blockIdx.y;
   const long long f_abs = p.first_frame + f;
+  pdl_wait();
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
     *p.stat_refined += *p.n_flagged;
     *p.n_flagged = 0;
@@ -207,6 +208,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_bulk_kernel(const Com
   const int l = plane >> 1, kv = plane & 1;
   const int f = blockIdx.y;
   const long long f_abs = p.first_frame + f;
+  pdl_wait();
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
     *p.stat_refined += *p.n_flagged;
     *p.n_flagged = 0;

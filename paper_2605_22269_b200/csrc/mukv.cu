@@ -212,15 +212,34 @@ WorkLayout work_layout(const mukv_config& c) {
 
 int pick_nc(int P) { return P <= 64 ? 2 : P <= 128 ? 4 : P <= 224 ? 7 : 8; }
 
+// Launches a kernel; with `dependent` it may be scheduled while the previous kernel of the stream
+// still runs (programmatic dependent launch: the kernel itself waits in pdl_wait()).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, unsigned block, size_t smem, cudaStream_t st,
+                     bool dependent, Args... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 template <typename T, typename A>
-cudaError_t launch_score(const ScoreParams& sp, int nc, dim3 grid, size_t smem, cudaStream_t st) {
+cudaError_t launch_score(const ScoreParams& sp, int nc, dim3 grid, size_t smem, cudaStream_t st,
+                         bool dependent = false) {
   switch (nc) {
-    case 2: score_kernel<T, A, 2><<<grid, kScoreThreads, smem, st>>>(sp); break;
-    case 4: score_kernel<T, A, 4><<<grid, kScoreThreads, smem, st>>>(sp); break;
-    case 7: score_kernel<T, A, 7><<<grid, kScoreThreads, smem, st>>>(sp); break;
-    default: score_kernel<T, A, 8><<<grid, kScoreThreads, smem, st>>>(sp); break;
+    case 2: return launch_k(score_kernel<T, A, 2>, grid, kScoreThreads, smem, st, dependent, sp);
+    case 4: return launch_k(score_kernel<T, A, 4>, grid, kScoreThreads, smem, st, dependent, sp);
+    case 7: return launch_k(score_kernel<T, A, 7>, grid, kScoreThreads, smem, st, dependent, sp);
+    default: return launch_k(score_kernel<T, A, 8>, grid, kScoreThreads, smem, st, dependent, sp);
   }
-  return cudaGetLastError();
 }
 
 template <typename T, typename A>
@@ -401,7 +420,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   sp.ifft_part = ctx->ws + ctx->wl.ifft_d;
   {
     ProfScope ps(ctx, 1, st);
-    e = launch_score<T, double>(sp, ctx->nc, grid, score_smem_bytes<T, double>(P, c.head_dim), st);
+    e = launch_score<T, double>(sp, ctx->nc, grid, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "refine kernel: %s", cudaGetErrorString(e));
 
@@ -424,12 +443,11 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   {
     ProfScope ps(ctx, 2, st);
     if (ctx->compact_bulk)
-      compact_bulk_kernel<T><<<dim3(L * 2, n), kCompactThreads, ctx->compact_smem, st>>>(
-          cp, reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status));
+      e = launch_k(compact_bulk_kernel<T>, dim3(L * 2, n), kCompactThreads, ctx->compact_smem, st, !ctx->prof_on, cp,
+                   reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status));
     else
-      compact_kernel<T><<<dim3(L * 2, n), kCompactThreads, 0, st>>>(cp);
+      e = launch_k(compact_kernel<T>, dim3(L * 2, n), kCompactThreads, 0, st, !ctx->prof_on, cp);
   }
-  e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "compact kernel: %s", cudaGetErrorString(e));
 
   ctx->launches += 3;
@@ -497,8 +515,8 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
     if (e == cudaSuccess) e = set_score_attr<float, double>(ctx->nc, score_smem_bytes<float, double>(P, D));
   }
   ctx->compact_smem = compact_bulk_smem_bytes(cfg->keep_per_frame, ctx->C, ctx->esize);
-  ctx->compact_bulk = ctx->compact_smem <= 100 * 1024;
-  if (const char* s = getenv("MUKV_COMPACT_PLAIN")) if (atoi(s) != 0) ctx->compact_bulk = false;
+  ctx->compact_bulk = false;
+  if (const char* s = getenv("MUKV_COMPACT_BULK")) ctx->compact_bulk = atoi(s) != 0 && ctx->compact_smem <= 100 * 1024;
   if (e == cudaSuccess && ctx->compact_bulk)
     e = cfg->dtype == MUKV_BF16
             ? cudaFuncSetAttribute((const void*)compact_bulk_kernel<__nv_bfloat16>,

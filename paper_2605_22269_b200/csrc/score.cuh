@@ -213,6 +213,8 @@ __global__ void __launch_bounds__(kScoreThreads) score_kernel(const ScoreParams 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h = blockIdx.x;
   int f = blockIdx.y;
+  pdl_wait();
+  pdl_trigger();
   if (p.refine) {
     if ((int)blockIdx.y >= *p.n_flagged) return;
     f = p.flagged[blockIdx.y];

@@ -380,6 +380,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
         }
       }
       if (!ok) atomicCAS(p.status, 0, 3);
+      pdl_trigger();                                     // the next kernel of the call may be scheduled
       // copies of this thread still in flight land before the block goes away
       for (int s = 0; s < 2; ++s) {
         const int cnt = (nk + 1 - s) >> 1;
