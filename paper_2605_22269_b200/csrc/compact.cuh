@@ -185,71 +185,117 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
   compact_segment_plane(p, l, kv);
 }
 
-// compact_bulk_kernel<T>: the same work with the copy done by the bulk-copy engine.  One block per
-// (layer, K|V, frame): the kappa kept rows are fetched with one bulk copy each into shared memory
-// (all in flight at once), leave as ONE contiguous bulk store into the frame's page, and are summed
-// for the pooled entry out of shared memory meanwhile.  Used when the plane fits in shared memory.
-constexpr int kCompactScratchBytes = 16384;      // cross-group partial sums (float or double)
-constexpr int kCompactTailBytes = 2048;          // kept ids, barrier
+// compact_stream_kernel<T>: the same work as a persistent, pipelined stream through the bulk-copy
+// engine.  One block per SM walks its share of the (layer, K|V, frame) planes.  The kappa kept rows
+// of a plane are fetched with one bulk copy each into one of `n_buf` shared-memory buffers, leave as
+// ONE contiguous bulk store into the frame's page, and are summed for the pooled entry out of shared
+// memory meanwhile; the rows of the next planes are already in flight.  Used when at least two
+// planes fit in shared memory.
+constexpr int kStreamScratchBytes = 8192;        // cross-group partial sums
+constexpr int kStreamMaxBufs = 4;
+constexpr int kStreamMaxItems = 64;              // planes per block
 
-__host__ inline size_t compact_bulk_smem_bytes(int kappa, int C, int esize) {
-  return ((size_t)kappa * C * esize + 127) / 128 * 128 + kCompactScratchBytes + kCompactTailBytes + 128;
+struct StreamShape {
+  int n_buf;                                     // 0: does not fit
+  int grid;
+  size_t smem;
+};
+
+__host__ inline StreamShape compact_stream_shape(int kappa, int C, int esize, int n_planes, int n_sms, size_t limit) {
+  StreamShape sh;
+  sh.n_buf = 0; sh.grid = 0; sh.smem = 0;
+  const size_t rows = ((size_t)kappa * C * esize + 127) / 128 * 128;
+  int grid = n_sms < n_planes ? n_sms : n_planes;
+  if (grid < 1) grid = 1;
+  const int per_block = (n_planes + grid - 1) / grid;
+  if (per_block > kStreamMaxItems) return sh;
+  const size_t fixed = kStreamScratchBytes + (size_t)per_block * kappa * sizeof(int) + 256 + 128;
+  for (int nb = kStreamMaxBufs; nb >= 2; --nb) {
+    if (nb * rows + fixed <= limit) { sh.n_buf = nb; sh.grid = grid; sh.smem = nb * rows + fixed; return sh; }
+  }
+  return sh;
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kCompactThreads) compact_bulk_kernel(const CompactParams p, int* status) {
+__global__ void __launch_bounds__(kCompactThreads, 1) compact_stream_kernel(const CompactParams p, int n_buf,
+                                                                           int* status) {
   constexpr int VE = 16 / sizeof(T);
   extern __shared__ unsigned char smem_raw[];
+  __shared__ int s_done[kStreamMaxItems];           // planes whose last frame this block finished
+  __shared__ int s_ndone;
   const uint32_t raw = tc::smem_u32(smem_raw);
   const uint32_t base = (raw + 127u) & ~127u;
   unsigned char* sm = smem_raw + (base - raw);
-  const int tid = threadIdx.x;
-  const int plane = blockIdx.x;                 // l*2 + kv
-  const int l = plane >> 1, kv = plane & 1;
-  const int f = blockIdx.y;
-  const long long f_abs = p.first_frame + f;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int kappa = p.kappa, C = p.C;
+  const int n_planes = p.L * 2 * p.n_frames;
+  const uint32_t row_bytes = (uint32_t)C * sizeof(T);
+  const uint32_t rows_bytes = ((uint32_t)kappa * row_bytes + 127u) / 128u * 128u;
+  const int n_my = (n_planes - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // items b, b+grid, ...
+  unsigned char* s_scratch = sm + (size_t)n_buf * rows_bytes;
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_scratch + kStreamScratchBytes);        // [kStreamMaxBufs]
+  int* s_kept = reinterpret_cast<int*>(s_scratch + kStreamScratchBytes + 256);           // [n_my][kappa]
   pdl_wait();
-  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
+  if (blockIdx.x == 0 && tid == 0) {
     *p.stat_refined += *p.n_flagged;
     *p.n_flagged = 0;
   }
-  const int kappa = p.kappa, C = p.C;
-  const uint32_t row_bytes = (uint32_t)C * sizeof(T);
-  const uint32_t rows_bytes = ((uint32_t)kappa * row_bytes + 127u) / 128u * 128u;
-  unsigned char* s_rows = sm;
-  unsigned char* s_scratch = sm + rows_bytes;
-  int* s_kept = reinterpret_cast<int*>(sm + rows_bytes + kCompactScratchBytes);
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(sm + rows_bytes + kCompactScratchBytes + 1024);
-  const uint32_t bar = tc::smem_u32(s_bar);
-  for (int r = tid; r < kappa; r += kCompactThreads) s_kept[r] = p.kept_store[f_abs * kappa + r];
   if (tid == 0) {
-    tc::mbar_init(bar, 1);
+    for (int b = 0; b < kStreamMaxBufs; ++b) tc::mbar_init(tc::smem_u32(&s_bar[b]), 1);
     tc::fence_mbar_init();
-    tc::mbar_expect_tx(bar, (uint32_t)kappa * row_bytes);
+    s_ndone = 0;
+  }
+  // item k of this block is plane (blockIdx.x + k*gridDim.x): frame-major, so neighbouring blocks
+  // work on the same frame
+  for (int i = tid; i < n_my * kappa; i += kCompactThreads) {
+    const int k = i / kappa, r = i % kappa;
+    const int item = blockIdx.x + k * gridDim.x;
+    const int f = item / (p.L * 2);
+    s_kept[i] = p.kept_store[(p.first_frame + f) * kappa + r];
   }
   __syncthreads();
-  const unsigned char* src_base =
-      reinterpret_cast<const unsigned char*>(kv ? p.v : p.k) + ((long long)l * p.n_frames + f) * p.P * (long long)row_bytes;
-  for (int r = tid; r < kappa; r += kCompactThreads)
-    tc::bulk_load(base + (uint32_t)r * row_bytes, src_base + (long long)s_kept[r] * row_bytes, row_bytes, bar);
-  const bool landed = tc::mbar_wait(bar, 0) || tc::mbar_wait(bar, 0);
-  const int bad = __syncthreads_or(landed ? 0 : 1);
-  unsigned char* page = p.store + p.page_table[f_abs];
-  if (bad) {
-    if (tid == 0) atomicCAS(status, 0, 6);
-  } else if (tid == 0) {
-    tc::bulk_store(page + (long long)plane * kappa * row_bytes, base, (uint32_t)kappa * row_bytes);
-  }
-  // ---- pooled entry out of shared memory: thread = (row group, 16-byte column)
-  const int NV = C / VE;                        // vectors per row (power of two, <= 256)
+
+  // warp 0 issues the row copies of item k into buffer k % n_buf
+  auto issue_loads = [&](int k) {
+    const int item = blockIdx.x + k * gridDim.x;
+    const int f = item / (p.L * 2), plane = item % (p.L * 2);
+    const int l = plane >> 1, kv = plane & 1;
+    const uint32_t bar = tc::smem_u32(&s_bar[k % n_buf]);
+    const uint32_t dst = base + (uint32_t)(k % n_buf) * rows_bytes;
+    const unsigned char* src_base = reinterpret_cast<const unsigned char*>(kv ? p.v : p.k) +
+                                    ((long long)l * p.n_frames + f) * p.P * (long long)row_bytes;
+    if (lane == 0) tc::mbar_expect_tx(bar, (uint32_t)kappa * row_bytes);
+    __syncwarp();
+    for (int r = lane; r < kappa; r += 32)
+      tc::bulk_load(dst + (uint32_t)r * row_bytes, src_base + (long long)s_kept[k * kappa + r] * row_bytes, row_bytes, bar);
+  };
+  if (warp == 0)
+    for (int k = 0; k < n_buf && k < n_my; ++k) issue_loads(k);
+
+  const int NV = C / VE;                        // 16-byte vectors per row (power of two, <= 256)
   const int rows_per_pass = kCompactThreads / NV;
   const int c = tid % NV, r0 = tid / NV;
-  const bool exact = (l == p.L - 1) && (kv == 0);
-  float acc[VE];
-  double acc64[VE];
+  bool failed = false;
+  int pend_plane = -1, pend_old = 0;            // arrival of the previous item, looked at one item later
+  for (int k = 0; k < n_my; ++k) {
+    const int item = blockIdx.x + k * gridDim.x;
+    const int f = item / (p.L * 2), plane = item % (p.L * 2);
+    const int l = plane >> 1, kv = plane & 1;
+    const long long f_abs = p.first_frame + f;
+    const int b = k % n_buf;
+    const uint32_t ph = (uint32_t)((k / n_buf) & 1);
+    const bool landed = tc::mbar_wait(tc::smem_u32(&s_bar[b]), ph) || tc::mbar_wait(tc::smem_u32(&s_bar[b]), ph);
+    if (__syncthreads_or(landed ? 0 : 1)) { failed = true; break; }
+    const unsigned char* s_rows = sm + (size_t)b * rows_bytes;
+    if (tid == 0)
+      tc::bulk_store(p.store + p.page_table[f_abs] + (long long)plane * kappa * row_bytes,
+                     base + (uint32_t)b * rows_bytes, (uint32_t)kappa * row_bytes);
+    // ---- pooled entry out of shared memory: thread = (row group, 16-byte column)
+    const bool exact = (l == p.L - 1) && (kv == 0);
+    float acc[VE];
+    double acc64[VE];
 #pragma unroll
-  for (int e = 0; e < VE; ++e) { acc[e] = 0.f; acc64[e] = 0.0; }
-  if (!bad) {
+    for (int e = 0; e < VE; ++e) { acc[e] = 0.f; acc64[e] = 0.0; }
     for (int r = r0; r < kappa; r += rows_per_pass) {
       const uint4 x = *reinterpret_cast<const uint4*>(s_rows + (size_t)r * row_bytes + (size_t)c * 16);
       const uint32_t w[4] = {x.x, x.y, x.z, x.w};
@@ -269,49 +315,71 @@ __global__ void __launch_bounds__(kCompactThreads) compact_bulk_kernel(const Com
         for (int i = 0; i < VE; ++i) acc[i] += e[i];
       }
     }
-  }
-  // reduce the row groups (fixed order) and write the mean
-  float* s_red = reinterpret_cast<float*>(s_scratch);
-  double* s_red64 = reinterpret_cast<double*>(s_scratch);
-  if (exact) {
+    float* fe = p.frame_entry + ((f_abs * p.L + l) * 2 + kv) * C;
+    if (!exact) {
+      float* s_red = reinterpret_cast<float*>(s_scratch);           // [256 threads][VE] <= 8 KB
 #pragma unroll
-    for (int i = 0; i < VE; ++i) s_red64[tid * VE + i] = acc64[i];
-  } else {
-#pragma unroll
-    for (int i = 0; i < VE; ++i) s_red[tid * VE + i] = acc[i];
-  }
-  __syncthreads();
-  float* fe = p.frame_entry + ((f_abs * p.L + l) * 2 + kv) * C;
-  for (int col = tid; col < C; col += kCompactThreads) {
-    const int cv = col / VE, ce = col % VE;
-    if (exact) {
-      double t = 0.0;
-      for (int g = 0; g < rows_per_pass; ++g) t += s_red64[(g * NV + cv) * VE + ce];
-      p.frame_ksum[f_abs * C + col] = t;
-      const float m = (float)(t / (double)kappa);
-      fe[col] = m;
-      p.frame_key[f_abs * C + col] = m;
+      for (int i = 0; i < VE; ++i) s_red[tid * VE + i] = acc[i];
+      __syncthreads();
+      for (int col = tid; col < C; col += kCompactThreads) {
+        const int cv = col / VE, ce = col % VE;
+        float t = 0.f;
+        for (int g = 0; g < rows_per_pass; ++g) t += s_red[(g * NV + cv) * VE + ce];
+        fe[col] = t / (float)kappa;
+      }
     } else {
-      float t = 0.f;
-      for (int g = 0; g < rows_per_pass; ++g) t += s_red[(g * NV + cv) * VE + ce];
-      fe[col] = t / (float)kappa;
+      // the last-layer keys are summed in double (their mean ranks blocks later); the scratch holds
+      // half of the threads' partial sums at a time
+      double* s_red64 = reinterpret_cast<double*>(s_scratch);       // [128 threads][VE] <= 8 KB
+      for (int half = 0; half < 2; ++half) {
+        if ((tid & 1) == half) {
+#pragma unroll
+          for (int i = 0; i < VE; ++i) s_red64[(tid >> 1) * VE + i] = acc64[i];
+        }
+        __syncthreads();
+        // thread t = g*NV + cv wrote slot t>>1 when (t & 1) == half: columns with (cv & 1) == half
+        for (int col = tid; col < C; col += kCompactThreads) {
+          const int cv = col / VE, ce = col % VE;
+          if ((cv & 1) != half) continue;
+          double t = 0.0;
+          for (int g = 0; g < rows_per_pass; ++g) t += s_red64[((g * NV + cv) >> 1) * VE + ce];
+          p.frame_ksum[f_abs * C + col] = t;
+          const float m = (float)(t / (double)kappa);
+          fe[col] = m;
+          p.frame_key[f_abs * C + col] = m;
+        }
+        __syncthreads();
+      }
+    }
+    // ---- the plane's arrival counter (the result is looked at during the next item)
+    __threadfence();
+    __syncthreads();                            // every thread has read the buffer and written its entries
+    if (tid == 0) {
+      if (pend_plane >= 0 && pend_old == p.n_frames - 1) s_done[s_ndone++] = pend_plane;
+      pend_old = atomicAdd(p.plane_counter + plane, 1);
+      pend_plane = plane;
+      // refill the buffer once the store has read it
+      tc::bulk_store_wait_read();
+    }
+    if (k + n_buf < n_my) {
+      __syncthreads();                          // thread 0 has seen the store leave shared memory
+      if (warp == 0) issue_loads(k + n_buf);
     }
   }
-  if (tid == 0 && !bad) tc::bulk_store_wait_read();      // shared memory stays valid until the store has read it
-
-  // ---- segment entries of this plane, by the block that completes the plane
-  __shared__ int s_last;
-  __threadfence();
-  __syncthreads();
   if (tid == 0) {
-    const int old = atomicAdd(p.plane_counter + plane, 1);
-    s_last = (old == p.n_frames - 1);
-    if (s_last) p.plane_counter[plane] = 0;            // ready for the next launch
+    if (failed) atomicCAS(status, 0, 6);
+    if (pend_plane >= 0 && pend_old == p.n_frames - 1) s_done[s_ndone++] = pend_plane;
+    tc::bulk_store_wait_read();
   }
   __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  compact_segment_plane(p, l, kv);
+  // ---- segment entries of the planes this block completed
+  const int nd = s_ndone;
+  if (nd > 0) __threadfence();
+  for (int i = 0; i < nd; ++i) {
+    const int plane = s_done[i];
+    if (tid == 0) p.plane_counter[plane] = 0;          // ready for the next launch
+    compact_segment_plane(p, plane >> 1, plane & 1);
+  }
 }
 
 }  // namespace mukv

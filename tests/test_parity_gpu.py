@@ -157,9 +157,9 @@ def test_chunk7b_tile_block_scoring(monkeypatch):
     assert run.ctx.mukv_get_stats().device_status == 0
 
 
-def test_chunk7b_bulk_copy_compaction(monkeypatch):
-    # compaction through the bulk-copy engine (optional variant) instead of register copies
-    monkeypatch.setenv("MUKV_COMPACT_BULK", "1")
+def test_chunk7b_plain_compaction(monkeypatch):
+    # compaction with register copies (the kernel used when two planes do not fit in shared memory)
+    monkeypatch.setenv("MUKV_COMPACT_PLAIN", "1")
     run = H.GpuRun("chunk7b", n_frames=5)
     full_compress_check(run)
 
