@@ -194,6 +194,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
 constexpr int kStreamScratchBytes = 8192;        // cross-group partial sums
 constexpr int kStreamMaxBufs = 4;
 constexpr int kStreamMaxItems = 64;              // planes per block
+constexpr int kStreamSmemLimit = 226 * 1024;     // dynamic shared memory (the kernel also has a little static)
 
 struct StreamShape {
   int n_buf;                                     // 0: does not fit

@@ -442,7 +442,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   {
     ProfScope ps(ctx, 2, st);
     const StreamShape sh = ctx->compact_stream
-                               ? compact_stream_shape(c.keep_per_frame, C, ctx->esize, L * 2 * n, ctx->n_sms, 227 * 1024)
+                               ? compact_stream_shape(c.keep_per_frame, C, ctx->esize, L * 2 * n, ctx->n_sms, kStreamSmemLimit)
                                : StreamShape{0, 0, 0};
     if (sh.n_buf >= 2)
       e = launch_k(compact_stream_kernel<T>, dim3(sh.grid), kCompactThreads, sh.smem, st, !ctx->prof_on, cp, sh.n_buf,
@@ -521,9 +521,9 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
   if (e == cudaSuccess && ctx->compact_stream)
     e = cfg->dtype == MUKV_BF16
             ? cudaFuncSetAttribute((const void*)compact_stream_kernel<__nv_bfloat16>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemLimit)
             : cudaFuncSetAttribute((const void*)compact_stream_kernel<float>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemLimit);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute((const void*)rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRankStageBytes);
   if (e == cudaSuccess && ctx->tcs.ok) {
