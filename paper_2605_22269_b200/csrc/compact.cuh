@@ -6,11 +6,12 @@
 // token order, to the frame's page; the same registers feed the mean over the kept rows.
 // The last-layer key plane is summed in double: its mean is the retrieval key (Eq. 5) that
 // later ranks blocks, so it is kept free of accumulation-order noise.
+// compact_kernel keeps the rows in registers between load and store (any plane size);
+// compact_async_kernel lands them in shared memory first (planes that fit).
 // The block that finishes a (layer, K|V) plane of the chunk last (arrival counter, nobody waits)
 // refreshes that plane of every segment entry the chunk touches: mean over the frames present.
 #pragma once
 #include "common.cuh"
-#include "tc.cuh"
 
 namespace mukv {
 
@@ -185,202 +186,119 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
   compact_segment_plane(p, l, kv);
 }
 
-// compact_stream_kernel<T>: the same work as a persistent, pipelined stream through the bulk-copy
-// engine.  One block per SM walks its share of the (layer, K|V, frame) planes.  The kappa kept rows
-// of a plane are fetched with one bulk copy each into one of `n_buf` shared-memory buffers, leave as
-// ONE contiguous bulk store into the frame's page, and are summed for the pooled entry out of shared
-// memory meanwhile; the rows of the next planes are already in flight.  Used when at least two
-// planes fit in shared memory.
-constexpr int kStreamScratchBytes = 8192;        // cross-group partial sums
-constexpr int kStreamMaxBufs = 4;
-constexpr int kStreamMaxItems = 64;              // planes per block
-constexpr int kStreamSmemLimit = 226 * 1024;     // dynamic shared memory (the kernel also has a little static)
-
-struct StreamShape {
-  int n_buf;                                     // 0: does not fit
-  int grid;
-  size_t smem;
-};
-
-__host__ inline StreamShape compact_stream_shape(int kappa, int C, int esize, int n_planes, int n_sms, size_t limit) {
-  StreamShape sh;
-  sh.n_buf = 0; sh.grid = 0; sh.smem = 0;
-  const size_t rows = ((size_t)kappa * C * esize + 127) / 128 * 128;
-  int grid = n_sms < n_planes ? n_sms : n_planes;
-  if (grid < 1) grid = 1;
-  const int per_block = (n_planes + grid - 1) / grid;
-  if (per_block > kStreamMaxItems) return sh;
-  const size_t fixed = kStreamScratchBytes + (size_t)per_block * kappa * sizeof(int) + 256 + 128;
-  for (int nb = kStreamMaxBufs; nb >= 2; --nb) {
-    if (nb * rows + fixed <= limit) { sh.n_buf = nb; sh.grid = grid; sh.smem = nb * rows + fixed; return sh; }
-  }
-  return sh;
+// compact_async_kernel<T>: the same work with the kept rows of a plane landed in shared memory by
+// asynchronous 16-byte copies (cp.async), all of them in flight at once, four blocks per SM.  From
+// shared memory each row leaves for the frame's page as streaming 16-byte stores, and each thread
+// sums its own 32-bit column over the rows in row order: no registers tied up by loads in flight
+// and no cross-thread reduction.  Used when the plane fits in shared memory.
+__host__ inline size_t compact_async_smem_bytes(int kappa, int C, int esize) {
+  return ((size_t)kappa * C * esize + 127) / 128 * 128 + (size_t)kappa * sizeof(int) + 256;
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kCompactThreads, 1) compact_stream_kernel(const CompactParams p, int n_buf,
-                                                                           int* status) {
-  constexpr int VE = 16 / sizeof(T);
-  extern __shared__ unsigned char smem_raw[];
-  __shared__ int s_done[kStreamMaxItems];           // planes whose last frame this block finished
-  __shared__ int s_ndone;
-  const uint32_t raw = tc::smem_u32(smem_raw);
-  const uint32_t base = (raw + 127u) & ~127u;
-  unsigned char* sm = smem_raw + (base - raw);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int kappa = p.kappa, C = p.C;
-  const int n_planes = p.L * 2 * p.n_frames;
-  const uint32_t row_bytes = (uint32_t)C * sizeof(T);
-  const uint32_t rows_bytes = ((uint32_t)kappa * row_bytes + 127u) / 128u * 128u;
-  const int n_my = (n_planes - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // items b, b+grid, ...
-  unsigned char* s_scratch = sm + (size_t)n_buf * rows_bytes;
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(s_scratch + kStreamScratchBytes);        // [kStreamMaxBufs]
-  int* s_kept = reinterpret_cast<int*>(s_scratch + kStreamScratchBytes + 256);           // [n_my][kappa]
+__global__ void __launch_bounds__(kCompactThreads) compact_async_kernel(const CompactParams p) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int tid = threadIdx.x;
+  const int plane = blockIdx.x;                 // l*2 + kv
+  const int l = plane >> 1, kv = plane & 1;
+  const int f = blockIdx.y;
+  const long long f_abs = p.first_frame + f;
   pdl_wait();
-  if (blockIdx.x == 0 && tid == 0) {
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
     *p.stat_refined += *p.n_flagged;
     *p.n_flagged = 0;
   }
-  if (tid == 0) {
-    for (int b = 0; b < kStreamMaxBufs; ++b) tc::mbar_init(tc::smem_u32(&s_bar[b]), 1);
-    tc::fence_mbar_init();
-    s_ndone = 0;
-  }
-  // item k of this block is plane (blockIdx.x + k*gridDim.x): frame-major, so neighbouring blocks
-  // work on the same frame
-  for (int i = tid; i < n_my * kappa; i += kCompactThreads) {
-    const int k = i / kappa, r = i % kappa;
-    const int item = blockIdx.x + k * gridDim.x;
-    const int f = item / (p.L * 2);
-    s_kept[i] = p.kept_store[(p.first_frame + f) * kappa + r];
-  }
+  const int kappa = p.kappa, C = p.C;
+  const uint32_t row_bytes = (uint32_t)C * sizeof(T);
+  const uint32_t rows_bytes = ((uint32_t)kappa * row_bytes + 127u) / 128u * 128u;
+  unsigned char* s_rows = smem_raw;
+  int* s_kept = reinterpret_cast<int*>(smem_raw + rows_bytes);
+  for (int r = tid; r < kappa; r += kCompactThreads) s_kept[r] = p.kept_store[f_abs * kappa + r];
+  unsigned char* page = p.store + p.page_table[f_abs];
   __syncthreads();
-
-  // warp 0 issues the row copies of item k into buffer k % n_buf
-  auto issue_loads = [&](int k) {
-    const int item = blockIdx.x + k * gridDim.x;
-    const int f = item / (p.L * 2), plane = item % (p.L * 2);
-    const int l = plane >> 1, kv = plane & 1;
-    const uint32_t bar = tc::smem_u32(&s_bar[k % n_buf]);
-    const uint32_t dst = base + (uint32_t)(k % n_buf) * rows_bytes;
-    const unsigned char* src_base = reinterpret_cast<const unsigned char*>(kv ? p.v : p.k) +
-                                    ((long long)l * p.n_frames + f) * p.P * (long long)row_bytes;
-    if (lane == 0) tc::mbar_expect_tx(bar, (uint32_t)kappa * row_bytes);
-    __syncwarp();
-    for (int r = lane; r < kappa; r += 32)
-      tc::bulk_load(dst + (uint32_t)r * row_bytes, src_base + (long long)s_kept[k * kappa + r] * row_bytes, row_bytes, bar);
-  };
-  if (warp == 0)
-    for (int k = 0; k < n_buf && k < n_my; ++k) issue_loads(k);
-
-  const int NV = C / VE;                        // 16-byte vectors per row (power of two, <= 256)
-  const int rows_per_pass = kCompactThreads / NV;
-  const int c = tid % NV, r0 = tid / NV;
-  bool failed = false;
-  int pend_plane = -1, pend_old = 0;            // arrival of the previous item, looked at one item later
-  for (int k = 0; k < n_my; ++k) {
-    const int item = blockIdx.x + k * gridDim.x;
-    const int f = item / (p.L * 2), plane = item % (p.L * 2);
-    const int l = plane >> 1, kv = plane & 1;
-    const long long f_abs = p.first_frame + f;
-    const int b = k % n_buf;
-    const uint32_t ph = (uint32_t)((k / n_buf) & 1);
-    const bool landed = tc::mbar_wait(tc::smem_u32(&s_bar[b]), ph) || tc::mbar_wait(tc::smem_u32(&s_bar[b]), ph);
-    if (__syncthreads_or(landed ? 0 : 1)) { failed = true; break; }
-    const unsigned char* s_rows = sm + (size_t)b * rows_bytes;
-    if (tid == 0)
-      tc::bulk_store(p.store + p.page_table[f_abs] + (long long)plane * kappa * row_bytes,
-                     base + (uint32_t)b * rows_bytes, (uint32_t)kappa * row_bytes);
-    // ---- pooled entry out of shared memory: thread = (row group, 16-byte column)
-    const bool exact = (l == p.L - 1) && (kv == 0);
-    float acc[VE];
-    double acc64[VE];
-#pragma unroll
-    for (int e = 0; e < VE; ++e) { acc[e] = 0.f; acc64[e] = 0.0; }
-    for (int r = r0; r < kappa; r += rows_per_pass) {
-      const uint4 x = *reinterpret_cast<const uint4*>(s_rows + (size_t)r * row_bytes + (size_t)c * 16);
-      const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-      float e[VE];
-      if constexpr (sizeof(T) == 2) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { e[(2 * i) % VE] = bf16_lo(w[i]); e[(2 * i + 1) % VE] = bf16_hi(w[i]); }
-      } else {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) e[i % VE] = __uint_as_float(w[i]);
-      }
+  const unsigned char* src_base = reinterpret_cast<const unsigned char*>(kv ? p.v : p.k) +
+                                  ((long long)l * p.n_frames + f) * p.P * (long long)row_bytes;
+  const int vec_per_row = (int)(row_bytes >> 4);
+  const int n_vec = kappa * vec_per_row;
+  const uint32_t s_base = (uint32_t)__cvta_generic_to_shared(s_rows);
+  for (int v = tid; v < n_vec; v += kCompactThreads) {
+    const int r = v / vec_per_row, cvec = v % vec_per_row;
+    const unsigned char* src = src_base + (long long)s_kept[r] * row_bytes + ((long long)cvec << 4);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s_base + ((uint32_t)v << 4)), "l"(src) : "memory");
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+  // ---- the rows leave for the page (one contiguous run: kept rows in ascending token order)
+  unsigned char* dst = page + (long long)plane * kappa * row_bytes;
+  for (int v = tid; v < n_vec; v += kCompactThreads)
+    st_stream(dst + ((long long)v << 4), *reinterpret_cast<const uint4*>(s_rows + ((size_t)v << 4)));
+  // ---- pooled entry: thread = one 32-bit column, rows added in order
+  const bool exact = (l == p.L - 1) && (kv == 0);
+  const int words = (int)(row_bytes >> 2);
+  float* fe = p.frame_entry + ((f_abs * p.L + l) * 2 + kv) * C;
+  const uint32_t* s_w = reinterpret_cast<const uint32_t*>(s_rows);
+  for (int w = tid; w < words; w += kCompactThreads) {
+    if constexpr (sizeof(T) == 2) {
       if (exact) {
-#pragma unroll
-        for (int i = 0; i < VE; ++i) acc64[i] += (double)e[i];
+        double a = 0.0, b = 0.0;
+        for (int r = 0; r < kappa; ++r) {
+          const uint32_t x = s_w[(size_t)r * words + w];
+          a += (double)bf16_lo(x);
+          b += (double)bf16_hi(x);
+        }
+        p.frame_ksum[f_abs * C + 2 * w] = a;
+        p.frame_ksum[f_abs * C + 2 * w + 1] = b;
+        const float ma = (float)(a / (double)kappa), mb = (float)(b / (double)kappa);
+        fe[2 * w] = ma; fe[2 * w + 1] = mb;
+        p.frame_key[f_abs * C + 2 * w] = ma;
+        p.frame_key[f_abs * C + 2 * w + 1] = mb;
       } else {
-#pragma unroll
-        for (int i = 0; i < VE; ++i) acc[i] += e[i];
-      }
-    }
-    float* fe = p.frame_entry + ((f_abs * p.L + l) * 2 + kv) * C;
-    if (!exact) {
-      float* s_red = reinterpret_cast<float*>(s_scratch);           // [256 threads][VE] <= 8 KB
-#pragma unroll
-      for (int i = 0; i < VE; ++i) s_red[tid * VE + i] = acc[i];
-      __syncthreads();
-      for (int col = tid; col < C; col += kCompactThreads) {
-        const int cv = col / VE, ce = col % VE;
-        float t = 0.f;
-        for (int g = 0; g < rows_per_pass; ++g) t += s_red[(g * NV + cv) * VE + ce];
-        fe[col] = t / (float)kappa;
+        float a0 = 0.f, b0 = 0.f, a1 = 0.f, b1 = 0.f;        // two partial sums per column: shorter add chains
+        int r = 0;
+        for (; r + 1 < kappa; r += 2) {
+          const uint32_t x = s_w[(size_t)r * words + w], y = s_w[(size_t)(r + 1) * words + w];
+          a0 += bf16_lo(x); b0 += bf16_hi(x);
+          a1 += bf16_lo(y); b1 += bf16_hi(y);
+        }
+        if (r < kappa) { const uint32_t x = s_w[(size_t)r * words + w]; a0 += bf16_lo(x); b0 += bf16_hi(x); }
+        fe[2 * w] = (a0 + a1) / (float)kappa;
+        fe[2 * w + 1] = (b0 + b1) / (float)kappa;
       }
     } else {
-      // the last-layer keys are summed in double (their mean ranks blocks later); the scratch holds
-      // half of the threads' partial sums at a time
-      double* s_red64 = reinterpret_cast<double*>(s_scratch);       // [128 threads][VE] <= 8 KB
-      for (int half = 0; half < 2; ++half) {
-        if ((tid & 1) == half) {
-#pragma unroll
-          for (int i = 0; i < VE; ++i) s_red64[(tid >> 1) * VE + i] = acc64[i];
+      if (exact) {
+        double a = 0.0;
+        for (int r = 0; r < kappa; ++r) a += (double)__uint_as_float(s_w[(size_t)r * words + w]);
+        p.frame_ksum[f_abs * C + w] = a;
+        const float m = (float)(a / (double)kappa);
+        fe[w] = m;
+        p.frame_key[f_abs * C + w] = m;
+      } else {
+        float a0 = 0.f, a1 = 0.f;
+        int r = 0;
+        for (; r + 1 < kappa; r += 2) {
+          a0 += __uint_as_float(s_w[(size_t)r * words + w]);
+          a1 += __uint_as_float(s_w[(size_t)(r + 1) * words + w]);
         }
-        __syncthreads();
-        // thread t = g*NV + cv wrote slot t>>1 when (t & 1) == half: columns with (cv & 1) == half
-        for (int col = tid; col < C; col += kCompactThreads) {
-          const int cv = col / VE, ce = col % VE;
-          if ((cv & 1) != half) continue;
-          double t = 0.0;
-          for (int g = 0; g < rows_per_pass; ++g) t += s_red64[((g * NV + cv) >> 1) * VE + ce];
-          p.frame_ksum[f_abs * C + col] = t;
-          const float m = (float)(t / (double)kappa);
-          fe[col] = m;
-          p.frame_key[f_abs * C + col] = m;
-        }
-        __syncthreads();
+        if (r < kappa) a0 += __uint_as_float(s_w[(size_t)r * words + w]);
+        fe[w] = (a0 + a1) / (float)kappa;
       }
     }
-    // ---- the plane's arrival counter (the result is looked at during the next item)
-    __threadfence();
-    __syncthreads();                            // every thread has read the buffer and written its entries
-    if (tid == 0) {
-      if (pend_plane >= 0 && pend_old == p.n_frames - 1) s_done[s_ndone++] = pend_plane;
-      pend_old = atomicAdd(p.plane_counter + plane, 1);
-      pend_plane = plane;
-      // refill the buffer once the store has read it
-      tc::bulk_store_wait_read();
-    }
-    if (k + n_buf < n_my) {
-      __syncthreads();                          // thread 0 has seen the store leave shared memory
-      if (warp == 0) issue_loads(k + n_buf);
-    }
   }
+
+  // ---- segment entries of this plane, by the block that completes the plane
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
   if (tid == 0) {
-    if (failed) atomicCAS(status, 0, 6);
-    if (pend_plane >= 0 && pend_old == p.n_frames - 1) s_done[s_ndone++] = pend_plane;
-    tc::bulk_store_wait_read();
+    const int old = atomicAdd(p.plane_counter + plane, 1);
+    s_last = (old == p.n_frames - 1);
+    if (s_last) p.plane_counter[plane] = 0;            // ready for the next launch
   }
   __syncthreads();
-  // ---- segment entries of the planes this block completed
-  const int nd = s_ndone;
-  if (nd > 0) __threadfence();
-  for (int i = 0; i < nd; ++i) {
-    const int plane = s_done[i];
-    if (tid == 0) p.plane_counter[plane] = 0;          // ready for the next launch
-    compact_segment_plane(p, plane >> 1, plane & 1);
-  }
+  if (!s_last) return;
+  __threadfence();
+  compact_segment_plane(p, l, kv);
 }
 
 }  // namespace mukv

@@ -65,7 +65,8 @@ struct mukv_ctx {
   float flag_margin, flat_ratio;
   TcShape tcs;                           // tcs.ok: the chunk is scored on the tensor cores
   int n_sms;
-  bool compact_stream;                   // compaction as a pipelined stream through the bulk-copy engine
+  bool compact_async;                    // compaction through shared memory (the plane fits)
+  size_t compact_smem;
   CUtensorMap wmap;                      // DFT matrix terms [3*D][D] bf16
   std::string err;
   // optional per-kernel timing (host objects only)
@@ -441,12 +442,8 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   cp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
   {
     ProfScope ps(ctx, 2, st);
-    const StreamShape sh = ctx->compact_stream
-                               ? compact_stream_shape(c.keep_per_frame, C, ctx->esize, L * 2 * n, ctx->n_sms, kStreamSmemLimit)
-                               : StreamShape{0, 0, 0};
-    if (sh.n_buf >= 2)
-      e = launch_k(compact_stream_kernel<T>, dim3(sh.grid), kCompactThreads, sh.smem, st, !ctx->prof_on, cp, sh.n_buf,
-                   reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status));
+    if (ctx->compact_async)
+      e = launch_k(compact_async_kernel<T>, dim3(L * 2, n), kCompactThreads, ctx->compact_smem, st, !ctx->prof_on, cp);
     else
       e = launch_k(compact_kernel<T>, dim3(L * 2, n), kCompactThreads, 0, st, !ctx->prof_on, cp);
   }
@@ -516,14 +513,15 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
     e = set_score_attr<float, float>(ctx->nc, score_smem_bytes<float, float>(P, D));
     if (e == cudaSuccess) e = set_score_attr<float, double>(ctx->nc, score_smem_bytes<float, double>(P, D));
   }
-  ctx->compact_stream = true;
-  if (const char* s = getenv("MUKV_COMPACT_PLAIN")) if (atoi(s) != 0) ctx->compact_stream = false;
-  if (e == cudaSuccess && ctx->compact_stream)
+  ctx->compact_smem = compact_async_smem_bytes(cfg->keep_per_frame, ctx->C, ctx->esize);
+  ctx->compact_async = ctx->compact_smem <= 110 * 1024;              // at least two blocks per SM
+  if (const char* s = getenv("MUKV_COMPACT_PLAIN")) if (atoi(s) != 0) ctx->compact_async = false;
+  if (e == cudaSuccess && ctx->compact_async)
     e = cfg->dtype == MUKV_BF16
-            ? cudaFuncSetAttribute((const void*)compact_stream_kernel<__nv_bfloat16>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemLimit)
-            : cudaFuncSetAttribute((const void*)compact_stream_kernel<float>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemLimit);
+            ? cudaFuncSetAttribute((const void*)compact_async_kernel<__nv_bfloat16>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->compact_smem)
+            : cudaFuncSetAttribute((const void*)compact_async_kernel<float>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->compact_smem);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute((const void*)rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRankStageBytes);
   if (e == cudaSuccess && ctx->tcs.ok) {

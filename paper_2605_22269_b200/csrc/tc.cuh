@@ -100,23 +100,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, 
       : "memory");
 }
 
-// ---------------------------------------------------------------- bulk copies (untiled TMA)
-// size a multiple of 16 bytes, both addresses 16-byte aligned
-__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-__device__ __forceinline__ void bulk_store(void* dst, uint32_t src_smem, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes)
-               : "memory");
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-// the bulk stores of this thread have finished reading shared memory
-__device__ __forceinline__ void bulk_store_wait_read() {
-  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-}
-
 // ---------------------------------------------------------------- tensor memory
 // ncols: power of two in [32, 512]; executed by one whole warp
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {

@@ -157,8 +157,8 @@ def test_chunk7b_tile_block_scoring(monkeypatch):
     assert run.ctx.mukv_get_stats().device_status == 0
 
 
-def test_chunk7b_plain_compaction(monkeypatch):
-    # compaction with register copies (the kernel used when two planes do not fit in shared memory)
+def test_chunk7b_register_compaction(monkeypatch):
+    # compaction with the rows held in registers (the kernel used when a plane does not fit in shared memory)
     monkeypatch.setenv("MUKV_COMPACT_PLAIN", "1")
     run = H.GpuRun("chunk7b", n_frames=5)
     full_compress_check(run)
