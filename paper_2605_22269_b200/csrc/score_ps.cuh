@@ -122,8 +122,8 @@ __device__ __forceinline__ float ps_chunk_exp(uint32_t (&r)[16], float c, float 
 
 // Eq. 4 and the selection for frame f, run by the epilogue warps of the block that finished the
 // frame last.  It sits on the critical path at the end of the launch, so it is written for speed:
-// the partial sums are added in double and in block order, everything after that is single
-// precision (double-precision arithmetic is slow on this part), few barriers, and the rank counting
+// everything is single precision (double-precision arithmetic is slow on this part), the partial
+// sums are added in a fixed order, few barriers, and the rank counting
 // runs on the scores' bit patterns (scores lie in [0, 1], so the patterns order like the values),
 // two threads per token.  Single precision adds about 1e-7 to the score error, which the safety
 // test below covers: a frame whose lowest kept and highest dropped score are closer than
@@ -141,22 +141,29 @@ __device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c
     // the blocks' column sums, sixteen loads in flight at a time, added in block order
     const float* cp = reinterpret_cast<const float*>(sp.colsum_part) + et;
     const float* fp = reinterpret_cast<const float*>(sp.ifft_part) + (long long)f * Hkv * P + et;
-    double a64 = 0.0, f64 = 0.0;
+    // single-precision sums in a fixed pairwise order (double-precision adds are slow on this part)
     float y[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) y[i] = i < Hkv ? __ldcg(fp + (long long)i * P) : 0.f;
+    float a32 = 0.f;
     for (int cc = c_first; cc <= c_last; cc += 16) {
       float x[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) x[i] = cc + i <= c_last ? __ldcg(cp + (long long)(cc + i + f) * P) : 0.f;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) a64 += (double)x[i];
+      for (int w = 8; w >= 1; w >>= 1)
+#pragma unroll
+        for (int i = 0; i < w; ++i) x[i] += x[i + w];
+      a32 += x[0];
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) f64 += (double)y[i];
-    for (int gg = 8; gg < Hkv; ++gg) f64 += (double)__ldcg(fp + (long long)gg * P);
-    att = (float)a64 * (1.f / (float)((long long)sp.Hq * P));
-    fft = (float)f64 * (1.f / (float)((long long)Hkv * sp.D));
+    for (int w = 4; w >= 1; w >>= 1)
+#pragma unroll
+      for (int i = 0; i < w; ++i) y[i] += y[i + w];
+    float f32 = y[0];
+    for (int gg = 8; gg < Hkv; ++gg) f32 += __ldcg(fp + (long long)gg * P);
+    att = a32 * (1.f / (float)((long long)sp.Hq * P));
+    fft = f32 * (1.f / (float)((long long)Hkv * sp.D));
   }
   // ---- min / max of both signals over the frame (the tokens live in the first eight warps)
   if (warp < 8) {
@@ -189,6 +196,7 @@ __device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c
     if (t < P) {
       const int key = __float_as_int(s_sc[t]);
       const int4* v = reinterpret_cast<const int4*>(s_sc);
+#pragma unroll 4
       for (int j = j0; j < j1; ++j) {
         const int4 o = v[j];
         gt += (o.x > key) + (o.y > key) + (o.z > key) + (o.w > key);
