@@ -6,8 +6,6 @@
 // token order, to the frame's page; the same registers feed the mean over the kept rows.
 // The last-layer key plane is summed in double: its mean is the retrieval key (Eq. 5) that
 // later ranks blocks, so it is kept free of accumulation-order noise.
-// compact_kernel keeps the rows in registers between load and store (any plane size);
-// compact_async_kernel lands them in shared memory first (planes that fit).
 // The block that finishes a (layer, K|V) plane of the chunk last (arrival counter, nobody waits)
 // refreshes that plane of every segment entry the chunk touches: mean over the frames present.
 #pragma once
@@ -168,121 +166,6 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
       float t = 0.f;
       for (int g = 0; g < rows_per_pass; ++g) t += s_red[(g * NV + cv) * VE + ce];
       fe[col] = t / (float)kappa;
-    }
-  }
-
-  // ---- segment entries of this plane, by the block that completes the plane
-  __shared__ int s_last;
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int old = atomicAdd(p.plane_counter + plane, 1);
-    s_last = (old == p.n_frames - 1);
-    if (s_last) p.plane_counter[plane] = 0;            // ready for the next launch
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  compact_segment_plane(p, l, kv);
-}
-
-// compact_async_kernel<T>: the same work with the kept rows of a plane landed in shared memory by
-// asynchronous 16-byte copies (cp.async), all of them in flight at once, four blocks per SM.  From
-// shared memory each row leaves for the frame's page as streaming 16-byte stores, and each thread
-// sums its own 32-bit column over the rows in row order: no registers tied up by loads in flight
-// and no cross-thread reduction.  Used when the plane fits in shared memory.
-__host__ inline size_t compact_async_smem_bytes(int kappa, int C, int esize) {
-  return ((size_t)kappa * C * esize + 127) / 128 * 128 + (size_t)kappa * sizeof(int) + 256;
-}
-
-template <typename T>
-__global__ void __launch_bounds__(kCompactThreads) compact_async_kernel(const CompactParams p) {
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  const int tid = threadIdx.x;
-  const int plane = blockIdx.x;                 // l*2 + kv
-  const int l = plane >> 1, kv = plane & 1;
-  const int f = blockIdx.y;
-  const long long f_abs = p.first_frame + f;
-  pdl_wait();
-  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
-    *p.stat_refined += *p.n_flagged;
-    *p.n_flagged = 0;
-  }
-  const int kappa = p.kappa, C = p.C;
-  const uint32_t row_bytes = (uint32_t)C * sizeof(T);
-  const uint32_t rows_bytes = ((uint32_t)kappa * row_bytes + 127u) / 128u * 128u;
-  unsigned char* s_rows = smem_raw;
-  int* s_kept = reinterpret_cast<int*>(smem_raw + rows_bytes);
-  for (int r = tid; r < kappa; r += kCompactThreads) s_kept[r] = p.kept_store[f_abs * kappa + r];
-  unsigned char* page = p.store + p.page_table[f_abs];
-  __syncthreads();
-  const unsigned char* src_base = reinterpret_cast<const unsigned char*>(kv ? p.v : p.k) +
-                                  ((long long)l * p.n_frames + f) * p.P * (long long)row_bytes;
-  const int vec_per_row = (int)(row_bytes >> 4);
-  const int n_vec = kappa * vec_per_row;
-  const uint32_t s_base = (uint32_t)__cvta_generic_to_shared(s_rows);
-  for (int v = tid; v < n_vec; v += kCompactThreads) {
-    const int r = v / vec_per_row, cvec = v % vec_per_row;
-    const unsigned char* src = src_base + (long long)s_kept[r] * row_bytes + ((long long)cvec << 4);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s_base + ((uint32_t)v << 4)), "l"(src) : "memory");
-  }
-  asm volatile("cp.async.commit_group;" ::: "memory");
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
-  __syncthreads();
-  // ---- the rows leave for the page (one contiguous run: kept rows in ascending token order)
-  unsigned char* dst = page + (long long)plane * kappa * row_bytes;
-  for (int v = tid; v < n_vec; v += kCompactThreads)
-    st_stream(dst + ((long long)v << 4), *reinterpret_cast<const uint4*>(s_rows + ((size_t)v << 4)));
-  // ---- pooled entry: thread = one 32-bit column, rows added in order
-  const bool exact = (l == p.L - 1) && (kv == 0);
-  const int words = (int)(row_bytes >> 2);
-  float* fe = p.frame_entry + ((f_abs * p.L + l) * 2 + kv) * C;
-  const uint32_t* s_w = reinterpret_cast<const uint32_t*>(s_rows);
-  for (int w = tid; w < words; w += kCompactThreads) {
-    if constexpr (sizeof(T) == 2) {
-      if (exact) {
-        double a = 0.0, b = 0.0;
-        for (int r = 0; r < kappa; ++r) {
-          const uint32_t x = s_w[(size_t)r * words + w];
-          a += (double)bf16_lo(x);
-          b += (double)bf16_hi(x);
-        }
-        p.frame_ksum[f_abs * C + 2 * w] = a;
-        p.frame_ksum[f_abs * C + 2 * w + 1] = b;
-        const float ma = (float)(a / (double)kappa), mb = (float)(b / (double)kappa);
-        fe[2 * w] = ma; fe[2 * w + 1] = mb;
-        p.frame_key[f_abs * C + 2 * w] = ma;
-        p.frame_key[f_abs * C + 2 * w + 1] = mb;
-      } else {
-        float a0 = 0.f, b0 = 0.f, a1 = 0.f, b1 = 0.f;        // two partial sums per column: shorter add chains
-        int r = 0;
-        for (; r + 1 < kappa; r += 2) {
-          const uint32_t x = s_w[(size_t)r * words + w], y = s_w[(size_t)(r + 1) * words + w];
-          a0 += bf16_lo(x); b0 += bf16_hi(x);
-          a1 += bf16_lo(y); b1 += bf16_hi(y);
-        }
-        if (r < kappa) { const uint32_t x = s_w[(size_t)r * words + w]; a0 += bf16_lo(x); b0 += bf16_hi(x); }
-        fe[2 * w] = (a0 + a1) / (float)kappa;
-        fe[2 * w + 1] = (b0 + b1) / (float)kappa;
-      }
-    } else {
-      if (exact) {
-        double a = 0.0;
-        for (int r = 0; r < kappa; ++r) a += (double)__uint_as_float(s_w[(size_t)r * words + w]);
-        p.frame_ksum[f_abs * C + w] = a;
-        const float m = (float)(a / (double)kappa);
-        fe[w] = m;
-        p.frame_key[f_abs * C + w] = m;
-      } else {
-        float a0 = 0.f, a1 = 0.f;
-        int r = 0;
-        for (; r + 1 < kappa; r += 2) {
-          a0 += __uint_as_float(s_w[(size_t)r * words + w]);
-          a1 += __uint_as_float(s_w[(size_t)(r + 1) * words + w]);
-        }
-        if (r < kappa) a0 += __uint_as_float(s_w[(size_t)r * words + w]);
-        fe[w] = (a0 + a1) / (float)kappa;
-      }
     }
   }
 

@@ -65,8 +65,6 @@ struct mukv_ctx {
   float flag_margin, flat_ratio;
   TcShape tcs;                           // tcs.ok: the chunk is scored on the tensor cores
   int n_sms;
-  bool compact_async;                    // compaction through shared memory (the plane fits)
-  size_t compact_smem;
   CUtensorMap wmap;                      // DFT matrix terms [3*D][D] bf16
   std::string err;
   // optional per-kernel timing (host objects only)
@@ -442,10 +440,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   cp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
   {
     ProfScope ps(ctx, 2, st);
-    if (ctx->compact_async)
-      e = launch_k(compact_async_kernel<T>, dim3(L * 2, n), kCompactThreads, ctx->compact_smem, st, !ctx->prof_on, cp);
-    else
-      e = launch_k(compact_kernel<T>, dim3(L * 2, n), kCompactThreads, 0, st, !ctx->prof_on, cp);
+    e = launch_k(compact_kernel<T>, dim3(L * 2, n), kCompactThreads, 0, st, !ctx->prof_on, cp);
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "compact kernel: %s", cudaGetErrorString(e));
 
@@ -513,15 +508,6 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
     e = set_score_attr<float, float>(ctx->nc, score_smem_bytes<float, float>(P, D));
     if (e == cudaSuccess) e = set_score_attr<float, double>(ctx->nc, score_smem_bytes<float, double>(P, D));
   }
-  ctx->compact_smem = compact_async_smem_bytes(cfg->keep_per_frame, ctx->C, ctx->esize);
-  ctx->compact_async = ctx->compact_smem <= 110 * 1024;              // at least two blocks per SM
-  if (const char* s = getenv("MUKV_COMPACT_PLAIN")) if (atoi(s) != 0) ctx->compact_async = false;
-  if (e == cudaSuccess && ctx->compact_async)
-    e = cfg->dtype == MUKV_BF16
-            ? cudaFuncSetAttribute((const void*)compact_async_kernel<__nv_bfloat16>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->compact_smem)
-            : cudaFuncSetAttribute((const void*)compact_async_kernel<float>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->compact_smem);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute((const void*)rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRankStageBytes);
   if (e == cudaSuccess && ctx->tcs.ok) {

@@ -157,13 +157,6 @@ def test_chunk7b_tile_block_scoring(monkeypatch):
     assert run.ctx.mukv_get_stats().device_status == 0
 
 
-def test_chunk7b_register_compaction(monkeypatch):
-    # compaction with the rows held in registers (the kernel used when a plane does not fit in shared memory)
-    monkeypatch.setenv("MUKV_COMPACT_PLAIN", "1")
-    run = H.GpuRun("chunk7b", n_frames=5)
-    full_compress_check(run)
-
-
 def test_chunk7b_cuda_core_scoring(monkeypatch):
     # bf16 inputs scored by the plain multiply-add kernel (the one fp32 inputs always use)
     monkeypatch.setenv("MUKV_SCORE_FMA", "1")
