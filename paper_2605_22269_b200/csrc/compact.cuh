@@ -6,8 +6,7 @@
 // token order, to the frame's page; the same registers feed the mean over the kept rows.
 // The last-layer key plane is summed in double: its mean is the retrieval key (Eq. 5) that
 // later ranks blocks, so it is kept free of accumulation-order noise.
-// The block that finishes a (layer, K|V) plane of the chunk last (arrival counter, nobody waits)
-// refreshes that plane of every segment entry the chunk touches: mean over the frames present.
+// segment_kernel: refreshes every segment entry the chunk touches: mean over the frames present.
 #pragma once
 #include "common.cuh"
 
@@ -31,7 +30,6 @@ struct CompactParams {
   long long* stat_refined;        // device counter
   // segment entries (Eq. 5 at segment level)
   int fseg;                       // frames per segment
-  int* plane_counter;             // [L*2] arrivals per plane, zero between launches
   float* seg_entry;               // [max_segs][L][2][C]
   float* seg_key;                 // [max_segs][C]
 };
@@ -93,6 +91,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
   const int f = blockIdx.y;
   const long long f_abs = p.first_frame + f;
   pdl_wait();
+  pdl_trigger();
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
     *p.stat_refined += *p.n_flagged;
     *p.n_flagged = 0;
@@ -168,20 +167,13 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
       fe[col] = t / (float)kappa;
     }
   }
+}
 
-  // ---- segment entries of this plane, by the block that completes the plane
-  __shared__ int s_last;
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int old = atomicAdd(p.plane_counter + plane, 1);
-    s_last = (old == p.n_frames - 1);
-    if (s_last) p.plane_counter[plane] = 0;            // ready for the next launch
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  compact_segment_plane(p, l, kv);
+// segment_kernel: one block per (layer, K|V) plane; refreshes that plane of every segment entry the
+// chunk touches.  Launched right after compact_kernel (programmatic dependent launch).
+__global__ void __launch_bounds__(kCompactThreads) segment_kernel(const CompactParams p) {
+  pdl_wait();
+  compact_segment_plane(p, blockIdx.x >> 1, blockIdx.x & 1);
 }
 
 }  // namespace mukv

@@ -36,7 +36,7 @@ struct StoreLayout {
 };
 
 struct WorkLayout {
-  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, stat_refined, dev_status, plane_counter;
+  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, stat_refined, dev_status;
   size_t q64, qnorm, s_frm, s_seg, wtab, total;
   size_t zero_begin, zero_end;          // region that must start as zeros
 };
@@ -197,7 +197,6 @@ WorkLayout work_layout(const mukv_config& c) {
   w.n_flagged = off;      off = align_up(off + sizeof(int));
   w.stat_refined = off;   off = align_up(off + sizeof(long long));
   w.dev_status = off;     off = align_up(off + sizeof(int));
-  w.plane_counter = off;  off = align_up(off + (size_t)c.n_layers * 2 * sizeof(int));
   w.zero_end = off;
   w.q64 = off;            off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * C * sizeof(double));
   w.qnorm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * sizeof(double));
@@ -435,7 +434,6 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   cp.n_flagged = sp.n_flagged;
   cp.stat_refined = reinterpret_cast<long long*>(ctx->ws + ctx->wl.stat_refined);
   cp.fseg = c.frames_per_segment;
-  cp.plane_counter = reinterpret_cast<int*>(ctx->ws + ctx->wl.plane_counter);
   cp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
   cp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
   {
@@ -443,8 +441,13 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
     e = launch_k(compact_kernel<T>, dim3(L * 2, n), kCompactThreads, 0, st, !ctx->prof_on, cp);
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "compact kernel: %s", cudaGetErrorString(e));
+  {
+    ProfScope ps(ctx, 3, st);
+    e = launch_k(segment_kernel, dim3(L * 2), kCompactThreads, 0, st, !ctx->prof_on, cp);
+  }
+  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "segment kernel: %s", cudaGetErrorString(e));
 
-  ctx->launches += 3;
+  ctx->launches += 4;
   ctx->frames = t0 + n;
   return MUKV_OK;
 }
@@ -679,7 +682,7 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "rank kernel: %s", cudaGetErrorString(e));
-    ctx->launches += 3;
+    ctx->launches += 4;
     return MUKV_OK;
   } catch (...) {
     return fail(ctx, MUKV_E_INVALID, "unexpected exception");
