@@ -20,9 +20,11 @@ struct QMeta {
 };
 
 // ------------------------------------------------------------------------------ Eq. 6
-// One block per question.  The question's tokens are dealt to kPoolSlices groups of threads so that
-// many loads are in flight; the slices are added in a fixed order.  The pooled query is written
-// transposed, q64t[c][question] (row stride MUKV_MAX_QUESTIONS), the layout scan_kernel stages.
+// One block per question.  Thread (slice, vector) sums one 16-byte vector of channels over the
+// tokens n = slice, slice + kPoolSlices, ... and the G query heads of its key group: every load is
+// a full 16-byte vector and all of a thread's loads are independent.  The slices are added in a
+// fixed order.  The pooled query is written transposed, q64t[c][question] (row stride
+// MUKV_MAX_QUESTIONS), the layout scan_kernel stages.
 constexpr int kPoolThreads = 1024;
 constexpr int kPoolSmemDoubles = 5632;
 
@@ -30,27 +32,45 @@ template <typename T>
 __global__ void __launch_bounds__(kPoolThreads) qpool_kernel(const T* __restrict__ qtok, const QMeta meta, int Hq,
                                                              int Hkv, int D, double* __restrict__ q64t,
                                                              double* __restrict__ qnorm) {
+  constexpr int VE = 16 / sizeof(T);
   __shared__ double s_acc[kPoolSmemDoubles];
   __shared__ double s_part[kPoolThreads / 32];
   const int qi = blockIdx.x;
   const int C = Hkv * D, G = Hq / Hkv;
   const int n0 = meta.off[qi], n1 = meta.off[qi + 1];
-  int nsl = kPoolSmemDoubles / C;
-  nsl = nsl > 4 ? 4 : (nsl < 1 ? 1 : nsl);
-  for (int idx = threadIdx.x; idx < nsl * C; idx += kPoolThreads) {
-    const int sl = idx / C, col = idx % C;
-    const int g = col / D, d = col % D;
-    double t0 = 0.0, t1 = 0.0;
+  const int NV = C / VE, DV = D / VE;                       // vectors per pooled row / per head
+  int nsl = kPoolSmemDoubles / C;                           // token slices whose partial sums fit
+  if (nsl > kPoolThreads / NV) nsl = kPoolThreads / NV;
+  if (nsl < 1) nsl = 1;
+  for (int idx = threadIdx.x; idx < nsl * NV; idx += kPoolThreads) {
+    const int sl = idx / NV, cv = idx % NV;
+    const int g = cv / DV, dv = cv % DV;
+    double tot[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) tot[e] = 0.0;
     for (int n = n0 + sl; n < n1; n += nsl) {
-      const T* row = qtok + ((long long)n * Hq + (long long)g * G) * D + d;
-      int j = 0;
-      for (; j + 1 < G; j += 2) {
-        t0 += (double)elem_to_float<T>(row[(long long)j * D]);
-        t1 += (double)elem_to_float<T>(row[(long long)(j + 1) * D]);
+      const T* row = qtok + ((long long)n * Hq + (long long)g * G) * D + dv * VE;
+#pragma unroll 1
+      for (int j0 = 0; j0 < G; j0 += 8) {
+        uint4 x[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          x[j] = j0 + j < G ? *reinterpret_cast<const uint4*>(row + (long long)(j0 + j) * D) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t w[4] = {x[j].x, x[j].y, x[j].z, x[j].w};
+          if constexpr (sizeof(T) == 2) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { tot[2 * i] += (double)bf16_lo(w[i]); tot[2 * i + 1] += (double)bf16_hi(w[i]); }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) tot[i] += (double)__uint_as_float(w[i]);
+          }
+        }
       }
-      if (j < G) t0 += (double)elem_to_float<T>(row[(long long)j * D]);
     }
-    s_acc[idx] = t0 + t1;
+#pragma unroll
+    for (int e = 0; e < VE; ++e) s_acc[sl * C + cv * VE + e] = tot[e];
   }
   __syncthreads();
   double sq = 0.0;
