@@ -328,22 +328,55 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
     tc::prefetch_tmap(&kmap);
     tc::prefetch_tmap(&wmap);
   }
+  // ---- TMA producer (thread 0).  produce(limit) issues loads in item order until `limit` operand
+  // stages have been filled in total; the first call runs before the block-wide barrier below, so
+  // that the first operands are on their way while tensor memory is being allocated.
+  int pr_i = i0, pr_t = 0, pr_nk = 0, pr_ns = 0, pr_unit = -1;
+  bool pr_ok = true;
+  auto produce = [&](int limit) {
+    while (pr_i < i1 && pr_ok && pr_ns < limit) {
+      const int unit = pr_i / ipu, x = pr_i % ipu;
+      const int f = unit / Hkv, g = unit % Hkv;
+      if (unit != pr_unit) {
+        const int kb_i = pr_nk & 1;
+        pr_ok = tc::mbar_wait(PS_BAR_KE(kb_i), (uint32_t)(((pr_nk >> 1) & 1) ^ 1));
+        if (!pr_ok) break;
+        tc::mbar_expect_tx(PS_BAR_KF(kb_i), k_buf);
+        for (int kb = 0; kb < KB; ++kb)
+          tc::tma_load_3d(sK + (uint32_t)kb_i * k_buf + kb * k_kb, &kmap, kb * 64, g, f * P, PS_BAR_KF(kb_i));
+        ++pr_nk;
+        pr_unit = unit;
+      }
+      const int n_ld = x < p.n_mt ? 3 : 1;               // DFT item: the three matrix terms, smallest first
+      while (pr_t < n_ld && pr_ns < limit) {
+        const int s = pr_ns % NS;
+        pr_ok = tc::mbar_wait(PS_BAR_SE(s), (uint32_t)(((pr_ns / NS) & 1) ^ 1));
+        if (!pr_ok) break;
+        const uint32_t dst = sS + (uint32_t)s * st_buf;
+        if (x < p.n_mt) {
+          tc::mbar_expect_tx(PS_BAR_SF(s), (uint32_t)KB * (uint32_t)D * 128u);
+          for (int kb = 0; kb < KB; ++kb)
+            tc::tma_load_2d(dst + kb * st_kb, &wmap, kb * 64, (2 - pr_t) * D, PS_BAR_SF(s));
+        } else {
+          tc::mbar_expect_tx(PS_BAR_SF(s), (uint32_t)KB * (uint32_t)rows_q * 128u);
+          for (int kb = 0; kb < KB; ++kb)
+            tc::tma_load_3d(dst + kb * st_kb, &qmap, kb * 64, g * G, f * P + (x - p.n_mt) * p.tpt, PS_BAR_SF(s));
+        }
+        ++pr_ns;
+        ++pr_t;
+      }
+      if (!pr_ok) break;
+      if (pr_t == n_ld) { ++pr_i; pr_t = 0; }
+    }
+  };
+  if (tid == 0) produce(NS);
   if (warp == 1) {
     __syncwarp();
     tc::tmem_alloc(tc::smem_u32(tmem_slot), 512u);
   }
-  // Rows of a stage that a Q box never writes (rows_q .. 127) are read by the MMA as rows of the
-  // tile; they only produce rows of the product that are never used, but they must be finite.
-  // A DFT term fills all D rows of a stage it uses, so a stage may hold old matrix rows there: finite too.
-  {
-    const int pad_rows = 128 - rows_q;
-    uint4* s4 = reinterpret_cast<uint4*>(sm + 2u * k_buf);
-    for (int i = tid; i < NS * KB * pad_rows * 8; i += kPsThreads) {
-      const int blk = i / (pad_rows * 8), rem = i % (pad_rows * 8);
-      s4[(size_t)blk * (st_kb / 16) + (size_t)rows_q * 8 + rem] = make_uint4(0u, 0u, 0u, 0u);
-    }
-  }
-  tc::fence_proxy_async_smem();
+  // Rows of a stage that a Q box never writes (rows_q .. 127) hold whatever the stage held before.
+  // The MMA reads them as rows of the tile: they only produce rows of the product that belong to
+  // no token, and the epilogue discards those rows whatever their bits are.
   tc::tc_fence_before_sync();
   __syncthreads();
   tc::tc_fence_after_sync();
@@ -353,49 +386,18 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
     // the control warpgroup (warps 2 and 3 have no other job) hands its registers over
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kPsCtrlRegs));
   if (warp == 0) {
-    // ================================================================== TMA producer
+    // ================================================================== TMA producer (continued)
     if (lane == 0) {
-      bool ok = true;
-      int nk = 0, ns = 0, last_unit = -1;
-      for (int i = i0; i < i1 && ok; ++i) {
-        const int unit = i / ipu, x = i % ipu;
-        const int f = unit / Hkv, g = unit % Hkv;
-        if (unit != last_unit) {
-          const int kb_i = nk & 1;
-          ok = tc::mbar_wait(PS_BAR_KE(kb_i), (uint32_t)(((nk >> 1) & 1) ^ 1));
-          if (!ok) break;
-          tc::mbar_expect_tx(PS_BAR_KF(kb_i), k_buf);
-          for (int kb = 0; kb < KB; ++kb)
-            tc::tma_load_3d(sK + (uint32_t)kb_i * k_buf + kb * k_kb, &kmap, kb * 64, g, f * P, PS_BAR_KF(kb_i));
-          ++nk;
-          last_unit = unit;
-        }
-        const int n_ld = x < p.n_mt ? 3 : 1;             // DFT item: the three matrix terms, smallest first
-        for (int t = 0; t < n_ld && ok; ++t) {
-          const int s = ns % NS;
-          ok = tc::mbar_wait(PS_BAR_SE(s), (uint32_t)(((ns / NS) & 1) ^ 1));
-          if (!ok) break;
-          const uint32_t dst = sS + (uint32_t)s * st_buf;
-          if (x < p.n_mt) {
-            tc::mbar_expect_tx(PS_BAR_SF(s), (uint32_t)KB * (uint32_t)D * 128u);
-            for (int kb = 0; kb < KB; ++kb) tc::tma_load_2d(dst + kb * st_kb, &wmap, kb * 64, (2 - t) * D, PS_BAR_SF(s));
-          } else {
-            tc::mbar_expect_tx(PS_BAR_SF(s), (uint32_t)KB * (uint32_t)rows_q * 128u);
-            for (int kb = 0; kb < KB; ++kb)
-              tc::tma_load_3d(dst + kb * st_kb, &qmap, kb * 64, g * G, f * P + (x - p.n_mt) * p.tpt, PS_BAR_SF(s));
-          }
-          ++ns;
-        }
-      }
-      if (!ok) atomicCAS(p.status, 0, 3);
+      produce(0x7fffffff);
+      if (!pr_ok) atomicCAS(p.status, 0, 3);
       pdl_trigger();                                     // the next kernel of the call may be scheduled
       // copies of this thread still in flight land before the block goes away
       for (int s = 0; s < 2; ++s) {
-        const int cnt = (nk + 1 - s) >> 1;
+        const int cnt = (pr_nk + 1 - s) >> 1;
         if (cnt) tc::mbar_wait(PS_BAR_KF(s), (uint32_t)((cnt - 1) & 1));
       }
       for (int s = 0; s < NS; ++s) {
-        const int cnt = (ns + NS - 1 - s) / NS;
+        const int cnt = (pr_ns + NS - 1 - s) / NS;
         if (cnt) tc::mbar_wait(PS_BAR_SF(s), (uint32_t)((cnt - 1) & 1));
       }
     }
