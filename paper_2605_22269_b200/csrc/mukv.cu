@@ -417,7 +417,8 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   sp.ifft_part = ctx->ws + ctx->wl.ifft_d;
   {
     ProfScope ps(ctx, 1, st);
-    e = launch_score<T, double>(sp, ctx->nc, grid, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
+    const dim3 rgrid(c.n_q_heads, n < 2 ? n : 2);          // its blocks walk the flagged frames
+    e = launch_score<T, double>(sp, ctx->nc, rgrid, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "refine kernel: %s", cudaGetErrorString(e));
 

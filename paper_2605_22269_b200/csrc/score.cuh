@@ -207,18 +207,10 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
   }
 }
 
+// The work of one block: query head h of frame f (a frame slot of the chunk).
 template <typename T, typename A, int NC>
-__global__ void __launch_bounds__(kScoreThreads) score_kernel(const ScoreParams p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+__device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, int f, unsigned char* smem_raw) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int h = blockIdx.x;
-  int f = blockIdx.y;
-  pdl_wait();
-  pdl_trigger();
-  if (p.refine) {
-    if ((int)blockIdx.y >= *p.n_flagged) return;
-    f = p.flagged[blockIdx.y];
-  }
   const int P = p.P, D = p.D, Hq = p.Hq, Hkv = p.Hkv, G = p.G;
   const int g = h / G;
   constexpr int EPW = ElemTraits<T>::kPerWord;
@@ -394,6 +386,25 @@ __global__ void __launch_bounds__(kScoreThreads) score_kernel(const ScoreParams 
   }
   __syncthreads();
   select_frame<1>(p, f, att, fft, s_sc, s_int, s_misc);
+}
+
+// Normal pass: block (h, f) of a grid (Hq, n_frames).  Double-precision pass (p.refine): the grid
+// has few rows of blocks, which walk the list of flagged frames; with nothing flagged they return
+// at once.
+template <typename T, typename A, int NC>
+__global__ void __launch_bounds__(kScoreThreads) score_kernel(const ScoreParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_wait();
+  pdl_trigger();
+  if (!p.refine) {
+    score_frame_block<T, A, NC>(p, blockIdx.x, blockIdx.y, smem_raw);
+    return;
+  }
+  const int n = *p.n_flagged;
+  for (int slot = blockIdx.y; slot < n; slot += gridDim.y) {
+    score_frame_block<T, A, NC>(p, blockIdx.x, p.flagged[slot], smem_raw);
+    __syncthreads();
+  }
 }
 
 }  // namespace mukv

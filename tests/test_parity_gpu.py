@@ -157,6 +157,14 @@ def test_chunk7b_tile_block_scoring(monkeypatch):
     assert run.ctx.mukv_get_stats().device_status == 0
 
 
+def test_chunk7b_every_frame_through_the_double_pass(monkeypatch):
+    # a huge safety margin flags every frame: the double-precision pass has to walk a list longer than its grid
+    monkeypatch.setenv("MUKV_FLAG_MARGIN", "1.0")
+    run = H.GpuRun("chunk7b", n_frames=5)
+    full_compress_check(run)
+    assert run.ctx.mukv_get_stats().refined_frames == 5
+
+
 def test_chunk7b_cuda_core_scoring(monkeypatch):
     # bf16 inputs scored by the plain multiply-add kernel (the one fp32 inputs always use)
     monkeypatch.setenv("MUKV_SCORE_FMA", "1")
