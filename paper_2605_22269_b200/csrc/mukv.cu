@@ -177,6 +177,8 @@ TcShape tc_shape(const mukv_config& c) {
   return t;
 }
 
+constexpr int kRefineSplit = 4;     // blocks per query head in the double-precision pass
+
 WorkLayout work_layout(const mukv_config& c) {
   WorkLayout w;
   const size_t F = c.max_frames_per_chunk, P = c.tokens_per_frame;
@@ -189,7 +191,7 @@ WorkLayout work_layout(const mukv_config& c) {
   w.colsum_f = off;       off = align_up(off + F * parts * P * sizeof(float));
   w.colsum_p = off;       off = align_up(off + (ts.persistent ? (kPsMaxBlocks + F) * P * sizeof(float) : 0));
   w.ifft_f = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(float));
-  w.colsum_d = off;       off = align_up(off + F * c.n_q_heads * P * sizeof(double));
+  w.colsum_d = off;       off = align_up(off + F * c.n_q_heads * kRefineSplit * P * sizeof(double));
   w.ifft_d = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(double));
   w.zero_begin = off;
   w.frame_counter = off;  off = align_up(off + F * sizeof(int));
@@ -399,6 +401,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   sp.pages_off = (long long)ctx->sl.pages;
   sp.page_bytes = (long long)ctx->sl.page_bytes;
   sp.refine = 0;
+  sp.row_split = 1;
   const dim3 grid(c.n_q_heads, n);
   cudaError_t e;
   const char* what = "score kernel";
@@ -413,11 +416,12 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   // frames too close to a tie boundary: same computation in double (blocks beyond the flagged
   // count return at once)
   sp.refine = 1;
+  sp.row_split = kRefineSplit;
   sp.colsum_part = ctx->ws + ctx->wl.colsum_d;
   sp.ifft_part = ctx->ws + ctx->wl.ifft_d;
   {
     ProfScope ps(ctx, 1, st);
-    const dim3 rgrid(c.n_q_heads, n < 2 ? n : 2);          // its blocks walk the flagged frames
+    const dim3 rgrid(c.n_q_heads * kRefineSplit, n < 2 ? n : 2);   // its blocks walk the flagged frames
     e = launch_score<T, double>(sp, ctx->nc, rgrid, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "refine kernel: %s", cudaGetErrorString(e));
@@ -868,6 +872,7 @@ mukv_status noalloc_impl(const mukv_config& c, const void* d_q, const void* d_k_
   sp.frame_ts = reinterpret_cast<long long*>(base + kNaTs);
   sp.page_table = reinterpret_cast<long long*>(base + kNaPt);
   sp.refine = 0;
+  sp.row_split = 1;
   const dim3 grid(c.n_q_heads, n);
   e = launch_score<T, float>(sp, nc, grid, score_smem_bytes<T, float>(P, D), st);
   if (e != cudaSuccess) return fail(nullptr, MUKV_E_CUDA, "score kernel: %s", cudaGetErrorString(e));

@@ -30,7 +30,7 @@ struct ScoreParams {
   const void* q;                // [n][P][Hq][D]
   const void* k_last;           // [n][P][Hkv][D]  (last layer of K)
   // scratch
-  void* colsum_part;            // A [F][Hq][P]
+  void* colsum_part;            // A [F][Hq * row_split][P]
   void* ifft_part;              // A [F][Hkv][P]
   int* frame_counter;           // [F], zero between launches
   int* flagged;                 // [F] frame slots needing the double pass
@@ -43,6 +43,7 @@ struct ScoreParams {
   long long* page_table;        // [max_frames]
   long long pages_off, page_bytes;
   int refine;                   // 1: frames come from the flagged list, no further flagging
+  int row_split;                // blocks that share a query head, each a range of query rows (>= 1)
 };
 
 template <typename T>
@@ -207,9 +208,11 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
   }
 }
 
-// The work of one block: query head h of frame f (a frame slot of the chunk).
+// The work of one block: part q (of p.row_split) of the query rows of head h of frame f (a frame
+// slot of the chunk).
 template <typename T, typename A, int NC>
-__device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, int f, unsigned char* smem_raw) {
+__device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, int q, int f,
+                                                  unsigned char* smem_raw) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = p.P, D = p.D, Hq = p.Hq, Hkv = p.Hkv, G = p.G;
   const int g = h / G;
@@ -270,8 +273,11 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, i
 #pragma unroll
   for (int c = 0; c < NC; ++c) jrow[c] = min(lane + 32 * c, P - 1) * WS;
 
+  const int RS = p.row_split;
   const int n_steps = (P + kRowsPerStep - 1) / kRowsPerStep;
-  for (int rb = warp; rb < n_steps; rb += kScoreWarps) {
+  const int n_per = (n_steps + RS - 1) / RS;
+  const int rb_end = (q + 1) * n_per < n_steps ? (q + 1) * n_per : n_steps;
+  for (int rb = q * n_per + warp; rb < rb_end; rb += kScoreWarps) {
     __syncwarp();
 #pragma unroll
     for (int r = 0; r < kRowsPerStep; ++r) {
@@ -329,14 +335,14 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, i
   if (tid < P) {
     A t = (A)0;
     for (int w = 0; w < kScoreWarps; ++w) t += red[w * 256 + tid];
-    reinterpret_cast<A*>(p.colsum_part)[((long long)f * Hq + h) * P + tid] = t;
+    reinterpret_cast<A*>(p.colsum_part)[(((long long)f * Hq + h) * RS + q) * P + tid] = t;
   }
 
   // ---- Eq. 2-3: sum over the D bins of |DFT(k_j)| for this block's share of head g's tokens
   {
-    const int hg = h % G;
+    const int hg = (h % G) * RS + q;                 // the G * RS blocks that hold key head g share its tokens
     const int half = D / 2;
-    for (int j = hg + warp * G; j < P; j += kScoreWarps * G) {
+    for (int j = hg + warp * G * RS; j < P; j += kScoreWarps * G * RS) {
       const T* kr = Ks + (size_t)j * DS;
       A total = (A)0;
       // bins 1 .. D/2-1 (twice, by conjugate symmetry) and bin 0
@@ -369,16 +375,16 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, i
   __syncthreads();
   if (tid == 0) {
     const int old = atomicAdd(p.frame_counter + f, 1);
-    s_int[63] = (old == Hq - 1);
-    if (old == Hq - 1) p.frame_counter[f] = 0;      // ready for the next launch
+    s_int[63] = (old == Hq * RS - 1);
+    if (old == Hq * RS - 1) p.frame_counter[f] = 0;  // ready for the next launch
   }
   __syncthreads();
   if (!s_int[63]) return;
   __threadfence();
   double att[1] = {0.0}, fft[1] = {0.0};
   if (tid < P) {
-    const A* cp = reinterpret_cast<const A*>(p.colsum_part) + (long long)f * Hq * P + tid;
-    for (int hh = 0; hh < Hq; ++hh) att[0] += (double)__ldcg(cp + (long long)hh * P);
+    const A* cp = reinterpret_cast<const A*>(p.colsum_part) + (long long)f * Hq * RS * P + tid;
+    for (int hh = 0; hh < Hq * RS; ++hh) att[0] += (double)__ldcg(cp + (long long)hh * P);
     att[0] = att[0] / (double)((long long)Hq * P);
     const A* fp = reinterpret_cast<const A*>(p.ifft_part) + (long long)f * Hkv * P + tid;
     for (int gg = 0; gg < Hkv; ++gg) fft[0] += (double)__ldcg(fp + (long long)gg * P);
@@ -388,21 +394,21 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, i
   select_frame<1>(p, f, att, fft, s_sc, s_int, s_misc);
 }
 
-// Normal pass: block (h, f) of a grid (Hq, n_frames).  Double-precision pass (p.refine): the grid
-// has few rows of blocks, which walk the list of flagged frames; with nothing flagged they return
-// at once.
+// Grid (Hq * row_split, frames).  Normal pass: block row = frame slot of the chunk.  Double-precision
+// pass (p.refine): the grid has few rows of blocks, which walk the list of flagged frames; with
+// nothing flagged they return at once.
 template <typename T, typename A, int NC>
 __global__ void __launch_bounds__(kScoreThreads) score_kernel(const ScoreParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_wait();
   pdl_trigger();
   if (!p.refine) {
-    score_frame_block<T, A, NC>(p, blockIdx.x, blockIdx.y, smem_raw);
+    score_frame_block<T, A, NC>(p, blockIdx.x / p.row_split, blockIdx.x % p.row_split, blockIdx.y, smem_raw);
     return;
   }
   const int n = *p.n_flagged;
   for (int slot = blockIdx.y; slot < n; slot += gridDim.y) {
-    score_frame_block<T, A, NC>(p, blockIdx.x, p.flagged[slot], smem_raw);
+    score_frame_block<T, A, NC>(p, blockIdx.x / p.row_split, blockIdx.x % p.row_split, p.flagged[slot], smem_raw);
     __syncthreads();
   }
 }
