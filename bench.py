@@ -174,7 +174,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--frames", type=int, default=0, help="shorten the stream (debugging / profiling only)")
-    ap.add_argument("--oracle-frames", type=int, default=8)
+    ap.add_argument("--oracle-frames", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--l2", default="inputs", choices=["inputs", "flush"],
