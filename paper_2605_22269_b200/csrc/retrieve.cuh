@@ -6,7 +6,7 @@
 // summation order.  Kernels:
 //   qpool_kernel    Eq. 6   one block per question
 //   scan_kernel     Eq. 7   cosine of every question with every frame key and segment key (a skinny
-//                           double-precision product, tiled through shared memory)
+//                           double-precision product on the fp64 tensor-core instruction)
 //   rank_kernel     stage-1 candidates, Eq. 8 rerank, final top-k; one block per question
 //   gather_kernel   Eq. 9   copies the selected pages into the per-question decode buffers
 #pragma once
@@ -94,11 +94,21 @@ __global__ void __launch_bounds__(kPoolThreads) qpool_kernel(const T* __restrict
 // ------------------------------------------------------------------------------ Eq. 7
 // Rows 0..n_frm-1 are frame keys, rows n_frm..n_frm+n_seg-1 segment keys.  A block owns
 // kScanRows rows and walks the feature axis in chunks of kScanCC: the rows' chunk (float) and the
-// chunk of up to kScanQB pooled queries (double) are staged in shared memory, thread
-// (row pair, question quad) keeps a 2 x 4 tile of double dot products.
+// chunk of up to kScanQB pooled queries (double) are staged in shared memory.  The product itself
+// is a dense double-precision contraction [rows x C] . [C x questions] and runs on the
+// double-precision tensor-core instruction (mma.sync m8n8k4 f64): warp w owns rows 8*(w%4).. and
+// questions 32*(w/4).., four 8 x 8 accumulator tiles.  (Plain double-precision FMAs are slow on
+// this part; the scores have to be double because indices are ranked on them.)
 constexpr int kScanRows = 32;
 constexpr int kScanCC = 64;
 constexpr int kScanQB = 64;
+constexpr int kScanQPad = kScanQB + 4;
+
+__device__ __forceinline__ void dmma_m8n8k4(double (&c)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(c[0]), "+d"(c[1])
+               : "d"(a), "d"(b));
+}
 
 __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ frame_key,
                                                    const float* __restrict__ seg_key, long long n_frm,
@@ -107,22 +117,21 @@ __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ fra
                                                    double* __restrict__ s_seg, long long frm_stride,
                                                    long long seg_stride) {
   __shared__ float rows[kScanRows][kScanCC + 1];
-  __shared__ __align__(16) double qs[kScanCC][kScanQB];
+  __shared__ __align__(16) double qs[kScanCC][kScanQPad];
   __shared__ double s_knorm[kScanRows];
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const long long row0 = (long long)blockIdx.x * kScanRows;
   const long long n_rows = n_frm + n_seg;
   const int lr = tid >> 3, lc = (tid & 7) * 8;               // staging: row, first column of 8
   const long long my_row = row0 + lr;
   const float* src = my_row < n_frm ? frame_key + my_row * C
                                     : (my_row < n_rows ? seg_key + (my_row - n_frm) * C : nullptr);
-  const int rp = tid >> 4, qd = tid & 15;                    // compute: rows rp, rp+16; questions 4qd..4qd+3
+  const int wr = (warp & 3) * 8, wq = (warp >> 2) * 32;      // this warp's rows and questions
+  const int fr = lane >> 2, fk = lane & 3;                   // fragment row / k (A), k / column (B)
   for (int qb = 0; qb < nq; qb += kScanQB) {
-    double acc[2][4];
+    double acc[4][2];
 #pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+    for (int i = 0; i < 4; ++i) { acc[i][0] = 0.0; acc[i][1] = 0.0; }
     double kk = 0.0;
     for (int c0 = 0; c0 < C; c0 += kScanCC) {
       __syncthreads();                                       // the previous chunk has been consumed
@@ -138,15 +147,11 @@ __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ fra
         qs[cc][qq] = (c0 + cc < C && qb + qq < nq) ? q64t[(long long)(c0 + cc) * MUKV_MAX_QUESTIONS + qb + qq] : 0.0;
       }
       __syncthreads();
-#pragma unroll 8
-      for (int cc = 0; cc < kScanCC; ++cc) {
-        const double a0 = (double)rows[rp][cc], a1 = (double)rows[rp + 16][cc];
-        const double2 q01 = *reinterpret_cast<const double2*>(&qs[cc][4 * qd]);
-        const double2 q23 = *reinterpret_cast<const double2*>(&qs[cc][4 * qd + 2]);
-        acc[0][0] = fma(a0, q01.x, acc[0][0]); acc[0][1] = fma(a0, q01.y, acc[0][1]);
-        acc[0][2] = fma(a0, q23.x, acc[0][2]); acc[0][3] = fma(a0, q23.y, acc[0][3]);
-        acc[1][0] = fma(a1, q01.x, acc[1][0]); acc[1][1] = fma(a1, q01.y, acc[1][1]);
-        acc[1][2] = fma(a1, q23.x, acc[1][2]); acc[1][3] = fma(a1, q23.y, acc[1][3]);
+#pragma unroll 4
+      for (int cc = 0; cc < kScanCC; cc += 4) {
+        const double a = (double)rows[wr + fr][cc + fk];     // A[row fr][k fk]
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) dmma_m8n8k4(acc[nt], a, qs[cc + fk][wq + nt * 8 + fr]);   // B[k fk][col fr]
       }
     }
     if (qb == 0) {
@@ -157,21 +162,23 @@ __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ fra
       if ((tid & 7) == 0) s_knorm[lr] = sqrt(kk);
     }
     __syncthreads();
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int r = rp + 16 * i;
-      const long long row = row0 + r;
-      if (row >= n_rows) continue;
+    // accumulator tile: row fr, columns 2*fk and 2*fk + 1
+    const int r = wr + fr;
+    const long long row = row0 + r;
+    if (row < n_rows) {
       const double knorm = s_knorm[r];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int qi = qb + 4 * qd + j;
-        if (qi >= nq) continue;
-        double den = knorm * qnorm[qi];
-        den = den > 1e-12 ? den : 1e-12;
-        const double sc = acc[i][j] / den;
-        if (row < n_frm) s_frm[(long long)qi * frm_stride + row] = sc;
-        else s_seg[(long long)qi * seg_stride + (row - n_frm)] = sc;
+      for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int qi = qb + wq + nt * 8 + 2 * fk + j;
+          if (qi >= nq) continue;
+          double den = knorm * qnorm[qi];
+          den = den > 1e-12 ? den : 1e-12;
+          const double sc = acc[nt][j] / den;
+          if (row < n_frm) s_frm[(long long)qi * frm_stride + row] = sc;
+          else s_seg[(long long)qi * seg_stride + (row - n_frm)] = sc;
+        }
       }
     }
   }
