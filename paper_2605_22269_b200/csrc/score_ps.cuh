@@ -36,7 +36,7 @@ constexpr int kPsThreads = 640;           // warpgroup 0: control, warpgroups 1-
 constexpr int kPsEpiThreads = 512;
 constexpr int kPsSplit = 4;                // warps that share a row (32-lane quarter), each a column range
 constexpr int kPsEpiOff = 128;             // first epilogue thread
-constexpr int kPsMiscBytes = 20480;
+constexpr int kPsMiscBytes = 24576;
 constexpr int kPsMaxBlocks = 256;          // bound on the grid (slots of partial sums)
 constexpr int kPsAccCols = 64;             // accumulator columns per epilogue thread: P <= 4 * 64
 // Twenty warps put five on each scheduler, whose 16 K registers allow 96 per thread at launch.
@@ -47,6 +47,7 @@ constexpr int kPsCtrlRegs = 32;
 constexpr int kPsEpiRegs = 112;
 static_assert(128 * (96 - kPsCtrlRegs) >= 512 * (kPsEpiRegs - 96), "register hand-over does not balance");
 typedef NamedGroup<5, kPsEpiThreads, kPsEpiOff> PsEpiGroup;
+static_assert(sizeof(ScoreParams) <= 1536, "the shared-memory copy of the parameters has 1536 bytes");
 
 struct ScorePsParams {
   ScoreParams sp;            // colsum_part: float [grid + n_frames][P] slots, ifft_part: float [F][Hkv][P]
@@ -74,23 +75,30 @@ __device__ __forceinline__ int ps_owner(long long i, long long n, long long nb) 
   return (int)(((i + 1) * nb - 1) / n);
 }
 
+// square root to about one unit in the last place (one special-function instruction and a multiply)
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float y;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ float ps_chunk_max(const uint32_t (&r)[16], int col0, int P, bool causal, int i_tok) {
-  float m0 = -INFINITY, m1 = -INFINITY;
   if (!causal && col0 + 16 <= P) {
-#pragma unroll
-    for (int k = 0; k < 16; k += 4) {
-      m0 = fmaxf(m0, fmaxf(__uint_as_float(r[k]), __uint_as_float(r[k + 1])));
-      m1 = fmaxf(m1, fmaxf(__uint_as_float(r[k + 2]), __uint_as_float(r[k + 3])));
-    }
-  } else {
-#pragma unroll
-    for (int k = 0; k < 16; ++k) {
-      const int j = col0 + k;
-      const bool ok = (j < P) && (!causal || j <= i_tok);
-      m0 = ok ? fmaxf(m0, __uint_as_float(r[k])) : m0;
-    }
+    const float a = tc::fmax3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
+    const float b = tc::fmax3(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
+    const float c = tc::fmax3(__uint_as_float(r[6]), __uint_as_float(r[7]), __uint_as_float(r[8]));
+    const float d = tc::fmax3(__uint_as_float(r[9]), __uint_as_float(r[10]), __uint_as_float(r[11]));
+    const float e = tc::fmax3(__uint_as_float(r[12]), __uint_as_float(r[13]), __uint_as_float(r[14]));
+    return fmaxf(tc::fmax3(a, b, c), tc::fmax3(d, e, __uint_as_float(r[15])));
   }
-  return fmaxf(m0, m1);
+  float m = -INFINITY;
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+    const int j = col0 + k;
+    const bool ok = (j < P) && (!causal || j <= i_tok);
+    m = ok ? fmaxf(m, __uint_as_float(r[k])) : m;
+  }
+  return m;
 }
 
 // r <- exp2(r * c - mc) (0 where masked); returns the sum
@@ -293,15 +301,18 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
   const uint32_t sS = sK + 2u * k_buf;                   // NS operand stages
   const uint32_t misc_off = 2u * k_buf + (uint32_t)NS * st_buf;
   float* s_col = reinterpret_cast<float*>(sm + misc_off);                     // [4][256]
-  float* s_mx = reinterpret_cast<float*>(sm + misc_off + 4096);               // [kPsSplit][128]
-  float* s_sum = s_mx + kPsSplit * 128;                                       // [kPsSplit][128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + misc_off + 8192);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + misc_off + 8192 + 192);
-  int* s_flag = reinterpret_cast<int*>(sm + misc_off + 8192 + 196);
-  float* s_mref = reinterpret_cast<float*>(sm + misc_off + 10240);            // [4 chunks][512 threads]
+  // (reference, sum) of a row's four warps, one copy per accumulator: a copy is rewritten two items
+  // later, after the row's warps have met again at the barrier of the item in between
+  float* s_mx = reinterpret_cast<float*>(sm + misc_off + 4096);               // [2][kPsSplit][128]
+  float* s_sum = s_mx + 2 * kPsSplit * 128;                                   // [2][kPsSplit][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + misc_off + 12288);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + misc_off + 12288 + 192);
+  int* s_flag = reinterpret_cast<int*>(sm + misc_off + 12288 + 196);
   // the selection routine is a real call: it reads the parameters from this copy, so that the
   // kernel's own parameter block never has its address taken (which would move it to local memory)
-  ScoreParams* s_sp = reinterpret_cast<ScoreParams*>(sm + misc_off + 8704);
+  ScoreParams* s_sp = reinterpret_cast<ScoreParams*>(sm + misc_off + 12800);
+  int* s_cnt = reinterpret_cast<int*>(sm + misc_off + 14336);                 // [512], selection only
+  float* s_mref = reinterpret_cast<float*>(sm + misc_off + 16384);            // [4 chunks][512 threads]
   const uint32_t b0 = tc::smem_u32(bars);
   // key buffer full / empty, accumulator full / empty (2 each), stage full / empty (kPsMaxStages each)
 #define PS_BAR_KF(s) (b0 + 8u * (uint32_t)(s))
@@ -459,8 +470,10 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
     const int et = tid - kPsEpiOff, ew = et >> 5;
     const int q = warp & 3, h = ew >> 2;                 // TMEM lane quarter, column range
     const int row = q * 32 + lane;
+    const int row_tok = row / G;                         // token of this row inside its tile
     const uint32_t tlane = (uint32_t)(q * 32) << 16;
-    const int nch16 = p.npad >> 4, ch_base = nch16 / kPsSplit, ch_rem = nch16 % kPsSplit;
+    // the columns of a row go to its four warps in chunks of 16
+    const int nch16 = (P + 15) >> 4, ch_base = nch16 / kPsSplit, ch_rem = nch16 % kPsSplit;
     const int my_c0 = h * ch_base + (h < ch_rem ? h : ch_rem), my_nch = ch_base + (h < ch_rem ? 1 : 0);
     const bool causal = sp.causal != 0;
     const float c = p.exp2_scale;
@@ -470,50 +483,49 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
     for (int k = 0; k < kPsAccCols; ++k) acc[k] = 0.f;
     bool ok = true;
     int it = 0;
+    int x = i0 % ipu, g = (i0 / ipu) % Hkv, f = (i0 / ipu) / Hkv;
     for (int i = i0; i < i1; ++i, ++it) {
-      const int unit = i / ipu, x = i % ipu;
-      const int f = unit / Hkv, g = unit % Hkv;
       const int b = it & 1;
-      const bool done = tc::mbar_wait(PS_BAR_AF(b), (uint32_t)((it >> 1) & 1));
-      ok = tc::named_sync_and(5, kPsEpiThreads, done);
-      if (!ok) break;
+      // A wait that runs out is recorded; the warp then goes on without waiting (every read
+      // below stays inside the accumulators), so that the warps of a row keep meeting at their barrier.
+      if (ok) ok = __all_sync(kFull, tc::mbar_wait(PS_BAR_AF(b), (uint32_t)((it >> 1) & 1)));
       tc::tc_fence_after_sync();
       const uint32_t tb = tmem + (uint32_t)b * 256u + tlane;
       if (x < p.n_mt) {
-        // ---- Eq. 2-3: this thread's half of the bins of its token
+        // ---- Eq. 2-3: this thread's share of the bins of its token
         const int H2 = D >> 1;
         const int bins = H2 / kPsSplit >= 16 ? H2 / kPsSplit : 16;   // per warp of the row, a multiple of 16
         const int bin0 = h * bins;
         float tot = 0.f;
         if (bin0 < H2) {
 #pragma unroll 1
-          for (int cc = 0; cc < bins; cc += 16) {
-            uint32_t re[16], im[16];
-            tc::tmem_ld16(tb + bin0 + cc, re);
-            tc::tmem_ld16(tb + H2 + bin0 + cc, im);
-            tc::tmem_wait_ld16x2(re, im);
+          for (int cc = 0; cc < bins; cc += 8) {
+            uint32_t re[8], im[8];
+            tc::tmem_ld8(tb + bin0 + cc, re);
+            tc::tmem_ld8(tb + H2 + bin0 + cc, im);
+            tc::tmem_wait_ld8x2(re, im);
 #pragma unroll
-            for (int k = 0; k < 16; ++k) {
+            for (int k = 0; k < 8; ++k) {
               const float a = __uint_as_float(re[k]), bb = __uint_as_float(im[k]);
-              const float mag = sqrtf(fmaf(a, a, bb * bb));
+              const float mag = sqrt_approx(fmaf(a, a, bb * bb));
               // bins 0 and D/2 are real: their two values sit in the re/im slots of "bin 0"
               tot += (bin0 + cc + k == 0) ? fabsf(a) + fabsf(bb) : 2.f * mag;
             }
           }
         }
-        s_sum[h * 128 + row] = tot;
+        float* xs = s_sum + b * kPsSplit * 128;
+        xs[h * 128 + row] = tot;
         tc::named_sync(1 + q, 32 * kPsSplit);
         const int token = x * 128 + row;
         if (h == 0 && token < P) {
           float t4 = 0.f;
 #pragma unroll
-          for (int hh = 0; hh < kPsSplit; ++hh) t4 += s_sum[hh * 128 + row];
+          for (int hh = 0; hh < kPsSplit; ++hh) t4 += xs[hh * 128 + row];
           reinterpret_cast<float*>(sp.ifft_part)[((long long)f * Hkv + g) * P + token] = t4;
         }
       } else {
         // ---- Eq. 1
-        const int tile = x - p.n_mt;
-        const int i_tok = tile * p.tpt + row / G;
+        const int i_tok = (x - p.n_mt) * p.tpt + row_tok;
         const bool valid = (row < rows_q) && (i_tok < P);
         // sweep 1: running maximum, e = exp(z - running max) back into tensor memory, row sum.
         // One 16-column chunk per trip; the other warps of the scheduler cover the load latency.
@@ -533,16 +545,18 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
           m_run = m_new;
         }
         tc::tmem_wait_st();
-        s_mx[h * 128 + row] = m_run;
-        s_sum[h * 128 + row] = l;
+        float* xm = s_mx + b * kPsSplit * 128;
+        float* xs = s_sum + b * kPsSplit * 128;
+        xm[h * 128 + row] = m_run;
+        xs[h * 128 + row] = l;
         tc::named_sync(1 + q, 32 * kPsSplit);
-        float m = s_mx[row];
+        float m = xm[row];
 #pragma unroll
-        for (int hh = 1; hh < kPsSplit; ++hh) m = fmaxf(m, s_mx[hh * 128 + row]);
+        for (int hh = 1; hh < kPsSplit; ++hh) m = fmaxf(m, xm[hh * 128 + row]);
         float lsum = 0.f;
 #pragma unroll
-        for (int hh = 0; hh < kPsSplit; ++hh) lsum += s_sum[hh * 128 + row] * ex2_approx((s_mx[hh * 128 + row] - m) * c);
-        const float inv = valid ? 1.f / lsum : 0.f;
+        for (int hh = 0; hh < kPsSplit; ++hh) lsum += xs[hh * 128 + row] * ex2_approx((xm[hh * 128 + row] - m) * c);
+        const float inv = valid ? __fdividef(1.f, lsum) : 0.f;
         // sweep 2: acc[column] += e * 2^(ref - max) / sum
 #pragma unroll
         for (int ch = 0; ch < kMaxCh; ++ch) {
@@ -563,7 +577,8 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(PS_BAR_AE(b));
 
-      if (i + 1 == i1 || (i + 1) / ipf != f) {
+      const bool frame_ends = (i + 1 == i1) || (x == ipu - 1 && g == Hkv - 1);
+      if (frame_ends) {
         // ---- leaving frame f: publish this block's column sums, the last block selects
 #pragma unroll
         for (int pp = 0; pp < (kPsAccCols + 31) / 32; ++pp) {
@@ -574,7 +589,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
             else v[k] = 0.f;
           }
           const float s = warp_column_sums(v, lane);
-          if (2 * pp + (lane >> 4) < my_nch) s_col[q * 256 + (my_c0 + 2 * pp) * 16 + lane] = s;
+          if (pp * 32 + lane < my_nch * 16) s_col[q * 256 + my_c0 * 16 + pp * 32 + lane] = s;
         }
         PsEpiGroup::sync();
         float* slot = reinterpret_cast<float*>(sp.colsum_part) + (long long)(cta + f) * P;
@@ -594,12 +609,16 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
         if (s_flag[0]) {
           __threadfence();
           ps_finish_frame(*s_sp, f, c_first, c_last, s_col, reinterpret_cast<int*>(sm + misc_off + 3072),
-                          reinterpret_cast<float*>(sm + misc_off + 2048), reinterpret_cast<int*>(s_mref));
+                          reinterpret_cast<float*>(sm + misc_off + 2048), s_cnt);
         }
         PsEpiGroup::sync();
       }
+      if (++x == ipu) {
+        x = 0;
+        if (++g == Hkv) { g = 0; ++f; }
+      }
     }
-    if (!ok && et == 0) atomicCAS(p.status, 0, 5);
+    if (!ok && lane == 0) atomicCAS(p.status, 0, 5);
   }
 #undef PS_BAR_KF
 #undef PS_BAR_KE
