@@ -1,14 +1,29 @@
 // KV compaction into the paged store and block pooling (Sec. 3.3 "selected KV slices ... are
-// stored", Sec. 3.4 Eq. 5).
+// stored", Sec. 3.4 Eq. 5), and the in-block selection that feeds it (Eq. 4 and the top-kappa rule).
 //
 // compact_kernel<T>: one thread block per (layer, K|V, frame).  The kappa kept rows of that
 // plane (C = Hkv*D elements each, one contiguous run in the input) are copied, in ascending
 // token order, to the frame's page; the same registers feed the mean over the kept rows.
 // The last-layer key plane is summed in double: its mean is the retrieval key (Eq. 5) that
 // later ranks blocks, so it is kept free of accumulation-order noise.
-// segment_kernel: refreshes every segment entry the chunk touches: mean over the frames present.
+//
+// Where do the kept ids come from?  After the persistent tensor-core scoring kernel every block
+// works them out itself (sel_mode 1): it adds the scoring blocks' partial column sums of its frame
+// in a fixed order, applies Eq. 4 and selects, all in single precision; the blocks of a frame run
+// the same arithmetic on the same numbers, so they agree, and the one with plane 0 writes the ids
+// and the index.  That costs a few microseconds at the start of each block, in parallel on the
+// whole device, where a selection inside the scoring kernel left one block per frame working while
+// all others had finished.  After the other scoring kernels the ids are read from the store
+// (sel_mode 0).  Either way a frame whose lowest kept and highest dropped score are closer than
+// tie_eps + flag_margin is skipped here: the double-precision pass that follows decides it, and
+// segment_kernel then compacts it.
+//
+// segment_kernel<T>: one block per (layer, K|V) plane: compacts the frames the double-precision
+// pass decided, then refreshes that plane of every segment entry the chunk touches (mean over the
+// frames present).
 #pragma once
 #include "common.cuh"
+#include "score.cuh"
 
 namespace mukv {
 
@@ -20,19 +35,200 @@ struct CompactParams {
   long long first_frame;
   const void* k;                  // [L][n][P][C]
   const void* v;
-  const int* kept_store;          // [max_frames][kappa]
   unsigned char* store;           // store base
-  const long long* page_table;    // [max_frames] byte offsets
   float* frame_entry;             // [max_frames][L][2][C]
   float* frame_key;               // [max_frames][C]
   double* frame_ksum;             // [max_frames][C]  exact sums of the last-layer kept keys
-  int* n_flagged;                 // reset here for the next chunk
   long long* stat_refined;        // device counter
+  int* seg_counter;               // arrival counter of segment_kernel's blocks, zero between launches
   // segment entries (Eq. 5 at segment level)
   int fseg;                       // frames per segment
   float* seg_entry;               // [max_segs][L][2][C]
   float* seg_key;                 // [max_segs][C]
+  // selection
+  int sel_mode;                   // 0: kept ids are in the store; 1: select here from the partial sums
+  int ps_grid, ps_items, ps_ipf;  // the scoring launch: blocks, items, items per frame
+  ScoreParams sp;                 // partial sums, Eq. 4 parameters, index and flag outputs
 };
+
+// owner of item i when n items are split into contiguous shares [c*n/nb, (c+1)*n/nb)
+__device__ __forceinline__ int share_owner(unsigned i, unsigned n, unsigned nb) { return (int)(((i + 1u) * nb - 1u) / n); }
+
+struct SelectScratch {
+  unsigned mm[kCompactThreads / 32][4];   // per-warp min / max keys of the two signals
+  int hist[256];
+  int list[256];                  // keys of the scores in the bin that holds the kappa-th largest
+  int cnt[kCompactThreads / 32][4];
+  unsigned ab[kCompactThreads / 32][2];
+  int bin, rank, n_list;
+  float tau;
+};
+
+// Eq. 4 and the top-kappa rule for frame f from the partial sums of the persistent scoring kernel,
+// run by a whole block of kCompactThreads threads (thread t owns token t; P <= 256).  The kept ids
+// go to s_kept in ascending order; with `write` also to the store and to the caller's outputs.
+// Returns true when single precision cannot decide the frame safely (see select_frame): nothing
+// of the frame may then be used, and with `write` the frame has been put on the flagged list.
+// Everything is single precision; scores lie in [0, 1], so their bit patterns order like the
+// values and the reductions run on them as integers.
+__device__ inline bool select_from_partials(const CompactParams& p, int f, bool write, int* s_kept, SelectScratch* sc) {
+  const ScoreParams& sp = p.sp;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int NW = kCompactThreads / 32;
+  const int P = sp.P, Hkv = sp.Hkv, kappa = sp.kappa;
+  const bool valid = tid < P;
+  float att = 0.f, fft = 0.f;
+  if (valid) {
+    // the scoring blocks' column sums, added in block order
+    const int c_first = share_owner((unsigned)(f * p.ps_ipf), (unsigned)p.ps_items, (unsigned)p.ps_grid);
+    const int c_last = share_owner((unsigned)((f + 1) * p.ps_ipf - 1), (unsigned)p.ps_items, (unsigned)p.ps_grid);
+    const float* cp = reinterpret_cast<const float*>(sp.colsum_part) + tid;
+    const float* fp = reinterpret_cast<const float*>(sp.ifft_part) + (long long)f * Hkv * P + tid;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    for (int cc = c_first; cc <= c_last; cc += 4) {
+      const float x0 = __ldcg(cp + (long long)(cc + f) * P);
+      const float x1 = cc + 1 <= c_last ? __ldcg(cp + (long long)(cc + 1 + f) * P) : 0.f;
+      const float x2 = cc + 2 <= c_last ? __ldcg(cp + (long long)(cc + 2 + f) * P) : 0.f;
+      const float x3 = cc + 3 <= c_last ? __ldcg(cp + (long long)(cc + 3 + f) * P) : 0.f;
+      a0 += x0; a1 += x1; a2 += x2; a3 += x3;
+    }
+    float f0 = 0.f, f1 = 0.f;
+    for (int g = 0; g < Hkv; g += 2) {
+      const float y0 = __ldcg(fp + (long long)g * P);
+      const float y1 = g + 1 < Hkv ? __ldcg(fp + (long long)(g + 1) * P) : 0.f;
+      f0 += y0; f1 += y1;
+    }
+    att = ((a0 + a1) + (a2 + a3)) * (1.f / (float)((long long)sp.Hq * P));
+    fft = (f0 + f1) * (1.f / (float)((long long)Hkv * sp.D));
+  }
+  // ---- min / max of both signals over the frame (both are sums of non-negative terms)
+  {
+    const unsigned ka = __float_as_uint(att), kf = __float_as_uint(fft);
+    const unsigned v0 = __reduce_min_sync(kFull, valid ? ka : 0xffffffffu), v1 = __reduce_max_sync(kFull, valid ? ka : 0u);
+    const unsigned v2 = __reduce_min_sync(kFull, valid ? kf : 0xffffffffu), v3 = __reduce_max_sync(kFull, valid ? kf : 0u);
+    if (lane == 0) { sc->mm[warp][0] = v0; sc->mm[warp][1] = v1; sc->mm[warp][2] = v2; sc->mm[warp][3] = v3; }
+    sc->hist[tid] = 0;
+    if (tid == 0) sc->n_list = 0;
+  }
+  __syncthreads();
+  unsigned m0 = 0xffffffffu, m1 = 0u, m2 = 0xffffffffu, m3 = 0u;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) {
+    m0 = min(m0, sc->mm[w][0]); m1 = max(m1, sc->mm[w][1]);
+    m2 = min(m2, sc->mm[w][2]); m3 = max(m3, sc->mm[w][3]);
+  }
+  const float amin = __uint_as_float(m0), amax = __uint_as_float(m1);
+  const float fmin_ = __uint_as_float(m2), fmax_ = __uint_as_float(m3);
+  // ---- Eq. 4
+  const float an = (amax == amin) ? 0.f : (att - amin) / (amax - amin);
+  float fn = (fmax_ == fmin_) ? 0.f : (fft - fmin_) / (fmax_ - fmin_);
+  if (sp.keep_low) fn = 1.f - fn;
+  const float s = sp.alpha * an + (1.f - sp.alpha) * fn;
+  const int key = __float_as_int(s);
+  // ---- tau = kappa-th largest score: a 256-bin histogram finds its bin, the scores of that bin
+  // are ranked among themselves
+  int bin = (int)(s * 256.f);
+  bin = bin < 0 ? 0 : (bin > 255 ? 255 : bin);
+  if (valid) atomicAdd(&sc->hist[bin], 1);
+  __syncthreads();
+  if (warp == 0) {
+    int c[8], T = 0;                                     // lane l owns bins 8l .. 8l+7
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { c[i] = sc->hist[8 * lane + i]; T += c[i]; }
+    int incl = T;                                        // scores in this lane's bins and all higher ones
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_down_sync(kFull, incl, o);
+      if (lane + o < 32) incl += v;
+    }
+    const int above = incl - T;
+    if (above < kappa && kappa <= above + T) {           // true for exactly one lane
+      int r = kappa - above, b = 7;
+      for (; b > 0; --b) {
+        if (r <= c[b]) break;
+        r -= c[b];
+      }
+      sc->bin = 8 * lane + b;
+      sc->rank = r;
+    }
+  }
+  __syncthreads();
+  const bool member = valid && bin == sc->bin;
+  if (member) sc->list[atomicAdd(&sc->n_list, 1)] = key;
+  __syncthreads();
+  if (member) {
+    const int n = sc->n_list, r = sc->rank;
+    int gt = 0, ge = 0;
+    for (int i = 0; i < n; ++i) {
+      const int o = sc->list[i];
+      gt += (o > key);
+      ge += (o >= key);
+    }
+    if (gt < r && r <= ge) sc->tau = s;                  // every writer holds the same value
+  }
+  __syncthreads();
+  const float tau = sc->tau;
+  const float delta = sp.tie_eps;
+  const bool sure = valid && (s > tau + delta);
+  const bool band = valid && !sure && (s >= tau - delta);
+  const unsigned lt = (1u << lane) - 1u;
+  const unsigned b_sure = __ballot_sync(kFull, sure), b_band = __ballot_sync(kFull, band);
+  if (lane == 0) { sc->cnt[warp][0] = __popc(b_sure); sc->cnt[warp][1] = __popc(b_band); }
+  __syncthreads();
+  int n_sure = 0, band_rank = __popc(b_band & lt);
+#pragma unroll
+  for (int w = 0; w < NW; ++w) {
+    n_sure += sc->cnt[w][0];
+    if (w < warp) band_rank += sc->cnt[w][1];
+  }
+  const bool keep = sure || (band && band_rank < kappa - n_sure);
+  const unsigned b_keep = __ballot_sync(kFull, keep);
+  {
+    // lowest kept and highest dropped score, for the safety test below
+    const unsigned ks = (unsigned)key;
+    const unsigned a = __reduce_min_sync(kFull, keep ? ks : 0xffffffffu);
+    const unsigned b = __reduce_max_sync(kFull, (valid && !keep) ? ks : 0u);
+    if (lane == 0) { sc->cnt[warp][2] = __popc(b_keep); sc->ab[warp][0] = a; sc->ab[warp][1] = b; }
+  }
+  __syncthreads();
+  int pos = __popc(b_keep & lt);
+  unsigned ka = 0xffffffffu, kb = 0u;
+  bool any_dropped = false;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) {
+    if (w < warp) pos += sc->cnt[w][2];
+    ka = min(ka, sc->ab[w][0]);
+    kb = max(kb, sc->ab[w][1]);
+  }
+  any_dropped = kappa < P;
+  // does single precision decide this frame safely?  (see select_frame)
+  const float a = __uint_as_float(ka), b = any_dropped ? __uint_as_float(kb) : -3.0e38f;
+  bool risky = any_dropped && (a - b <= delta + sp.flag_margin);
+  const float aabs = fmaxf(amax, -amin), fabs_ = fmaxf(fmax_, -fmin_);
+  if (amax != amin && (amax - amin) < sp.flat_ratio * aabs && sp.alpha != 0.f) risky = true;
+  if (fmax_ != fmin_ && (fmax_ - fmin_) < sp.flat_ratio * fabs_ && sp.alpha != 1.f) risky = true;
+  if (keep) s_kept[pos] = tid;
+  if (write) {
+    const long long f_abs = sp.first_frame + f;
+    if (keep) {
+      sp.kept_store[f_abs * kappa + pos] = tid;
+      if (sp.kept_out) sp.kept_out[(long long)f * kappa + pos] = tid;
+    }
+    if (sp.scores_out && valid) {
+      const long long np = (long long)sp.n_frames * P;
+      sp.scores_out[0 * np + (long long)f * P + tid] = att;
+      sp.scores_out[1 * np + (long long)f * P + tid] = fft;
+      sp.scores_out[2 * np + (long long)f * P + tid] = s;
+    }
+    if (tid == 0) {
+      sp.frame_ts[f_abs] = f_abs;
+      sp.page_table[f_abs] = sp.pages_off + f_abs * sp.page_bytes;
+      if (risky) sp.flagged[atomicAdd(sp.n_flagged, 1)] = f;
+    }
+  }
+  __syncthreads();
+  return risky;
+}
 
 // Segment entries (Eq. 5 at segment level) of one (layer, K|V) plane for every segment the chunk
 // touches: mean over the frames present.  Run by one whole block.
@@ -78,31 +274,26 @@ __device__ inline void compact_segment_plane(const CompactParams& p, int l, int 
   }
 }
 
+struct CompactScratch {
+  float red[kCompactThreads * 8];
+  double red64[kCompactThreads * 8];
+  int kept[MUKV_MAX_TOKENS];
+};
+
+// Copies the kept rows (ids in sc->kept, ascending) of plane (l, kv) of chunk frame f to the
+// frame's page and writes the plane's frame entry (Eq. 5).  Run by a whole block.
 // NV = 16-byte vectors per row; the block covers 256/NV rows per pass.
 template <typename T>
-__global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactParams p) {
+__device__ inline void compact_plane(const CompactParams& p, int plane, int f, CompactScratch* sc) {
   constexpr int VE = 16 / sizeof(T);
-  __shared__ float s_red[kCompactThreads * VE];
-  __shared__ double s_red64[kCompactThreads * VE];
-  __shared__ int s_kept[MUKV_MAX_TOKENS];
   const int tid = threadIdx.x;
-  const int plane = blockIdx.x;                 // l*2 + kv
   const int l = plane >> 1, kv = plane & 1;
-  const int f = blockIdx.y;
   const long long f_abs = p.first_frame + f;
-  pdl_wait();
-  pdl_trigger();
-  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) {
-    *p.stat_refined += *p.n_flagged;
-    *p.n_flagged = 0;
-  }
   const int kappa = p.kappa, C = p.C;
   const int NV = C / VE;                        // vectors per row (power of two, <= 256)
   const int rows_per_pass = kCompactThreads / NV;
-  for (int r = tid; r < kappa; r += kCompactThreads) s_kept[r] = p.kept_store[f_abs * kappa + r];
-  __syncthreads();
   const T* src_base = reinterpret_cast<const T*>(kv ? p.v : p.k) + ((long long)l * p.n_frames + f) * p.P * C;
-  unsigned char* page = p.store + p.page_table[f_abs];
+  unsigned char* page = p.store + p.sp.pages_off + f_abs * p.sp.page_bytes;
   T* dst_base = reinterpret_cast<T*>(page) + (long long)plane * kappa * C;
   const int c = tid % NV, r0 = tid / NV;
   const bool exact = (l == p.L - 1) && (kv == 0);
@@ -116,7 +307,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       const int rr = r + u * rows_per_pass;
-      if (rr < kappa) x[u] = ld_stream(src_base + (long long)s_kept[rr] * C + c * VE);
+      if (rr < kappa) x[u] = ld_stream(src_base + (long long)sc->kept[rr] * C + c * VE);
     }
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
@@ -145,10 +336,10 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
   // reduce the row groups (fixed order) and write the mean
   if (exact) {
 #pragma unroll
-    for (int i = 0; i < VE; ++i) s_red64[tid * VE + i] = acc64[i];
+    for (int i = 0; i < VE; ++i) sc->red64[tid * VE + i] = acc64[i];
   } else {
 #pragma unroll
-    for (int i = 0; i < VE; ++i) s_red[tid * VE + i] = acc[i];
+    for (int i = 0; i < VE; ++i) sc->red[tid * VE + i] = acc[i];
   }
   __syncthreads();
   float* fe = p.frame_entry + ((f_abs * p.L + l) * 2 + kv) * C;
@@ -156,24 +347,76 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
     const int cv = col / VE, ce = col % VE;
     if (exact) {
       double t = 0.0;
-      for (int g = 0; g < rows_per_pass; ++g) t += s_red64[(g * NV + cv) * VE + ce];
+      for (int g = 0; g < rows_per_pass; ++g) t += sc->red64[(g * NV + cv) * VE + ce];
       p.frame_ksum[f_abs * C + col] = t;
       const float m = (float)(t / (double)kappa);
       fe[col] = m;
       p.frame_key[f_abs * C + col] = m;
     } else {
       float t = 0.f;
-      for (int g = 0; g < rows_per_pass; ++g) t += s_red[(g * NV + cv) * VE + ce];
+      for (int g = 0; g < rows_per_pass; ++g) t += sc->red[(g * NV + cv) * VE + ce];
       fe[col] = t / (float)kappa;
     }
   }
 }
 
-// segment_kernel: one block per (layer, K|V) plane; refreshes that plane of every segment entry the
-// chunk touches.  Launched right after compact_kernel (programmatic dependent launch).
-__global__ void __launch_bounds__(kCompactThreads) segment_kernel(const CompactParams p) {
+// is chunk frame f on the flagged list (of n entries)?
+__device__ __forceinline__ bool frame_is_flagged(const int* flagged, int n, int f) {
+  bool hit = false;
+  for (int i = 0; i < n; ++i) hit |= (__ldcg(flagged + i) == f);
+  return hit;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactParams p) {
+  __shared__ CompactScratch cs;
+  __shared__ SelectScratch ss;
+  const int tid = threadIdx.x;
+  const int plane = blockIdx.x;                 // l*2 + kv
+  const int f = blockIdx.y;
   pdl_wait();
-  compact_segment_plane(p, blockIdx.x >> 1, blockIdx.x & 1);
+  pdl_trigger();
+  if (p.sel_mode == 1) {
+    if (select_from_partials(p, f, plane == 0, cs.kept, &ss)) return;
+  } else {
+    if (frame_is_flagged(p.sp.flagged, *p.sp.n_flagged, f)) return;
+    const long long f_abs = p.first_frame + f;
+    for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = p.sp.kept_store[f_abs * p.kappa + r];
+    __syncthreads();
+  }
+  compact_plane<T>(p, plane, f, &cs);
+}
+
+// segment_kernel: one block per (layer, K|V) plane.  First the frames that the double-precision
+// pass decided (their ids are in the store by now), then that plane of every segment entry the
+// chunk touches.  The block that finishes last clears the flagged list for the next chunk.
+template <typename T>
+__global__ void __launch_bounds__(kCompactThreads) segment_kernel(const CompactParams p) {
+  __shared__ CompactScratch cs;
+  const int tid = threadIdx.x, plane = blockIdx.x;
+  pdl_wait();
+  const int n_fl = *p.sp.n_flagged;
+  for (int i = 0; i < n_fl; ++i) {
+    const int f = p.sp.flagged[i];
+    const long long f_abs = p.first_frame + f;
+    __syncthreads();
+    for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = __ldcg(p.sp.kept_store + f_abs * p.kappa + r);
+    __syncthreads();
+    compact_plane<T>(p, plane, f, &cs);
+  }
+  // the frame entries this block has just written are read below by other threads of the block
+  if (n_fl) __threadfence();
+  __syncthreads();
+  compact_segment_plane(p, plane >> 1, plane & 1);
+  __syncthreads();
+  if (tid == 0) {
+    const int old = atomicAdd(p.seg_counter, 1);
+    if (old == (int)gridDim.x - 1) {
+      *p.stat_refined += n_fl;
+      *p.sp.n_flagged = 0;
+      *p.seg_counter = 0;
+    }
+  }
 }
 
 }  // namespace mukv

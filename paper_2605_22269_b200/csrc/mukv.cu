@@ -36,7 +36,8 @@ struct StoreLayout {
 };
 
 struct WorkLayout {
-  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, stat_refined, dev_status;
+  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, seg_counter, stat_refined,
+      dev_status;
   size_t q64, qnorm, s_frm, s_seg, wtab, total;
   size_t zero_begin, zero_end;          // region that must start as zeros
 };
@@ -197,6 +198,7 @@ WorkLayout work_layout(const mukv_config& c) {
   w.frame_counter = off;  off = align_up(off + F * sizeof(int));
   w.flagged = off;        off = align_up(off + F * sizeof(int));
   w.n_flagged = off;      off = align_up(off + sizeof(int));
+  w.seg_counter = off;    off = align_up(off + sizeof(int));
   w.stat_refined = off;   off = align_up(off + sizeof(long long));
   w.dev_status = off;     off = align_up(off + sizeof(int));
   w.zero_end = off;
@@ -335,7 +337,8 @@ std::vector<uint16_t> dft_terms(int D) {
 
 // Scores a bf16 chunk on the tensor cores (Eq. 1-4 and the selection).
 cudaError_t launch_score_tc(mukv_ctx* ctx, const ScoreParams& sp, const void* d_q, const void* k_last, int n,
-                            cudaStream_t st, const char** why) {
+                            cudaStream_t st, const char** why, int* ps_grid, int* ps_items, int* ps_ipf) {
+  *ps_grid = 0;
   const mukv_config& c = ctx->cfg;
   const TcShape& t = ctx->tcs;
   const int P = c.tokens_per_frame, D = c.head_dim;
@@ -358,6 +361,7 @@ cudaError_t launch_score_tc(mukv_ctx* ctx, const ScoreParams& sp, const void* d_
     pp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
     int blocks = ctx->n_sms < kPsMaxBlocks ? ctx->n_sms : kPsMaxBlocks;
     if (blocks > pp.n_items) blocks = pp.n_items;
+    *ps_grid = blocks; *ps_items = pp.n_items; *ps_ipf = c.n_kv_heads * (t.n_mt + t.tiles);
     score_ps_kernel<<<blocks, kPsThreads, t.smem_ps, st>>>(pp, qmap, kmap, ctx->wmap);
     *why = "score_ps kernel";
     return cudaGetLastError();
@@ -405,16 +409,43 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   const dim3 grid(c.n_q_heads, n);
   cudaError_t e;
   const char* what = "score kernel";
+  int ps_grid = 0, ps_items = 0, ps_ipf = 0;
   {
     ProfScope ps(ctx, 0, st);
     if (ctx->tcs.ok)
-      e = launch_score_tc(ctx, sp, d_q, sp.k_last, n, st, &what);
+      e = launch_score_tc(ctx, sp, d_q, sp.k_last, n, st, &what, &ps_grid, &ps_items, &ps_ipf);
     else
       e = launch_score<T, float>(sp, ctx->nc, grid, score_smem_bytes<T, float>(P, c.head_dim), st);
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "%s: %s", what, cudaGetErrorString(e));
-  // frames too close to a tie boundary: same computation in double (blocks beyond the flagged
-  // count return at once)
+
+  // Compaction of every frame that single precision decides; after the persistent scoring kernel
+  // its blocks also do the selection (Eq. 4, top-kappa) from that kernel's partial sums.
+  CompactParams cp;
+  memset(&cp, 0, sizeof cp);
+  cp.L = L; cp.kappa = c.keep_per_frame; cp.C = C; cp.P = P; cp.n_frames = n; cp.first_frame = t0;
+  cp.k = d_k; cp.v = d_v;
+  cp.store = ctx->store;
+  cp.frame_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.frame_entry);
+  cp.frame_key = reinterpret_cast<float*>(ctx->store + ctx->sl.frame_key);
+  cp.frame_ksum = reinterpret_cast<double*>(ctx->store + ctx->sl.frame_ksum);
+  cp.stat_refined = reinterpret_cast<long long*>(ctx->ws + ctx->wl.stat_refined);
+  cp.seg_counter = reinterpret_cast<int*>(ctx->ws + ctx->wl.seg_counter);
+  cp.fseg = c.frames_per_segment;
+  cp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
+  cp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
+  cp.sel_mode = ps_grid > 0 ? 1 : 0;
+  cp.ps_grid = ps_grid; cp.ps_items = ps_items; cp.ps_ipf = ps_ipf;
+  cp.sp = sp;
+  if (ps_grid > 0) cp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
+  {
+    ProfScope ps(ctx, 2, st);
+    e = launch_k(compact_kernel<T>, dim3(L * 2, n), kCompactThreads, 0, st, !ctx->prof_on, cp);
+  }
+  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "compact kernel: %s", cudaGetErrorString(e));
+
+  // frames too close to a tie boundary: the scores again in double precision, and the selection
+  // (blocks beyond the flagged count return at once)
   sp.refine = 1;
   sp.row_split = kRefineSplit;
   sp.colsum_part = ctx->ws + ctx->wl.colsum_d;
@@ -425,30 +456,10 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
     e = launch_score<T, double>(sp, ctx->nc, rgrid, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "refine kernel: %s", cudaGetErrorString(e));
-
-  CompactParams cp;
-  memset(&cp, 0, sizeof cp);
-  cp.L = L; cp.kappa = c.keep_per_frame; cp.C = C; cp.P = P; cp.n_frames = n; cp.first_frame = t0;
-  cp.k = d_k; cp.v = d_v;
-  cp.kept_store = sp.kept_store;
-  cp.store = ctx->store;
-  cp.page_table = sp.page_table;
-  cp.frame_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.frame_entry);
-  cp.frame_key = reinterpret_cast<float*>(ctx->store + ctx->sl.frame_key);
-  cp.frame_ksum = reinterpret_cast<double*>(ctx->store + ctx->sl.frame_ksum);
-  cp.n_flagged = sp.n_flagged;
-  cp.stat_refined = reinterpret_cast<long long*>(ctx->ws + ctx->wl.stat_refined);
-  cp.fseg = c.frames_per_segment;
-  cp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
-  cp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
-  {
-    ProfScope ps(ctx, 2, st);
-    e = launch_k(compact_kernel<T>, dim3(L * 2, n), kCompactThreads, 0, st, !ctx->prof_on, cp);
-  }
-  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "compact kernel: %s", cudaGetErrorString(e));
+  // compaction of those frames, then the segment entries
   {
     ProfScope ps(ctx, 3, st);
-    e = launch_k(segment_kernel, dim3(L * 2), kCompactThreads, 0, st, !ctx->prof_on, cp);
+    e = launch_k(segment_kernel<T>, dim3(L * 2), kCompactThreads, 0, st, !ctx->prof_on, cp);
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "segment kernel: %s", cudaGetErrorString(e));
 

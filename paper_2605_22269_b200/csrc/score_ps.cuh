@@ -20,10 +20,12 @@
 //               (shuffle butterfly), so the per-tile cost is one fused multiply-add per logit.
 //               DFT item: magnitudes of the D bins of each key vector, summed.
 //
-// Per frame, every block that worked on it stores its column sums in a slot of its own; the
-// block that arrives last (counter, nobody waits) adds the slots in a fixed order, applies
-// Eq. 4 and selects the kappa tokens.  All mbarrier waits are bounded; a wait that runs out
-// makes the role record a code in the status word and leave its loop.
+// Per frame, every block that worked on it stores its column sums in a slot of its own (slot
+// index = block + frame).  Eq. 4 and the selection are left to the kernel that follows
+// (compact_kernel adds the slots in a fixed order): done here, by the block that finishes a frame
+// last, they kept one block per frame busy for microseconds after all others had finished.
+// All mbarrier waits are bounded; a wait that runs out makes the role record a code in the status
+// word and go on without waiting.
 #pragma once
 #include "common.cuh"
 #include "score.cuh"
@@ -36,7 +38,7 @@ constexpr int kPsThreads = 640;           // warpgroup 0: control, warpgroups 1-
 constexpr int kPsEpiThreads = 512;
 constexpr int kPsSplit = 4;                // warps that share a row (32-lane quarter), each a column range
 constexpr int kPsEpiOff = 128;             // first epilogue thread
-constexpr int kPsMiscBytes = 24576;
+constexpr int kPsMiscBytes = 12800 + 8192;
 constexpr int kPsMaxBlocks = 256;          // bound on the grid (slots of partial sums)
 constexpr int kPsAccCols = 64;             // accumulator columns per epilogue thread: P <= 4 * 64
 // Twenty warps put five on each scheduler, whose 16 K registers allow 96 per thread at launch.
@@ -47,7 +49,6 @@ constexpr int kPsCtrlRegs = 32;
 constexpr int kPsEpiRegs = 112;
 static_assert(128 * (96 - kPsCtrlRegs) >= 512 * (kPsEpiRegs - 96), "register hand-over does not balance");
 typedef NamedGroup<5, kPsEpiThreads, kPsEpiOff> PsEpiGroup;
-static_assert(sizeof(ScoreParams) <= 1536, "the shared-memory copy of the parameters has 1536 bytes");
 
 struct ScorePsParams {
   ScoreParams sp;            // colsum_part: float [grid + n_frames][P] slots, ifft_part: float [F][Hkv][P]
@@ -68,11 +69,6 @@ __host__ inline int score_ps_stages(int P, int D, size_t limit) {
   int n = kPsMaxStages;
   while (n >= 2 && score_ps_smem_bytes(P, D, n) > limit) --n;
   return n;                  // < 2: the kernel does not fit
-}
-
-// owner of item i when n items are split into contiguous shares [c*n/nb, (c+1)*n/nb)
-__device__ __forceinline__ int ps_owner(long long i, long long n, long long nb) {
-  return (int)(((i + 1) * nb - 1) / n);
 }
 
 // square root to about one unit in the last place (one special-function instruction and a multiply)
@@ -128,154 +124,6 @@ __device__ __forceinline__ float ps_chunk_exp(uint32_t (&r)[16], float c, float 
   return l0 + l1;
 }
 
-// Eq. 4 and the selection for frame f, run by the epilogue warps of the block that finished the
-// frame last.  It sits on the critical path at the end of the launch, so it is written for speed:
-// everything is single precision (double-precision arithmetic is slow on this part), the partial
-// sums are added in a fixed order, few barriers, and the rank counting
-// runs on the scores' bit patterns (scores lie in [0, 1], so the patterns order like the values),
-// two threads per token.  Single precision adds about 1e-7 to the score error, which the safety
-// test below covers: a frame whose lowest kept and highest dropped score are closer than
-// tie_eps + flag_margin is left to the double-precision pass (score_kernel<T, double> with
-// select_frame), which applies the same rule.  Kept out of line so that the tile loop's register
-// allocation is not disturbed.
-__device__ __noinline__ void ps_finish_frame(const ScoreParams& sp, int f, int c_first, int c_last, float* s_sc,
-                                             int* s_int, float* s_misc, int* s_cnt) {
-  const int et = PsEpiGroup::tid(), lane = et & 31, warp = et >> 5;
-  const int P = sp.P, Hkv = sp.Hkv, kappa = sp.kappa;
-  const bool valid = et < P;
-  const float big = 3.0e38f;
-  float att = 0.f, fft = 0.f;
-  if (valid) {
-    // the blocks' column sums, sixteen loads in flight at a time, added in block order
-    const float* cp = reinterpret_cast<const float*>(sp.colsum_part) + et;
-    const float* fp = reinterpret_cast<const float*>(sp.ifft_part) + (long long)f * Hkv * P + et;
-    // single-precision sums in a fixed pairwise order (double-precision adds are slow on this part)
-    float y[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) y[i] = i < Hkv ? __ldcg(fp + (long long)i * P) : 0.f;
-    float a32 = 0.f;
-    for (int cc = c_first; cc <= c_last; cc += 16) {
-      float x[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) x[i] = cc + i <= c_last ? __ldcg(cp + (long long)(cc + i + f) * P) : 0.f;
-#pragma unroll
-      for (int w = 8; w >= 1; w >>= 1)
-#pragma unroll
-        for (int i = 0; i < w; ++i) x[i] += x[i + w];
-      a32 += x[0];
-    }
-#pragma unroll
-    for (int w = 4; w >= 1; w >>= 1)
-#pragma unroll
-      for (int i = 0; i < w; ++i) y[i] += y[i + w];
-    float f32 = y[0];
-    for (int gg = 8; gg < Hkv; ++gg) f32 += __ldcg(fp + (long long)gg * P);
-    att = a32 * (1.f / (float)((long long)sp.Hq * P));
-    fft = f32 * (1.f / (float)((long long)Hkv * sp.D));
-  }
-  // ---- min / max of both signals over the frame (the tokens live in the first eight warps)
-  if (warp < 8) {
-    const float v0 = warp_min(valid ? att : big), v1 = warp_max(valid ? att : -big);
-    const float v2 = warp_min(valid ? fft : big), v3 = warp_max(valid ? fft : -big);
-    if (lane == 0) { s_misc[warp * 4] = v0; s_misc[warp * 4 + 1] = v1; s_misc[warp * 4 + 2] = v2; s_misc[warp * 4 + 3] = v3; }
-  }
-  PsEpiGroup::sync();
-  float amin = big, amax = -big, fmin_ = big, fmax_ = -big;
-#pragma unroll
-  for (int w = 0; w < 8; ++w) {
-    amin = fminf(amin, s_misc[w * 4 + 0]);
-    amax = fmaxf(amax, s_misc[w * 4 + 1]);
-    fmin_ = fminf(fmin_, s_misc[w * 4 + 2]);
-    fmax_ = fmaxf(fmax_, s_misc[w * 4 + 3]);
-  }
-  // ---- Eq. 4
-  const float an = (amax == amin) ? 0.f : (att - amin) / (amax - amin);
-  float fn = (fmax_ == fmin_) ? 0.f : (fft - fmin_) / (fmax_ - fmin_);
-  if (sp.keep_low) fn = 1.f - fn;
-  const float s = sp.alpha * an + (1.f - sp.alpha) * fn;
-  if (et < 256) s_sc[et] = valid ? s : -1.f;                 // slots past P hold -1: below every score
-  PsEpiGroup::sync();
-  // ---- tau = kappa-th largest score: rank counting, each token's scan split over two threads
-  {
-    const int t = et & 255, half = et >> 8;
-    const int n4 = (P + 3) >> 2, mid = (n4 + 1) >> 1;
-    const int j0 = half ? mid : 0, j1 = half ? n4 : mid;
-    int gt = 0, ge = 0;
-    if (t < P) {
-      const int key = __float_as_int(s_sc[t]);
-      const int4* v = reinterpret_cast<const int4*>(s_sc);
-#pragma unroll 4
-      for (int j = j0; j < j1; ++j) {
-        const int4 o = v[j];
-        gt += (o.x > key) + (o.y > key) + (o.z > key) + (o.w > key);
-        ge += (o.x >= key) + (o.y >= key) + (o.z >= key) + (o.w >= key);
-      }
-    }
-    s_cnt[half * 256 + t] = gt | (ge << 16);
-  }
-  PsEpiGroup::sync();
-  if (valid) {
-    const int c0 = s_cnt[et], c1 = s_cnt[256 + et];
-    const int gt = (c0 & 0xffff) + (c1 & 0xffff), ge = (c0 >> 16) + (c1 >> 16);
-    if (gt < kappa && kappa <= ge) s_misc[32] = s;          // every writer holds the same value
-  }
-  PsEpiGroup::sync();
-  const float tau = s_misc[32];
-  const float delta = sp.tie_eps;
-  const bool sure = valid && (s > tau + delta);
-  const bool band = valid && !sure && (s >= tau - delta);
-  const unsigned lt = (1u << lane) - 1u;
-  const unsigned b_sure = __ballot_sync(kFull, sure), b_band = __ballot_sync(kFull, band);
-  if (lane == 0 && warp < 8) { s_int[warp] = __popc(b_sure); s_int[8 + warp] = __popc(b_band); }
-  PsEpiGroup::sync();
-  int n_sure = 0, band_rank = __popc(b_band & lt);
-#pragma unroll
-  for (int w = 0; w < 8; ++w) {
-    n_sure += s_int[w];
-    if (w < warp) band_rank += s_int[8 + w];
-  }
-  const bool keep = sure || (band && band_rank < kappa - n_sure);
-  const unsigned b_keep = __ballot_sync(kFull, keep);
-  if (lane == 0 && warp < 8) s_int[16 + warp] = __popc(b_keep);
-  // lowest kept and highest dropped score, for the safety test below
-  if (warp < 8) {
-    const float a = warp_min(keep ? s : big), b = warp_max((valid && !keep) ? s : -big);
-    if (lane == 0) { s_misc[40 + warp * 2] = a; s_misc[41 + warp * 2] = b; }
-  }
-  PsEpiGroup::sync();
-  const long long f_abs = sp.first_frame + f;
-  if (keep) {
-    int pos = __popc(b_keep & lt);
-    for (int w = 0; w < warp; ++w) pos += s_int[16 + w];
-    sp.kept_store[f_abs * kappa + pos] = et;
-    if (sp.kept_out) sp.kept_out[(long long)f * kappa + pos] = et;
-  }
-  if (sp.scores_out && valid) {
-    const long long np = (long long)sp.n_frames * P;
-    sp.scores_out[0 * np + (long long)f * P + et] = att;
-    sp.scores_out[1 * np + (long long)f * P + et] = fft;
-    sp.scores_out[2 * np + (long long)f * P + et] = s;
-  }
-  if (et == 0) {
-    sp.frame_ts[f_abs] = f_abs;
-    sp.page_table[f_abs] = sp.pages_off + f_abs * sp.page_bytes;
-    // does single precision decide this frame safely?  (see select_frame)
-    float a = big, b = -big;
-    for (int w = 0; w < 8; ++w) {
-      a = fminf(a, s_misc[40 + w * 2]);
-      b = fmaxf(b, s_misc[41 + w * 2]);
-    }
-    bool risky = (kappa < P) && (a - b <= delta + sp.flag_margin);
-    const float aabs = fmaxf(amax, -amin), fabs_ = fmaxf(fmax_, -fmin_);
-    if (amax != amin && (amax - amin) < sp.flat_ratio * aabs && sp.alpha != 0.f) risky = true;
-    if (fmax_ != fmin_ && (fmax_ - fmin_) < sp.flat_ratio * fabs_ && sp.alpha != 1.f) risky = true;
-    if (risky) {
-      const int slot = atomicAdd(sp.n_flagged, 1);
-      sp.flagged[slot] = f;
-    }
-  }
-}
-
 __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
                                                  const __grid_constant__ CUtensorMap qmap,
                                                  const __grid_constant__ CUtensorMap kmap,
@@ -289,10 +137,10 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
   const int P = sp.P, D = sp.D, G = sp.G, Hkv = sp.Hkv, KB = D >> 6;
   const int NS = p.n_stages;
   const int ipu = p.n_mt + p.tiles;                      // items per (frame, key head)
-  const int ipf = Hkv * ipu;                             // items per frame
   const int n_cta = gridDim.x, cta = blockIdx.x;
-  const int i0 = (int)((long long)cta * p.n_items / n_cta);
-  const int i1 = (int)((long long)(cta + 1) * p.n_items / n_cta);
+  // contiguous shares [c*n/nb, (c+1)*n/nb); the compaction kernel finds the blocks of a frame from the same rule
+  const int i0 = (int)((unsigned)cta * (unsigned)p.n_items / (unsigned)n_cta);
+  const int i1 = (int)((unsigned)(cta + 1) * (unsigned)p.n_items / (unsigned)n_cta);
   const int rows_q = p.tpt * G;
 
   const uint32_t k_kb = (uint32_t)p.npad * 128u, st_kb = 128u * 128u;
@@ -307,12 +155,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
   float* s_sum = s_mx + 2 * kPsSplit * 128;                                   // [2][kPsSplit][128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + misc_off + 12288);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + misc_off + 12288 + 192);
-  int* s_flag = reinterpret_cast<int*>(sm + misc_off + 12288 + 196);
-  // the selection routine is a real call: it reads the parameters from this copy, so that the
-  // kernel's own parameter block never has its address taken (which would move it to local memory)
-  ScoreParams* s_sp = reinterpret_cast<ScoreParams*>(sm + misc_off + 12800);
-  int* s_cnt = reinterpret_cast<int*>(sm + misc_off + 14336);                 // [512], selection only
-  float* s_mref = reinterpret_cast<float*>(sm + misc_off + 16384);            // [4 chunks][512 threads]
+  float* s_mref = reinterpret_cast<float*>(sm + misc_off + 12800);            // [4 chunks][512 threads]
   const uint32_t b0 = tc::smem_u32(bars);
   // key buffer full / empty, accumulator full / empty (2 each), stage full / empty (kPsMaxStages each)
 #define PS_BAR_KF(s) (b0 + 8u * (uint32_t)(s))
@@ -334,7 +177,6 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
       tc::mbar_init(PS_BAR_SE(s), 1);
     }
     tc::fence_mbar_init();
-    *s_sp = p.sp;
     tc::prefetch_tmap(&qmap);
     tc::prefetch_tmap(&kmap);
     tc::prefetch_tmap(&wmap);
@@ -579,7 +421,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
 
       const bool frame_ends = (i + 1 == i1) || (x == ipu - 1 && g == Hkv - 1);
       if (frame_ends) {
-        // ---- leaving frame f: publish this block's column sums, the last block selects
+        // ---- leaving frame f: this block's column sums go to its slot of the frame
 #pragma unroll
         for (int pp = 0; pp < (kPsAccCols + 31) / 32; ++pp) {
           float v[32];
@@ -595,23 +437,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
         float* slot = reinterpret_cast<float*>(sp.colsum_part) + (long long)(cta + f) * P;
         for (int t = et; t < P; t += kPsEpiThreads)
           slot[t] = (s_col[t] + s_col[256 + t]) + (s_col[512 + t] + s_col[768 + t]);
-        __threadfence();
-        PsEpiGroup::sync();
-        const int c_first = ps_owner((long long)f * ipf, p.n_items, n_cta);
-        const int c_last = ps_owner((long long)(f + 1) * ipf - 1, p.n_items, n_cta);
-        if (et == 0) {
-          const int n_slots = c_last - c_first + 1;
-          const int old = atomicAdd(sp.frame_counter + f, 1);
-          s_flag[0] = (old == n_slots - 1);
-          if (old == n_slots - 1) sp.frame_counter[f] = 0;          // ready for the next launch
-        }
-        PsEpiGroup::sync();
-        if (s_flag[0]) {
-          __threadfence();
-          ps_finish_frame(*s_sp, f, c_first, c_last, s_col, reinterpret_cast<int*>(sm + misc_off + 3072),
-                          reinterpret_cast<float*>(sm + misc_off + 2048), s_cnt);
-        }
-        PsEpiGroup::sync();
+        PsEpiGroup::sync();                                // the sums may be overwritten
       }
       if (++x == ipu) {
         x = 0;
