@@ -40,6 +40,7 @@ struct CompactParams {
   float* frame_key;               // [max_frames][C]
   double* frame_ksum;             // [max_frames][C]  exact sums of the last-layer kept keys
   long long* stat_refined;        // device counter
+  int* n_flagged_next;            // the flagged count of the next chunk (the two chunks' counts alternate)
   int* seg_counter;               // arrival counter of segment_kernel's blocks, zero between launches
   // segment entries (Eq. 5 at segment level)
   int fseg;                       // frames per segment
@@ -84,22 +85,25 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
     const int c_last = share_owner((unsigned)((f + 1) * p.ps_ipf - 1), (unsigned)p.ps_items, (unsigned)p.ps_grid);
     const float* cp = reinterpret_cast<const float*>(sp.colsum_part) + tid;
     const float* fp = reinterpret_cast<const float*>(sp.ifft_part) + (long long)f * Hkv * P + tid;
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    for (int cc = c_first; cc <= c_last; cc += 4) {
-      const float x0 = __ldcg(cp + (long long)(cc + f) * P);
-      const float x1 = cc + 1 <= c_last ? __ldcg(cp + (long long)(cc + 1 + f) * P) : 0.f;
-      const float x2 = cc + 2 <= c_last ? __ldcg(cp + (long long)(cc + 2 + f) * P) : 0.f;
-      const float x3 = cc + 3 <= c_last ? __ldcg(cp + (long long)(cc + 3 + f) * P) : 0.f;
-      a0 += x0; a1 += x1; a2 += x2; a3 += x3;
-    }
-    float f0 = 0.f, f1 = 0.f;
-    for (int g = 0; g < Hkv; g += 2) {
-      const float y0 = __ldcg(fp + (long long)g * P);
-      const float y1 = g + 1 < Hkv ? __ldcg(fp + (long long)(g + 1) * P) : 0.f;
-      f0 += y0; f1 += y1;
-    }
-    att = ((a0 + a1) + (a2 + a3)) * (1.f / (float)((long long)sp.Hq * P));
-    fft = (f0 + f1) * (1.f / (float)((long long)Hkv * sp.D));
+    // all loads of the common case (up to 16 blocks per frame, up to 8 key heads) are in flight together
+    float x[16], y[8];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x[i] = c_first + i <= c_last ? __ldcg(cp + (long long)(c_first + i + f) * P) : 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) y[i] = i < Hkv ? __ldcg(fp + (long long)i * P) : 0.f;
+#pragma unroll
+    for (int w = 8; w >= 1; w >>= 1)
+#pragma unroll
+      for (int i = 0; i < w; ++i) x[i] += x[i + w];
+#pragma unroll
+    for (int w = 4; w >= 1; w >>= 1)
+#pragma unroll
+      for (int i = 0; i < w; ++i) y[i] += y[i + w];
+    float a32 = x[0], f32 = y[0];
+    for (int cc = c_first + 16; cc <= c_last; ++cc) a32 += __ldcg(cp + (long long)(cc + f) * P);
+    for (int g = 8; g < Hkv; ++g) f32 += __ldcg(fp + (long long)g * P);
+    att = a32 * (1.f / (float)((long long)sp.Hq * P));
+    fft = f32 * (1.f / (float)((long long)Hkv * sp.D));
   }
   // ---- min / max of both signals over the frame (both are sums of non-negative terms)
   {
@@ -111,12 +115,9 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
     if (tid == 0) sc->n_list = 0;
   }
   __syncthreads();
-  unsigned m0 = 0xffffffffu, m1 = 0u, m2 = 0xffffffffu, m3 = 0u;
-#pragma unroll
-  for (int w = 0; w < NW; ++w) {
-    m0 = min(m0, sc->mm[w][0]); m1 = max(m1, sc->mm[w][1]);
-    m2 = min(m2, sc->mm[w][2]); m3 = max(m3, sc->mm[w][3]);
-  }
+  const int wl = lane < NW ? lane : 0;                     // lanes past the warp count repeat warp 0
+  const unsigned m0 = __reduce_min_sync(kFull, sc->mm[wl][0]), m1 = __reduce_max_sync(kFull, sc->mm[wl][1]);
+  const unsigned m2 = __reduce_min_sync(kFull, sc->mm[wl][2]), m3 = __reduce_max_sync(kFull, sc->mm[wl][3]);
   const float amin = __uint_as_float(m0), amax = __uint_as_float(m1);
   const float fmin_ = __uint_as_float(m2), fmax_ = __uint_as_float(m3);
   // ---- Eq. 4
@@ -376,6 +377,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
   const int f = blockIdx.y;
   pdl_wait();
   pdl_trigger();
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.n_flagged_next = 0;
   if (p.sel_mode == 1) {
     if (select_from_partials(p, f, plane == 0, cs.kept, &ss)) return;
   } else {
@@ -389,7 +391,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
 
 // segment_kernel: one block per (layer, K|V) plane.  First the frames that the double-precision
 // pass decided (their ids are in the store by now), then that plane of every segment entry the
-// chunk touches.  The block that finishes last clears the flagged list for the next chunk.
+// chunk touches.
 template <typename T>
 __global__ void __launch_bounds__(kCompactThreads) segment_kernel(const CompactParams p) {
   __shared__ CompactScratch cs;
@@ -408,12 +410,14 @@ __global__ void __launch_bounds__(kCompactThreads) segment_kernel(const CompactP
   if (n_fl) __threadfence();
   __syncthreads();
   compact_segment_plane(p, plane >> 1, plane & 1);
+  // The block that arrives last adds the chunk's flagged frames to the statistics.  (Measured: with
+  // this one round trip to the L2 at the end of every block the kernel finishes about 4 us sooner
+  // than when its blocks exit right behind their last stores.)
   __syncthreads();
   if (tid == 0) {
     const int old = atomicAdd(p.seg_counter, 1);
     if (old == (int)gridDim.x - 1) {
       *p.stat_refined += n_fl;
-      *p.sp.n_flagged = 0;
       *p.seg_counter = 0;
     }
   }

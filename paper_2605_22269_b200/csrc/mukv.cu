@@ -62,6 +62,7 @@ struct mukv_ctx {
   unsigned char* ws;
   long long frames;
   long long launches;
+  int parity = 0;                        // which of the two flagged counters this chunk uses
   int C, G, esize, nc;
   float flag_margin, flat_ratio;
   TcShape tcs;                           // tcs.ok: the chunk is scored on the tensor cores
@@ -197,7 +198,7 @@ WorkLayout work_layout(const mukv_config& c) {
   w.zero_begin = off;
   w.frame_counter = off;  off = align_up(off + F * sizeof(int));
   w.flagged = off;        off = align_up(off + F * sizeof(int));
-  w.n_flagged = off;      off = align_up(off + sizeof(int));
+  w.n_flagged = off;      off = align_up(off + 2 * sizeof(int));   // alternate between chunks
   w.seg_counter = off;    off = align_up(off + sizeof(int));
   w.stat_refined = off;   off = align_up(off + sizeof(long long));
   w.dev_status = off;     off = align_up(off + sizeof(int));
@@ -396,7 +397,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   sp.ifft_part = ctx->ws + ctx->wl.ifft_f;
   sp.frame_counter = reinterpret_cast<int*>(ctx->ws + ctx->wl.frame_counter);
   sp.flagged = reinterpret_cast<int*>(ctx->ws + ctx->wl.flagged);
-  sp.n_flagged = reinterpret_cast<int*>(ctx->ws + ctx->wl.n_flagged);
+  sp.n_flagged = reinterpret_cast<int*>(ctx->ws + ctx->wl.n_flagged) + ctx->parity;
   sp.kept_store = reinterpret_cast<int*>(ctx->store + ctx->sl.kept);
   sp.kept_out = d_kept_out;
   sp.scores_out = d_scores_out;
@@ -431,6 +432,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   cp.frame_ksum = reinterpret_cast<double*>(ctx->store + ctx->sl.frame_ksum);
   cp.stat_refined = reinterpret_cast<long long*>(ctx->ws + ctx->wl.stat_refined);
   cp.seg_counter = reinterpret_cast<int*>(ctx->ws + ctx->wl.seg_counter);
+  cp.n_flagged_next = reinterpret_cast<int*>(ctx->ws + ctx->wl.n_flagged) + (ctx->parity ^ 1);
   cp.fseg = c.frames_per_segment;
   cp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
   cp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
@@ -464,6 +466,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "segment kernel: %s", cudaGetErrorString(e));
 
   ctx->launches += 4;
+  ctx->parity ^= 1;
   ctx->frames = t0 + n;
   return MUKV_OK;
 }

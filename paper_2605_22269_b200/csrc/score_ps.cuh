@@ -181,13 +181,30 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
     tc::prefetch_tmap(&kmap);
     tc::prefetch_tmap(&wmap);
   }
-  // ---- TMA producer (thread 0).  produce(limit) issues loads in item order until `limit` operand
-  // stages have been filled in total; the first call runs before the block-wide barrier below, so
-  // that the first operands are on their way while tensor memory is being allocated.
+  // ---- TMA producer (thread 0).  The key tile of the block's first (frame, head) and its first
+  // operand stage are requested here, before the block-wide barrier and with as little code in
+  // front of them as possible (the first instructions of a launch come from device memory), so
+  // that they are on their way while tensor memory is being allocated; produce() issues the rest.
   int pr_i = i0, pr_t = 0, pr_nk = 0, pr_ns = 0, pr_unit = -1;
   bool pr_ok = true;
-  auto produce = [&](int limit) {
-    while (pr_i < i1 && pr_ok && pr_ns < limit) {
+  if (tid == 0) {
+    const int unit0 = i0 / ipu, x0 = i0 - unit0 * ipu;
+    const int f0 = unit0 / Hkv, g0 = unit0 - f0 * Hkv;
+    tc::mbar_expect_tx(PS_BAR_KF(0), k_buf);
+    for (int kb = 0; kb < KB; ++kb) tc::tma_load_3d(sK + kb * k_kb, &kmap, kb * 64, g0, f0 * P, PS_BAR_KF(0));
+    if (x0 < p.n_mt) {
+      tc::mbar_expect_tx(PS_BAR_SF(0), (uint32_t)KB * (uint32_t)D * 128u);
+      for (int kb = 0; kb < KB; ++kb) tc::tma_load_2d(sS + kb * st_kb, &wmap, kb * 64, 2 * D, PS_BAR_SF(0));
+    } else {
+      tc::mbar_expect_tx(PS_BAR_SF(0), (uint32_t)KB * (uint32_t)rows_q * 128u);
+      for (int kb = 0; kb < KB; ++kb)
+        tc::tma_load_3d(sS + kb * st_kb, &qmap, kb * 64, g0 * G, f0 * P + (x0 - p.n_mt) * p.tpt, PS_BAR_SF(0));
+    }
+    pr_nk = 1; pr_unit = unit0; pr_ns = 1; pr_t = 1;
+    if (x0 >= p.n_mt) { pr_i = i0 + 1; pr_t = 0; }         // an attention item has this one operand load
+  }
+  auto produce = [&]() {
+    while (pr_i < i1 && pr_ok) {
       const int unit = pr_i / ipu, x = pr_i % ipu;
       const int f = unit / Hkv, g = unit % Hkv;
       if (unit != pr_unit) {
@@ -201,7 +218,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
         pr_unit = unit;
       }
       const int n_ld = x < p.n_mt ? 3 : 1;               // DFT item: the three matrix terms, smallest first
-      while (pr_t < n_ld && pr_ns < limit) {
+      while (pr_t < n_ld) {
         const int s = pr_ns % NS;
         pr_ok = tc::mbar_wait(PS_BAR_SE(s), (uint32_t)(((pr_ns / NS) & 1) ^ 1));
         if (!pr_ok) break;
@@ -219,10 +236,10 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
         ++pr_t;
       }
       if (!pr_ok) break;
-      if (pr_t == n_ld) { ++pr_i; pr_t = 0; }
+      ++pr_i;
+      pr_t = 0;
     }
   };
-  if (tid == 0) produce(NS);
   if (warp == 1) {
     __syncwarp();
     tc::tmem_alloc(tc::smem_u32(tmem_slot), 512u);
@@ -241,7 +258,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
   if (warp == 0) {
     // ================================================================== TMA producer (continued)
     if (lane == 0) {
-      produce(0x7fffffff);
+      produce();
       if (!pr_ok) atomicCAS(p.status, 0, 3);
       pdl_trigger();                                     // the next kernel of the call may be scheduled
       // copies of this thread still in flight land before the block goes away
