@@ -232,7 +232,9 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
 }
 
 // Segment entries (Eq. 5 at segment level) of one (layer, K|V) plane for every segment the chunk
-// touches: mean over the frames present.  Run by one whole block.
+// touches: mean over the frames present, added in frame order.  Run by one whole block.  The loads
+// of up to 16 frames (and, in single precision, of two columns) are in flight together: the
+// kernel is a chain of L2 round trips and little else.
 __device__ inline void compact_segment_plane(const CompactParams& p, int l, int kv) {
   const int tid = threadIdx.x;
   const int C = p.C, kappa = p.kappa;
@@ -244,33 +246,40 @@ __device__ inline void compact_segment_plane(const CompactParams& p, int l, int 
     long long t1 = t0 + p.fseg;
     if (t1 > frames_total) t1 = frames_total;
     const int nf = (int)(t1 - t0);
-    for (int col = tid; col < C; col += kCompactThreads) {
-      float m;
-      // eight loads in flight at a time, added in frame order
-      if (exact) {
+    if (exact) {
+      for (int col = tid; col < C; col += kCompactThreads) {
         double t = 0.0;
-        for (long long ff = t0; ff < t1; ff += 8) {
-          double x[8];
+        for (long long ff = t0; ff < t1; ff += 16) {
+          double x[16];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) x[i] = ff + i < t1 ? __ldcg(p.frame_ksum + (ff + i) * C + col) : 0.0;
+          for (int i = 0; i < 16; ++i) x[i] = ff + i < t1 ? __ldcg(p.frame_ksum + (ff + i) * C + col) : 0.0;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) t += x[i];
+          for (int i = 0; i < 16; ++i) t += x[i];
         }
-        m = (float)(t / ((double)nf * (double)kappa));
+        const float m = (float)(t / ((double)nf * (double)kappa));
         p.seg_key[u * C + col] = m;
-      } else {
-        float t = 0.f;
-        for (long long ff = t0; ff < t1; ff += 8) {
-          float x[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            x[i] = ff + i < t1 ? __ldcg(p.frame_entry + (((ff + i) * p.L + l) * 2 + kv) * C + col) : 0.f;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) t += x[i];
-        }
-        m = t / (float)nf;
+        p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = m;
       }
-      p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = m;
+    } else {
+      for (int col = tid; col < C; col += 2 * kCompactThreads) {
+        const int col1 = col + kCompactThreads;
+        const bool two = col1 < C;
+        float ta = 0.f, tb = 0.f;
+        for (long long ff = t0; ff < t1; ff += 16) {
+          float xa[16], xb[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float* src = p.frame_entry + (((ff + i) * p.L + l) * 2 + kv) * C;
+            xa[i] = ff + i < t1 ? __ldcg(src + col) : 0.f;
+            xb[i] = (two && ff + i < t1) ? __ldcg(src + col1) : 0.f;
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { ta += xa[i]; tb += xb[i]; }
+        }
+        float* dst = p.seg_entry + ((u * p.L + l) * 2 + kv) * C;
+        dst[col] = ta / (float)nf;
+        if (two) dst[col1] = tb / (float)nf;
+      }
     }
   }
 }
