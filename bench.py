@@ -25,9 +25,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one score_ps_kernel launch on a 16-frame chunk of this
-# workload (ncu capture summarised in profiles/score_ps_kernel_chunk16.md)
-SCORE_TRAFFIC_BYTES = 25892608
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch on a 16-frame chunk of this workload
+# (ncu capture summarised in profiles/score_ps_kernel_chunk16.md)
+SCORE_TRAFFIC_BYTES = 25857792
+COMPACT_TRAFFIC_BYTES = 45178112 + 4190976
 
 METRIC = "compressed_frames_per_s"
 UNIT = "frames/s"
@@ -319,8 +320,9 @@ def main():
                         frac=ach / peak_tf, traffic=None,
                         peak_source="148 SMs x 128 fp32 FMA lanes x 2 flop x sampled SM clock")
     else:
+        traffic = COMPACT_TRAFFIC_BYTES if dom == "compact" and cfg.dtype == 0 and T % chunk == 0 and chunk == 16 else None
         roofline = dict(kernel=dom + "_kernel", bound="hbm", achieved=kernels[dom]["achieved_gbs"],
-                        peak=peaks["hbm_gbs"], unit="GB/s", frac=kernels[dom]["frac_of_hbm_peak"], traffic=None,
+                        peak=peaks["hbm_gbs"], unit="GB/s", frac=kernels[dom]["frac_of_hbm_peak"], traffic=traffic,
                         peak_source=peaks["source"] + " copy bandwidth")
     path_gbs = ab["per_frame"] * fps / world / 1e9
     retr_gbs = (ab["gather_per_question"] + ab["index_row"] * T / nq) * rps / world / 1e9
