@@ -25,7 +25,8 @@
 // (compact_kernel adds the slots in a fixed order): done here, by the block that finishes a frame
 // last, they kept one block per frame busy for microseconds after all others had finished.
 // All mbarrier waits are bounded; a wait that runs out makes the role record a code in the status
-// word and go on without waiting.
+// word; the producer and the MMA issuer then leave their loops, the epilogue warps go on without
+// waiting (their reads stay inside the accumulators).
 #pragma once
 #include "common.cuh"
 #include "score.cuh"
