@@ -194,11 +194,19 @@ __device__ __forceinline__ double order_key_inv(unsigned long long k) {
   return __longlong_as_double((long long)b);
 }
 
+constexpr int kRankList = 64;      // keys left in the radix select below which they are ranked directly
+constexpr int kRankCand = 256;     // scores at or above the tie band that the short emission path can hold
+
 struct RankScratch {
   unsigned int hist[256];
   int scan[40];
   unsigned long long prefix;
   int remaining;
+  int bin_count, list_n, cand_n;
+  unsigned long long list[kRankList];
+  int cand_idx[kRankCand];
+  double cand_s[kRankCand];
+  unsigned char cand_band[kRankCand], cand_keep[kRankCand];
 };
 
 // Indices of the k highest scores among i in [0,n) with member(i) true, ascending by index, with
@@ -262,13 +270,83 @@ __device__ int block_topk_set(ScoreFn score, MemberFn member, int n, int k, doub
           }
           sc->prefix = prefix | ((unsigned long long)(8 * tid + b) << shift);
           sc->remaining = r;
+          sc->bin_count = c[b];
         }
       }
       __syncthreads();
+      if (pass < 7 && sc->bin_count <= kRankList) {
+        // few keys share the prefix found so far: collect them and rank them directly
+        const unsigned long long pre = sc->prefix, mask = ~0ull << shift;
+        if (tid == 0) sc->list_n = 0;
+        __syncthreads();
+        for (int i = tid; i < n; i += nt) {
+          if (!member(i)) continue;
+          const unsigned long long key = order_key(score(i));
+          if ((key & mask) == pre) sc->list[atomicAdd(&sc->list_n, 1)] = key;
+        }
+        __syncthreads();
+        const int m = sc->list_n, r = sc->remaining;
+        if (tid < m) {
+          const unsigned long long key = sc->list[tid];
+          int gt = 0, ge = 0;
+          for (int t = 0; t < m; ++t) {
+            gt += (sc->list[t] > key);
+            ge += (sc->list[t] >= key);
+          }
+          if (gt < r && r <= ge) sc->prefix = key;      // every writer holds the same value
+        }
+        __syncthreads();
+        break;
+      }
     }
     tau = order_key_inv(sc->prefix);
   }
   const bool all = (k == n_mem);
+  // Everything at or above the tie band, collected in any order.  When that is a short list (it
+  // holds k entries plus the ties), the band rule and the ascending output order are worked out
+  // on the list; the ordered walk over all n scores below is the fallback for a crowded band.
+  if (tid == 0) sc->cand_n = 0;
+  __syncthreads();
+  for (int i = tid; i < n; i += nt) {
+    if (!member(i)) continue;
+    const double s = score(i);
+    const bool sure = all || s > tau + delta;
+    const bool band = !sure && s >= tau - delta;
+    if (sure || band) {
+      const int c = atomicAdd(&sc->cand_n, 1);
+      if (c < kRankCand) {
+        sc->cand_idx[c] = i;
+        sc->cand_s[c] = s;
+        sc->cand_band[c] = band ? 1 : 0;
+      }
+    }
+  }
+  __syncthreads();
+  const int n_cand = sc->cand_n;
+  if (n_cand <= kRankCand) {
+    bool keep = false;
+    int my_idx = 0;
+    if (tid < n_cand) {
+      my_idx = sc->cand_idx[tid];
+      int n_sure = 0, band_before = 0;
+      for (int t = 0; t < n_cand; ++t) {
+        const bool bt = sc->cand_band[t] != 0;
+        n_sure += bt ? 0 : 1;
+        band_before += (bt && sc->cand_idx[t] < my_idx) ? 1 : 0;
+      }
+      keep = !sc->cand_band[tid] || band_before < k - n_sure;
+      sc->cand_keep[tid] = keep ? 1 : 0;
+    }
+    __syncthreads();
+    if (keep) {
+      int pos = 0;
+      for (int t = 0; t < n_cand; ++t) pos += (sc->cand_keep[t] && sc->cand_idx[t] < my_idx) ? 1 : 0;
+      out_idx[pos] = my_idx;
+      if (out_score) out_score[pos] = sc->cand_s[tid];
+    }
+    __syncthreads();
+    return k;
+  }
   // count the sure ones
   int cnt = 0;
   for (int i = tid; i < n; i += nt)
