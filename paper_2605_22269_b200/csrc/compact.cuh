@@ -121,8 +121,11 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
   const float amin = __uint_as_float(m0), amax = __uint_as_float(m1);
   const float fmin_ = __uint_as_float(m2), fmax_ = __uint_as_float(m3);
   // ---- Eq. 4
-  const float an = (amax == amin) ? 0.f : (att - amin) / (amax - amin);
-  float fn = (fmax_ == fmin_) ? 0.f : (fft - fmin_) / (fmax_ - fmin_);
+  // (one reciprocal per signal, the same in every thread, instead of a division per token)
+  const float inv_a = (amax == amin) ? 0.f : 1.f / (amax - amin);
+  const float inv_f = (fmax_ == fmin_) ? 0.f : 1.f / (fmax_ - fmin_);
+  const float an = (att - amin) * inv_a;
+  float fn = (fft - fmin_) * inv_f;
   if (sp.keep_low) fn = 1.f - fn;
   const float s = sp.alpha * an + (1.f - sp.alpha) * fn;
   const int key = __float_as_int(s);

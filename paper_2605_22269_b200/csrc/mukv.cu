@@ -675,11 +675,10 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
     const unsigned blocks = (unsigned)((rows + kScanRows - 1) / kScanRows);
     {
       ProfScope ps(ctx, 5, st);
-      scan_kernel<<<blocks, 256, 0, st>>>(frame_key, seg_key, n_frm, n_seg, C, nq,
-                                                                           q64, qnorm, s_frm, s_seg, c.max_frames,
-                                                                           ctx->sl.max_segs);
+      e = launch_k(scan_kernel, dim3(blocks), 256, 0, st, !ctx->prof_on, frame_key, seg_key, n_frm, n_seg, C, nq,
+                   (const double*)q64, (const double*)qnorm, s_frm, s_seg, (long long)c.max_frames,
+                   (long long)ctx->sl.max_segs);
     }
-    e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "scan kernel: %s", cudaGetErrorString(e));
     RankParams rp;
     memset(&rp, 0, sizeof rp);
@@ -697,9 +696,8 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
       const size_t staged = rank_smem + (size_t)(n_frm + n_seg) * sizeof(double);
       rp.stage = staged <= (size_t)kRankStageBytes ? 1 : 0;
       if (rp.stage) rank_smem = staged;
-      rank_kernel<<<nq, kRankThreads, rank_smem, st>>>(rp, meta);
+      e = launch_k(rank_kernel, dim3(nq), kRankThreads, rank_smem, st, !ctx->prof_on, rp, meta);
     }
-    e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "rank kernel: %s", cudaGetErrorString(e));
     ctx->launches += 4;
     return MUKV_OK;

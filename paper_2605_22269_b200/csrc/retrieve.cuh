@@ -120,6 +120,8 @@ __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ fra
   __shared__ __align__(16) double qs[kScanCC][kScanQPad];
   __shared__ double s_knorm[kScanRows];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_wait();                                                // the pooled questions are complete
+  pdl_trigger();
   const long long row0 = (long long)blockIdx.x * kScanRows;
   const long long n_rows = n_frm + n_seg;
   const int lr = tid >> 3, lc = (tid & 7) * 8;               // staging: row, first column of 8
@@ -421,6 +423,7 @@ __global__ void __launch_bounds__(kRankThreads) rank_kernel(const RankParams p, 
   __shared__ double s_gn;
 
   const int qi = blockIdx.x, tid = threadIdx.x;
+  pdl_wait();                                                // the scores of the scan are complete
   const int C = p.C;
   long long tl = meta.t_limit[qi];
   if (tl > p.n_frm) tl = p.n_frm;
