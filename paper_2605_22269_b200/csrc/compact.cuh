@@ -49,6 +49,8 @@ struct CompactParams {
   // selection
   int sel_mode;                   // 0: kept ids are in the store; 1: select here from the partial sums
   int ps_grid, ps_items, ps_ipf;  // the scoring launch: blocks, items, items per frame
+  unsigned* sel_flag;             // [F] (epoch << 1 | risky) once the plane-0 block has published its frame's ids
+  unsigned epoch;                 // number of this call, never repeated
   ScoreParams sp;                 // partial sums, Eq. 4 parameters, index and flag outputs
 };
 
@@ -384,17 +386,45 @@ template <typename T>
 __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactParams p) {
   __shared__ CompactScratch cs;
   __shared__ SelectScratch ss;
+  __shared__ unsigned s_seen;
   const int tid = threadIdx.x;
-  const int plane = blockIdx.x;                 // l*2 + kv
-  const int f = blockIdx.y;
+  // frame is the fast block index: the blocks that start first cover the low planes of every frame,
+  // the plane-0 blocks among them
+  const int f = blockIdx.x;
+  const int plane = blockIdx.y;                 // l*2 + kv
   pdl_wait();
   pdl_trigger();
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.n_flagged_next = 0;
+  const long long f_abs = p.first_frame + f;
   if (p.sel_mode == 1) {
-    if (select_from_partials(p, f, plane == 0, cs.kept, &ss)) return;
+    // A block that starts after its frame's plane-0 block has published the ids (the blocks beyond
+    // the first wave do) reads them; every other block selects itself.  Nobody waits.
+    if (tid == 0) {
+      unsigned v = 0u;
+      if (plane != 0) {
+        v = *reinterpret_cast<volatile unsigned*>(p.sel_flag + f);
+        __threadfence();
+      }
+      s_seen = v;
+    }
+    __syncthreads();
+    const unsigned seen = s_seen;
+    bool risky;
+    if ((seen >> 1) == p.epoch) {
+      risky = (seen & 1u) != 0u;
+      for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = __ldcg(p.sp.kept_store + f_abs * p.kappa + r);
+      __syncthreads();
+    } else {
+      risky = select_from_partials(p, f, plane == 0, cs.kept, &ss);
+      if (plane == 0) {
+        __threadfence();                        // this thread's ids are visible before the flag is
+        __syncthreads();
+        if (tid == 0) *reinterpret_cast<volatile unsigned*>(p.sel_flag + f) = (p.epoch << 1) | (risky ? 1u : 0u);
+      }
+    }
+    if (risky) return;
   } else {
     if (frame_is_flagged(p.sp.flagged, *p.sp.n_flagged, f)) return;
-    const long long f_abs = p.first_frame + f;
     for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = p.sp.kept_store[f_abs * p.kappa + r];
     __syncthreads();
   }

@@ -36,7 +36,7 @@ struct StoreLayout {
 };
 
 struct WorkLayout {
-  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, seg_counter, stat_refined,
+  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, seg_counter, sel_flag, stat_refined,
       dev_status;
   size_t q64, qnorm, s_frm, s_seg, wtab, total;
   size_t zero_begin, zero_end;          // region that must start as zeros
@@ -63,6 +63,7 @@ struct mukv_ctx {
   long long frames;
   long long launches;
   int parity = 0;                        // which of the two flagged counters this chunk uses
+  unsigned epoch = 0;                    // compress calls so far (tags the per-frame selection flags)
   int C, G, esize, nc;
   float flag_margin, flat_ratio;
   TcShape tcs;                           // tcs.ok: the chunk is scored on the tensor cores
@@ -200,6 +201,7 @@ WorkLayout work_layout(const mukv_config& c) {
   w.flagged = off;        off = align_up(off + F * sizeof(int));
   w.n_flagged = off;      off = align_up(off + 2 * sizeof(int));   // alternate between chunks
   w.seg_counter = off;    off = align_up(off + sizeof(int));
+  w.sel_flag = off;       off = align_up(off + F * sizeof(unsigned));
   w.stat_refined = off;   off = align_up(off + sizeof(long long));
   w.dev_status = off;     off = align_up(off + sizeof(int));
   w.zero_end = off;
@@ -432,6 +434,8 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   cp.frame_ksum = reinterpret_cast<double*>(ctx->store + ctx->sl.frame_ksum);
   cp.stat_refined = reinterpret_cast<long long*>(ctx->ws + ctx->wl.stat_refined);
   cp.seg_counter = reinterpret_cast<int*>(ctx->ws + ctx->wl.seg_counter);
+  cp.sel_flag = reinterpret_cast<unsigned*>(ctx->ws + ctx->wl.sel_flag);
+  cp.epoch = (++ctx->epoch) & 0x7fffffffu;
   cp.n_flagged_next = reinterpret_cast<int*>(ctx->ws + ctx->wl.n_flagged) + (ctx->parity ^ 1);
   cp.fseg = c.frames_per_segment;
   cp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
@@ -442,7 +446,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   if (ps_grid > 0) cp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
   {
     ProfScope ps(ctx, 2, st);
-    e = launch_k(compact_kernel<T>, dim3(L * 2, n), kCompactThreads, 0, st, !ctx->prof_on, cp);
+    e = launch_k(compact_kernel<T>, dim3(n, L * 2), kCompactThreads, 0, st, !ctx->prof_on, cp);
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "compact kernel: %s", cudaGetErrorString(e));
 
