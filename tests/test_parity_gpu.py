@@ -149,6 +149,15 @@ def test_chunk7b_causal():
     full_compress_check(run)
 
 
+@pytest.mark.parametrize("chunk", [1, 3])
+def test_chunk7b_small_chunks(chunk):
+    # a one-frame chunk spreads a frame over 52 scoring blocks (more partial sums than the selection
+    # loads in one batch); three-frame chunks leave block shares that straddle frames
+    run = H.GpuRun("chunk7b", n_frames=4)
+    full_compress_check(run, chunk=chunk)
+    assert run.ctx.mukv_get_stats().device_status == 0
+
+
 def test_chunk7b_tile_block_scoring(monkeypatch):
     # the one-tile-per-block tensor-core kernel (used when the persistent kernel's buffers do not fit)
     monkeypatch.setenv("MUKV_SCORE_TILE_BLOCKS", "1")
