@@ -98,7 +98,7 @@ class ClockSampler:
 
 
 def algorithmic_bytes(cfg, k_frm: int) -> dict:
-    """Bytes the method has to move, per unit ('Rooflines')."""
+    """Bytes the method has to move, per unit of work (frame, question, index row)."""
     es = 2 if cfg.dtype == 0 else 4
     C = cfg.n_kv_heads * cfg.head_dim
     P, L, kap = cfg.tokens_per_frame, cfg.n_layers, cfg.keep_per_frame
