@@ -206,7 +206,7 @@ WorkLayout work_layout(const mukv_config& c) {
   w.dev_status = off;     off = align_up(off + sizeof(int));
   w.zero_end = off;
   w.q64 = off;            off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * C * sizeof(double));
-  w.qnorm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * sizeof(double));
+  w.qnorm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * c.n_kv_heads * sizeof(double));
   w.s_frm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * c.max_frames * sizeof(double));
   w.s_seg = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * max_segs * sizeof(double));
   w.wtab = off;           off = align_up(off + (ts.ok ? (size_t)3 * c.head_dim * c.head_dim * 2 : 0));
@@ -667,10 +667,10 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
     {
       ProfScope ps(ctx, 4, st);
       if (c.dtype == MUKV_BF16)
-        qpool_kernel<__nv_bfloat16><<<nq, kPoolThreads, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(d_qtok), meta,
+        qpool_kernel<__nv_bfloat16><<<dim3(nq, c.n_kv_heads), kPoolThreads, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(d_qtok), meta,
                                                        c.n_q_heads, c.n_kv_heads, c.head_dim, q64, qnorm);
       else
-        qpool_kernel<float><<<nq, kPoolThreads, 0, st>>>(reinterpret_cast<const float*>(d_qtok), meta, c.n_q_heads,
+        qpool_kernel<float><<<dim3(nq, c.n_kv_heads), kPoolThreads, 0, st>>>(reinterpret_cast<const float*>(d_qtok), meta, c.n_q_heads,
                                                c.n_kv_heads, c.head_dim, q64, qnorm);
     }
     cudaError_t e = cudaGetLastError();
@@ -680,7 +680,7 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
     {
       ProfScope ps(ctx, 5, st);
       e = launch_k(scan_kernel, dim3(blocks), 256, 0, st, !ctx->prof_on, frame_key, seg_key, n_frm, n_seg, C, nq,
-                   (const double*)q64, (const double*)qnorm, s_frm, s_seg, (long long)c.max_frames,
+                   (const double*)q64, (const double*)qnorm, (int)c.n_kv_heads, s_frm, s_seg, (long long)c.max_frames,
                    (long long)ctx->sl.max_segs);
     }
     if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "scan kernel: %s", cudaGetErrorString(e));

@@ -4,7 +4,7 @@
 // All ranking arithmetic is double precision: the work is a few hundred MFLOP per batch of
 // questions, tiny next to the gather, and it makes the selected indices independent of
 // summation order.  Kernels:
-//   qpool_kernel    Eq. 6   one block per question
+//   qpool_kernel    Eq. 6   one block per (question, key head)
 //   scan_kernel     Eq. 7   cosine of every question with every frame key and segment key (a skinny
 //                           double-precision product on the fp64 tensor-core instruction)
 //   rank_kernel     stage-1 candidates, Eq. 8 rerank, final top-k; one block per question
@@ -20,31 +20,30 @@ struct QMeta {
 };
 
 // ------------------------------------------------------------------------------ Eq. 6
-// One block per question.  Thread (slice, vector) sums one 16-byte vector of channels over the
-// tokens n = slice, slice + kPoolSlices, ... and the G query heads of its key group: every load is
-// a full 16-byte vector and all of a thread's loads are independent.  The slices are added in a
-// fixed order.  The pooled query is written transposed, q64t[c][question] (row stride
-// MUKV_MAX_QUESTIONS), the layout scan_kernel stages.
+// One block per (question, key head).  Thread (slice, vector) sums one 16-byte vector of the head's
+// channels over the tokens n = slice, slice + slices, ... and the G query heads of the group: every
+// load is a full 16-byte vector and all of a thread's loads are independent.  The slices are added
+// in a fixed order.  The pooled query is written transposed, q64t[c][question] (row stride
+// MUKV_MAX_QUESTIONS), the layout scan_kernel stages; the head's share of the squared norm goes to
+// qn2[question][key head] (scan_kernel adds the shares in head order).
 constexpr int kPoolThreads = 1024;
-constexpr int kPoolSmemDoubles = 5632;
+constexpr int kPoolSmemDoubles = 4096;
 
 template <typename T>
 __global__ void __launch_bounds__(kPoolThreads) qpool_kernel(const T* __restrict__ qtok, const QMeta meta, int Hq,
                                                              int Hkv, int D, double* __restrict__ q64t,
-                                                             double* __restrict__ qnorm) {
+                                                             double* __restrict__ qn2) {
   constexpr int VE = 16 / sizeof(T);
   __shared__ double s_acc[kPoolSmemDoubles];
   __shared__ double s_part[kPoolThreads / 32];
-  const int qi = blockIdx.x;
-  const int C = Hkv * D, G = Hq / Hkv;
+  const int qi = blockIdx.x, g = blockIdx.y;
+  const int G = Hq / Hkv;
   const int n0 = meta.off[qi], n1 = meta.off[qi + 1];
-  const int NV = C / VE, DV = D / VE;                       // vectors per pooled row / per head
-  int nsl = kPoolSmemDoubles / C;                           // token slices whose partial sums fit
-  if (nsl > kPoolThreads / NV) nsl = kPoolThreads / NV;
-  if (nsl < 1) nsl = 1;
-  for (int idx = threadIdx.x; idx < nsl * NV; idx += kPoolThreads) {
-    const int sl = idx / NV, cv = idx % NV;
-    const int g = cv / DV, dv = cv % DV;
+  const int DV = D / VE;                                    // vectors per head
+  int nsl = kPoolThreads / DV;                              // token slices whose partial sums fit
+  if (nsl > kPoolSmemDoubles / D) nsl = kPoolSmemDoubles / D;
+  const int sl = threadIdx.x / DV, dv = threadIdx.x % DV;
+  if (sl < nsl) {
     double tot[VE];
 #pragma unroll
     for (int e = 0; e < VE; ++e) tot[e] = 0.0;
@@ -70,15 +69,15 @@ __global__ void __launch_bounds__(kPoolThreads) qpool_kernel(const T* __restrict
       }
     }
 #pragma unroll
-    for (int e = 0; e < VE; ++e) s_acc[sl * C + cv * VE + e] = tot[e];
+    for (int e = 0; e < VE; ++e) s_acc[sl * D + dv * VE + e] = tot[e];
   }
   __syncthreads();
   double sq = 0.0;
-  for (int col = threadIdx.x; col < C; col += kPoolThreads) {
+  for (int col = threadIdx.x; col < D; col += kPoolThreads) {
     double t = 0.0;
-    for (int sl = 0; sl < nsl; ++sl) t += s_acc[sl * C + col];
+    for (int k = 0; k < nsl; ++k) t += s_acc[k * D + col];
     t = t / (double)((long long)(n1 - n0) * G);
-    q64t[(long long)col * MUKV_MAX_QUESTIONS + qi] = t;
+    q64t[(long long)(g * D + col) * MUKV_MAX_QUESTIONS + qi] = t;
     sq += t * t;
   }
   sq = warp_sum(sq);
@@ -87,7 +86,7 @@ __global__ void __launch_bounds__(kPoolThreads) qpool_kernel(const T* __restrict
   if (threadIdx.x == 0) {
     double t = 0.0;
     for (int w = 0; w < kPoolThreads / 32; ++w) t += s_part[w];
-    qnorm[qi] = sqrt(t);
+    qn2[(long long)qi * Hkv + g] = t;
   }
 }
 
@@ -113,15 +112,21 @@ __device__ __forceinline__ void dmma_m8n8k4(double (&c)[2], double a, double b) 
 __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ frame_key,
                                                    const float* __restrict__ seg_key, long long n_frm,
                                                    long long n_seg, int C, int nq, const double* __restrict__ q64t,
-                                                   const double* __restrict__ qnorm, double* __restrict__ s_frm,
+                                                   const double* __restrict__ qn2, int Hkv, double* __restrict__ s_frm,
                                                    double* __restrict__ s_seg, long long frm_stride,
                                                    long long seg_stride) {
   __shared__ float rows[kScanRows][kScanCC + 1];
   __shared__ __align__(16) double qs[kScanCC][kScanQPad];
   __shared__ double s_knorm[kScanRows];
+  __shared__ double s_qn[MUKV_MAX_QUESTIONS];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_wait();                                                // the pooled questions are complete
   pdl_trigger();
+  for (int qq = tid; qq < nq; qq += 256) {                   // norms of the pooled questions (read after the barriers below)
+    double t = 0.0;
+    for (int gg = 0; gg < Hkv; ++gg) t += qn2[(long long)qq * Hkv + gg];
+    s_qn[qq] = sqrt(t);
+  }
   const long long row0 = (long long)blockIdx.x * kScanRows;
   const long long n_rows = n_frm + n_seg;
   const int lr = tid >> 3, lc = (tid & 7) * 8;               // staging: row, first column of 8
@@ -175,7 +180,7 @@ __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ fra
         for (int j = 0; j < 2; ++j) {
           const int qi = qb + wq + nt * 8 + 2 * fk + j;
           if (qi >= nq) continue;
-          double den = knorm * qnorm[qi];
+          double den = knorm * s_qn[qi];
           den = den > 1e-12 ? den : 1e-12;
           const double sc = acc[nt][j] / den;
           if (row < n_frm) s_frm[(long long)qi * frm_stride + row] = sc;
