@@ -26,7 +26,7 @@ struct QMeta {
 // in a fixed order.  The pooled query is written transposed, q64t[c][question] (row stride
 // MUKV_MAX_QUESTIONS), the layout scan_kernel stages; the head's share of the squared norm goes to
 // qn2[question][key head] (scan_kernel adds the shares in head order).
-constexpr int kPoolThreads = 1024;
+constexpr int kPoolThreads = 512;
 constexpr int kPoolSmemDoubles = 4096;
 
 template <typename T>
@@ -140,20 +140,37 @@ __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ fra
 #pragma unroll
     for (int i = 0; i < 4; ++i) { acc[i][0] = 0.0; acc[i][1] = 0.0; }
     double kk = 0.0;
+    // the chunk after the one being multiplied is already on its way into registers
+    float xr[8];
+    double xq[kScanCC * kScanQB / 256];
+    auto fetch = [&](int c0) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int cc = lc + i;
+        xr[i] = (src && c0 + cc < C) ? src[c0 + cc] : 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < kScanCC * kScanQB / 256; ++i) {
+        const int idx = tid + i * 256;
+        const int cc = idx / kScanQB, qq = idx % kScanQB;
+        xq[i] = (c0 + cc < C && qb + qq < nq) ? q64t[(long long)(c0 + cc) * MUKV_MAX_QUESTIONS + qb + qq] : 0.0;
+      }
+    };
+    fetch(0);
     for (int c0 = 0; c0 < C; c0 += kScanCC) {
       __syncthreads();                                       // the previous chunk has been consumed
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const int cc = lc + i;
-        const float x = (src && c0 + cc < C) ? src[c0 + cc] : 0.f;
-        rows[lr][cc] = x;
-        kk = fma((double)x, (double)x, kk);
+        rows[lr][lc + i] = xr[i];
+        kk = fma((double)xr[i], (double)xr[i], kk);
       }
-      for (int idx = tid; idx < kScanCC * kScanQB; idx += 256) {
-        const int cc = idx / kScanQB, qq = idx % kScanQB;
-        qs[cc][qq] = (c0 + cc < C && qb + qq < nq) ? q64t[(long long)(c0 + cc) * MUKV_MAX_QUESTIONS + qb + qq] : 0.0;
+#pragma unroll
+      for (int i = 0; i < kScanCC * kScanQB / 256; ++i) {
+        const int idx = tid + i * 256;
+        qs[idx / kScanQB][idx % kScanQB] = xq[i];
       }
       __syncthreads();
+      if (c0 + kScanCC < C) fetch(c0 + kScanCC);
 #pragma unroll 4
       for (int cc = 0; cc < kScanCC; cc += 4) {
         const double a = (double)rows[wr + fr][cc + fk];     // A[row fr][k fk]
@@ -220,8 +237,19 @@ struct RankScratch {
 // the tie band: tau = k-th largest; scores above tau+delta are taken; those within delta of tau
 // share the remaining places by lowest index.  Run by the whole block; returns the count
 // (= min(k, number of members)).  score(i) must be cheap and pure.
+// score(i) read from an array; every index a member.  One pair of types for the selections over
+// segments, frames and candidates, so that they share one copy of block_topk_set (kept out of
+// line: the ranking kernel is bound by instruction fetch, not by arithmetic).
+struct ArrScore {
+  const double* p;
+  __device__ double operator()(int i) const { return p[i]; }
+};
+struct AllMembers {
+  __device__ bool operator()(int) const { return true; }
+};
+
 template <typename ScoreFn, typename MemberFn>
-__device__ int block_topk_set(ScoreFn score, MemberFn member, int n, int k, double delta, int* out_idx,
+__device__ __noinline__ int block_topk_set(ScoreFn score, MemberFn member, int n, int k, double delta, int* out_idx,
                               double* out_score, RankScratch* sc) {
   const int tid = threadIdx.x, nt = blockDim.x;
   // how many members are there at all
@@ -450,9 +478,8 @@ __global__ void __launch_bounds__(kRankThreads) rank_kernel(const RankParams p, 
     sf = st_f;
     ss = st_s;
   }
-  auto seg_score = [&](int i) { return ss[i]; };
-  auto frm_score = [&](int i) { return sf[i]; };
-  auto always = [](int) { return true; };
+  const ArrScore seg_score{ss}, frm_score{sf};
+  const AllMembers always;
 
   // ---- segments: lambda = 0, final = stage-1 top-k
   const int c_seg = block_topk_set(seg_score, always, n_seg, p.k_seg, p.delta, s_sel_seg, s_sel_seg_score, &sc);
@@ -517,7 +544,7 @@ __global__ void __launch_bounds__(kRankThreads) rank_kernel(const RankParams p, 
       }
     }
     __syncthreads();
-    auto new_score = [&](int i) { return s_new[i]; };
+    const ArrScore new_score{s_new};
     c_frm = block_topk_set(new_score, always, n_cand, p.k_frm, p.delta, s_pick, s_pick_score, &sc);
     // s_pick holds positions in the candidate list (ascending position = ascending frame id)
     for (int i = tid; i < c_frm; i += kRankThreads) s_pick[i] = s_cand[s_pick[i]];
