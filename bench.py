@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch on a 16-frame chunk of this workload
 # (ncu capture summarised in profiles/score_ps_kernel_chunk16.md)
 SCORE_TRAFFIC_BYTES = 25857792
-COMPACT_TRAFFIC_BYTES = 45180416 + 4244480
+COMPACT_TRAFFIC_BYTES = 45182464 + 3919104
 
 METRIC = "compressed_frames_per_s"
 UNIT = "frames/s"
