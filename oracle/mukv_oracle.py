@@ -153,6 +153,19 @@ def keep_count(rho: float, n_tokens: int) -> int:
     return int(np.floor(rho * n_tokens + 1e-9))
 
 
+def select_tokens(I, kappa: int, delta: float = TIE_EPS) -> np.ndarray:
+    """Kept token ids of one block from its fused scores (Sec. 3.3, "Granularity Adaptive
+    Compression": the kappa highest scores stay), ascending.
+
+    The paper does not say what happens when a score is not a number (Inf or NaN among the
+    inputs).  Reading: such a block has no ranking, and its first kappa tokens are kept.
+    """
+    I = np.asarray(I, dtype=np.float64)
+    if not np.all(np.isfinite(I)):
+        return np.arange(min(int(kappa), I.shape[0]), dtype=np.int64)
+    return topk_set(I, kappa, delta)
+
+
 def score_frame(Q, K_last, alpha, causal=False, keep_low_freq=False):
     """(I_att, I_fft, I) for one frame."""
     ia = attention_importance(Q, K_last, causal)
@@ -234,7 +247,7 @@ def compress_chunk(store: Store, Q, K, V) -> None:
         Vf = np.asarray(V)[:, f]
         ia, ifr, I = score_frame(np.asarray(Q)[f], Kf[-1], cfg["alpha"],
                                  cfg.get("attn_causal", False), cfg.get("keep_low_freq", False))
-        kept = topk_set(I, cfg["keep_per_frame"], cfg.get("tie_eps", TIE_EPS))
+        kept = select_tokens(I, cfg["keep_per_frame"], cfg.get("tie_eps", TIE_EPS))
         pk = compact_rows(Kf, kept)
         pv = compact_rows(Vf, kept)
         store.kept.append(kept)

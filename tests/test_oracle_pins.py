@@ -182,6 +182,27 @@ def test_topk_set_budget_and_shape():
     assert O.topk_set(np.zeros(8), 3).tolist() == [0, 1, 2]
 
 
+def test_select_tokens_non_finite_rule():
+    # finite scores: the top-kappa rule; any Inf or NaN: no ranking, the first kappa tokens
+    rng = np.random.default_rng(8)
+    s = rng.random(40)
+    assert O.select_tokens(s, 7).tolist() == O.topk_set(s, 7).tolist()
+    for bad in (np.nan, np.inf, -np.inf):
+        t = s.copy()
+        t[33] = bad
+        assert O.select_tokens(t, 7).tolist() == list(range(7))
+    # through the whole frame path: one infinite key makes the frame's scores NaN
+    Q = rng.standard_normal((1, 12, 2, 8)).astype(np.float32)
+    K = rng.standard_normal((1, 1, 12, 2, 8)).astype(np.float32)
+    K[0, 0, 4, 1, 2] = np.inf
+    st = O.Store(dict(n_layers=1, n_q_heads=2, n_kv_heads=2, head_dim=8, tokens_per_frame=12, keep_per_frame=5,
+                      frames_per_segment=2, alpha=0.7))
+    with np.errstate(all="ignore"):
+        O.compress_chunk(st, Q, K, K)
+    assert st.kept[0].tolist() == [0, 1, 2, 3, 4]
+    assert not np.all(np.isfinite(st.scores[0][2]))
+
+
 def test_budget_matches_paper_token_counts():
     path = os.path.join(os.path.dirname(__file__), "golden", "paper_token_counts.txt")
     rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
