@@ -26,8 +26,13 @@
  *   - Errors: every entry point returns a mukv_status.  Argument errors are detected on the
  *     host before anything is enqueued and leave the store unchanged.  No C++ exception
  *     crosses this boundary.  mukv_last_error() gives a readable message.
- *   - Threading: one context is used by one host thread at a time.  mukv_retrieve and
- *     mukv_gather only read the store.
+ *   - Threading: one context is used by one host thread at a time, and the calls on one context
+ *     must also be ordered on the device (the same stream, or streams joined by events): every
+ *     call, mukv_retrieve included, keeps intermediate results in the context's workspace.
+ *     mukv_retrieve and mukv_gather do not modify the store.
+ *   - A launch failure in the middle of mukv_compress_chunk (MUKV_E_CUDA after part of the call
+ *     was enqueued) leaves the chunk half stored: the context then answers MUKV_E_STATE to every
+ *     call except mukv_reset, mukv_get_stats and mukv_destroy.
  *
  * Tensor layouts are token-major; element type is mukv_config.dtype (bf16 or fp32):
  *     Q   [n_frames][P][Hq][D]        last-layer queries of the chunk's visual tokens
@@ -97,7 +102,12 @@ typedef struct {
   int64_t refined_frames;        /* frames whose selection was redone in double         */
   int64_t refined_questions;     /* reserved (retrieval always scores in double)        */
   int64_t kernel_launches;       /* kernels launched by this context since creation     */
-  int32_t device_status;         /* 0, or a device-side consistency code                */
+  int32_t device_status;         /* 0, or the first device-side event code recorded:
+                                    3, 4, 5  a bounded wait inside the tensor-core scoring kernel
+                                             ran out (producer, MMA issuer, epilogue): the chunk's
+                                             scores are not to be trusted;
+                                    7        a frame's scores were not finite (Inf/NaN inputs):
+                                             its kappa lowest token ids were kept            */
   int32_t reserved;
 } mukv_stats;
 
@@ -114,8 +124,22 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
                         void* d_workspace, size_t workspace_bytes, mukv_ctx** out);
 void mukv_destroy(mukv_ctx* ctx);
 
-/* Forgets every stored frame (capacity and buffers are kept).  Stream-ordered. */
+/* Forgets every stored frame (capacity and buffers are kept) and clears the counters behind
+ * mukv_get_stats (refined_frames, device_status).  The host-side frame counter is reset at once;
+ * the device-side counters are cleared by a memset enqueued on `stream`, so the call must be
+ * ordered after the context's earlier work like any other call. */
 mukv_status mukv_reset(mukv_ctx* ctx, mukv_stream stream);
+
+/* Options of a context.  They exist for tests and experiments; the defaults are what the
+ * parity guarantees are stated for.
+ *   MUKV_OPT_FLAG_MARGIN  frames whose lowest kept and highest dropped fused score differ by less
+ *                         than tie_eps + margin are re-scored in double precision.  The built-in
+ *                         margin (3e-6) can only be raised: smaller values return MUKV_E_INVALID.
+ *   MUKV_OPT_SCORE_PATH   0 (default): bf16 chunks are scored on the tensor cores, fp32 chunks by
+ *                         the multiply-add kernel;  1: the multiply-add kernel for every dtype.
+ * Takes effect from the next mukv_compress_chunk. */
+typedef enum { MUKV_OPT_FLAG_MARGIN = 0, MUKV_OPT_SCORE_PATH = 1 } mukv_option;
+mukv_status mukv_set_option(mukv_ctx* ctx, int32_t option, double value);
 
 /* Sec. 3.3 + Eq. 5.  Compresses frames first_frame .. first_frame+n_frames-1.
  *   d_q [n_frames][P][Hq][D], d_k / d_v [L][n_frames][P][Hkv][D]: inputs, read only.
@@ -129,6 +153,8 @@ mukv_status mukv_reset(mukv_ctx* ctx, mukv_stream stream);
  * entry of every segment the chunk touches (mean over the frames present so far).
  * Frames whose selection lies too close to a tie boundary for single precision are
  * re-scored in double precision on the device before they are stored.
+ * A frame whose fused scores are not all finite (Inf or NaN among its inputs) has no ranking:
+ * its kappa lowest token ids are kept and device_status 7 is recorded.
  * Errors: INVALID, ALIGN, STATE (first_frame), CAPACITY (n_frames, store full), CUDA. */
 mukv_status mukv_compress_chunk(mukv_ctx* ctx, const void* d_q, const void* d_k, const void* d_v,
                                 int32_t n_frames, int64_t first_frame,
@@ -201,7 +227,7 @@ mukv_status mukv_profile_read(mukv_ctx* ctx, double* ms, int64_t* launches);
  * frame the method would keep.
  *
  *   cfg        shapes and method parameters; n_layers, frames_per_segment, max_frames and
- *              max_frames_per_chunk are ignored.  Limits: n_frames <= MUKV_NOALLOC_MAX_FRAMES,
+ *              max_frames_per_chunk are ignored (whatever they hold).  Limits: n_frames <= MUKV_NOALLOC_MAX_FRAMES,
  *              n_q_heads <= MUKV_NOALLOC_MAX_Q_HEADS, n_kv_heads <= MUKV_NOALLOC_MAX_KV_HEADS,
  *              tokens_per_frame <= MUKV_MAX_TOKENS; larger requests return MUKV_E_CAPACITY.
  *   d_q        [n_frames][P][Hq][D] last-layer queries;  d_k_last [n_frames][P][Hkv][D] last-layer

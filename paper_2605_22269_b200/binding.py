@@ -17,13 +17,14 @@ from . import build as _build
 
 BF16, FP32 = 0, 1
 RETR_PARALLEL, RETR_HIER, RETR_SEMI = 0, 1, 2
+OPT_FLAG_MARGIN, OPT_SCORE_PATH = 0, 1
 MAX_QUESTIONS, MAX_TOPK, MAX_TOKENS = 128, 256, 256
 NOALLOC_MAX_FRAMES, NOALLOC_MAX_Q_HEADS, NOALLOC_MAX_KV_HEADS = 16, 32, 8
 
 STATUS_NAMES = {0: "MUKV_OK", -1: "MUKV_E_INVALID", -2: "MUKV_E_SHAPE", -3: "MUKV_E_DTYPE", -4: "MUKV_E_ALIGN",
                 -5: "MUKV_E_CAPACITY", -6: "MUKV_E_STATE", -7: "MUKV_E_CUDA", -8: "MUKV_E_UNSUPPORTED"}
 
-EXPORTS = ["mukv_store_bytes", "mukv_workspace_bytes", "mukv_create", "mukv_destroy", "mukv_reset",
+EXPORTS = ["mukv_store_bytes", "mukv_workspace_bytes", "mukv_create", "mukv_destroy", "mukv_reset", "mukv_set_option",
            "mukv_compress_chunk", "mukv_retrieve", "mukv_gather", "mukv_store_region", "mukv_get_stats",
            "mukv_last_error", "mukv_profile_enable", "mukv_profile_read", "mukv_score_frames_noalloc"]
 PROF_KINDS = ["score", "refine", "compact", "segment", "qpool", "scan", "rank", "gather"]
@@ -75,6 +76,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.mukv_destroy.argtypes = [vp]
     lib.mukv_reset.restype = i32
     lib.mukv_reset.argtypes = [vp, vp]
+    lib.mukv_set_option.restype = i32
+    lib.mukv_set_option.argtypes = [vp, i32, C.c_double]
     lib.mukv_compress_chunk.restype = i32
     lib.mukv_compress_chunk.argtypes = [vp, vp, vp, vp, i32, i64, vp, vp, vp]
     lib.mukv_retrieve.restype = i32
@@ -169,6 +172,9 @@ class MukvContext:
     # ---- the calls of include/mukv.h --------------------------------------------------------
     def mukv_reset(self, stream=None):
         self._check(self.lib.mukv_reset(self.handle, _stream(stream)))
+
+    def mukv_set_option(self, option: int, value: float):
+        self._check(self.lib.mukv_set_option(self.handle, option, float(value)))
 
     def mukv_compress_chunk(self, q, k, v, n_frames: int, first_frame: int, kept_out=None, scores_out=None,
                             stream=None):

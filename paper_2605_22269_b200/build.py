@@ -12,7 +12,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
 
 TARGETS = {
     "libmukv.so": (os.path.join(HERE, "csrc", "mukv.cu"),
-                   [os.path.join(HERE, "csrc", n) for n in ("common.cuh", "score.cuh", "score_tc.cuh", "score_ps.cuh", "tc.cuh", "compact.cuh", "retrieve.cuh")]
+                   [os.path.join(HERE, "csrc", n) for n in ("common.cuh", "score.cuh", "score_ps.cuh", "tc.cuh", "compact.cuh", "retrieve.cuh")]
                    + [os.path.join(os.path.dirname(HERE), "include", "mukv.h")]),
     "libmukv_synth.so": (os.path.join(HERE, "synth", "synth.cu"), []),
 }

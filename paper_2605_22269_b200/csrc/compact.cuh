@@ -54,6 +54,9 @@ struct CompactParams {
   ScoreParams sp;                 // partial sums, Eq. 4 parameters, index and flag outputs
 };
 
+// a token id read back from memory, forced into the frame (row addresses are computed from it)
+__device__ __forceinline__ int token_id(int id, int P) { return (unsigned)id < (unsigned)P ? id : 0; }
+
 // owner of item i when n items are split into contiguous shares [c*n/nb, (c+1)*n/nb)
 __device__ __forceinline__ int share_owner(unsigned i, unsigned n, unsigned nb) { return (int)(((i + 1u) * nb - 1u) / n); }
 
@@ -116,7 +119,9 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
     sc->hist[tid] = 0;
     if (tid == 0) sc->n_list = 0;
   }
-  __syncthreads();
+  // a frame with a score that is not a number has no ranking: every score counts as 0 below, so
+  // that the lowest kappa ids are kept (every block of the frame sees the same sums and agrees)
+  const bool bad = __syncthreads_or(valid && !(isfinite(att) && isfinite(fft))) != 0;
   const int wl = lane < NW ? lane : 0;                     // lanes past the warp count repeat warp 0
   const unsigned m0 = __reduce_min_sync(kFull, sc->mm[wl][0]), m1 = __reduce_max_sync(kFull, sc->mm[wl][1]);
   const unsigned m2 = __reduce_min_sync(kFull, sc->mm[wl][2]), m3 = __reduce_max_sync(kFull, sc->mm[wl][3]);
@@ -129,7 +134,7 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
   const float an = (att - amin) * inv_a;
   float fn = (fft - fmin_) * inv_f;
   if (sp.keep_low) fn = 1.f - fn;
-  const float s = sp.alpha * an + (1.f - sp.alpha) * fn;
+  const float s = bad ? 0.f : sp.alpha * an + (1.f - sp.alpha) * fn;
   const int key = __float_as_int(s);
   // ---- tau = kappa-th largest score: a 256-bin histogram finds its bin, the scores of that bin
   // are ranked among themselves
@@ -213,6 +218,7 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
   const float aabs = fmaxf(amax, -amin), fabs_ = fmaxf(fmax_, -fmin_);
   if (amax != amin && (amax - amin) < sp.flat_ratio * aabs && sp.alpha != 0.f) risky = true;
   if (fmax_ != fmin_ && (fmax_ - fmin_) < sp.flat_ratio * fabs_ && sp.alpha != 1.f) risky = true;
+  if (bad) risky = false;                                 // double precision would not rank it either
   if (keep) s_kept[pos] = tid;
   if (write) {
     const long long f_abs = sp.first_frame + f;
@@ -230,6 +236,7 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
       sp.frame_ts[f_abs] = f_abs;
       sp.page_table[f_abs] = sp.pages_off + f_abs * sp.page_bytes;
       if (risky) sp.flagged[atomicAdd(sp.n_flagged, 1)] = f;
+      if (bad && sp.status) atomicCAS(sp.status, 0, kStatusNonFinite);
     }
   }
   __syncthreads();
@@ -415,7 +422,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
     bool risky;
     if ((seen >> 1) == p.epoch) {
       risky = (seen & 1u) != 0u;
-      for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = __ldcg(p.sp.kept_store + f_abs * p.kappa + r);
+      for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(__ldcg(p.sp.kept_store + f_abs * p.kappa + r), p.P);
       __syncthreads();
     } else {
       risky = select_from_partials(p, f, plane == 0, cs.kept, &ss);
@@ -428,7 +435,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
     if (risky) return;
   } else {
     if (frame_is_flagged(p.sp.flagged, *p.sp.n_flagged, f)) return;
-    for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = p.sp.kept_store[f_abs * p.kappa + r];
+    for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(p.sp.kept_store[f_abs * p.kappa + r], p.P);
     __syncthreads();
   }
   compact_plane<T>(p, plane, f, &cs);
@@ -447,7 +454,7 @@ __global__ void __launch_bounds__(kCompactThreads) segment_kernel(const CompactP
     const int f = p.sp.flagged[i];
     const long long f_abs = p.first_frame + f;
     __syncthreads();
-    for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = __ldcg(p.sp.kept_store + f_abs * p.kappa + r);
+    for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(__ldcg(p.sp.kept_store + f_abs * p.kappa + r), p.P);
     __syncthreads();
     compact_plane<T>(p, plane, f, &cs);
   }

@@ -11,6 +11,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -20,7 +21,6 @@
 #include "retrieve.cuh"
 #include "score.cuh"
 #include "score_ps.cuh"
-#include "score_tc.cuh"
 
 using namespace mukv;
 
@@ -44,10 +44,9 @@ struct WorkLayout {
 
 // Tiling of the tensor-core scoring kernel (bf16 inputs only).
 struct TcShape {
-  bool ok;                 // bf16 chunk scored on the tensor cores
-  bool persistent;         // by the persistent kernel (its operand buffers fit in shared memory)
-  int tpt, tiles, npad, n_mt, tmem_cols, ps_stages;
-  size_t smem, smem_ps;
+  bool ok;                 // bf16 chunk scored on the tensor cores (every supported bf16 shape fits)
+  int tpt, tiles, npad, n_mt, ps_stages;
+  size_t smem_ps;
 };
 
 thread_local std::string g_create_error;
@@ -66,6 +65,8 @@ struct mukv_ctx {
   unsigned epoch = 0;                    // compress calls so far (tags the per-frame selection flags)
   int C, G, esize, nc;
   float flag_margin, flat_ratio;
+  bool force_fma = false;                // MUKV_OPT_SCORE_PATH 1: multiply-add scoring for every dtype
+  bool failed = false;                   // a compress call broke off half way: only reset / stats / destroy
   TcShape tcs;                           // tcs.ok: the chunk is scored on the tensor cores
   int n_sms;
   CUtensorMap wmap;                      // DFT matrix terms [3*D][D] bf16
@@ -86,6 +87,13 @@ mukv_status fail(mukv_ctx* ctx, mukv_status st, const char* fmt, ...) {
   va_end(ap);
   if (ctx) ctx->err = buf; else g_create_error = buf;
   return st;
+}
+
+// A launch failed after part of a compress call was enqueued: the chunk is half stored and the
+// device-side counters no longer match the host's, so the context stops until mukv_reset.
+mukv_status broke_off(mukv_ctx* ctx, const char* what, cudaError_t e) {
+  ctx->failed = true;
+  return fail(ctx, MUKV_E_CUDA, "%s: %s (the chunk is half stored: call mukv_reset)", what, cudaGetErrorString(e));
 }
 
 // Brackets one kernel launch with a pair of events when profiling is on.
@@ -169,18 +177,19 @@ TcShape tc_shape(const mukv_config& c) {
   t.tiles = (c.tokens_per_frame + t.tpt - 1) / t.tpt;
   t.npad = (c.tokens_per_frame + 15) / 16 * 16;
   t.n_mt = (c.tokens_per_frame + 127) / 128;
-  int need = t.npad > c.head_dim ? t.npad : c.head_dim;
-  t.tmem_cols = 32;
-  while (t.tmem_cols < need) t.tmem_cols *= 2;
-  t.smem = score_tc_smem_bytes(c.tokens_per_frame, c.head_dim);
   t.ps_stages = score_ps_stages(c.tokens_per_frame, c.head_dim, 227 * 1024);
   t.smem_ps = score_ps_smem_bytes(c.tokens_per_frame, c.head_dim, t.ps_stages < 2 ? 2 : t.ps_stages);
-  t.ok = t.smem <= 227 * 1024;
-  t.persistent = t.ok && t.ps_stages >= 2 && t.npad <= kPsSplit * kPsAccCols;
+  t.ok = t.ps_stages >= 2 && t.npad <= kPsSplit * kPsAccCols;
   return t;
 }
 
 constexpr int kRefineSplit = 4;     // blocks per query head in the double-precision pass
+// Single precision decides a frame only when its lowest kept and highest dropped fused score are
+// further apart than tie_eps + kFlagMargin; a signal whose range is below kFlatRatio of its
+// magnitude (the min-max division then amplifies rounding noise) also sends the frame to the
+// double-precision pass.
+constexpr float kFlagMargin = 3e-6f;
+constexpr float kFlatRatio = 1e-3f;
 
 WorkLayout work_layout(const mukv_config& c) {
   WorkLayout w;
@@ -189,10 +198,8 @@ WorkLayout work_layout(const mukv_config& c) {
   const size_t max_segs = (c.max_frames + c.frames_per_segment - 1) / c.frames_per_segment;
   size_t off = 0;
   const TcShape ts = tc_shape(c);
-  const size_t parts = ts.ok && (size_t)c.n_kv_heads * ts.tiles > (size_t)c.n_q_heads
-                           ? (size_t)c.n_kv_heads * ts.tiles : (size_t)c.n_q_heads;
-  w.colsum_f = off;       off = align_up(off + F * parts * P * sizeof(float));
-  w.colsum_p = off;       off = align_up(off + (ts.persistent ? (kPsMaxBlocks + F) * P * sizeof(float) : 0));
+  w.colsum_f = off;       off = align_up(off + F * (size_t)c.n_q_heads * P * sizeof(float));
+  w.colsum_p = off;       off = align_up(off + (ts.ok ? (kPsMaxBlocks + F) * P * sizeof(float) : 0));
   w.ifft_f = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(float));
   w.colsum_d = off;       off = align_up(off + F * c.n_q_heads * kRefineSplit * P * sizeof(double));
   w.ifft_d = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(double));
@@ -246,16 +253,53 @@ cudaError_t launch_score(const ScoreParams& sp, int nc, dim3 grid, size_t smem, 
   }
 }
 
+// Raises a kernel's dynamic shared-memory limit to everything the device allows beside the
+// kernel's static shared memory.
+cudaError_t raise_smem_limit(const void* fn, int optin) {
+  cudaFuncAttributes fa;
+  cudaError_t e = cudaFuncGetAttributes(&fa, fn);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - (int)fa.sharedSizeBytes);
+}
+
 template <typename T, typename A>
-cudaError_t set_score_attr(int nc, size_t smem) {
-  const void* fn = nullptr;
-  switch (nc) {
-    case 2: fn = (const void*)score_kernel<T, A, 2>; break;
-    case 4: fn = (const void*)score_kernel<T, A, 4>; break;
-    case 7: fn = (const void*)score_kernel<T, A, 7>; break;
-    default: fn = (const void*)score_kernel<T, A, 8>; break;
+cudaError_t raise_score_limits(int optin) {
+  cudaError_t e = raise_smem_limit((const void*)score_kernel<T, A, 2>, optin);
+  if (e == cudaSuccess) e = raise_smem_limit((const void*)score_kernel<T, A, 4>, optin);
+  if (e == cudaSuccess) e = raise_smem_limit((const void*)score_kernel<T, A, 7>, optin);
+  if (e == cudaSuccess) e = raise_smem_limit((const void*)score_kernel<T, A, 8>, optin);
+  return e;
+}
+
+constexpr int kMaxDevices = 64;
+std::mutex g_dev_mutex;
+bool g_limits_raised[kMaxDevices];
+
+// Once per device (that device current): the dynamic shared-memory limit of every kernel that
+// needs more than the default goes to the device's maximum.  The limit belongs to the kernel,
+// not to a context, so it is never set to one context's need: a second context of another
+// shape, or the allocation-free entry point, would otherwise find it too low.
+cudaError_t raise_kernel_limits(int* n_sms) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (n_sms) {
+    e = cudaDeviceGetAttribute(n_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
   }
-  return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_dev_mutex);
+  if (g_limits_raised[dev]) return cudaSuccess;
+  int optin = 0;
+  e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e == cudaSuccess) e = raise_score_limits<__nv_bfloat16, float>(optin);
+  if (e == cudaSuccess) e = raise_score_limits<__nv_bfloat16, double>(optin);
+  if (e == cudaSuccess) e = raise_score_limits<float, float>(optin);
+  if (e == cudaSuccess) e = raise_score_limits<float, double>(optin);
+  if (e == cudaSuccess) e = raise_smem_limit((const void*)rank_kernel, optin);
+  if (e == cudaSuccess) e = raise_smem_limit((const void*)score_ps_kernel, optin);
+  if (e == cudaSuccess) g_limits_raised[dev] = true;
+  return e;
 }
 
 // ---------------------------------------------------------------- TMA descriptors
@@ -338,47 +382,33 @@ std::vector<uint16_t> dft_terms(int D) {
   return w;
 }
 
-// Scores a bf16 chunk on the tensor cores (Eq. 1-4 and the selection).
-cudaError_t launch_score_tc(mukv_ctx* ctx, const ScoreParams& sp, const void* d_q, const void* k_last, int n,
+// Scores a bf16 chunk on the tensor cores (Eq. 1-3; Eq. 4 and the selection follow in compact_kernel).
+cudaError_t launch_score_ps(mukv_ctx* ctx, const ScoreParams& sp, const void* d_q, const void* k_last, int n,
                             cudaStream_t st, const char** why, int* ps_grid, int* ps_items, int* ps_ipf) {
   *ps_grid = 0;
   const mukv_config& c = ctx->cfg;
   const TcShape& t = ctx->tcs;
   const int P = c.tokens_per_frame, D = c.head_dim;
-  CUtensorMap qmap, kmap, kmap_dft;
+  CUtensorMap qmap, kmap;
   const long long rows = (long long)n * P;
   if (!encode_map3(&qmap, d_q, D, c.n_q_heads, rows, ctx->G, t.tpt) ||
-      !encode_map3(&kmap, k_last, D, c.n_kv_heads, rows, 1, t.npad) ||
-      !encode_map3(&kmap_dft, k_last, D, c.n_kv_heads, rows, 1, 128)) {
+      !encode_map3(&kmap, k_last, D, c.n_kv_heads, rows, 1, t.npad)) {
     *why = "cuTensorMapEncodeTiled failed";
     return cudaErrorInvalidValue;
   }
-  if (t.persistent) {
-    ScorePsParams pp;
-    memset(&pp, 0, sizeof pp);
-    pp.sp = sp;
-    pp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
-    pp.tiles = t.tiles; pp.tpt = t.tpt; pp.npad = t.npad; pp.n_mt = t.n_mt; pp.n_stages = t.ps_stages;
-    pp.n_items = n * c.n_kv_heads * (t.n_mt + t.tiles);
-    pp.exp2_scale = (float)(1.4426950408889634 / std::sqrt((double)D));
-    pp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
-    int blocks = ctx->n_sms < kPsMaxBlocks ? ctx->n_sms : kPsMaxBlocks;
-    if (blocks > pp.n_items) blocks = pp.n_items;
-    *ps_grid = blocks; *ps_items = pp.n_items; *ps_ipf = c.n_kv_heads * (t.n_mt + t.tiles);
-    score_ps_kernel<<<blocks, kPsThreads, t.smem_ps, st>>>(pp, qmap, kmap, ctx->wmap);
-    *why = "score_ps kernel";
-    return cudaGetLastError();
-  }
-  ScoreTcParams tp;
-  memset(&tp, 0, sizeof tp);
-  tp.sp = sp;
-  tp.tiles = t.tiles; tp.tpt = t.tpt; tp.npad = t.npad; tp.n_mt = t.n_mt; tp.tmem_cols = t.tmem_cols;
-  tp.op_bytes = score_tc_op_bytes(P, D);
-  tp.exp2_scale = (float)(1.4426950408889634 / std::sqrt((double)D));
-  tp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
-  const dim3 grid(t.n_mt + t.tiles, c.n_kv_heads, n);
-  score_tc_kernel<<<grid, kTcThreads, t.smem, st>>>(tp, qmap, kmap, kmap_dft, ctx->wmap);
-  *why = "score_tc kernel";
+  ScorePsParams pp;
+  memset(&pp, 0, sizeof pp);
+  pp.sp = sp;
+  pp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
+  pp.tiles = t.tiles; pp.tpt = t.tpt; pp.npad = t.npad; pp.n_mt = t.n_mt; pp.n_stages = t.ps_stages;
+  pp.n_items = n * c.n_kv_heads * (t.n_mt + t.tiles);
+  pp.exp2_scale = (float)(1.4426950408889634 / std::sqrt((double)D));
+  pp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
+  int blocks = ctx->n_sms < kPsMaxBlocks ? ctx->n_sms : kPsMaxBlocks;
+  if (blocks > pp.n_items) blocks = pp.n_items;
+  *ps_grid = blocks; *ps_items = pp.n_items; *ps_ipf = c.n_kv_heads * (t.n_mt + t.tiles);
+  score_ps_kernel<<<blocks, kPsThreads, t.smem_ps, st>>>(pp, qmap, kmap, ctx->wmap);
+  *why = "score_ps kernel";
   return cudaGetLastError();
 }
 
@@ -407,6 +437,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   sp.page_table = reinterpret_cast<long long*>(ctx->store + ctx->sl.page_table);
   sp.pages_off = (long long)ctx->sl.pages;
   sp.page_bytes = (long long)ctx->sl.page_bytes;
+  sp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
   sp.refine = 0;
   sp.row_split = 1;
   const dim3 grid(c.n_q_heads, n);
@@ -415,8 +446,8 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   int ps_grid = 0, ps_items = 0, ps_ipf = 0;
   {
     ProfScope ps(ctx, 0, st);
-    if (ctx->tcs.ok)
-      e = launch_score_tc(ctx, sp, d_q, sp.k_last, n, st, &what, &ps_grid, &ps_items, &ps_ipf);
+    if (ctx->tcs.ok && !ctx->force_fma)
+      e = launch_score_ps(ctx, sp, d_q, sp.k_last, n, st, &what, &ps_grid, &ps_items, &ps_ipf);
     else
       e = launch_score<T, float>(sp, ctx->nc, grid, score_smem_bytes<T, float>(P, c.head_dim), st);
   }
@@ -448,7 +479,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
     ProfScope ps(ctx, 2, st);
     e = launch_k(compact_kernel<T>, dim3(n, L * 2), kCompactThreads, 0, st, !ctx->prof_on, cp);
   }
-  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "compact kernel: %s", cudaGetErrorString(e));
+  if (e != cudaSuccess) return broke_off(ctx, "compact kernel", e);
 
   // frames too close to a tie boundary: the scores again in double precision, and the selection
   // (blocks beyond the flagged count return at once)
@@ -461,13 +492,13 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
     const dim3 rgrid(c.n_q_heads * kRefineSplit, n < 2 ? n : 2);   // its blocks walk the flagged frames
     e = launch_score<T, double>(sp, ctx->nc, rgrid, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
   }
-  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "refine kernel: %s", cudaGetErrorString(e));
+  if (e != cudaSuccess) return broke_off(ctx, "refine kernel", e);
   // compaction of those frames, then the segment entries
   {
     ProfScope ps(ctx, 3, st);
     e = launch_k(segment_kernel<T>, dim3(L * 2), kCompactThreads, 0, st, !ctx->prof_on, cp);
   }
-  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "segment kernel: %s", cudaGetErrorString(e));
+  if (e != cudaSuccess) return broke_off(ctx, "segment kernel", e);
 
   ctx->launches += 4;
   ctx->parity ^= 1;
@@ -518,37 +549,15 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
   ctx->esize = cfg->dtype == MUKV_BF16 ? 2 : 4;
   ctx->nc = pick_nc(cfg->tokens_per_frame);
   ctx->tcs = tc_shape(*cfg);
-  if (const char* s = getenv("MUKV_SCORE_FMA")) if (atoi(s) != 0) ctx->tcs.ok = ctx->tcs.persistent = false;
-  if (const char* s = getenv("MUKV_SCORE_TILE_BLOCKS")) if (atoi(s) != 0) ctx->tcs.persistent = false;
   ctx->n_sms = 1;
-  ctx->flag_margin = 3e-6f;
-  ctx->flat_ratio = 1e-3f;
-  if (const char* s = getenv("MUKV_FLAG_MARGIN")) ctx->flag_margin = (float)atof(s);
-  if (const char* s = getenv("MUKV_FLAT_RATIO")) ctx->flat_ratio = (float)atof(s);
-  const int P = cfg->tokens_per_frame, D = cfg->head_dim;
-  cudaError_t e;
-  if (cfg->dtype == MUKV_BF16) {
-    e = set_score_attr<__nv_bfloat16, float>(ctx->nc, score_smem_bytes<__nv_bfloat16, float>(P, D));
-    if (e == cudaSuccess) e = set_score_attr<__nv_bfloat16, double>(ctx->nc, score_smem_bytes<__nv_bfloat16, double>(P, D));
-  } else {
-    e = set_score_attr<float, float>(ctx->nc, score_smem_bytes<float, float>(P, D));
-    if (e == cudaSuccess) e = set_score_attr<float, double>(ctx->nc, score_smem_bytes<float, double>(P, D));
-  }
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute((const void*)rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRankStageBytes);
+  ctx->flag_margin = kFlagMargin;
+  ctx->flat_ratio = kFlatRatio;
+  const int D = cfg->head_dim;
+  cudaError_t e = raise_kernel_limits(&ctx->n_sms);
   if (e == cudaSuccess && ctx->tcs.ok) {
     const std::vector<uint16_t> w = dft_terms(D);
     e = cudaMemcpy(ctx->ws + ctx->wl.wtab, w.data(), w.size() * 2, cudaMemcpyHostToDevice);
     if (e == cudaSuccess && !encode_map2(&ctx->wmap, ctx->ws + ctx->wl.wtab, D, 3LL * D, D)) e = cudaErrorInvalidValue;
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute((const void*)score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)ctx->tcs.smem);
-    if (e == cudaSuccess && ctx->tcs.persistent)
-      e = cudaFuncSetAttribute((const void*)score_ps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)ctx->tcs.smem_ps);
-    int dev = 0;
-    if (e == cudaSuccess) e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, dev);
   }
   if (e == cudaSuccess)
     e = cudaMemset(ctx->ws + ctx->wl.zero_begin, 0, ctx->wl.zero_end - ctx->wl.zero_begin);
@@ -591,10 +600,32 @@ mukv_status mukv_profile_read(mukv_ctx* ctx, double* ms, int64_t* launches) {
 }
 
 mukv_status mukv_reset(mukv_ctx* ctx, mukv_stream stream) {
-  (void)stream;
   if (!ctx) return MUKV_E_INVALID;
+  // arrival counters, flagged lists, selection flags, statistics and the event word start over
+  cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->wl.zero_begin, 0, ctx->wl.zero_end - ctx->wl.zero_begin,
+                                  static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "mukv_reset: %s", cudaGetErrorString(e));
   ctx->frames = 0;
+  ctx->parity = 0;
+  ctx->failed = false;
   return MUKV_OK;
+}
+
+mukv_status mukv_set_option(mukv_ctx* ctx, int32_t option, double value) {
+  if (!ctx) return MUKV_E_INVALID;
+  switch (option) {
+    case MUKV_OPT_FLAG_MARGIN:
+      if (!(value >= (double)kFlagMargin) || !(value <= 4.0))
+        return fail(ctx, MUKV_E_INVALID, "the safety margin can only be raised above %g (got %g)", (double)kFlagMargin, value);
+      ctx->flag_margin = (float)value;
+      return MUKV_OK;
+    case MUKV_OPT_SCORE_PATH:
+      if (value != 0.0 && value != 1.0) return fail(ctx, MUKV_E_INVALID, "score path must be 0 or 1");
+      ctx->force_fma = value == 1.0;
+      return MUKV_OK;
+    default:
+      return fail(ctx, MUKV_E_INVALID, "unknown option %d", option);
+  }
 }
 
 mukv_status mukv_compress_chunk(mukv_ctx* ctx, const void* d_q, const void* d_k, const void* d_v, int32_t n_frames,
@@ -602,6 +633,7 @@ mukv_status mukv_compress_chunk(mukv_ctx* ctx, const void* d_q, const void* d_k,
                                 mukv_stream stream) {
   if (!ctx) return MUKV_E_INVALID;
   try {
+    if (ctx->failed) return fail(ctx, MUKV_E_STATE, "an earlier call broke off half way: call mukv_reset");
     if (!d_q || !d_k || !d_v) return fail(ctx, MUKV_E_INVALID, "null input pointer");
     if (!aligned16(d_q) || !aligned16(d_k) || !aligned16(d_v) || !aligned4(d_kept_out) || !aligned4(d_scores_out))
       return fail(ctx, MUKV_E_ALIGN, "d_q, d_k, d_v must be 16-byte aligned, the outputs 4-byte aligned");
@@ -630,6 +662,7 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
                           int32_t* d_counts, mukv_stream stream) {
   if (!ctx) return MUKV_E_INVALID;
   try {
+    if (ctx->failed) return fail(ctx, MUKV_E_STATE, "an earlier call broke off half way: call mukv_reset");
     if (!d_qtok || !h_q_offsets || !d_seg_idx || !d_frm_idx || !d_counts)
       return fail(ctx, MUKV_E_INVALID, "null argument");
     if (!aligned16(d_qtok) || !aligned4(d_seg_idx) || !aligned4(d_frm_idx) || !aligned4(d_seg_score) ||
@@ -714,6 +747,7 @@ mukv_status mukv_gather(mukv_ctx* ctx, const int32_t* d_frm_idx, const int32_t* 
                         void* d_decode, int64_t decode_stride_bytes, int32_t* d_tok_meta, mukv_stream stream) {
   if (!ctx) return MUKV_E_INVALID;
   try {
+    if (ctx->failed) return fail(ctx, MUKV_E_STATE, "an earlier call broke off half way: call mukv_reset");
     if (!d_frm_idx || !d_counts || !d_decode) return fail(ctx, MUKV_E_INVALID, "null argument");
     if (!aligned4(d_frm_idx) || !aligned4(d_counts) || !aligned16(d_decode) || !aligned4(d_tok_meta))
       return fail(ctx, MUKV_E_ALIGN, "d_decode must be 16-byte aligned, index arrays 4-byte aligned");
@@ -828,26 +862,17 @@ constexpr size_t kNaTotal = kNaCtrl + kNaCtrlBytes;
 // In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaTotal];
 
-constexpr int kNaMaxDevices = 64;
-unsigned char* g_noalloc_ptr[kNaMaxDevices];             // device address of the array, per device
+unsigned char* g_noalloc_ptr[kMaxDevices];               // device address of the array, per device
 
-// Once per device, with that device current: resolves the array's device address and raises the
-// dynamic shared-memory limit of every variant of the scoring kernel to what the largest
-// supported frame needs.  Allocates nothing.
+// Once per device, with that device current: resolves the array's device address and makes sure the
+// scoring kernels may use the shared memory the largest supported frame needs.  Allocates nothing.
 cudaError_t noalloc_setup(int dev, unsigned char** out) {
+  cudaError_t e = raise_kernel_limits(nullptr);
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> lock(g_dev_mutex);
   if (!g_noalloc_ptr[dev]) {
     void* ptr = nullptr;
-    cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
-    if (e != cudaSuccess) return e;
-    const int ncs[4] = {2, 4, 7, 8};
-    for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
-      const int nc = ncs[i];
-      e = set_score_attr<__nv_bfloat16, float>(nc, score_smem_bytes<__nv_bfloat16, float>(kNaP, 128));
-      if (e == cudaSuccess)
-        e = set_score_attr<__nv_bfloat16, double>(nc, score_smem_bytes<__nv_bfloat16, double>(kNaP, 128));
-      if (e == cudaSuccess) e = set_score_attr<float, float>(nc, score_smem_bytes<float, float>(kNaP, 128));
-      if (e == cudaSuccess) e = set_score_attr<float, double>(nc, score_smem_bytes<float, double>(kNaP, 128));
-    }
+    e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
     if (e != cudaSuccess) return e;
     g_noalloc_ptr[dev] = static_cast<unsigned char*>(ptr);
   }
@@ -861,7 +886,7 @@ mukv_status noalloc_impl(const mukv_config& c, const void* d_q, const void* d_k_
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return fail(nullptr, MUKV_E_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
-  if (dev < 0 || dev >= kNaMaxDevices) return fail(nullptr, MUKV_E_CAPACITY, "device index %d not supported", dev);
+  if (dev < 0 || dev >= kMaxDevices) return fail(nullptr, MUKV_E_CAPACITY, "device index %d not supported", dev);
   const int P = c.tokens_per_frame, D = c.head_dim, nc = pick_nc(P);
   unsigned char* base = nullptr;
   e = noalloc_setup(dev, &base);
@@ -873,7 +898,7 @@ mukv_status noalloc_impl(const mukv_config& c, const void* d_q, const void* d_k_
   memset(&sp, 0, sizeof sp);
   sp.P = P; sp.Hq = c.n_q_heads; sp.Hkv = c.n_kv_heads; sp.D = D; sp.G = c.n_q_heads / c.n_kv_heads;
   sp.kappa = c.keep_per_frame; sp.n_frames = n; sp.causal = c.attn_causal; sp.keep_low = c.keep_low_freq;
-  sp.alpha = c.alpha; sp.tie_eps = c.tie_eps; sp.flag_margin = 3e-6f; sp.flat_ratio = 1e-3f;
+  sp.alpha = c.alpha; sp.tie_eps = c.tie_eps; sp.flag_margin = kFlagMargin; sp.flat_ratio = kFlatRatio;
   sp.first_frame = 0;
   sp.q = d_q;
   sp.k_last = d_k_last;
@@ -909,10 +934,10 @@ extern "C" mukv_status mukv_score_frames_noalloc(const mukv_config* cfg, const v
     if (!cfg || !d_q || !d_k_last) return fail(nullptr, MUKV_E_INVALID, "null argument");
     if (!d_kept_out && !d_scores_out) return fail(nullptr, MUKV_E_INVALID, "no output requested");
     mukv_config c = *cfg;
-    if (c.max_frames < 1) c.max_frames = 1;                      // not used here
-    if (c.max_frames_per_chunk < 1) c.max_frames_per_chunk = 1;
-    if (c.n_layers < 1) c.n_layers = 1;
-    if (c.frames_per_segment < 1) c.frames_per_segment = 1;
+    c.max_frames = 1;                                            // fields this entry point ignores
+    c.max_frames_per_chunk = 1;
+    c.n_layers = 1;
+    c.frames_per_segment = 1;
     if (const char* why = check_config(&c))
       return fail(nullptr, (c.dtype != MUKV_BF16 && c.dtype != MUKV_FP32) ? MUKV_E_DTYPE : MUKV_E_SHAPE, "%s", why);
     if (n_frames < 1) return fail(nullptr, MUKV_E_INVALID, "n_frames must be >= 1");

@@ -17,6 +17,7 @@
 namespace mukv {
 
 constexpr int kScoreThreads = 256;
+constexpr int kStatusNonFinite = 7;   // a frame's scores were not finite: its lowest kappa ids were kept
 constexpr int kScoreWarps = kScoreThreads / 32;
 constexpr int kRowsPerStep = 4;
 
@@ -42,6 +43,7 @@ struct ScoreParams {
   long long* frame_ts;          // [max_frames]
   long long* page_table;        // [max_frames]
   long long pages_off, page_bytes;
+  int* status;                  // device event word (0 = nothing recorded); see mukv_stats.device_status
   int refine;                   // 1: frames come from the flagged list, no further flagging
   int row_split;                // blocks that share a query head, each a range of query rows (>= 1)
 };
@@ -76,6 +78,14 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
   bool valid[TOK];
 #pragma unroll
   for (int k = 0; k < TOK; ++k) { tok[k] = tid + k * nt; valid[k] = tok[k] < P; }
+  // ---- a frame with a score that is not a number has no ranking: every score counts as 0 below,
+  // so that the lowest kappa ids are kept, and the event is recorded
+  bool bad_here = false;
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) bad_here |= valid[k] && !(isfinite(att_raw[k]) && isfinite(fft_raw[k]));
+  int n_bad;
+  group_excl_count<Grp>(bad_here, s_int, n_bad);
+  const bool bad = n_bad != 0;
   // ---- min / max of both signals over the frame
   A v[4] = {big, -big, big, -big};
 #pragma unroll
@@ -109,7 +119,7 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
     A an = (amax == amin) ? (A)0 : (att_raw[k] - amin) / (amax - amin);
     A fn = (fmax_ == fmin_) ? (A)0 : (fft_raw[k] - fmin_) / (fmax_ - fmin_);
     if (p.keep_low) fn = (A)1 - fn;
-    s[k] = alpha * an + ((A)1 - alpha) * fn;
+    s[k] = bad ? (A)0 : alpha * an + ((A)1 - alpha) * fn;
     if (valid[k]) s_sc[tok[k]] = s[k];
   }
   Grp::sync();
@@ -169,13 +179,14 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
   if (tid == 0) {
     p.frame_ts[f_abs] = f_abs;
     p.page_table[f_abs] = p.pages_off + f_abs * p.page_bytes;
+    if (bad && p.status) atomicCAS(p.status, 0, kStatusNonFinite);
   }
   // ---- does single precision decide this frame safely?
   // With a = lowest kept score and b = highest dropped score, the kept set is the same for every
   // perturbation of the scores below flag_margin / 2 as long as a - b > tie_eps + flag_margin: no
   // dropped token can then enter the tie band of the kappa-th score.  Anything closer is redone
   // in double precision.
-  if (!p.refine) {
+  if (!p.refine && !bad) {
     A a = big, b = -big;
 #pragma unroll
     for (int k = 0; k < TOK; ++k) {

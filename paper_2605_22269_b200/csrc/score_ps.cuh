@@ -2,8 +2,9 @@
 //
 // score_ps_kernel: one block of 640 threads per SM.  The chunk is a list of items, ordered by
 // (frame, key head): first the DFT row tiles of that head's keys (Eq. 2-3), then the attention
-// row tiles (Eq. 1; the G query heads of the group are flattened with the tokens into rows, as
-// in score_tc_kernel).  Each block takes a contiguous share of the list.
+// row tiles (Eq. 1; the G query heads of the group are flattened with the tokens into rows: one
+// TMA box of tpt = 128/G tokens x G heads x 64 channels lands as up to 128 rows of a K-major,
+// 128-byte-swizzled operand).  Each block takes a contiguous share of the list.
 //
 //   warp 0      TMA producer.  The key tile K_g of a (frame, head) goes to one of two buffers when
 //               the head changes; everything else streams through a ring of 32 KB operand stages:
@@ -30,7 +31,6 @@
 #pragma once
 #include "common.cuh"
 #include "score.cuh"
-#include "score_tc.cuh"
 #include "tc.cuh"
 
 namespace mukv {
@@ -70,6 +70,27 @@ __host__ inline int score_ps_stages(int P, int D, size_t limit) {
   int n = kPsMaxStages;
   while (n >= 2 && score_ps_smem_bytes(P, D, n) > limit) --n;
   return n;                  // < 2: the kernel does not fit
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// v[c] summed over the 32 lanes of the warp, for 32 columns c at once: lane c ends with column c.
+__device__ __forceinline__ float warp_column_sums(float (&v)[32], int lane) {
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) {
+    const bool up = (lane & s) != 0;
+#pragma unroll
+    for (int k = 0; k < s; ++k) {
+      const float send = up ? v[k] : v[k + s];
+      const float keep = up ? v[k + s] : v[k];
+      v[k] = keep + __shfl_xor_sync(kFull, send, s);
+    }
+  }
+  return v[0];
 }
 
 // square root to about one unit in the last place (one special-function instruction and a multiply)

@@ -13,6 +13,7 @@ from paper_2605_22269_b200 import binding as B
 from paper_2605_22269_b200.synth.cpu import StreamSpec, workload
 
 RTOL, ATOL = 1e-3, 1e-5          # floating-point tolerance of the parity tests
+FLAG_MARGIN = 3e-6               # the library's built-in safety margin of the single-precision selection
 
 
 def spec_config(spec: StreamSpec, wl: dict, max_frames: int | None = None, **over) -> B.MukvConfig:
@@ -96,13 +97,16 @@ def oracle_stream(spec: StreamSpec, ocfg: dict, frames, last_only: bool, workers
 class GpuRun:
     """Compresses a whole synthetic stream on the GPU, chunk by chunk, through the C ABI."""
 
-    def __init__(self, name_or_wl, max_frames=None, n_frames=None, device="cuda:0", want_scores=True, **cfg_over):
+    def __init__(self, name_or_wl, max_frames=None, n_frames=None, device="cuda:0", want_scores=True, options=None,
+                 **cfg_over):
         from paper_2605_22269_b200.synth.gpu import GpuStream
         self.wl = workload(name_or_wl) if isinstance(name_or_wl, str) else name_or_wl
         self.spec = self.wl["spec"]
         self.n_frames = n_frames or self.spec.n_frames
         self.cfg = spec_config(self.spec, self.wl, max_frames or self.n_frames, **cfg_over)
         self.ctx = B.MukvContext(self.cfg, device)
+        for opt, val in (options or {}).items():
+            self.ctx.mukv_set_option(opt, val)
         self.gs = GpuStream(self.spec, device)
         self.device = device
         self.want_scores = want_scores

@@ -139,6 +139,8 @@ def test_chunk7b_full_parity():
     worst = np.abs(run.scores[2] - np.stack([s[2] for s in st.scores])).max()
     print(f"chunk7b: max |fused score - oracle| = {worst:.3e}; refined frames = "
           f"{run.ctx.mukv_get_stats().refined_frames}")
+    # what keeps the single-precision selection exact: the score error stays below half the safety margin
+    assert worst < H.FLAG_MARGIN / 2
     qtok, offs, _ = questions(run)
     wl = run.wl
     retrieval_check(run, st, qtok, offs, wl["k_seg"], wl["k_frm"], wl["lam"], B.RETR_SEMI)
@@ -158,27 +160,121 @@ def test_chunk7b_small_chunks(chunk):
     assert run.ctx.mukv_get_stats().device_status == 0
 
 
-def test_chunk7b_tile_block_scoring(monkeypatch):
-    # the one-tile-per-block tensor-core kernel (used when the persistent kernel's buffers do not fit)
-    monkeypatch.setenv("MUKV_SCORE_TILE_BLOCKS", "1")
-    run = H.GpuRun("chunk7b", n_frames=5)
-    full_compress_check(run)
-    assert run.ctx.mukv_get_stats().device_status == 0
-
-
-def test_chunk7b_every_frame_through_the_double_pass(monkeypatch):
+def test_chunk7b_every_frame_through_the_double_pass():
     # a huge safety margin flags every frame: the double-precision pass has to walk a list longer than its grid
-    monkeypatch.setenv("MUKV_FLAG_MARGIN", "1.0")
-    run = H.GpuRun("chunk7b", n_frames=5)
+    run = H.GpuRun("chunk7b", n_frames=5, options={B.OPT_FLAG_MARGIN: 1.0})
     full_compress_check(run)
     assert run.ctx.mukv_get_stats().refined_frames == 5
 
 
-def test_chunk7b_cuda_core_scoring(monkeypatch):
+def test_chunk7b_cuda_core_scoring():
     # bf16 inputs scored by the plain multiply-add kernel (the one fp32 inputs always use)
-    monkeypatch.setenv("MUKV_SCORE_FMA", "1")
-    run = H.GpuRun("chunk7b", n_frames=3)
+    run = H.GpuRun("chunk7b", n_frames=3, options={B.OPT_SCORE_PATH: 1})
     full_compress_check(run)
+
+
+def test_safety_margin_can_only_be_raised():
+    run = H.GpuRun("tiny")
+    with pytest.raises(B.MukvError) as e:
+        run.ctx.mukv_set_option(B.OPT_FLAG_MARGIN, 0.0)
+    assert e.value.status == -1
+    with pytest.raises(B.MukvError):
+        run.ctx.mukv_set_option(99, 1.0)
+
+
+# The production path for bf16 chunks selects inside compact_kernel from the tensor-core kernel's
+# partial sums, in single precision: every variant of Eq. 4 and of the top-kappa rule has to hold
+# there too (paper: the low / high frequency ablation, the attention-only and frequency-only rows of
+# the compression ablation, alpha per granularity).
+@pytest.mark.parametrize("over", [dict(keep_low_freq=1), dict(alpha=0.0), dict(alpha=1.0), dict(alpha=0.5),
+                                  dict(alpha=0.8), dict(keep_per_frame=1), dict(keep_per_frame=196),
+                                  dict(keep_per_frame=19), dict(keep_low_freq=1, alpha=0.0, attn_causal=1)])
+def test_chunk7b_variants_on_the_tensor_core_path(over):
+    run = H.GpuRun("chunk7b", n_frames=5, **over)
+    full_compress_check(run, chunk=3)
+    st = run.ctx.mukv_get_stats()
+    assert st.device_status == 0 and st.refined_frames <= 1
+
+
+def _flat_chunk(run, n, q_val, k_mode):
+    """A hand-made bf16 chunk: zero or constant queries; keys constant over tokens ("const"), or
+    constant except for one token ("spike")."""
+    c = run.cfg
+    P, L = c.tokens_per_frame, c.n_layers
+    dev = run.device
+    q = torch.full((n, P, c.n_q_heads, c.head_dim), q_val, dtype=torch.bfloat16, device=dev)
+    k = torch.full((L, n, P, c.n_kv_heads, c.head_dim), 0.5, dtype=torch.bfloat16, device=dev)
+    if k_mode == "spike":
+        k[:, :, 100] = 2.0
+    v = torch.arange(P, dtype=torch.float32, device=dev).to(torch.bfloat16).view(1, 1, P, 1, 1).expand_as(k).contiguous()
+    return q, k, v
+
+
+@pytest.mark.parametrize("k_mode,alpha", [("const", 0.7), ("const", 0.0), ("const", 1.0), ("spike", 0.7),
+                                          ("spike", 1.0)])
+def test_flat_signals_on_the_tensor_core_path(k_mode, alpha):
+    # zero queries and constant keys: both signals flat, every fused score equal (all of them land
+    # in one histogram bin), the lowest ids are kept.  With one different key the frequency signal
+    # has a single peak and the attention signal stays flat.
+    run = H.GpuRun("chunk7b", n_frames=3, alpha=alpha)
+    c = run.cfg
+    q, k, v = _flat_chunk(run, 3, 0.0, k_mode)
+    kept = torch.zeros((3, c.keep_per_frame), dtype=torch.int32, device=run.device)
+    sc = torch.zeros((3, 3, c.tokens_per_frame), dtype=torch.float32, device=run.device)
+    run.ctx.mukv_compress_chunk(q, k, v, 3, 0, kept, sc)
+    torch.cuda.synchronize()
+    st = O.Store(H.oracle_cfg(c))
+    O.compress_chunk(st, H.to_numpy_bits(q), H.to_numpy_bits(k), H.to_numpy_bits(v))
+    got = kept.cpu().numpy()
+    for f in range(3):
+        assert got[f].tolist() == st.kept[f].tolist(), f"kept ids differ at frame {f}"
+        for i in range(3):
+            H.close(sc[i, f].cpu().numpy(), st.scores[f][i], f"score[{i}] frame {f}")
+    pages = H.to_numpy_bits(run.ctx.region(0)[:3])
+    for f in range(3):
+        assert pages[f][:, 0].tobytes() == st.page_k[f].tobytes() and pages[f][:, 1].tobytes() == st.page_v[f].tobytes()
+    assert run.ctx.mukv_get_stats().device_status == 0
+
+
+def test_non_finite_inputs_keep_the_lowest_ids():
+    # one Inf key: every fused score of that frame is NaN; the frame keeps ids 0..kappa-1, the event
+    # is recorded, the neighbouring frames are not disturbed
+    run = H.GpuRun("chunk7b", n_frames=3)
+    c = run.cfg
+    q, k, v = run.gs.chunk(0, 3)
+    k[c.n_layers - 1, 1, 5, 0, 3] = float("inf")
+    kept = torch.zeros((3, c.keep_per_frame), dtype=torch.int32, device=run.device)
+    run.ctx.mukv_compress_chunk(q, k, v, 3, 0, kept, None)
+    torch.cuda.synchronize()
+    st = O.Store(H.oracle_cfg(c))
+    with np.errstate(all="ignore"):
+        O.compress_chunk(st, H.to_numpy_bits(q), H.to_numpy_bits(k), H.to_numpy_bits(v))
+    got = kept.cpu().numpy()
+    assert got[1].tolist() == list(range(c.keep_per_frame)) == st.kept[1].tolist()
+    assert got[0].tolist() == st.kept[0].tolist() and got[2].tolist() == st.kept[2].tolist()
+    pages = H.to_numpy_bits(run.ctx.region(0)[:3])
+    for f in range(3):
+        assert pages[f][:, 0].tobytes() == st.page_k[f].tobytes()
+    assert run.ctx.mukv_get_stats().device_status == 7
+    run.ctx.mukv_reset()
+    assert run.ctx.mukv_get_stats().device_status == 0 and run.ctx.mukv_get_stats().frames == 0
+
+
+def test_two_contexts_of_different_shape():
+    # kernel attributes belong to the kernel, not to a context: a second, smaller context must not
+    # take shared memory away from the first one's launches (the double-precision pass included)
+    big = H.GpuRun("chunk7b", n_frames=4, options={B.OPT_FLAG_MARGIN: 1.0})
+    spec = StreamSpec(seed=31, n_layers=2, n_q_heads=8, n_kv_heads=4, head_dim=64, tokens_per_frame=130, bf16=True,
+                      n_outlier=2, n_frames=3, scene_sigma=1.0, frame_sigma=0.5, scene_min=2, scene_max=3)
+    small = H.GpuRun(dict(spec=spec, keep=33, fseg=2, chunk=3, alpha=0.7), options={B.OPT_FLAG_MARGIN: 1.0})
+    full_compress_check(small)
+    full_compress_check(big)
+    assert big.ctx.mukv_get_stats().refined_frames == 4
+    spec32 = StreamSpec(seed=32, n_layers=1, n_q_heads=2, n_kv_heads=2, head_dim=64, tokens_per_frame=40, bf16=False,
+                        n_outlier=0, n_frames=2, scene_sigma=1.0, frame_sigma=0.5, scene_min=2, scene_max=3)
+    tiny = H.GpuRun(dict(spec=spec32, keep=7, fseg=2, chunk=2, alpha=0.7))
+    full_compress_check(tiny)
+    full_compress_check(H.GpuRun("tiny"))
 
 
 @pytest.mark.parametrize("shape", [dict(n_q_heads=8, n_kv_heads=8, head_dim=64, tokens_per_frame=130, keep=33),
@@ -206,6 +302,7 @@ def test_stream_1h():
     st = H.oracle_stream(spec, H.oracle_cfg(cfg), range(T), last_only=True)
     worst = H.check_frames_against_oracle(run, st, range(T), full_layers=False)
     print(f"stream_1h: max |fused score - oracle| = {worst:.3e}; refined = {run.ctx.mukv_get_stats().refined_frames}")
+    assert worst < H.FLAG_MARGIN / 2 and run.ctx.mukv_get_stats().refined_frames <= T // 200
     fkey = run.ctx.region(4).cpu().numpy()[:T]
     assert fkey.tobytes() == st.frame_keys().tobytes()
     skey = run.ctx.region(5).cpu().numpy()[:113]

@@ -1,4 +1,4 @@
-"""mukv_score_frames_noalloc against mukv_compress_chunk.
+"""mukv_score_frames_noalloc against mukv_compress_chunk and against the CPU oracle.
 
 The entry point under test serves callers that cannot allocate device memory (everything was given
 to another pool at start-up, or the allocator is off limits while they run): its scratch is a
@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import mukv_oracle as O
 from paper_2605_22269_b200 import binding as B
 from tests import harness as H
 
@@ -41,6 +42,35 @@ def test_noalloc_matches_compress_chunk_twice_in_a_row():
     _both_ways("chunk7b", 5, 0)          # bf16, 28 query heads over 4 key heads
     _both_ways("chunk7b", 3, 2)          # fewer frames than the call before: stale scratch must not matter
     _both_ways("tiny", 8, 0)             # fp32
+
+
+def test_noalloc_against_the_oracle_with_another_context_created_in_between():
+    # the oracle decides, not the other entry point; and a context of a smaller shape created
+    # between two calls must not take the scoring kernels' shared memory away
+    wl = H.workload("chunk7b")
+    spec = wl["spec"]
+    cfg = H.spec_config(spec, wl)
+    n = 5
+    from paper_2605_22269_b200.synth.gpu import GpuStream
+    gs = GpuStream(spec, "cuda:0")
+    q, k, v = gs.chunk(0, n)
+    st = O.Store(dict(H.oracle_cfg(cfg), n_layers=1))
+    O.compress_chunk(st, H.to_numpy_bits(q), H.to_numpy_bits(k[-1:]), H.to_numpy_bits(v[-1:]))
+    for round_ in range(2):
+        kept = torch.full((n, cfg.keep_per_frame), -2, dtype=torch.int32, device="cuda:0")
+        sc = torch.full((3, n, cfg.tokens_per_frame), -2.0, dtype=torch.float32, device="cuda:0")
+        B.mukv_score_frames_noalloc(cfg, q, k[cfg.n_layers - 1], n, kept, sc)
+        torch.cuda.synchronize()
+        for f in range(n):
+            assert kept[f].cpu().numpy().tolist() == st.kept[f].tolist(), f"round {round_}: kept ids differ at frame {f}"
+            for i in range(3):
+                H.close(sc[i, f].cpu().numpy(), st.scores[f][i], f"round {round_}: score[{i}] frame {f}")
+        if round_ == 0:
+            small = H.GpuRun("tiny")                 # fp32, P = 64, D = 64: the smallest shared-memory need
+            small.compress()
+            B.MukvContext(H.spec_config(H.StreamSpec(seed=5, n_layers=1, n_q_heads=4, n_kv_heads=4, head_dim=64,
+                                                     tokens_per_frame=196, bf16=True, n_outlier=0, n_frames=2),
+                                        dict(keep=9, fseg=2, chunk=2, alpha=0.7)), "cuda:0").close()
 
 
 def test_noalloc_rejects_what_does_not_fit():
