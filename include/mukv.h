@@ -160,6 +160,17 @@ mukv_status mukv_compress_chunk(mukv_ctx* ctx, const void* d_q, const void* d_k,
                                 int32_t n_frames, int64_t first_frame,
                                 int32_t* d_kept_out, float* d_scores_out, mukv_stream stream);
 
+/* Like mukv_compress_chunk, but each frame's tokens are ranked by numbers the caller supplies
+ * instead of Eq. 1-4: d_select_scores [n_frames][P] float (device), higher = kept first, ties and
+ * near-ties (within tie_eps) to the lowest token id.  This is how the "Rand(50%)" row of the paper's
+ * compression-ablation table is reproduced (uniform random scores, kappa = P/2), and it lets a
+ * caller plug in an indicator of its own.  No queries are needed.  The ranking runs in double
+ * precision on the given floats, so it equals the exact rule; scores that are not finite make the
+ * frame keep its kappa lowest ids (device_status 7).  Errors: as mukv_compress_chunk. */
+mukv_status mukv_compress_chunk_scored(mukv_ctx* ctx, const float* d_select_scores, const void* d_k,
+                                       const void* d_v, int32_t n_frames, int64_t first_frame,
+                                       int32_t* d_kept_out, mukv_stream stream);
+
 /* Sec. 3.4.  Serves nq questions in one batch.
  *   d_qtok      [sum Nq][Hq][D] last-layer query tokens of all questions, concatenated.
  *   h_q_offsets [nq+1] token offsets of each question in d_qtok (host, ascending, [0]=0).
@@ -202,6 +213,26 @@ mukv_status mukv_gather(mukv_ctx* ctx, const int32_t* d_frm_idx, const int32_t* 
  *        7 page table (int64 byte offsets from the store base) [max_frames]
  * Returns NULL for an unknown region; *bytes (if not NULL) receives the region size. */
 void* mukv_store_region(const mukv_ctx* ctx, int32_t which, size_t* bytes);
+
+/* Moving a store (the paper's "offline memory" outlives the questions; it prints no format).
+ * The store buffer is position independent: every reference inside it is an offset from its
+ * base.  mukv_export_header fills a small plain header (configuration, frames stored); the caller
+ * copies the store's bytes wherever it likes (cudaMemcpy to another buffer, another device, the
+ * host) once the stream has finished.  mukv_import builds a context over such a copy: like
+ * mukv_create, but the store's contents are kept and the stream continues at header->frames.
+ * Errors of mukv_import: INVALID (null, bad magic / version), SHAPE/DTYPE, ALIGN, CAPACITY
+ * (store_bytes below header->store_bytes, workspace too small). */
+#define MUKV_STORE_MAGIC 0x564B754Du   /* "MuKV" */
+#define MUKV_STORE_VERSION 1u
+typedef struct {
+  uint32_t magic, version;
+  mukv_config cfg;
+  int64_t frames;
+  uint64_t store_bytes;            /* what mukv_store_bytes(&cfg) returned */
+} mukv_store_header;
+mukv_status mukv_export_header(const mukv_ctx* ctx, mukv_store_header* out);
+mukv_status mukv_import(const mukv_store_header* header, void* d_store, size_t store_bytes,
+                        void* d_workspace, size_t workspace_bytes, mukv_ctx** out);
 
 /* Reads counters.  Copies a few device words: synchronises the given stream. */
 mukv_status mukv_get_stats(mukv_ctx* ctx, mukv_stats* out, mukv_stream stream);

@@ -238,15 +238,24 @@ class Store:
         return np.stack([self.segment_key(u) for u in range(self.n_segments)])
 
 
-def compress_chunk(store: Store, Q, K, V) -> None:
-    """Append one chunk.  Q[n][P][Hq][D] (last layer), K,V[L][n][P][Hkv][D]."""
+def compress_chunk(store: Store, Q, K, V, select_scores=None) -> None:
+    """Append one chunk.  Q[n][P][Hq][D] (last layer), K,V[L][n][P][Hkv][D].
+
+    With select_scores[n][P] the tokens are ranked by those numbers instead of the dual signal:
+    the "Rand(50%)" row of the paper's compression ablation (tokens dropped at random) is this
+    with uniform random scores and kappa = P/2; Q is not used then.
+    """
     cfg = store.cfg
-    n = np.asarray(Q).shape[0]
+    n = np.asarray(K).shape[1]
     for f in range(n):
         Kf = np.asarray(K)[:, f]
         Vf = np.asarray(V)[:, f]
-        ia, ifr, I = score_frame(np.asarray(Q)[f], Kf[-1], cfg["alpha"],
-                                 cfg.get("attn_causal", False), cfg.get("keep_low_freq", False))
+        if select_scores is not None:
+            I = np.asarray(select_scores, dtype=np.float64)[f]
+            ia = ifr = np.zeros_like(I)
+        else:
+            ia, ifr, I = score_frame(np.asarray(Q)[f], Kf[-1], cfg["alpha"],
+                                     cfg.get("attn_causal", False), cfg.get("keep_low_freq", False))
         kept = select_tokens(I, cfg["keep_per_frame"], cfg.get("tie_eps", TIE_EPS))
         pk = compact_rows(Kf, kept)
         pv = compact_rows(Vf, kept)

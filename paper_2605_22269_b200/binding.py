@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "MUKV_OK", -1: "MUKV_E_INVALID", -2: "MUKV_E_SHAPE", -3: "MUK
                 -5: "MUKV_E_CAPACITY", -6: "MUKV_E_STATE", -7: "MUKV_E_CUDA", -8: "MUKV_E_UNSUPPORTED"}
 
 EXPORTS = ["mukv_store_bytes", "mukv_workspace_bytes", "mukv_create", "mukv_destroy", "mukv_reset", "mukv_set_option",
-           "mukv_compress_chunk", "mukv_retrieve", "mukv_gather", "mukv_store_region", "mukv_get_stats",
+           "mukv_compress_chunk", "mukv_compress_chunk_scored", "mukv_export_header", "mukv_import", "mukv_retrieve", "mukv_gather", "mukv_store_region", "mukv_get_stats",
            "mukv_last_error", "mukv_profile_enable", "mukv_profile_read", "mukv_score_frames_noalloc"]
 PROF_KINDS = ["score", "refine", "compact", "segment", "qpool", "scan", "rank", "gather"]
 
@@ -50,6 +50,11 @@ class MukvStats(C.Structure):
                 ("page_bytes", C.c_int64), ("store_bytes_used", C.c_int64), ("refined_frames", C.c_int64),
                 ("refined_questions", C.c_int64), ("kernel_launches", C.c_int64),
                 ("device_status", C.c_int32), ("reserved", C.c_int32)]
+
+
+class MukvStoreHeader(C.Structure):
+    _fields_ = [("magic", C.c_uint32), ("version", C.c_uint32), ("cfg", MukvConfig), ("frames", C.c_int64),
+                ("store_bytes", C.c_uint64)]
 
 
 _LIB = None
@@ -80,6 +85,12 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.mukv_set_option.argtypes = [vp, i32, C.c_double]
     lib.mukv_compress_chunk.restype = i32
     lib.mukv_compress_chunk.argtypes = [vp, vp, vp, vp, i32, i64, vp, vp, vp]
+    lib.mukv_compress_chunk_scored.restype = i32
+    lib.mukv_compress_chunk_scored.argtypes = [vp, vp, vp, vp, i32, i64, vp, vp]
+    lib.mukv_export_header.restype = i32
+    lib.mukv_export_header.argtypes = [vp, C.POINTER(MukvStoreHeader)]
+    lib.mukv_import.restype = i32
+    lib.mukv_import.argtypes = [C.POINTER(MukvStoreHeader), vp, C.c_size_t, vp, C.c_size_t, C.POINTER(vp)]
     lib.mukv_retrieve.restype = i32
     lib.mukv_retrieve.argtypes = [vp, vp, C.POINTER(i32), C.POINTER(i64), i32, i32, i32, i32, f32, i32,
                                   vp, vp, vp, vp, vp, vp]
@@ -133,7 +144,7 @@ def mukv_score_frames_noalloc(cfg: MukvConfig, q, k_last, n_frames: int, kept_ou
 class MukvContext:
     """Owns the torch buffers behind one ``mukv_ctx`` and forwards calls to the C ABI."""
 
-    def __init__(self, cfg: MukvConfig, device="cuda:0"):
+    def __init__(self, cfg: MukvConfig, device="cuda:0", _header=None, _store=None):
         self.lib = load_library()
         self.cfg = cfg
         self.device = torch.device(device)
@@ -143,16 +154,36 @@ class MukvContext:
             # let mukv_create produce the message
             sb = wb = 256
         with torch.cuda.device(self.device):
-            self.store = torch.empty(sb, dtype=torch.uint8, device=self.device)
+            self.store = torch.empty(sb, dtype=torch.uint8, device=self.device) if _store is None else _store
             self.workspace = torch.empty(wb, dtype=torch.uint8, device=self.device)
             h = C.c_void_p()
-            st = self.lib.mukv_create(C.byref(cfg), self.store.data_ptr(), sb, self.workspace.data_ptr(), wb,
-                                      C.byref(h))
+            if _header is None:
+                st = self.lib.mukv_create(C.byref(cfg), self.store.data_ptr(), sb, self.workspace.data_ptr(), wb,
+                                          C.byref(h))
+            else:
+                st = self.lib.mukv_import(C.byref(_header), self.store.data_ptr(), self.store.numel(),
+                                          self.workspace.data_ptr(), wb, C.byref(h))
         if st != 0:
             raise MukvError(st, (self.lib.mukv_last_error(None) or b"").decode())
         self.handle = h
         self.C = cfg.n_kv_heads * cfg.head_dim
         self.torch_dtype = torch.bfloat16 if cfg.dtype == BF16 else torch.float32
+
+    @classmethod
+    def from_copy(cls, header: MukvStoreHeader, store: torch.Tensor) -> "MukvContext":
+        """mukv_import: a context over `store`, a uint8 device tensor holding a copy of an exported store."""
+        cfg = MukvConfig.from_buffer_copy(header.cfg)
+        return cls(cfg, store.device, _header=header, _store=store)
+
+    def mukv_export_header(self) -> MukvStoreHeader:
+        h = MukvStoreHeader()
+        self._check(self.lib.mukv_export_header(self.handle, C.byref(h)))
+        return h
+
+    def mukv_compress_chunk_scored(self, select_scores, k, v, n_frames: int, first_frame: int, kept_out=None,
+                                   stream=None):
+        self._check(self.lib.mukv_compress_chunk_scored(self.handle, _ptr(select_scores), _ptr(k), _ptr(v), n_frames,
+                                                        first_frame, _ptr(kept_out), _stream(stream)))
 
     def close(self):
         if getattr(self, "handle", None):

@@ -18,9 +18,14 @@
 // tie_eps + flag_margin is skipped here: the double-precision pass that follows decides it, and
 // segment_kernel then compacts it.
 //
-// segment_kernel<T>: one block per (layer, K|V) plane: compacts the frames the double-precision
-// pass decided, then refreshes that plane of every segment entry the chunk touches (mean over the
-// frames present).
+// tail_kernel<T, NC>: what has to wait for every frame of the chunk.  Normally that is only the
+// segment entries (Eq. 5 at segment level): blocks 0 .. 2L-1 refresh one (layer, K|V) plane each of
+// every segment entry the chunk touches (mean over the frames present), the other blocks leave at
+// once.  When frames were flagged (about one chunk in fifty on the synthetic streams) all blocks
+// first score those frames in double precision and select; once every block has finished that,
+// the flagged frames are compacted and then the segment entries written, one plane per block.
+// (Segment pooling by the compaction block that finishes a plane last was measured: the fence
+// every block then needs before it signs off costs more than this launch.)
 #pragma once
 #include "common.cuh"
 #include "score.cuh"
@@ -28,6 +33,7 @@
 namespace mukv {
 
 constexpr int kCompactThreads = 256;
+static_assert(kCompactThreads == kScoreThreads, "tail_kernel runs the scoring and the compaction code in one block");
 
 struct CompactParams {
   int L, kappa, C, P;             // C = Hkv*D elements per row
@@ -41,13 +47,15 @@ struct CompactParams {
   double* frame_ksum;             // [max_frames][C]  exact sums of the last-layer kept keys
   long long* stat_refined;        // device counter
   int* n_flagged_next;            // the flagged count of the next chunk (the two chunks' counts alternate)
-  int* seg_counter;               // arrival counter of segment_kernel's blocks, zero between launches
+  int* tail_ctr;                  // [2] tail_kernel: blocks done with the double-precision scores / with everything
   // segment entries (Eq. 5 at segment level)
   int fseg;                       // frames per segment
   float* seg_entry;               // [max_segs][L][2][C]
   float* seg_key;                 // [max_segs][C]
   // selection
-  int sel_mode;                   // 0: kept ids are in the store; 1: select here from the partial sums
+  int sel_mode;                   // 0: kept ids are in the store; 1: select here from the partial sums;
+                                  // 2: select here by the caller's scores
+  const float* ext_scores;        // [n_frames][P] (sel_mode 2)
   int ps_grid, ps_items, ps_ipf;  // the scoring launch: blocks, items, items per frame
   unsigned* sel_flag;             // [F] (epoch << 1 | risky) once the plane-0 block has published its frame's ids
   unsigned epoch;                 // number of this call, never repeated
@@ -68,6 +76,10 @@ struct SelectScratch {
   unsigned ab[kCompactThreads / 32][2];
   int bin, rank, n_list;
   float tau;
+  // scratch of select_by_score (ranking by the caller's scores)
+  double sc64[MUKV_MAX_TOKENS];
+  double misc64[4 * (kCompactThreads / 32)];
+  int cnt64[kCompactThreads / 32 + 1];
 };
 
 // Eq. 4 and the top-kappa rule for frame f from the partial sums of the persistent scoring kernel,
@@ -243,11 +255,29 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
   return risky;
 }
 
+// What compact_segment_plane needs, small enough to travel in registers (the function is kept out
+// of line so that its 32 loads in flight do not set the register count of the kernels that call it;
+// a reference to the kernel's parameter block would force a per-thread copy of the block instead).
+struct SegmentArgs {
+  int L, kappa, C, fseg, n_frames;
+  long long first_frame;
+  const float* frame_entry;
+  const double* frame_ksum;
+  float* seg_entry;
+  float* seg_key;
+};
+__device__ __forceinline__ SegmentArgs segment_args(const CompactParams& p) {
+  SegmentArgs a;
+  a.L = p.L; a.kappa = p.kappa; a.C = p.C; a.fseg = p.fseg; a.n_frames = p.n_frames; a.first_frame = p.first_frame;
+  a.frame_entry = p.frame_entry; a.frame_ksum = p.frame_ksum; a.seg_entry = p.seg_entry; a.seg_key = p.seg_key;
+  return a;
+}
+
 // Segment entries (Eq. 5 at segment level) of one (layer, K|V) plane for every segment the chunk
 // touches: mean over the frames present, added in frame order.  Run by one whole block.  The loads
 // of up to 16 frames (and, in single precision, of two columns) are in flight together: the
-// kernel is a chain of L2 round trips and little else.
-__device__ inline void compact_segment_plane(const CompactParams& p, int l, int kv) {
+// work is a chain of L2 round trips and little else.
+__device__ __noinline__ void compact_segment_plane(const SegmentArgs p, int l, int kv) {
   const int tid = threadIdx.x;
   const int C = p.C, kappa = p.kappa;
   const bool exact = (l == p.L - 1) && (kv == 0);
@@ -393,7 +423,7 @@ __device__ __forceinline__ bool frame_is_flagged(const int* flagged, int n, int 
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactParams p) {
+__global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(const CompactParams p) {
   __shared__ CompactScratch cs;
   __shared__ SelectScratch ss;
   __shared__ unsigned s_seen;
@@ -406,6 +436,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
   pdl_trigger();
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.n_flagged_next = 0;
   const long long f_abs = p.first_frame + f;
+  bool risky;
   if (p.sel_mode == 1) {
     // A block that starts after its frame's plane-0 block has published the ids (the blocks beyond
     // the first wave do) reads them; every other block selects itself.  Nobody waits.
@@ -419,7 +450,6 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
     }
     __syncthreads();
     const unsigned seen = s_seen;
-    bool risky;
     if ((seen >> 1) == p.epoch) {
       risky = (seen & 1u) != 0u;
       for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(__ldcg(p.sp.kept_store + f_abs * p.kappa + r), p.P);
@@ -432,45 +462,103 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
         if (tid == 0) *reinterpret_cast<volatile unsigned*>(p.sel_flag + f) = (p.epoch << 1) | (risky ? 1u : 0u);
       }
     }
-    if (risky) return;
+  } else if (p.sel_mode == 2) {
+    // Ranking by numbers the caller supplies (no Eq. 1-4): every block ranks its frame itself, in
+    // double precision on exact inputs, so nothing is ever too close to call; plane 0 writes the ids.
+    double sx[1] = {tid < p.P ? (double)__ldg(p.ext_scores + (long long)f * p.P + tid) : 0.0};
+    const bool bad = __syncthreads_or(tid < p.P && !isfinite(sx[0])) != 0;
+    if (bad) sx[0] = 0.0;
+    bool keep[1];
+    select_by_score<1>(p.sp, f, sx, plane == 0, cs.kept, keep, ss.sc64, ss.cnt64, ss.misc64);
+    if (bad && plane == 0 && tid == 0 && p.sp.status) atomicCAS(p.sp.status, 0, kStatusNonFinite);
+    risky = false;
+    __syncthreads();
   } else {
-    if (frame_is_flagged(p.sp.flagged, *p.sp.n_flagged, f)) return;
+    risky = frame_is_flagged(p.sp.flagged, *p.sp.n_flagged, f);
     for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(p.sp.kept_store[f_abs * p.kappa + r], p.P);
     __syncthreads();
   }
-  compact_plane<T>(p, plane, f, &cs);
+  if (!risky) compact_plane<T>(p, plane, f, &cs);
 }
 
-// segment_kernel: one block per (layer, K|V) plane.  First the frames that the double-precision
-// pass decided (their ids are in the store by now), then that plane of every segment entry the
-// chunk touches.
-template <typename T>
-__global__ void __launch_bounds__(kCompactThreads) segment_kernel(const CompactParams p) {
-  __shared__ CompactScratch cs;
-  const int tid = threadIdx.x, plane = blockIdx.x;
-  pdl_wait();
-  const int n_fl = *p.sp.n_flagged;
-  for (int i = 0; i < n_fl; ++i) {
-    const int f = p.sp.flagged[i];
-    const long long f_abs = p.first_frame + f;
-    __syncthreads();
-    for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(__ldcg(p.sp.kept_store + f_abs * p.kappa + r), p.P);
-    __syncthreads();
-    compact_plane<T>(p, plane, f, &cs);
+// Bounded wait until *ctr reaches `target` (other blocks of the same grid add to it; the grid is
+// sized so that all its blocks are resident).  False after about 1.5 s.
+__device__ inline bool wait_counter(const int* ctr, int target) {
+  const volatile int* c = ctr;
+  unsigned long long t0 = 0;
+  for (long long spin = 0;; ++spin) {
+    if (*c >= target) return true;
+    if ((spin & 63) == 63) {
+      unsigned long long now;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 1500000000ull) return false;
+    }
+    __nanosleep(200);
   }
-  // the frame entries this block has just written are read below by other threads of the block
-  if (n_fl) __threadfence();
-  __syncthreads();
-  compact_segment_plane(p, plane >> 1, plane & 1);
-  // The block that arrives last adds the chunk's flagged frames to the statistics.  (Measured: with
-  // this one round trip to the L2 at the end of every block the kernel finishes about 4 us sooner
-  // than when its blocks exit right behind their last stores.)
+}
+
+constexpr int kStatusTailWait = 6;   // tail_kernel: the wait for the double-precision scores ran out
+
+// tail_kernel: see the head of this file.  sp is the scoring configuration of the double-precision
+// pass (its partial-sum buffers, refine = 1); the grid is a multiple of nothing in particular: blocks
+// stride over the work, and the host keeps the grid within what is resident at once.
+template <typename T, int NC>
+__global__ void __launch_bounds__(kScoreThreads, 2) tail_kernel(const ScoreParams sp, const CompactParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ CompactScratch cs;
+  __shared__ int s_ok;
+  const int tid = threadIdx.x;
+  pdl_wait();
+  const int n_fl = *sp.n_flagged;
+  if (n_fl == 0) {
+    // the common case: segment entries only
+    for (int plane = blockIdx.x; plane < 2 * p.L; plane += gridDim.x)
+      compact_segment_plane(segment_args(p), plane >> 1, plane & 1);
+    return;
+  }
+  // ---- scores of the flagged frames in double precision; the block that finishes a frame last selects
+  const int units = sp.Hq * sp.row_split;
+  for (int w = blockIdx.x; w < n_fl * units; w += gridDim.x) {
+    const int u = w % units;
+    score_frame_block<T, double, NC>(sp, u / sp.row_split, u % sp.row_split, sp.flagged[w / units], smem_raw);
+    __syncthreads();
+  }
+  // ---- every block waits for all selections
+  __threadfence();
   __syncthreads();
   if (tid == 0) {
-    const int old = atomicAdd(p.seg_counter, 1);
+    atomicAdd(p.tail_ctr, 1);
+    s_ok = wait_counter(p.tail_ctr, (int)gridDim.x) ? 1 : 0;
+    __threadfence();
+  }
+  __syncthreads();
+  if (!s_ok) {
+    if (tid == 0 && sp.status) atomicCAS(sp.status, 0, kStatusTailWait);
+  } else {
+    // ---- the flagged frames' compaction, then the segment entries, plane by plane
+    for (int plane = blockIdx.x; plane < 2 * p.L; plane += gridDim.x) {
+      for (int i = 0; i < n_fl; ++i) {
+        const int f = sp.flagged[i];
+        const long long f_abs = p.first_frame + f;
+        __syncthreads();
+        for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(__ldcg(sp.kept_store + f_abs * p.kappa + r), p.P);
+        __syncthreads();
+        compact_plane<T>(p, plane, f, &cs);
+      }
+      __threadfence();                          // the frame entries just written are read below by other threads
+      __syncthreads();
+      compact_segment_plane(segment_args(p), plane >> 1, plane & 1);
+    }
+  }
+  // ---- the block that leaves last resets the counters and adds to the statistics
+  __syncthreads();
+  if (tid == 0) {
+    const int old = atomicAdd(p.tail_ctr + 1, 1);
     if (old == (int)gridDim.x - 1) {
       *p.stat_refined += n_fl;
-      *p.seg_counter = 0;
+      p.tail_ctr[0] = 0;
+      p.tail_ctr[1] = 0;
     }
   }
 }

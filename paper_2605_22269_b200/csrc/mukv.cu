@@ -36,8 +36,8 @@ struct StoreLayout {
 };
 
 struct WorkLayout {
-  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, seg_counter, sel_flag, stat_refined,
-      dev_status;
+  size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, tail_ctr, sel_flag,
+      stat_refined, dev_status;
   size_t q64, qnorm, s_frm, s_seg, wtab, total;
   size_t zero_begin, zero_end;          // region that must start as zeros
 };
@@ -69,6 +69,7 @@ struct mukv_ctx {
   bool failed = false;                   // a compress call broke off half way: only reset / stats / destroy
   TcShape tcs;                           // tcs.ok: the chunk is scored on the tensor cores
   int n_sms;
+  int tail_capacity = 1;                 // blocks of tail_kernel that are resident at once on this device
   CUtensorMap wmap;                      // DFT matrix terms [3*D][D] bf16
   std::string err;
   // optional per-kernel timing (host objects only)
@@ -207,7 +208,7 @@ WorkLayout work_layout(const mukv_config& c) {
   w.frame_counter = off;  off = align_up(off + F * sizeof(int));
   w.flagged = off;        off = align_up(off + F * sizeof(int));
   w.n_flagged = off;      off = align_up(off + 2 * sizeof(int));   // alternate between chunks
-  w.seg_counter = off;    off = align_up(off + sizeof(int));
+  w.tail_ctr = off;       off = align_up(off + 2 * sizeof(int));
   w.sel_flag = off;       off = align_up(off + F * sizeof(unsigned));
   w.stat_refined = off;   off = align_up(off + sizeof(long long));
   w.dev_status = off;     off = align_up(off + sizeof(int));
@@ -240,6 +241,27 @@ cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, unsigned block, size_t
   cfg.attrs = attr;
   cfg.numAttrs = dependent ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+template <typename T>
+const void* tail_fn(int nc) {
+  switch (nc) {
+    case 2: return (const void*)tail_kernel<T, 2>;
+    case 4: return (const void*)tail_kernel<T, 4>;
+    case 7: return (const void*)tail_kernel<T, 7>;
+    default: return (const void*)tail_kernel<T, 8>;
+  }
+}
+
+template <typename T>
+cudaError_t launch_tail(const ScoreParams& sp, const CompactParams& cp, int nc, int grid, size_t smem, cudaStream_t st,
+                        bool dependent) {
+  switch (nc) {
+    case 2: return launch_k(tail_kernel<T, 2>, dim3(grid), kScoreThreads, smem, st, dependent, sp, cp);
+    case 4: return launch_k(tail_kernel<T, 4>, dim3(grid), kScoreThreads, smem, st, dependent, sp, cp);
+    case 7: return launch_k(tail_kernel<T, 7>, dim3(grid), kScoreThreads, smem, st, dependent, sp, cp);
+    default: return launch_k(tail_kernel<T, 8>, dim3(grid), kScoreThreads, smem, st, dependent, sp, cp);
+  }
 }
 
 template <typename T, typename A>
@@ -296,6 +318,11 @@ cudaError_t raise_kernel_limits(int* n_sms) {
   if (e == cudaSuccess) e = raise_score_limits<__nv_bfloat16, double>(optin);
   if (e == cudaSuccess) e = raise_score_limits<float, float>(optin);
   if (e == cudaSuccess) e = raise_score_limits<float, double>(optin);
+  const int ncs[4] = {2, 4, 7, 8};
+  for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+    e = raise_smem_limit(tail_fn<__nv_bfloat16>(ncs[i]), optin);
+    if (e == cudaSuccess) e = raise_smem_limit(tail_fn<float>(ncs[i]), optin);
+  }
   if (e == cudaSuccess) e = raise_smem_limit((const void*)rank_kernel, optin);
   if (e == cudaSuccess) e = raise_smem_limit((const void*)score_ps_kernel, optin);
   if (e == cudaSuccess) g_limits_raised[dev] = true;
@@ -413,8 +440,8 @@ cudaError_t launch_score_ps(mukv_ctx* ctx, const ScoreParams& sp, const void* d_
 }
 
 template <typename T>
-mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const void* d_v, int n, long long t0,
-                          int* d_kept_out, float* d_scores_out, cudaStream_t st) {
+mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, const void* d_k, const void* d_v, int n,
+                          long long t0, int* d_kept_out, float* d_scores_out, cudaStream_t st) {
   const mukv_config& c = ctx->cfg;
   const int P = c.tokens_per_frame, L = c.n_layers, C = ctx->C;
   ScoreParams sp;
@@ -441,10 +468,10 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   sp.refine = 0;
   sp.row_split = 1;
   const dim3 grid(c.n_q_heads, n);
-  cudaError_t e;
+  cudaError_t e = cudaSuccess;
   const char* what = "score kernel";
   int ps_grid = 0, ps_items = 0, ps_ipf = 0;
-  {
+  if (!d_ext) {
     ProfScope ps(ctx, 0, st);
     if (ctx->tcs.ok && !ctx->force_fma)
       e = launch_score_ps(ctx, sp, d_q, sp.k_last, n, st, &what, &ps_grid, &ps_items, &ps_ipf);
@@ -464,14 +491,15 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   cp.frame_key = reinterpret_cast<float*>(ctx->store + ctx->sl.frame_key);
   cp.frame_ksum = reinterpret_cast<double*>(ctx->store + ctx->sl.frame_ksum);
   cp.stat_refined = reinterpret_cast<long long*>(ctx->ws + ctx->wl.stat_refined);
-  cp.seg_counter = reinterpret_cast<int*>(ctx->ws + ctx->wl.seg_counter);
+  cp.tail_ctr = reinterpret_cast<int*>(ctx->ws + ctx->wl.tail_ctr);
   cp.sel_flag = reinterpret_cast<unsigned*>(ctx->ws + ctx->wl.sel_flag);
   cp.epoch = (++ctx->epoch) & 0x7fffffffu;
   cp.n_flagged_next = reinterpret_cast<int*>(ctx->ws + ctx->wl.n_flagged) + (ctx->parity ^ 1);
   cp.fseg = c.frames_per_segment;
   cp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
   cp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
-  cp.sel_mode = ps_grid > 0 ? 1 : 0;
+  cp.sel_mode = d_ext ? 2 : ps_grid > 0 ? 1 : 0;
+  cp.ext_scores = d_ext;
   cp.ps_grid = ps_grid; cp.ps_items = ps_items; cp.ps_ipf = ps_ipf;
   cp.sp = sp;
   if (ps_grid > 0) cp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
@@ -481,28 +509,41 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const void* d_k, const
   }
   if (e != cudaSuccess) return broke_off(ctx, "compact kernel", e);
 
-  // frames too close to a tie boundary: the scores again in double precision, and the selection
-  // (blocks beyond the flagged count return at once)
+  // What needs every frame of the chunk: the segment entries; before them, for frames too close to
+  // a tie boundary, scores and selection again in double precision and their compaction.
   sp.refine = 1;
   sp.row_split = kRefineSplit;
   sp.colsum_part = ctx->ws + ctx->wl.colsum_d;
   sp.ifft_part = ctx->ws + ctx->wl.ifft_d;
   {
     ProfScope ps(ctx, 1, st);
-    const dim3 rgrid(c.n_q_heads * kRefineSplit, n < 2 ? n : 2);   // its blocks walk the flagged frames
-    e = launch_score<T, double>(sp, ctx->nc, rgrid, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
+    int grid_t = c.n_q_heads * kRefineSplit * (n < 2 ? n : 2);
+    if (grid_t < 2 * L) grid_t = 2 * L;
+    if (grid_t > ctx->tail_capacity) grid_t = ctx->tail_capacity;
+    e = launch_tail<T>(sp, cp, ctx->nc, grid_t, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
   }
-  if (e != cudaSuccess) return broke_off(ctx, "refine kernel", e);
-  // compaction of those frames, then the segment entries
-  {
-    ProfScope ps(ctx, 3, st);
-    e = launch_k(segment_kernel<T>, dim3(L * 2), kCompactThreads, 0, st, !ctx->prof_on, cp);
-  }
-  if (e != cudaSuccess) return broke_off(ctx, "segment kernel", e);
+  if (e != cudaSuccess) return broke_off(ctx, "tail kernel", e);
 
-  ctx->launches += 4;
+  ctx->launches += d_ext ? 2 : 3;
   ctx->parity ^= 1;
   ctx->frames = t0 + n;
+  return MUKV_OK;
+}
+
+mukv_status create_impl(const mukv_config* cfg, void* d_store, size_t store_bytes, void* d_workspace,
+                        size_t workspace_bytes, long long frames0, mukv_ctx** out);
+
+mukv_status check_chunk_args(mukv_ctx* ctx, int n_frames, long long first_frame) {
+  if (n_frames < 1) return fail(ctx, MUKV_E_INVALID, "n_frames must be >= 1");
+  if (n_frames > ctx->cfg.max_frames_per_chunk)
+    return fail(ctx, MUKV_E_CAPACITY, "n_frames %d exceeds max_frames_per_chunk %d", n_frames,
+                ctx->cfg.max_frames_per_chunk);
+  if (first_frame != ctx->frames)
+    return fail(ctx, MUKV_E_STATE, "first_frame %lld does not continue the stream (%lld frames stored)", first_frame,
+                ctx->frames);
+  if (first_frame + n_frames > ctx->cfg.max_frames)
+    return fail(ctx, MUKV_E_CAPACITY, "store full: %lld + %d frames > max_frames %lld", ctx->frames, n_frames,
+                (long long)ctx->cfg.max_frames);
   return MUKV_OK;
 }
 
@@ -522,6 +563,39 @@ size_t mukv_workspace_bytes(const mukv_config* cfg) {
 
 mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_bytes, void* d_workspace,
                         size_t workspace_bytes, mukv_ctx** out) {
+  return create_impl(cfg, d_store, store_bytes, d_workspace, workspace_bytes, 0, out);
+}
+
+mukv_status mukv_export_header(const mukv_ctx* ctx, mukv_store_header* out) {
+  if (!ctx || !out) return MUKV_E_INVALID;
+  memset(out, 0, sizeof *out);
+  out->magic = MUKV_STORE_MAGIC;
+  out->version = MUKV_STORE_VERSION;
+  out->cfg = ctx->cfg;
+  out->frames = ctx->frames;
+  out->store_bytes = ctx->sl.total;
+  return MUKV_OK;
+}
+
+mukv_status mukv_import(const mukv_store_header* header, void* d_store, size_t store_bytes, void* d_workspace,
+                        size_t workspace_bytes, mukv_ctx** out) {
+  if (!out) return fail(nullptr, MUKV_E_INVALID, "out is null");
+  *out = nullptr;
+  if (!header) return fail(nullptr, MUKV_E_INVALID, "null header");
+  if (header->magic != MUKV_STORE_MAGIC || header->version != MUKV_STORE_VERSION)
+    return fail(nullptr, MUKV_E_INVALID, "not a store header of this library version");
+  if (header->frames < 0 || header->frames > header->cfg.max_frames)
+    return fail(nullptr, MUKV_E_INVALID, "header: frame count out of range");
+  if (check_config(&header->cfg) == nullptr && header->store_bytes != store_layout(header->cfg).total)
+    return fail(nullptr, MUKV_E_INVALID, "header: store size does not match its configuration");
+  return create_impl(&header->cfg, d_store, store_bytes, d_workspace, workspace_bytes, header->frames, out);
+}
+
+}  // extern "C"
+
+namespace {
+mukv_status create_impl(const mukv_config* cfg, void* d_store, size_t store_bytes, void* d_workspace,
+                        size_t workspace_bytes, long long frames0, mukv_ctx** out) {
   if (!out) return fail(nullptr, MUKV_E_INVALID, "out is null");
   *out = nullptr;
   if (!cfg || !d_store || !d_workspace) return fail(nullptr, MUKV_E_INVALID, "null argument");
@@ -542,7 +616,7 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
   }
   ctx->store = static_cast<unsigned char*>(d_store);
   ctx->ws = static_cast<unsigned char*>(d_workspace);
-  ctx->frames = 0;
+  ctx->frames = frames0;
   ctx->launches = 0;
   ctx->C = cfg->n_kv_heads * cfg->head_dim;
   ctx->G = cfg->n_q_heads / cfg->n_kv_heads;
@@ -554,6 +628,17 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
   ctx->flat_ratio = kFlatRatio;
   const int D = cfg->head_dim;
   cudaError_t e = raise_kernel_limits(&ctx->n_sms);
+  if (e == cudaSuccess) {
+    // the blocks of tail_kernel wait for one another: its grid must be resident as a whole
+    int per_sm = 0;
+    const bool bf = cfg->dtype == MUKV_BF16;
+    const size_t dyn = bf ? score_smem_bytes<__nv_bfloat16, double>(cfg->tokens_per_frame, D)
+                          : score_smem_bytes<float, double>(cfg->tokens_per_frame, D);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bf ? tail_fn<__nv_bfloat16>(ctx->nc) : tail_fn<float>(ctx->nc),
+                                                      kScoreThreads, dyn);
+    if (e == cudaSuccess && per_sm < 1) e = cudaErrorInvalidConfiguration;
+    ctx->tail_capacity = per_sm * ctx->n_sms;
+  }
   if (e == cudaSuccess && ctx->tcs.ok) {
     const std::vector<uint16_t> w = dft_terms(D);
     e = cudaMemcpy(ctx->ws + ctx->wl.wtab, w.data(), w.size() * 2, cudaMemcpyHostToDevice);
@@ -570,6 +655,9 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
   *out = ctx;
   return MUKV_OK;
 }
+}  // namespace
+
+extern "C" {
 
 void mukv_destroy(mukv_ctx* ctx) {
   if (!ctx) return;
@@ -637,20 +725,31 @@ mukv_status mukv_compress_chunk(mukv_ctx* ctx, const void* d_q, const void* d_k,
     if (!d_q || !d_k || !d_v) return fail(ctx, MUKV_E_INVALID, "null input pointer");
     if (!aligned16(d_q) || !aligned16(d_k) || !aligned16(d_v) || !aligned4(d_kept_out) || !aligned4(d_scores_out))
       return fail(ctx, MUKV_E_ALIGN, "d_q, d_k, d_v must be 16-byte aligned, the outputs 4-byte aligned");
-    if (n_frames < 1) return fail(ctx, MUKV_E_INVALID, "n_frames must be >= 1");
-    if (n_frames > ctx->cfg.max_frames_per_chunk)
-      return fail(ctx, MUKV_E_CAPACITY, "n_frames %d exceeds max_frames_per_chunk %d", n_frames,
-                  ctx->cfg.max_frames_per_chunk);
-    if (first_frame != ctx->frames)
-      return fail(ctx, MUKV_E_STATE, "first_frame %lld does not continue the stream (%lld frames stored)",
-                  (long long)first_frame, ctx->frames);
-    if (first_frame + n_frames > ctx->cfg.max_frames)
-      return fail(ctx, MUKV_E_CAPACITY, "store full: %lld + %d frames > max_frames %lld", ctx->frames, n_frames,
-                  (long long)ctx->cfg.max_frames);
+    if (const mukv_status st = check_chunk_args(ctx, n_frames, first_frame)) return st;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (ctx->cfg.dtype == MUKV_BF16)
-      return compress_impl<__nv_bfloat16>(ctx, d_q, d_k, d_v, n_frames, first_frame, d_kept_out, d_scores_out, st);
-    return compress_impl<float>(ctx, d_q, d_k, d_v, n_frames, first_frame, d_kept_out, d_scores_out, st);
+      return compress_impl<__nv_bfloat16>(ctx, d_q, nullptr, d_k, d_v, n_frames, first_frame, d_kept_out, d_scores_out, st);
+    return compress_impl<float>(ctx, d_q, nullptr, d_k, d_v, n_frames, first_frame, d_kept_out, d_scores_out, st);
+  } catch (...) {
+    return fail(ctx, MUKV_E_INVALID, "unexpected exception");
+  }
+}
+
+mukv_status mukv_compress_chunk_scored(mukv_ctx* ctx, const float* d_select_scores, const void* d_k, const void* d_v,
+                                       int32_t n_frames, int64_t first_frame, int32_t* d_kept_out,
+                                       mukv_stream stream) {
+  if (!ctx) return MUKV_E_INVALID;
+  try {
+    if (ctx->failed) return fail(ctx, MUKV_E_STATE, "an earlier call broke off half way: call mukv_reset");
+    if (!d_select_scores || !d_k || !d_v) return fail(ctx, MUKV_E_INVALID, "null input pointer");
+    if (!aligned4(d_select_scores) || !aligned16(d_k) || !aligned16(d_v) || !aligned4(d_kept_out))
+      return fail(ctx, MUKV_E_ALIGN, "d_k, d_v must be 16-byte aligned, scores and outputs 4-byte aligned");
+    if (const mukv_status st = check_chunk_args(ctx, n_frames, first_frame)) return st;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->cfg.dtype == MUKV_BF16)
+      return compress_impl<__nv_bfloat16>(ctx, nullptr, d_select_scores, d_k, d_v, n_frames, first_frame, d_kept_out,
+                                          nullptr, st);
+    return compress_impl<float>(ctx, nullptr, d_select_scores, d_k, d_v, n_frames, first_frame, d_kept_out, nullptr, st);
   } catch (...) {
     return fail(ctx, MUKV_E_INVALID, "unexpected exception");
   }

@@ -61,6 +61,83 @@ __host__ inline size_t score_smem_bytes(int P, int D) {
   return ((ks + 15) / 16) * 16 + qs + tw + red + sel + 64;
 }
 
+// The top-kappa rule for one frame on final scores s (double), run by all threads of the group Grp.
+// Thread tid owns the tokens tid + k*size, k < TOK (TOK*size >= P).  tau is the kappa-th largest
+// score (rank counting: P <= 256); scores above tau + tie_eps are kept, the scores within tie_eps
+// of tau share the remaining places by lowest token id.  keep[k] says which of the thread's tokens
+// stay; the kept ids go, ascending, to s_kept (shared memory, may be null) and, with `write`, to
+// the store, to the caller's output and the frame's time stamp and page-table entry are set.
+// s_sc (P doubles), s_int (one int per warp + 1), s_misc (4 doubles per warp) are shared scratch.
+template <int TOK, class Grp = BlockGroup>
+__device__ inline void select_by_score(const ScoreParams& p, int f, const double (&s)[TOK], bool write, int* s_kept,
+                                       bool (&keep)[TOK], double* s_sc, int* s_int, double* s_misc) {
+  const int tid = Grp::tid();
+  const int nt = Grp::size();
+  const int P = p.P;
+  int tok[TOK];
+  bool valid[TOK];
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    tok[k] = tid + k * nt;
+    valid[k] = tok[k] < P;
+    if (valid[k]) s_sc[tok[k]] = s[k];
+  }
+  Grp::sync();
+  const int kappa = p.kappa;
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    if (valid[k]) {
+      int gt = 0, ge = 0;
+      for (int i = 0; i < P; ++i) {
+        const double o = s_sc[i];
+        gt += (o > s[k]);
+        ge += (o >= s[k]);
+      }
+      if (gt < kappa && kappa <= ge) s_misc[0] = s[k];      // every writer holds the same value
+    }
+  }
+  Grp::sync();
+  const double tau = s_misc[0];
+  const double delta = (double)p.tie_eps;
+  bool sure[TOK], band[TOK];
+  int n_sure = 0;
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    sure[k] = valid[k] && (s[k] > tau + delta);
+    band[k] = valid[k] && !sure[k] && (s[k] >= tau - delta);
+    int t;
+    group_excl_count<Grp>(sure[k], s_int, t);
+    n_sure += t;
+  }
+  int band_before = 0;
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    int t;
+    const int band_rank = band_before + group_excl_count<Grp>(band[k], s_int, t);
+    band_before += t;
+    keep[k] = sure[k] || (band[k] && band_rank < kappa - n_sure);
+  }
+  const long long f_abs = p.first_frame + f;
+  int out_before = 0;
+#pragma unroll
+  for (int k = 0; k < TOK; ++k) {
+    int t;
+    const int pos = out_before + group_excl_count<Grp>(keep[k], s_int, t);
+    out_before += t;
+    if (keep[k]) {
+      if (s_kept) s_kept[pos] = tok[k];
+      if (write) {
+        p.kept_store[f_abs * kappa + pos] = tok[k];
+        if (p.kept_out) p.kept_out[(long long)f * kappa + pos] = tok[k];
+      }
+    }
+  }
+  if (write && tid == 0) {
+    p.frame_ts[f_abs] = f_abs;
+    p.page_table[f_abs] = p.pages_off + f_abs * p.page_bytes;
+  }
+}
+
 // Eq. 4 and the top-kappa rule for one frame, run by all threads of the group Grp.  Thread tid owns
 // the tokens tid + k*size, k < TOK (TOK*size >= P); att_raw / fft_raw are their I_att and I_fft;
 // s_sc (P doubles), s_int (one int per warp + 1), s_misc (4 doubles per warp) are shared scratch.
@@ -120,73 +197,29 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
     A fn = (fmax_ == fmin_) ? (A)0 : (fft_raw[k] - fmin_) / (fmax_ - fmin_);
     if (p.keep_low) fn = (A)1 - fn;
     s[k] = bad ? (A)0 : alpha * an + ((A)1 - alpha) * fn;
-    if (valid[k]) s_sc[tok[k]] = s[k];
   }
-  Grp::sync();
-  // ---- tau = kappa-th largest score (rank counting; P <= 256)
-  const int kappa = p.kappa;
+  bool keep[TOK];
+  select_by_score<TOK, Grp>(p, f, s, true, nullptr, keep, s_sc, s_int, s_misc);
+  if (p.scores_out) {
+    const long long np = (long long)p.n_frames * P;
 #pragma unroll
-  for (int k = 0; k < TOK; ++k) {
-    if (valid[k]) {
-      int gt = 0, ge = 0;
-      for (int i = 0; i < P; ++i) {
-        const A o = s_sc[i];
-        gt += (o > s[k]);
-        ge += (o >= s[k]);
+    for (int k = 0; k < TOK; ++k) {
+      if (valid[k]) {
+        p.scores_out[0 * np + (long long)f * P + tok[k]] = (float)att_raw[k];
+        p.scores_out[1 * np + (long long)f * P + tok[k]] = (float)fft_raw[k];
+        p.scores_out[2 * np + (long long)f * P + tok[k]] = (float)s[k];
       }
-      if (gt < kappa && kappa <= ge) s_misc[0] = s[k];      // every writer holds the same value
     }
   }
-  Grp::sync();
-  const A tau = s_misc[0];
-  const A delta = (A)p.tie_eps;
-  bool sure[TOK], band[TOK], keep[TOK];
-  int n_sure = 0;
-#pragma unroll
-  for (int k = 0; k < TOK; ++k) {
-    sure[k] = valid[k] && (s[k] > tau + delta);
-    band[k] = valid[k] && !sure[k] && (s[k] >= tau - delta);
-    int t;
-    group_excl_count<Grp>(sure[k], s_int, t);
-    n_sure += t;
-  }
-  int band_before = 0;
-#pragma unroll
-  for (int k = 0; k < TOK; ++k) {
-    int t;
-    const int band_rank = band_before + group_excl_count<Grp>(band[k], s_int, t);
-    band_before += t;
-    keep[k] = sure[k] || (band[k] && band_rank < kappa - n_sure);
-  }
-  const long long f_abs = p.first_frame + f;
-  int out_before = 0;
-#pragma unroll
-  for (int k = 0; k < TOK; ++k) {
-    int t;
-    const int pos = out_before + group_excl_count<Grp>(keep[k], s_int, t);
-    out_before += t;
-    if (keep[k]) {
-      p.kept_store[f_abs * kappa + pos] = tok[k];
-      if (p.kept_out) p.kept_out[(long long)f * kappa + pos] = tok[k];
-    }
-    if (p.scores_out && valid[k]) {
-      const long long np = (long long)p.n_frames * P;
-      p.scores_out[0 * np + (long long)f * P + tok[k]] = (float)att_raw[k];
-      p.scores_out[1 * np + (long long)f * P + tok[k]] = (float)fft_raw[k];
-      p.scores_out[2 * np + (long long)f * P + tok[k]] = (float)s[k];
-    }
-  }
-  if (tid == 0) {
-    p.frame_ts[f_abs] = f_abs;
-    p.page_table[f_abs] = p.pages_off + f_abs * p.page_bytes;
-    if (bad && p.status) atomicCAS(p.status, 0, kStatusNonFinite);
-  }
+  if (tid == 0 && bad && p.status) atomicCAS(p.status, 0, kStatusNonFinite);
   // ---- does single precision decide this frame safely?
   // With a = lowest kept score and b = highest dropped score, the kept set is the same for every
   // perturbation of the scores below flag_margin / 2 as long as a - b > tie_eps + flag_margin: no
   // dropped token can then enter the tie band of the kappa-th score.  Anything closer is redone
   // in double precision.
   if (!p.refine && !bad) {
+    const int kappa = p.kappa;
+    const A delta = (A)p.tie_eps;
     A a = big, b = -big;
 #pragma unroll
     for (int k = 0; k < TOK; ++k) {

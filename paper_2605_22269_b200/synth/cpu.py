@@ -25,7 +25,7 @@ GOLD = 0x9E3779B97F4A7C15
 M1 = 0xBF58476D1CE4E5B9
 M2 = 0x94D049BB133111EB
 
-TAG_K, TAG_V, TAG_Q, TAG_OUT, TAG_MU, TAG_NU, TAG_SCENE, TAG_QUEST = 1, 2, 3, 4, 5, 6, 7, 8
+TAG_K, TAG_V, TAG_Q, TAG_OUT, TAG_MU, TAG_NU, TAG_SCENE, TAG_QUEST, TAG_RAND = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
 TABLE_BITS = 16
 
@@ -191,6 +191,18 @@ class StreamSpec:
             ks.append(k)
             vs.append(v)
         return np.stack(qs, 0), np.stack(ks, 1), np.stack(vs, 1)
+
+    def select_scores(self, n: int, t0: int = 0) -> np.ndarray:
+        """Uniform [0, 1) float32 numbers [n][P] (24 random bits each), one per token of frames
+        t0..t0+n-1: the random ranking of a random-drop baseline."""
+        P = self.tokens_per_frame
+        out = np.empty((n, P), dtype=np.float32)
+        for i in range(n):
+            words = np.arange(P, dtype=np.uint64)
+            with np.errstate(over="ignore"):
+                h = _mix64_np(np.uint64(stream_key(self.seed, TAG_RAND, t0 + i)) + (words + np.uint64(1)) * np.uint64(GOLD))
+            out[i] = ((h >> np.uint64(40)).astype(np.float64) / float(1 << 24)).astype(np.float32)
+        return out
 
     def questions(self, n_q: int, len_min: int, len_max: int, noise: float = 0.5):
         """Ragged question query tokens near random scene means.

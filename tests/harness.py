@@ -113,6 +113,9 @@ class GpuRun:
         self.kept = None
         self.scores = None
 
+    def store_bytes(self) -> int:
+        return self.ctx.store.numel()
+
     def compress(self, chunk=None):
         chunk = chunk or self.wl["chunk"]
         c = self.cfg

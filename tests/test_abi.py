@@ -37,7 +37,7 @@ def test_exports_match_header(lib):
 
 
 def test_struct_sizes_match_header():
-    assert C.sizeof(B.MukvConfig) == 64 and C.sizeof(B.MukvStats) == 72
+    assert C.sizeof(B.MukvConfig) == 64 and C.sizeof(B.MukvStats) == 72 and C.sizeof(B.MukvStoreHeader) == 88
 
 
 def test_store_size_of_the_three_hour_stream(lib):

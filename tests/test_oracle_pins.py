@@ -244,6 +244,22 @@ def test_compress_keeps_budget_and_copies_bytes():
                 assert st.page_v[t][l, r].tobytes() == V[l, t, j].tobytes()
 
 
+def test_random_drop_fixture():
+    # the "Rand(50%)" row of the compression ablation: selection by caller-given random scores
+    cfg = dict(CFG, keep_per_frame=O.keep_count(0.5, CFG["tokens_per_frame"]))
+    L, Hkv, D, P = cfg["n_layers"], cfg["n_kv_heads"], cfg["head_dim"], cfg["tokens_per_frame"]
+    K, V = rand(L, 4, P, Hkv, D), rand(L, 4, P, Hkv, D)
+    r = np.random.default_rng(3).random((4, P)).astype(np.float32)
+    st = O.Store(cfg)
+    O.compress_chunk(st, None, K, V, select_scores=r)
+    for t in range(4):
+        want = np.sort(np.argsort(-r[t].astype(np.float64), kind="stable")[:P // 2])
+        assert st.kept[t].tolist() == want.tolist() and len(want) == P // 2
+        assert st.page_k[t].tobytes() == K[:, t][:, want].tobytes()
+    # half of the memory tokens, as the table prints: 59K -> 29K
+    assert abs(300 * O.keep_count(0.5, 196) / 1000.0 - 29) <= 1.0
+
+
 def test_chunking_does_not_change_the_store():
     a, Q, K, V = make_store(5, chunk=2)
     b = O.Store(CFG)

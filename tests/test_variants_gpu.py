@@ -1,0 +1,82 @@
+"""Variants beyond the default path, through the C ABI against the CPU oracle: ranking by
+caller-supplied scores (the random-drop row of the paper's compression ablation) and moving a
+store between buffers (export / import)."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mukv_oracle as O
+from paper_2605_22269_b200 import binding as B
+from paper_2605_22269_b200.synth.cpu import workload
+from tests import harness as H
+from tests.test_parity_gpu import full_compress_check, retrieval_check
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,n,keep", [("chunk7b", 5, 98), ("tiny", 8, 32), ("chunk7b", 3, 49)])
+def test_random_drop_fixture(name, n, keep):
+    # "Rand(50%)": uniform random scores from the seeded generator, half of the tokens kept
+    run = H.GpuRun(name, n_frames=n, keep_per_frame=keep)
+    c = run.cfg
+    P = c.tokens_per_frame
+    r = run.spec.select_scores(n)                               # [n][P] float32, seeded
+    if name == "tiny":
+        r[1, 5] = r[1, 9]                                       # an exact tie and a near-tie inside the band
+        r[2, 7] = np.float32(r[2, 11] + 4e-7)
+    q, k, v = run.gs.chunk(0, n)
+    kept = torch.full((n, c.keep_per_frame), -1, dtype=torch.int32, device=run.device)
+    run.ctx.mukv_compress_chunk_scored(torch.from_numpy(r).to(run.device), k, v, n, 0, kept)
+    torch.cuda.synchronize()
+    st = O.Store(H.oracle_cfg(c))
+    O.compress_chunk(st, None, H.to_numpy_bits(k), H.to_numpy_bits(v), select_scores=r)
+    run.kept = kept.cpu().numpy()
+    run.scores = None
+    H.check_frames_against_oracle(run, st, range(n), full_layers=True)
+    seg = run.ctx.region(3).cpu().numpy()
+    for u in range(st.n_segments):
+        sk, sv = st.segment_entry(u)
+        H.close(seg[u][:, 0], sk, f"segment entry K {u}")
+    assert run.ctx.mukv_get_stats().device_status == 0 and run.ctx.mukv_get_stats().refined_frames == 0
+
+
+def test_export_import_continues_the_stream():
+    # 11 frames: 6 stored, store copied to a new buffer, imported, the other 5 appended there;
+    # the result must equal the oracle's uninterrupted stream, and retrieval must work on the copy
+    wl = dict(workload("chunk7b"))
+    wl["fseg"] = 4
+    a = H.GpuRun(wl, n_frames=11, max_frames=11)
+    c = a.cfg
+    q, k, v = a.gs.chunk(0, 6)
+    a.ctx.mukv_compress_chunk(q, k, v, 6, 0)
+    torch.cuda.synchronize()
+    hdr = a.ctx.mukv_export_header()
+    assert hdr.frames == 6 and hdr.store_bytes == a.store_bytes()
+    b_ctx = B.MukvContext.from_copy(hdr, a.ctx.store.clone())
+    a.ctx.close()
+    kept = torch.full((11, c.keep_per_frame), -1, dtype=torch.int32, device=a.device)
+    q2, k2, v2 = a.gs.chunk(6, 5)
+    b_ctx.mukv_compress_chunk(q2, k2, v2, 5, 6, kept[6:])
+    torch.cuda.synchronize()
+    run = a
+    run.ctx = b_ctx
+    st = H.oracle_stream(run.spec, H.oracle_cfg(c), range(11), last_only=False, workers=1)
+    kept[:6] = b_ctx.region(1)[:6]
+    run.kept = kept.cpu().numpy()
+    run.scores = None
+    H.check_frames_against_oracle(run, st, range(11), full_layers=True)
+    seg = b_ctx.region(3).cpu().numpy()
+    for u in range(st.n_segments):
+        sk, sv = st.segment_entry(u)
+        H.close(seg[u][:, 0], sk, f"segment entry K {u}")
+        H.close(seg[u][:, 1], sv, f"segment entry V {u}")
+        assert b_ctx.region(5)[u].cpu().numpy().tobytes() == st.segment_key(u).tobytes()
+    qtok, offs, _ = run.spec.questions(3, 4, 9)
+    retrieval_check(run, st, qtok, offs, 2, 3, 0.3, B.RETR_SEMI)
+    # a header that does not belong to the buffer is refused on the host
+    bad = B.MukvStoreHeader.from_buffer_copy(hdr)
+    bad.magic = 1
+    with pytest.raises(B.MukvError):
+        B.MukvContext.from_copy(bad, b_ctx.store)
