@@ -74,6 +74,7 @@ typedef enum { MUKV_RETR_PARALLEL = 0, MUKV_RETR_HIER = 1, MUKV_RETR_SEMI = 2 } 
 #define MUKV_MAX_QUESTIONS 128   /* questions per mukv_retrieve / mukv_gather call */
 #define MUKV_MAX_TOPK 256        /* upper bound for k_seg, k_frm (2*k candidates <= 512) */
 #define MUKV_MAX_TOKENS 256      /* upper bound for P (tokens per frame) */
+#define MUKV_MAX_PATCH_SPLIT 4   /* upper bound for patch_split (16 super patches per frame) */
 
 typedef struct {
   int32_t n_layers;              /* L                                                   */
@@ -89,7 +90,12 @@ typedef struct {
   float   alpha;                 /* Eq. 4 weight of the attention signal                */
   float   tie_eps;               /* scores within tie_eps of the k-th count as tied     */
   int32_t dtype;                 /* mukv_dtype of Q, K, V and of the stored pages       */
-  int32_t reserved;              /* set to 0                                            */
+  int32_t patch_split;           /* s: patch-level blocks = the kept tokens inside each of
+                                    the s x s super patches of a frame (Sec. 3.2); 0 = no
+                                    patch level; at most 4                               */
+  int32_t grid_width;            /* tokens per row of the frame's token grid (only read
+                                    when patch_split > 0; must divide P)                 */
+  int32_t reserved[3];           /* set to 0                                            */
   int64_t max_frames;            /* capacity of the store, in frames                    */
 } mukv_config;
 
@@ -191,6 +197,47 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
                           float* d_seg_score, float* d_frm_score, int32_t* d_counts,
                           mukv_stream stream);
 
+/* Sec. 3.4 over all three granularities (patch-, frame- and segment-level blocks), each with its
+ * own k_g and lambda_g; the paper's values are k_g = {20, 32, 12}, lambda_g = {0.3, 0.3, 0}.
+ * Stage 1 ranks every visible block of a granularity by cosine (Eq. 7) and keeps 2 k_g candidates;
+ * stage 2 re-scores them against the mean of the top_n segment keys (Eq. 8) and keeps k_g
+ * (lambda_g = 0: the k_g best of stage 1).  PARALLEL stops after stage 1; HIER looks for frame- and
+ * patch-level blocks only inside the selected segments.  A patch-level block is (frame, super
+ * patch), id = frame * S + super patch with S = patch_split^2; super patches that kept no token are
+ * no blocks.  The store must have been created with patch_split > 0 when k_patch > 0.
+ *   d_patch_idx [nq][k_patch] / d_patch_score: like the frame outputs; may be NULL when k_patch = 0.
+ *   d_counts [nq][3]: valid (segments, frames, patch blocks).
+ * Other arguments and errors as mukv_retrieve. */
+typedef struct {
+  int32_t k_patch, k_frm, k_seg;
+  float lambda_patch, lambda_frm, lambda_seg;
+  int32_t top_n;                 /* segment keys averaged into the global query; 0 = k_seg */
+  int32_t mode;                  /* mukv_retr_mode */
+} mukv_retr_params;
+mukv_status mukv_retrieve3(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_offsets,
+                           const int64_t* h_t_limit, int32_t nq, const mukv_retr_params* params,
+                           int32_t* d_seg_idx, int32_t* d_frm_idx, int32_t* d_patch_idx,
+                           float* d_seg_score, float* d_frm_score, float* d_patch_score,
+                           int32_t* d_counts, mukv_stream stream);
+
+/* Sec. 3.4 (first paragraph) / Sec. 3.5: the decode context when the selected blocks of all three
+ * granularities are loaded.  For question i, per layer l, K then V:
+ *   d_decode + i*decode_stride_bytes : [L][2][tok_cap][Hkv][D] in the store dtype, with
+ *   tok_cap = mukv_decode3_tokens(ctx, k_seg, k_frm, k_patch).  Token slots, in this order: one
+ *   summary token per selected segment (the segment's pooled entry, Eq. 5, rounded to the store
+ *   dtype), the kept tokens of the selected frames, the kept tokens of the selected patch-level
+ *   blocks; every group ascending by block id.  Only the first d_ntok[i] slots are written.
+ *   d_seg_idx / d_frm_idx / d_patch_idx / d_counts: as written by mukv_retrieve3 (device).
+ *   d_ntok [nq] int32: valid token slots per question.   d_tok_meta [nq][tok_cap][2] int32 or NULL:
+ *   (frame id, token id) per slot, (-1 - segment id, -1) for a summary token.
+ * Errors: INVALID, ALIGN, CAPACITY (nq, k, stride too small), STATE (k_patch > 0 without patch level). */
+int64_t mukv_decode3_tokens(const mukv_ctx* ctx, int32_t k_seg, int32_t k_frm, int32_t k_patch);
+mukv_status mukv_gather3(mukv_ctx* ctx, const int32_t* d_seg_idx, const int32_t* d_frm_idx,
+                         const int32_t* d_patch_idx, const int32_t* d_counts, int32_t nq,
+                         int32_t k_seg, int32_t k_frm, int32_t k_patch, void* d_decode,
+                         int64_t decode_stride_bytes, int32_t* d_ntok, int32_t* d_tok_meta,
+                         mukv_stream stream);
+
 /* Sec. 3.5.  For question i and layer l the kept K rows of the selected frames (ascending
  * frame id, ascending token id inside a frame) are concatenated, then the V rows:
  *   d_decode + i*decode_stride_bytes : [L][2 (K,V)][k_frm*kappa][Hkv][D] in the store dtype.
@@ -211,6 +258,8 @@ mukv_status mukv_gather(mukv_ctx* ctx, const int32_t* d_frm_idx, const int32_t* 
  *        5 segment keys (float)    [max_segments][C]
  *        6 frame timestamps (int64)[max_frames]
  *        7 page table (int64 byte offsets from the store base) [max_frames]
+ *        8 patch-level keys (float) [max_frames][S][C]     (patch_split > 0)
+ *        9 patch-level token counts (int32) [max_frames][S]
  * Returns NULL for an unknown region; *bytes (if not NULL) receives the region size. */
 void* mukv_store_region(const mukv_ctx* ctx, int32_t which, size_t* bytes);
 

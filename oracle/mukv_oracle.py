@@ -173,6 +173,17 @@ def score_frame(Q, K_last, alpha, causal=False, keep_low_freq=False):
     return ia, ifr, fuse(ia, ifr, alpha, keep_low_freq)
 
 
+def super_patch_of(token_ids, P: int, grid_width: int, split: int) -> np.ndarray:
+    """Super patch (0 .. split*split-1, row-major) of each token id of a frame whose P tokens are a
+    grid of grid_width columns, cut into split x split rectangles of ceil(rows/split) x
+    ceil(grid_width/split) tokens."""
+    ids = np.asarray(token_ids, dtype=np.int64)
+    rows = P // grid_width
+    rh = -(-rows // split)
+    cw = -(-grid_width // split)
+    return (ids // grid_width) // rh * split + (ids % grid_width) // cw
+
+
 def compact_rows(X, kept):
     """X[L][P][Hkv][D] -> X[L][kappa][Hkv][D] in ascending token order (bytes untouched)."""
     return np.ascontiguousarray(np.asarray(X)[:, kept, :, :])
@@ -215,6 +226,39 @@ class Store:
     def frame_key(self, t: int) -> np.ndarray:
         """Retrieval key of frame t: mean of the last-layer kept keys, heads concatenated."""
         return self.frame_entry(t)[0][-1]
+
+    # Sec. 3.2 / Eq. 5 "similarly k_{p_ft}": patch-level blocks.  The frame's P tokens form a grid of
+    # grid_width columns; the grid is cut into patch_split x patch_split super patches, and the kept
+    # tokens of a frame that fall into one super patch are one patch-level block.  Its key is the
+    # mean of their last-layer keys (heads concatenated); a super patch that kept no token has no block.
+    def n_patches(self) -> int:
+        return int(self.cfg.get("patch_split", 0)) ** 2
+
+    def patch_tokens(self, t: int, sp: int) -> np.ndarray:
+        """Positions (in the frame's kept list) of the kept tokens inside super patch sp."""
+        ids = self.kept[t]
+        return np.nonzero(super_patch_of(ids, self.cfg["tokens_per_frame"], self.cfg["grid_width"],
+                                         self.cfg["patch_split"]) == sp)[0]
+
+    def patch_count(self, t: int, sp: int) -> int:
+        return int(self.patch_tokens(t, sp).shape[0])
+
+    def patch_key(self, t: int, sp: int) -> np.ndarray:
+        pos = self.patch_tokens(t, sp)
+        C = self.sum_k[t].shape[1]
+        if pos.shape[0] == 0:
+            return np.zeros(C, dtype=np.float32)
+        rows = as_f64(self.page_k[t][-1][pos]).reshape(pos.shape[0], C)
+        return (rows.sum(axis=0) / float(pos.shape[0])).astype(np.float32)
+
+    def patch_keys(self, n_frm: int) -> np.ndarray:
+        S = self.n_patches()
+        C = self.sum_k[0].shape[1]
+        out = np.zeros((n_frm * S, C), dtype=np.float32)
+        for t in range(n_frm):
+            for sp in range(S):
+                out[t * S + sp] = self.patch_key(t, sp)
+        return out
 
     def segment_frames(self, u: int):
         fs = self.cfg["frames_per_segment"]
@@ -347,6 +391,80 @@ def retrieve(store: Store, Qq, k_seg: int, k_frm: int, top_n: int = 0, lam: floa
     }
 
 
+def _rerank(s_stage1, keys, cand, g, lam, k, delta):
+    """Eq. 8 on one granularity's candidates: returns (positions in cand, their calibrated scores)."""
+    gamma = cosine(g, keys[cand]) if g is not None else np.zeros(cand.shape[0])
+    s_new = (1.0 - lam) * s_stage1[cand] + lam * gamma
+    pick = topk_set(s_new, min(k, cand.shape[0]), delta)
+    return pick, s_new[pick]
+
+
+def retrieve3(store: Store, Qq, k_g, lambda_g, top_n: int = 0, mode: int = MODE_SEMI, t_limit=None,
+              delta: float = TIE_EPS):
+    """Sec. 3.4 over all three granularities.  k_g = (k_patch, k_frm, k_seg) and lambda_g =
+    (lambda_patch, lambda_frm, lambda_seg) in the paper's order (patch-, frame-, segment-level); the
+    paper's values are k_g = {20, 32, 12}, lambda_g = {0.3, 0.3, 0}.
+
+    Stage 1: cosine of the pooled question with every visible block key of each granularity (Eq. 7),
+    top-2k_g candidates per granularity.  Stage 2: the global query is the mean of the top-N
+    segment-level keys; every candidate of a granularity with lambda_g > 0 gets Eq. 8 and the best
+    k_g are kept (lambda_g = 0: the best k_g by cosine).  PARALLEL keeps the best k_g by cosine at every
+    granularity; HIER looks for frame- and patch-level blocks only inside the selected segments.
+    Patch-level block ids are frame * S + super patch; a super patch that kept no token is no block.
+    """
+    cfg = store.cfg
+    T = store.n_frames
+    t_limit = T if t_limit is None else min(int(t_limit), T)
+    fs = cfg["frames_per_segment"]
+    S = store.n_patches()
+    k_pat, k_frm, k_seg = (int(x) for x in k_g)
+    lam_pat, lam_frm, lam_seg = (float(x) for x in lambda_g)
+    n_frm = max(t_limit, 0)
+    n_seg = sum(1 for u in range(store.n_segments) if min((u + 1) * fs, T) <= t_limit)
+    q = pool_question(Qq, cfg["n_kv_heads"])
+    C = q.shape[0]
+    key_f = store.frame_keys()[:n_frm].astype(np.float64) if n_frm else np.zeros((0, C))
+    key_s = store.segment_keys()[:n_seg].astype(np.float64) if n_seg else np.zeros((0, C))
+    key_p = store.patch_keys(n_frm).astype(np.float64) if n_frm and S else np.zeros((0, C))
+    s_frm, s_seg, s_pat = cosine(q, key_f), cosine(q, key_s), cosine(q, key_p)
+    exists = np.array([store.patch_count(b // S, b % S) > 0 for b in range(n_frm * S)], dtype=bool) \
+        if S else np.zeros(0, dtype=bool)
+
+    # segment level; its own lambda is applied too (the paper sets it to 0: the global query comes from them)
+    N = k_seg if top_n <= 0 else top_n
+    top = topk_set(s_seg, min(N, n_seg), delta)
+    g = key_s[top].sum(axis=0) / float(top.shape[0]) if top.shape[0] > 0 else None
+    if mode == MODE_SEMI and lam_seg > 0.0:
+        cand = topk_set(s_seg, min(2 * k_seg, n_seg), delta)
+        pick, sc = _rerank(s_seg, key_s, cand, g, lam_seg, k_seg, delta)
+        sel_seg, seg_sc = cand[pick], sc
+    else:
+        sel_seg = topk_set(s_seg, min(k_seg, n_seg), delta)
+        seg_sc = s_seg[sel_seg]
+
+    def lower(s1, keys, member, k, lam):
+        ids = np.nonzero(member)[0]
+        if mode == MODE_HIER:
+            inside = set(sel_seg.tolist())
+            ids = np.array([b for b in ids if (owner(b) // fs) in inside], dtype=np.int64)
+        if mode == MODE_SEMI:
+            cand = ids[topk_set(s1[ids], min(2 * k, ids.shape[0]), delta)]
+            pick, sc = _rerank(s1, keys, cand, g, lam, k, delta)
+            return cand[pick], sc
+        pick = topk_set(s1[ids], min(k, ids.shape[0]), delta)
+        return ids[pick], s1[ids[pick]]
+
+    owner = lambda b: b
+    sel_frm, frm_sc = lower(s_frm, key_f, np.ones(n_frm, dtype=bool), k_frm, lam_frm)
+    owner = lambda b: b // S
+    if S:
+        sel_pat, pat_sc = lower(s_pat, key_p, exists, k_pat, lam_pat)
+    else:
+        sel_pat, pat_sc = np.zeros(0, dtype=np.int64), np.zeros(0)
+    return {"q": q, "seg_idx": sel_seg, "seg_score": seg_sc, "frm_idx": sel_frm, "frm_score": frm_sc,
+            "patch_idx": sel_pat, "patch_score": pat_sc}
+
+
 # --------------------------------------------------------------------------
 # Sec. 3.5, Eq. 9: the retrieved context R_k, R_v
 # --------------------------------------------------------------------------
@@ -361,3 +479,46 @@ def gather(store: Store, frm_idx):
     dec = np.stack([Rk, Rv], axis=1)                                     # [L][2][n*kappa][Hkv][D]
     meta = np.array([(t, int(j)) for t in frm_idx for j in store.kept[t]], dtype=np.int32)
     return dec, meta
+
+
+def round_to_dtype(x: np.ndarray, like: np.ndarray) -> np.ndarray:
+    """float32 values in the storage type of `like`: bfloat16 bit patterns (round to nearest even)
+    or float32."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    if like.dtype == np.uint16:
+        b = x.view(np.uint32)
+        return ((b + np.uint32(0x7FFF) + ((b >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)).astype(np.uint16)
+    return x
+
+
+def gather3(store: Store, seg_idx, frm_idx, patch_idx):
+    """The decode context when the selected blocks of all three granularities are loaded
+    (Sec. 3.4, first paragraph; Sec. 3.5).  Per layer, K then V, token slots in this order:
+    one summary token per selected segment (its pooled entry, Eq. 5, rounded to the cache's storage
+    type), the kept tokens of the selected frames, the kept tokens of the selected patch-level
+    blocks; every group ascending by block id, tokens ascending inside a block.
+    Returns (decode [L][2][n_tok][Hkv][D], meta [n_tok][2]): meta is (frame, token id), and
+    (-1 - segment, -1) for a summary token."""
+    S = store.n_patches()
+    L = store.page_k[0].shape[0]
+    Hkv, D = store.page_k[0].shape[2], store.page_k[0].shape[3]
+    ks, vs, meta = [], [], []
+    for u in [int(u) for u in seg_idx]:
+        ek, ev = store.segment_entry(u)
+        ks.append(round_to_dtype(ek, store.page_k[0]).reshape(L, 1, Hkv, D))
+        vs.append(round_to_dtype(ev, store.page_v[0]).reshape(L, 1, Hkv, D))
+        meta.append((-1 - u, -1))
+    for t in [int(t) for t in frm_idx]:
+        ks.append(store.page_k[t])
+        vs.append(store.page_v[t])
+        meta += [(t, int(j)) for j in store.kept[t]]
+    for b in [int(b) for b in patch_idx]:
+        t, sp = b // S, b % S
+        pos = store.patch_tokens(t, sp)
+        ks.append(store.page_k[t][:, pos])
+        vs.append(store.page_v[t][:, pos])
+        meta += [(t, int(store.kept[t][r])) for r in pos]
+    if not ks:
+        return None, np.zeros((0, 2), dtype=np.int32)
+    dec = np.stack([np.concatenate(ks, axis=1), np.concatenate(vs, axis=1)], axis=1)
+    return dec, np.array(meta, dtype=np.int32).reshape(-1, 2)

@@ -25,7 +25,8 @@ STATUS_NAMES = {0: "MUKV_OK", -1: "MUKV_E_INVALID", -2: "MUKV_E_SHAPE", -3: "MUK
                 -5: "MUKV_E_CAPACITY", -6: "MUKV_E_STATE", -7: "MUKV_E_CUDA", -8: "MUKV_E_UNSUPPORTED"}
 
 EXPORTS = ["mukv_store_bytes", "mukv_workspace_bytes", "mukv_create", "mukv_destroy", "mukv_reset", "mukv_set_option",
-           "mukv_compress_chunk", "mukv_compress_chunk_scored", "mukv_export_header", "mukv_import", "mukv_retrieve", "mukv_gather", "mukv_store_region", "mukv_get_stats",
+           "mukv_compress_chunk", "mukv_compress_chunk_scored", "mukv_export_header", "mukv_import",
+           "mukv_retrieve3", "mukv_gather3", "mukv_decode3_tokens", "mukv_retrieve", "mukv_gather", "mukv_store_region", "mukv_get_stats",
            "mukv_last_error", "mukv_profile_enable", "mukv_profile_read", "mukv_score_frames_noalloc"]
 PROF_KINDS = ["score", "refine", "compact", "segment", "qpool", "scan", "rank", "gather"]
 
@@ -42,7 +43,14 @@ class MukvConfig(C.Structure):
                 ("frames_per_segment", C.c_int32), ("max_frames_per_chunk", C.c_int32),
                 ("attn_causal", C.c_int32), ("keep_low_freq", C.c_int32),
                 ("alpha", C.c_float), ("tie_eps", C.c_float),
-                ("dtype", C.c_int32), ("reserved", C.c_int32), ("max_frames", C.c_int64)]
+                ("dtype", C.c_int32), ("patch_split", C.c_int32), ("grid_width", C.c_int32),
+                ("reserved", C.c_int32 * 3), ("max_frames", C.c_int64)]
+
+
+class MukvRetrParams(C.Structure):
+    _fields_ = [("k_patch", C.c_int32), ("k_frm", C.c_int32), ("k_seg", C.c_int32),
+                ("lambda_patch", C.c_float), ("lambda_frm", C.c_float), ("lambda_seg", C.c_float),
+                ("top_n", C.c_int32), ("mode", C.c_int32)]
 
 
 class MukvStats(C.Structure):
@@ -94,6 +102,13 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.mukv_retrieve.restype = i32
     lib.mukv_retrieve.argtypes = [vp, vp, C.POINTER(i32), C.POINTER(i64), i32, i32, i32, i32, f32, i32,
                                   vp, vp, vp, vp, vp, vp]
+    lib.mukv_retrieve3.restype = i32
+    lib.mukv_retrieve3.argtypes = [vp, vp, C.POINTER(i32), C.POINTER(i64), i32, C.POINTER(MukvRetrParams),
+                                   vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.mukv_decode3_tokens.restype = i64
+    lib.mukv_decode3_tokens.argtypes = [vp, i32, i32, i32]
+    lib.mukv_gather3.restype = i32
+    lib.mukv_gather3.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp, i64, vp, vp, vp]
     lib.mukv_gather.restype = i32
     lib.mukv_gather.argtypes = [vp, vp, vp, i32, i32, vp, i64, vp, vp]
     lib.mukv_store_region.restype = vp
@@ -124,10 +139,10 @@ def _stream(stream) -> int:
 
 def make_config(*, n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, keep_per_frame,
                 frames_per_segment, max_frames_per_chunk, max_frames, dtype=BF16, alpha=0.7, tie_eps=1e-6,
-                attn_causal=0, keep_low_freq=0) -> MukvConfig:
+                attn_causal=0, keep_low_freq=0, patch_split=0, grid_width=0) -> MukvConfig:
     return MukvConfig(n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, keep_per_frame,
                       frames_per_segment, max_frames_per_chunk, attn_causal, keep_low_freq,
-                      alpha, tie_eps, dtype, 0, max_frames)
+                      alpha, tie_eps, dtype, patch_split, grid_width, (C.c_int32 * 3)(0, 0, 0), max_frames)
 
 
 def mukv_score_frames_noalloc(cfg: MukvConfig, q, k_last, n_frames: int, kept_out=None, scores_out=None,
@@ -223,6 +238,26 @@ class MukvContext:
             nq, k_seg, k_frm, top_n, lambda_frm, mode, _ptr(seg_idx), _ptr(frm_idx), _ptr(seg_score),
             _ptr(frm_score), _ptr(counts), _stream(stream)))
 
+    def mukv_retrieve3(self, qtok, q_offsets, t_limit, params: MukvRetrParams, seg_idx, frm_idx, patch_idx,
+                       seg_score, frm_score, patch_score, counts, stream=None):
+        offs = np.ascontiguousarray(q_offsets, dtype=np.int32)
+        nq = offs.shape[0] - 1
+        tl = None if t_limit is None else np.ascontiguousarray(t_limit, dtype=np.int64)
+        self._check(self.lib.mukv_retrieve3(
+            self.handle, _ptr(qtok), offs.ctypes.data_as(C.POINTER(C.c_int32)),
+            None if tl is None else tl.ctypes.data_as(C.POINTER(C.c_int64)), nq, C.byref(params),
+            _ptr(seg_idx), _ptr(frm_idx), _ptr(patch_idx), _ptr(seg_score), _ptr(frm_score), _ptr(patch_score),
+            _ptr(counts), _stream(stream)))
+
+    def mukv_decode3_tokens(self, k_seg: int, k_frm: int, k_patch: int) -> int:
+        return int(self.lib.mukv_decode3_tokens(self.handle, k_seg, k_frm, k_patch))
+
+    def mukv_gather3(self, seg_idx, frm_idx, patch_idx, counts, nq: int, k_seg: int, k_frm: int, k_patch: int, decode,
+                     decode_stride_bytes: int, ntok, tok_meta=None, stream=None):
+        self._check(self.lib.mukv_gather3(self.handle, _ptr(seg_idx), _ptr(frm_idx), _ptr(patch_idx), _ptr(counts), nq,
+                                          k_seg, k_frm, k_patch, _ptr(decode), decode_stride_bytes, _ptr(ntok),
+                                          _ptr(tok_meta), _stream(stream)))
+
     def mukv_gather(self, frm_idx, counts, nq: int, k_frm: int, decode, decode_stride_bytes: int, tok_meta=None,
                     stream=None):
         self._check(self.lib.mukv_gather(self.handle, _ptr(frm_idx), _ptr(counts), nq, k_frm, _ptr(decode),
@@ -267,6 +302,10 @@ class MukvContext:
             return raw.view(torch.float32).view(T, self.C)
         if which == 5:
             return raw.view(torch.float32).view(segs, self.C)
+        if which == 8:
+            return raw.view(torch.float32).view(T, c.patch_split ** 2, self.C)
+        if which == 9:
+            return raw.view(torch.int32).view(T, c.patch_split ** 2)
         return raw.view(torch.int64).view(T)
 
     def decode_stride_bytes(self, k_frm: int) -> int:

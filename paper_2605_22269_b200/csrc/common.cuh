@@ -127,6 +127,14 @@ __device__ __forceinline__ int block_excl_count(bool flag, int* scratch, int& to
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// super patch (row-major, split x split) of token id j in a frame of P tokens laid out as a grid
+// with grid_width tokens per row: rectangles of ceil(rows/split) x ceil(grid_width/split) tokens
+__device__ __forceinline__ int super_patch_index(int j, int P, int grid_width, int split) {
+  const int rows = P / grid_width;
+  const int rh = (rows + split - 1) / split, cw = (grid_width + split - 1) / split;
+  return (j / grid_width) / rh * split + (j % grid_width) / cw;
+}
+
 // 16-byte streaming copies
 __device__ __forceinline__ uint4 ld_stream(const void* p) {
   uint4 v;

@@ -53,6 +53,10 @@ struct CompactParams {
   float* seg_entry;               // [max_segs][L][2][C]
   float* seg_key;                 // [max_segs][C]
   // selection
+  // patch-level blocks (Sec. 3.2; Eq. 5 "similarly"): S = patch_split^2 super patches per frame
+  int patch_split, grid_width;    // 0: no patch level
+  float* patch_key;               // [max_frames][S][C]
+  int* patch_cnt;                 // [max_frames][S]
   int sel_mode;                   // 0: kept ids are in the store; 1: select here from the partial sums;
                                   // 2: select here by the caller's scores
   const float* ext_scores;        // [n_frames][P] (sel_mode 2)
@@ -415,6 +419,32 @@ __device__ inline void compact_plane(const CompactParams& p, int plane, int f, C
   }
 }
 
+// Patch-level block keys of chunk frame f (Eq. 5 on the kept tokens of each super patch): mean of
+// their last-layer keys, summed in double like the frame key; kept ids in sc->kept.  Run by a
+// whole block; thread t owns columns t, t + 256, ...  sc->red is used as scratch.
+template <typename T>
+__device__ inline void pool_patches(const CompactParams& p, int f, CompactScratch* sc) {
+  const int tid = threadIdx.x;
+  const int S = p.patch_split * p.patch_split, C = p.C, kappa = p.kappa;
+  const long long f_abs = p.first_frame + f;
+  int* sp_of = reinterpret_cast<int*>(sc->red);          // super patch of each kept row
+  __syncthreads();
+  for (int r = tid; r < kappa; r += kCompactThreads) sp_of[r] = super_patch_index(sc->kept[r], p.P, p.grid_width, p.patch_split);
+  __syncthreads();
+  const T* src = reinterpret_cast<const T*>(p.k) + ((long long)(p.L - 1) * p.n_frames + f) * p.P * C;
+  for (int sp = 0; sp < S; ++sp) {
+    int cnt = 0;
+    for (int r = 0; r < kappa; ++r) cnt += (sp_of[r] == sp);
+    for (int col = tid; col < C; col += kCompactThreads) {
+      double t = 0.0;
+      for (int r = 0; r < kappa; ++r)
+        if (sp_of[r] == sp) t += (double)elem_to_float<T>(src[(long long)sc->kept[r] * C + col]);
+      p.patch_key[((f_abs * S) + sp) * C + col] = cnt ? (float)(t / (double)cnt) : 0.f;
+    }
+    if (tid == 0) p.patch_cnt[f_abs * S + sp] = cnt;
+  }
+}
+
 // is chunk frame f on the flagged list (of n entries)?
 __device__ __forceinline__ bool frame_is_flagged(const int* flagged, int n, int f) {
   bool hit = false;
@@ -478,7 +508,9 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(const Compa
     for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(p.sp.kept_store[f_abs * p.kappa + r], p.P);
     __syncthreads();
   }
-  if (!risky) compact_plane<T>(p, plane, f, &cs);
+  if (risky) return;
+  if (plane < 2 * p.L) compact_plane<T>(p, plane, f, &cs);
+  else pool_patches<T>(p, f, &cs);                // the extra row of blocks when there is a patch level
 }
 
 // Bounded wait until *ctr reaches `target` (other blocks of the same grid add to it; the grid is
@@ -537,15 +569,18 @@ __global__ void __launch_bounds__(kScoreThreads, 2) tail_kernel(const ScoreParam
     if (tid == 0 && sp.status) atomicCAS(sp.status, 0, kStatusTailWait);
   } else {
     // ---- the flagged frames' compaction, then the segment entries, plane by plane
-    for (int plane = blockIdx.x; plane < 2 * p.L; plane += gridDim.x) {
+    const int n_planes = 2 * p.L + (p.patch_split > 0 ? 1 : 0);
+    for (int plane = blockIdx.x; plane < n_planes; plane += gridDim.x) {
       for (int i = 0; i < n_fl; ++i) {
         const int f = sp.flagged[i];
         const long long f_abs = p.first_frame + f;
         __syncthreads();
         for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(__ldcg(sp.kept_store + f_abs * p.kappa + r), p.P);
         __syncthreads();
-        compact_plane<T>(p, plane, f, &cs);
+        if (plane < 2 * p.L) compact_plane<T>(p, plane, f, &cs);
+        else pool_patches<T>(p, f, &cs);
       }
+      if (plane >= 2 * p.L) continue;
       __threadfence();                          // the frame entries just written are read below by other threads
       __syncthreads();
       compact_segment_plane(segment_args(p), plane >> 1, plane & 1);

@@ -30,7 +30,8 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct StoreLayout {
-  size_t pages, kept, frame_entry, seg_entry, frame_key, seg_key, frame_ts, page_table, frame_ksum, total;
+  size_t pages, kept, frame_entry, seg_entry, frame_key, seg_key, frame_ts, page_table, frame_ksum, patch_key, patch_cnt,
+      total;
   size_t page_bytes;
   long long max_segs;
 };
@@ -38,7 +39,7 @@ struct StoreLayout {
 struct WorkLayout {
   size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, tail_ctr, sel_flag,
       stat_refined, dev_status;
-  size_t q64, qnorm, s_frm, s_seg, wtab, total;
+  size_t q64, qnorm, s_frm, s_seg, s_pat, wtab, total;
   size_t zero_begin, zero_end;          // region that must start as zeros
 };
 
@@ -137,6 +138,10 @@ const char* check_config(const mukv_config* c) {
   if (c->max_frames < 1) return "max_frames must be positive";
   if (!(c->alpha >= 0.f && c->alpha <= 1.f)) return "alpha must lie in [0, 1]";
   if (!(c->tie_eps >= 0.f)) return "tie_eps must be >= 0";
+  if (c->patch_split < 0 || c->patch_split > MUKV_MAX_PATCH_SPLIT) return "patch_split out of range";
+  if (c->patch_split > 0 && (c->grid_width < 1 || c->tokens_per_frame % c->grid_width != 0))
+    return "grid_width must divide tokens_per_frame when patch_split > 0";
+  if (c->reserved[0] != 0 || c->reserved[1] != 0 || c->reserved[2] != 0) return "reserved fields must be 0";
   const long long esize = c->dtype == MUKV_BF16 ? 2 : 4;
   const long long row_vec = (long long)c->n_kv_heads * c->head_dim * esize / 16;
   if (!is_pow2(row_vec) || row_vec > 256) return "Hkv*D*sizeof(element)/16 must be a power of two <= 256";
@@ -165,6 +170,9 @@ StoreLayout store_layout(const mukv_config& c) {
   s.frame_ts = off;     off = align_up(off + T * sizeof(long long));
   s.page_table = off;   off = align_up(off + T * sizeof(long long));
   s.frame_ksum = off;   off = align_up(off + T * C * sizeof(double));
+  const size_t S = (size_t)c.patch_split * c.patch_split;
+  s.patch_key = off;    off = align_up(off + T * S * C * sizeof(float));
+  s.patch_cnt = off;    off = align_up(off + T * S * sizeof(int));
   s.total = off;
   return s;
 }
@@ -217,6 +225,8 @@ WorkLayout work_layout(const mukv_config& c) {
   w.qnorm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * c.n_kv_heads * sizeof(double));
   w.s_frm = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * c.max_frames * sizeof(double));
   w.s_seg = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * max_segs * sizeof(double));
+  w.s_pat = off;          off = align_up(off + (size_t)MUKV_MAX_QUESTIONS * c.max_frames * c.patch_split * c.patch_split *
+                                               sizeof(double));
   w.wtab = off;           off = align_up(off + (ts.ok ? (size_t)3 * c.head_dim * c.head_dim * 2 : 0));
   w.total = off;
   return w;
@@ -498,6 +508,9 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   cp.fseg = c.frames_per_segment;
   cp.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
   cp.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
+  cp.patch_split = c.patch_split; cp.grid_width = c.grid_width;
+  cp.patch_key = reinterpret_cast<float*>(ctx->store + ctx->sl.patch_key);
+  cp.patch_cnt = reinterpret_cast<int*>(ctx->store + ctx->sl.patch_cnt);
   cp.sel_mode = d_ext ? 2 : ps_grid > 0 ? 1 : 0;
   cp.ext_scores = d_ext;
   cp.ps_grid = ps_grid; cp.ps_items = ps_items; cp.ps_ipf = ps_ipf;
@@ -505,7 +518,8 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   if (ps_grid > 0) cp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
   {
     ProfScope ps(ctx, 2, st);
-    e = launch_k(compact_kernel<T>, dim3(n, L * 2), kCompactThreads, 0, st, !ctx->prof_on, cp);
+    e = launch_k(compact_kernel<T>, dim3(n, L * 2 + (c.patch_split > 0 ? 1 : 0)), kCompactThreads, 0, st, !ctx->prof_on,
+                 cp);
   }
   if (e != cudaSuccess) return broke_off(ctx, "compact kernel", e);
 
@@ -518,7 +532,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   {
     ProfScope ps(ctx, 1, st);
     int grid_t = c.n_q_heads * kRefineSplit * (n < 2 ? n : 2);
-    if (grid_t < 2 * L) grid_t = 2 * L;
+    if (grid_t < 2 * L + 1) grid_t = 2 * L + 1;
     if (grid_t > ctx->tail_capacity) grid_t = ctx->tail_capacity;
     e = launch_tail<T>(sp, cp, ctx->nc, grid_t, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
   }
@@ -532,6 +546,113 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
 
 mukv_status create_impl(const mukv_config* cfg, void* d_store, size_t store_bytes, void* d_workspace,
                         size_t workspace_bytes, long long frames0, mukv_ctx** out);
+
+mukv_status retrieve_impl(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_offsets, const int64_t* h_t_limit,
+                          int32_t nq, const mukv_retr_params& prm, int32_t* d_seg_idx, int32_t* d_frm_idx,
+                          int32_t* d_pat_idx, float* d_seg_score, float* d_frm_score, float* d_pat_score,
+                          int32_t* d_counts, int counts_stride, mukv_stream stream) {
+  try {
+    const int k_seg = prm.k_seg, k_frm = prm.k_frm, k_pat = prm.k_patch, top_n = prm.top_n, mode = prm.mode;
+    if (ctx->failed) return fail(ctx, MUKV_E_STATE, "an earlier call broke off half way: call mukv_reset");
+    if (!d_qtok || !h_q_offsets || !d_seg_idx || !d_frm_idx || !d_counts)
+      return fail(ctx, MUKV_E_INVALID, "null argument");
+    if (!aligned16(d_qtok) || !aligned4(d_seg_idx) || !aligned4(d_frm_idx) || !aligned4(d_seg_score) ||
+        !aligned4(d_frm_score) || !aligned4(d_counts))
+      return fail(ctx, MUKV_E_ALIGN, "d_qtok must be 16-byte aligned, the outputs 4-byte aligned");
+    if (nq < 1) return fail(ctx, MUKV_E_INVALID, "nq must be >= 1");
+    if (nq > MUKV_MAX_QUESTIONS) return fail(ctx, MUKV_E_CAPACITY, "nq %d exceeds %d", nq, MUKV_MAX_QUESTIONS);
+    if (k_seg < 1 || k_frm < 1 || k_pat < 0 || top_n < 0)
+      return fail(ctx, MUKV_E_INVALID, "k_seg, k_frm must be >= 1, k_patch and top_n >= 0");
+    if (k_seg > MUKV_MAX_TOPK || k_frm > MUKV_MAX_TOPK || k_pat > MUKV_MAX_TOPK || top_n > MUKV_MAX_TOPK)
+      return fail(ctx, MUKV_E_CAPACITY, "k_seg / k_frm / k_patch / top_n exceed %d", MUKV_MAX_TOPK);
+    if (k_pat > 0 && ctx->cfg.patch_split == 0) return fail(ctx, MUKV_E_STATE, "the store has no patch level");
+    if (k_pat > 0 && !d_pat_idx) return fail(ctx, MUKV_E_INVALID, "d_patch_idx is null");
+    if (!aligned4(d_pat_idx) || !aligned4(d_pat_score)) return fail(ctx, MUKV_E_ALIGN, "outputs must be 4-byte aligned");
+    if (mode != MUKV_RETR_PARALLEL && mode != MUKV_RETR_HIER && mode != MUKV_RETR_SEMI)
+      return fail(ctx, MUKV_E_INVALID, "unknown retrieval mode %d", mode);
+    for (float lam : {prm.lambda_patch, prm.lambda_frm, prm.lambda_seg})
+      if (!(lam >= 0.f && lam <= 1.f)) return fail(ctx, MUKV_E_INVALID, "every lambda must lie in [0, 1]");
+    if (ctx->frames < 1) return fail(ctx, MUKV_E_STATE, "the store is empty");
+    QMeta meta;
+    if (h_q_offsets[0] != 0) return fail(ctx, MUKV_E_INVALID, "q_offsets[0] must be 0");
+    for (int i = 0; i < nq; ++i) {
+      if (h_q_offsets[i + 1] <= h_q_offsets[i])
+        return fail(ctx, MUKV_E_INVALID, "question %d has no tokens (offsets must ascend)", i);
+      if (h_t_limit && h_t_limit[i] < 0) return fail(ctx, MUKV_E_INVALID, "t_limit[%d] is negative", i);
+    }
+    for (int i = 0; i <= nq; ++i) meta.off[i] = h_q_offsets[i];
+    for (int i = 0; i < nq; ++i) meta.t_limit[i] = h_t_limit ? (long long)h_t_limit[i] : ctx->frames;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const mukv_config& c = ctx->cfg;
+    const int C = ctx->C;
+    double* q64 = reinterpret_cast<double*>(ctx->ws + ctx->wl.q64);
+    double* qnorm = reinterpret_cast<double*>(ctx->ws + ctx->wl.qnorm);
+    double* s_frm = reinterpret_cast<double*>(ctx->ws + ctx->wl.s_frm);
+    double* s_seg = reinterpret_cast<double*>(ctx->ws + ctx->wl.s_seg);
+    const float* frame_key = reinterpret_cast<const float*>(ctx->store + ctx->sl.frame_key);
+    const float* seg_key = reinterpret_cast<const float*>(ctx->store + ctx->sl.seg_key);
+    const long long n_frm = ctx->frames;
+    const long long n_seg = (n_frm + c.frames_per_segment - 1) / c.frames_per_segment;
+    {
+      ProfScope ps(ctx, 4, st);
+      if (c.dtype == MUKV_BF16)
+        qpool_kernel<__nv_bfloat16><<<dim3(nq, c.n_kv_heads), kPoolThreads, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(d_qtok), meta,
+                                                       c.n_q_heads, c.n_kv_heads, c.head_dim, q64, qnorm);
+      else
+        qpool_kernel<float><<<dim3(nq, c.n_kv_heads), kPoolThreads, 0, st>>>(reinterpret_cast<const float*>(d_qtok), meta, c.n_q_heads,
+                                               c.n_kv_heads, c.head_dim, q64, qnorm);
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "qpool kernel: %s", cudaGetErrorString(e));
+    const int S = c.patch_split * c.patch_split;
+    const long long n_pat = k_pat > 0 ? n_frm * S : 0;
+    const long long rows = n_frm + n_seg + n_pat;
+    const unsigned blocks = (unsigned)((rows + kScanRows - 1) / kScanRows);
+    double* s_pat = reinterpret_cast<double*>(ctx->ws + ctx->wl.s_pat);
+    const float* patch_key = reinterpret_cast<const float*>(ctx->store + ctx->sl.patch_key);
+    {
+      ProfScope ps(ctx, 5, st);
+      ScanParams sc;
+      memset(&sc, 0, sizeof sc);
+      sc.frame_key = frame_key; sc.seg_key = seg_key; sc.patch_key = patch_key;
+      sc.n_frm = n_frm; sc.n_seg = n_seg; sc.n_pat = n_pat;
+      sc.C = C; sc.nq = nq; sc.Hkv = c.n_kv_heads; sc.q64t = q64; sc.qn2 = qnorm;
+      sc.s_frm = s_frm; sc.s_seg = s_seg; sc.s_pat = s_pat;
+      sc.frm_stride = c.max_frames; sc.seg_stride = ctx->sl.max_segs; sc.pat_stride = (long long)c.max_frames * S;
+      e = launch_k(scan_kernel, dim3(blocks), 256, 0, st, !ctx->prof_on, sc);
+    }
+    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "scan kernel: %s", cudaGetErrorString(e));
+    RankParams rp;
+    memset(&rp, 0, sizeof rp);
+    rp.nq = nq; rp.C = C; rp.fseg = c.frames_per_segment;
+    rp.k_seg = k_seg; rp.k_frm = k_frm; rp.k_pat = k_pat; rp.top_n = top_n; rp.mode = mode; rp.S = S;
+    rp.lam_seg = (double)prm.lambda_seg; rp.lam_frm = (double)prm.lambda_frm; rp.lam_pat = (double)prm.lambda_patch;
+    rp.delta = (double)c.tie_eps;
+    rp.n_frm = n_frm; rp.n_seg = n_seg;
+    rp.s_frm = s_frm; rp.s_seg = s_seg; rp.s_pat = s_pat;
+    rp.frm_stride = c.max_frames; rp.seg_stride = ctx->sl.max_segs; rp.pat_stride = (long long)c.max_frames * S;
+    rp.frame_key = frame_key; rp.seg_key = seg_key; rp.patch_key = patch_key;
+    rp.patch_cnt = reinterpret_cast<const int*>(ctx->store + ctx->sl.patch_cnt);
+    rp.seg_idx = d_seg_idx; rp.frm_idx = d_frm_idx; rp.pat_idx = d_pat_idx;
+    rp.seg_score = d_seg_score; rp.frm_score = d_frm_score; rp.pat_score = d_pat_score;
+    rp.counts = d_counts; rp.counts_stride = counts_stride;
+    {
+      ProfScope ps(ctx, 6, st);
+      size_t rank_smem = (size_t)C * sizeof(double);
+      const size_t staged = rank_smem + (size_t)(n_frm + n_seg) * sizeof(double);
+      rp.stage = staged <= (size_t)kRankStageBytes ? 1 : 0;
+      if (rp.stage) rank_smem = staged;
+      e = launch_k(rank_kernel, dim3(nq), kRankThreads, rank_smem, st, !ctx->prof_on, rp, meta);
+    }
+    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "rank kernel: %s", cudaGetErrorString(e));
+    ctx->launches += 4;
+    return MUKV_OK;
+  } catch (...) {
+    return fail(ctx, MUKV_E_INVALID, "unexpected exception");
+  }
+}
+
+
 
 mukv_status check_chunk_args(mukv_ctx* ctx, int n_frames, long long first_frame) {
   if (n_frames < 1) return fail(ctx, MUKV_E_INVALID, "n_frames must be >= 1");
@@ -760,82 +881,84 @@ mukv_status mukv_retrieve(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
                           int32_t* d_seg_idx, int32_t* d_frm_idx, float* d_seg_score, float* d_frm_score,
                           int32_t* d_counts, mukv_stream stream) {
   if (!ctx) return MUKV_E_INVALID;
+  mukv_retr_params rp;
+  memset(&rp, 0, sizeof rp);
+  rp.k_seg = k_seg; rp.k_frm = k_frm; rp.k_patch = 0;
+  rp.lambda_frm = lambda_frm; rp.top_n = top_n; rp.mode = mode;
+  return retrieve_impl(ctx, d_qtok, h_q_offsets, h_t_limit, nq, rp, d_seg_idx, d_frm_idx, nullptr, d_seg_score,
+                       d_frm_score, nullptr, d_counts, 2, stream);
+}
+
+mukv_status mukv_retrieve3(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_offsets, const int64_t* h_t_limit,
+                           int32_t nq, const mukv_retr_params* params, int32_t* d_seg_idx, int32_t* d_frm_idx,
+                           int32_t* d_patch_idx, float* d_seg_score, float* d_frm_score, float* d_patch_score,
+                           int32_t* d_counts, mukv_stream stream) {
+  if (!ctx) return MUKV_E_INVALID;
+  if (!params) return fail(ctx, MUKV_E_INVALID, "null params");
+  return retrieve_impl(ctx, d_qtok, h_q_offsets, h_t_limit, nq, *params, d_seg_idx, d_frm_idx, d_patch_idx, d_seg_score,
+                       d_frm_score, d_patch_score, d_counts, 3, stream);
+}
+
+int64_t mukv_decode3_tokens(const mukv_ctx* ctx, int32_t k_seg, int32_t k_frm, int32_t k_patch) {
+  if (!ctx || k_seg < 0 || k_frm < 0 || k_patch < 0) return 0;
+  const mukv_config& c = ctx->cfg;
+  long long pmax = 0;
+  if (c.patch_split > 0) {
+    const int rows = c.tokens_per_frame / c.grid_width;
+    pmax = (long long)((rows + c.patch_split - 1) / c.patch_split) * ((c.grid_width + c.patch_split - 1) / c.patch_split);
+    if (pmax > c.keep_per_frame) pmax = c.keep_per_frame;
+  }
+  return (long long)k_seg + (long long)k_frm * c.keep_per_frame + (long long)k_patch * pmax;
+}
+
+mukv_status mukv_gather3(mukv_ctx* ctx, const int32_t* d_seg_idx, const int32_t* d_frm_idx, const int32_t* d_patch_idx,
+                         const int32_t* d_counts, int32_t nq, int32_t k_seg, int32_t k_frm, int32_t k_patch,
+                         void* d_decode, int64_t decode_stride_bytes, int32_t* d_ntok, int32_t* d_tok_meta,
+                         mukv_stream stream) {
+  if (!ctx) return MUKV_E_INVALID;
   try {
     if (ctx->failed) return fail(ctx, MUKV_E_STATE, "an earlier call broke off half way: call mukv_reset");
-    if (!d_qtok || !h_q_offsets || !d_seg_idx || !d_frm_idx || !d_counts)
-      return fail(ctx, MUKV_E_INVALID, "null argument");
-    if (!aligned16(d_qtok) || !aligned4(d_seg_idx) || !aligned4(d_frm_idx) || !aligned4(d_seg_score) ||
-        !aligned4(d_frm_score) || !aligned4(d_counts))
-      return fail(ctx, MUKV_E_ALIGN, "d_qtok must be 16-byte aligned, the outputs 4-byte aligned");
-    if (nq < 1) return fail(ctx, MUKV_E_INVALID, "nq must be >= 1");
-    if (nq > MUKV_MAX_QUESTIONS) return fail(ctx, MUKV_E_CAPACITY, "nq %d exceeds %d", nq, MUKV_MAX_QUESTIONS);
-    if (k_seg < 1 || k_frm < 1 || top_n < 0) return fail(ctx, MUKV_E_INVALID, "k_seg, k_frm must be >= 1, top_n >= 0");
-    if (k_seg > MUKV_MAX_TOPK || k_frm > MUKV_MAX_TOPK || top_n > MUKV_MAX_TOPK)
-      return fail(ctx, MUKV_E_CAPACITY, "k_seg / k_frm / top_n exceed %d", MUKV_MAX_TOPK);
-    if (mode != MUKV_RETR_PARALLEL && mode != MUKV_RETR_HIER && mode != MUKV_RETR_SEMI)
-      return fail(ctx, MUKV_E_INVALID, "unknown retrieval mode %d", mode);
-    if (!(lambda_frm >= 0.f && lambda_frm <= 1.f)) return fail(ctx, MUKV_E_INVALID, "lambda_frm must lie in [0, 1]");
-    if (ctx->frames < 1) return fail(ctx, MUKV_E_STATE, "the store is empty");
-    QMeta meta;
-    if (h_q_offsets[0] != 0) return fail(ctx, MUKV_E_INVALID, "q_offsets[0] must be 0");
-    for (int i = 0; i < nq; ++i) {
-      if (h_q_offsets[i + 1] <= h_q_offsets[i])
-        return fail(ctx, MUKV_E_INVALID, "question %d has no tokens (offsets must ascend)", i);
-      if (h_t_limit && h_t_limit[i] < 0) return fail(ctx, MUKV_E_INVALID, "t_limit[%d] is negative", i);
-    }
-    for (int i = 0; i <= nq; ++i) meta.off[i] = h_q_offsets[i];
-    for (int i = 0; i < nq; ++i) meta.t_limit[i] = h_t_limit ? (long long)h_t_limit[i] : ctx->frames;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!d_seg_idx || !d_frm_idx || !d_counts || !d_decode || !d_ntok) return fail(ctx, MUKV_E_INVALID, "null argument");
+    if (k_patch > 0 && !d_patch_idx) return fail(ctx, MUKV_E_INVALID, "d_patch_idx is null");
+    if (!aligned4(d_seg_idx) || !aligned4(d_frm_idx) || !aligned4(d_patch_idx) || !aligned4(d_counts) ||
+        !aligned16(d_decode) || !aligned4(d_ntok) || !aligned4(d_tok_meta))
+      return fail(ctx, MUKV_E_ALIGN, "d_decode must be 16-byte aligned, index arrays 4-byte aligned");
+    if (nq < 1 || k_seg < 1 || k_frm < 1 || k_patch < 0) return fail(ctx, MUKV_E_INVALID, "nq, k_seg, k_frm must be >= 1");
+    if (nq > MUKV_MAX_QUESTIONS || k_seg > MUKV_MAX_TOPK || k_frm > MUKV_MAX_TOPK || k_patch > MUKV_MAX_TOPK)
+      return fail(ctx, MUKV_E_CAPACITY, "nq or a k too large");
     const mukv_config& c = ctx->cfg;
-    const int C = ctx->C;
-    double* q64 = reinterpret_cast<double*>(ctx->ws + ctx->wl.q64);
-    double* qnorm = reinterpret_cast<double*>(ctx->ws + ctx->wl.qnorm);
-    double* s_frm = reinterpret_cast<double*>(ctx->ws + ctx->wl.s_frm);
-    double* s_seg = reinterpret_cast<double*>(ctx->ws + ctx->wl.s_seg);
-    const float* frame_key = reinterpret_cast<const float*>(ctx->store + ctx->sl.frame_key);
-    const float* seg_key = reinterpret_cast<const float*>(ctx->store + ctx->sl.seg_key);
-    const long long n_frm = ctx->frames;
-    const long long n_seg = (n_frm + c.frames_per_segment - 1) / c.frames_per_segment;
+    if (k_patch > 0 && c.patch_split == 0) return fail(ctx, MUKV_E_STATE, "the store has no patch level");
+    const long long tok_cap = mukv_decode3_tokens(ctx, k_seg, k_frm, k_patch);
+    const long long need = (long long)c.n_layers * 2 * tok_cap * ctx->C * ctx->esize;
+    if (decode_stride_bytes < need)
+      return fail(ctx, MUKV_E_CAPACITY, "decode_stride_bytes %lld < %lld needed per question",
+                  (long long)decode_stride_bytes, need);
+    if (decode_stride_bytes % 16 != 0) return fail(ctx, MUKV_E_ALIGN, "decode_stride_bytes must be a multiple of 16");
+    Gather3Params gp;
+    memset(&gp, 0, sizeof gp);
+    gp.nq = nq; gp.k_seg = k_seg; gp.k_frm = k_frm; gp.k_pat = k_patch; gp.L = c.n_layers; gp.kappa = c.keep_per_frame;
+    gp.C = ctx->C; gp.P = c.tokens_per_frame; gp.S = c.patch_split * c.patch_split; gp.grid_width = c.grid_width;
+    gp.patch_split = c.patch_split; gp.tok_cap = (int)tok_cap; gp.esize = ctx->esize;
+    gp.seg_idx = d_seg_idx; gp.frm_idx = d_frm_idx; gp.pat_idx = d_patch_idx; gp.counts = d_counts;
+    gp.store = ctx->store;
+    gp.page_table = reinterpret_cast<const long long*>(ctx->store + ctx->sl.page_table);
+    gp.kept_store = reinterpret_cast<const int*>(ctx->store + ctx->sl.kept);
+    gp.seg_entry = reinterpret_cast<const float*>(ctx->store + ctx->sl.seg_entry);
+    gp.patch_cnt = reinterpret_cast<const int*>(ctx->store + ctx->sl.patch_cnt);
+    gp.decode = static_cast<unsigned char*>(d_decode);
+    gp.decode_stride = decode_stride_bytes;
+    gp.ntok = d_ntok; gp.tok_meta = d_tok_meta;
+    const long long units = (long long)nq * c.n_layers * 2 * (k_frm + 1);
+    const unsigned blocks = (unsigned)(units < 148 * 8 ? units : 148 * 8);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
     {
-      ProfScope ps(ctx, 4, st);
-      if (c.dtype == MUKV_BF16)
-        qpool_kernel<__nv_bfloat16><<<dim3(nq, c.n_kv_heads), kPoolThreads, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(d_qtok), meta,
-                                                       c.n_q_heads, c.n_kv_heads, c.head_dim, q64, qnorm);
-      else
-        qpool_kernel<float><<<dim3(nq, c.n_kv_heads), kPoolThreads, 0, st>>>(reinterpret_cast<const float*>(d_qtok), meta, c.n_q_heads,
-                                               c.n_kv_heads, c.head_dim, q64, qnorm);
+      ProfScope ps(ctx, 7, st);
+      if (c.dtype == MUKV_BF16) gather3_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(gp);
+      else gather3_kernel<float><<<blocks, 256, 0, st>>>(gp);
     }
     cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "qpool kernel: %s", cudaGetErrorString(e));
-    const long long rows = n_frm + n_seg;
-    const unsigned blocks = (unsigned)((rows + kScanRows - 1) / kScanRows);
-    {
-      ProfScope ps(ctx, 5, st);
-      e = launch_k(scan_kernel, dim3(blocks), 256, 0, st, !ctx->prof_on, frame_key, seg_key, n_frm, n_seg, C, nq,
-                   (const double*)q64, (const double*)qnorm, (int)c.n_kv_heads, s_frm, s_seg, (long long)c.max_frames,
-                   (long long)ctx->sl.max_segs);
-    }
-    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "scan kernel: %s", cudaGetErrorString(e));
-    RankParams rp;
-    memset(&rp, 0, sizeof rp);
-    rp.nq = nq; rp.C = C; rp.fseg = c.frames_per_segment;
-    rp.k_seg = k_seg; rp.k_frm = k_frm; rp.top_n = top_n; rp.mode = mode;
-    rp.lambda = (double)lambda_frm; rp.delta = (double)c.tie_eps;
-    rp.n_frm = n_frm; rp.n_seg = n_seg;
-    rp.s_frm = s_frm; rp.s_seg = s_seg; rp.frm_stride = c.max_frames; rp.seg_stride = ctx->sl.max_segs;
-    rp.frame_key = frame_key; rp.seg_key = seg_key;
-    rp.seg_idx = d_seg_idx; rp.frm_idx = d_frm_idx; rp.seg_score = d_seg_score; rp.frm_score = d_frm_score;
-    rp.counts = d_counts;
-    {
-      ProfScope ps(ctx, 6, st);
-      size_t rank_smem = (size_t)C * sizeof(double);
-      const size_t staged = rank_smem + (size_t)(n_frm + n_seg) * sizeof(double);
-      rp.stage = staged <= (size_t)kRankStageBytes ? 1 : 0;
-      if (rp.stage) rank_smem = staged;
-      e = launch_k(rank_kernel, dim3(nq), kRankThreads, rank_smem, st, !ctx->prof_on, rp, meta);
-    }
-    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "rank kernel: %s", cudaGetErrorString(e));
-    ctx->launches += 4;
+    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "gather3 kernel: %s", cudaGetErrorString(e));
+    ctx->launches += 1;
     return MUKV_OK;
   } catch (...) {
     return fail(ctx, MUKV_E_INVALID, "unexpected exception");
@@ -900,6 +1023,8 @@ void* mukv_store_region(const mukv_ctx* ctx, int32_t which, size_t* bytes) {
     case 5: off = s.seg_key; sz = (size_t)s.max_segs * C * sizeof(float); break;
     case 6: off = s.frame_ts; sz = T * sizeof(long long); break;
     case 7: off = s.page_table; sz = T * sizeof(long long); break;
+    case 8: off = s.patch_key; sz = T * c.patch_split * c.patch_split * C * sizeof(float); break;
+    case 9: off = s.patch_cnt; sz = T * c.patch_split * c.patch_split * sizeof(int); break;
     default: return nullptr;
   }
   if (bytes) *bytes = sz;

@@ -91,7 +91,8 @@ __global__ void __launch_bounds__(kPoolThreads) qpool_kernel(const T* __restrict
 }
 
 // ------------------------------------------------------------------------------ Eq. 7
-// Rows 0..n_frm-1 are frame keys, rows n_frm..n_frm+n_seg-1 segment keys.  A block owns
+// Rows 0..n_frm-1 are frame keys, rows n_frm..n_frm+n_seg-1 segment keys, then n_pat patch-level
+// keys (n_pat = 0 without a patch level).  A block owns
 // kScanRows rows and walks the feature axis in chunks of kScanCC: the rows' chunk (float) and the
 // chunk of up to kScanQB pooled queries (double) are staged in shared memory.  The product itself
 // is a dense double-precision contraction [rows x C] . [C x questions] and runs on the
@@ -109,12 +110,25 @@ __device__ __forceinline__ void dmma_m8n8k4(double (&c)[2], double a, double b) 
                : "d"(a), "d"(b));
 }
 
-__global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ frame_key,
-                                                   const float* __restrict__ seg_key, long long n_frm,
-                                                   long long n_seg, int C, int nq, const double* __restrict__ q64t,
-                                                   const double* __restrict__ qn2, int Hkv, double* __restrict__ s_frm,
-                                                   double* __restrict__ s_seg, long long frm_stride,
-                                                   long long seg_stride) {
+struct ScanParams {
+  const float* frame_key; const float* seg_key; const float* patch_key;
+  long long n_frm, n_seg, n_pat;
+  int C, nq, Hkv;
+  const double* q64t; const double* qn2;
+  double* s_frm; double* s_seg; double* s_pat;
+  long long frm_stride, seg_stride, pat_stride;
+};
+
+__global__ void __launch_bounds__(256) scan_kernel(const ScanParams sp) {
+  const float* __restrict__ frame_key = sp.frame_key;
+  const float* __restrict__ seg_key = sp.seg_key;
+  const long long n_frm = sp.n_frm, n_seg = sp.n_seg;
+  const int C = sp.C, nq = sp.nq, Hkv = sp.Hkv;
+  const double* __restrict__ q64t = sp.q64t;
+  const double* __restrict__ qn2 = sp.qn2;
+  double* __restrict__ s_frm = sp.s_frm;
+  double* __restrict__ s_seg = sp.s_seg;
+  const long long frm_stride = sp.frm_stride, seg_stride = sp.seg_stride;
   __shared__ float rows[kScanRows][kScanCC + 1];
   __shared__ __align__(16) double qs[kScanCC][kScanQPad];
   __shared__ double s_knorm[kScanRows];
@@ -128,11 +142,12 @@ __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ fra
     s_qn[qq] = sqrt(t);
   }
   const long long row0 = (long long)blockIdx.x * kScanRows;
-  const long long n_rows = n_frm + n_seg;
+  const long long n_rows = n_frm + n_seg + sp.n_pat;
   const int lr = tid >> 3, lc = (tid & 7) * 8;               // staging: row, first column of 8
   const long long my_row = row0 + lr;
   const float* src = my_row < n_frm ? frame_key + my_row * C
-                                    : (my_row < n_rows ? seg_key + (my_row - n_frm) * C : nullptr);
+                     : (my_row < n_frm + n_seg ? seg_key + (my_row - n_frm) * C
+                     : (my_row < n_rows ? sp.patch_key + (my_row - n_frm - n_seg) * C : nullptr));
   const int wr = (warp & 3) * 8, wq = (warp >> 2) * 32;      // this warp's rows and questions
   const int fr = lane >> 2, fk = lane & 3;                   // fragment row / k (A), k / column (B)
   for (int qb = 0; qb < nq; qb += kScanQB) {
@@ -201,7 +216,8 @@ __global__ void __launch_bounds__(256) scan_kernel(const float* __restrict__ fra
           den = den > 1e-12 ? den : 1e-12;
           const double sc = acc[nt][j] / den;
           if (row < n_frm) s_frm[(long long)qi * frm_stride + row] = sc;
-          else s_seg[(long long)qi * seg_stride + (row - n_frm)] = sc;
+          else if (row < n_frm + n_seg) s_seg[(long long)qi * seg_stride + (row - n_frm)] = sc;
+          else sp.s_pat[(long long)qi * sp.pat_stride + (row - n_frm - n_seg)] = sc;
         }
       }
     }
@@ -425,35 +441,95 @@ __device__ __noinline__ int block_topk_set(ScoreFn score, MemberFn member, int n
 
 struct RankParams {
   int nq, C, fseg;
-  int k_seg, k_frm, top_n, mode;
-  double lambda, delta;
+  int k_seg, k_frm, k_pat, top_n, mode;
+  int S;                                  // patch-level blocks per frame (0: none)
+  double lam_seg, lam_frm, lam_pat, delta;
   long long n_frm, n_seg;                 // stored
   const double* s_frm;                    // [nq][frm_stride]
   const double* s_seg;
-  long long frm_stride, seg_stride;
+  const double* s_pat;                    // [nq][pat_stride]
+  long long frm_stride, seg_stride, pat_stride;
   const float* frame_key;
   const float* seg_key;
-  int* seg_idx; int* frm_idx; float* seg_score; float* frm_score; int* counts;
-  int stage;                              // 1: the question's scores are copied to shared memory first
+  const float* patch_key;
+  const int* patch_cnt;                   // [frames][S]
+  int* seg_idx; int* frm_idx; int* pat_idx; float* seg_score; float* frm_score; float* pat_score;
+  int* counts; int counts_stride;         // 2 or 3 ints per question
+  int stage;                              // 1: the question's frame and segment scores are copied to shared memory first
 };
 
 constexpr int kRankThreads = 512;
 constexpr int kRankStageBytes = 192 * 1024;       // dynamic shared memory the kernel may be given
 constexpr int kMaxCand = 2 * MUKV_MAX_TOPK;
 
+struct RankShared {
+  RankScratch sc;
+  int sel_seg[MUKV_MAX_TOPK];
+  double sel_seg_score[MUKV_MAX_TOPK];
+  int top[MUKV_MAX_TOPK];
+  int cand[kMaxCand];
+  double cand_score[kMaxCand];
+  double s_new[kMaxCand];
+  int pick[MUKV_MAX_TOPK];
+  double pick_score[MUKV_MAX_TOPK];
+  double gn;
+};
+
+// Stage 1 + stage 2 of one granularity for one question, run by the whole block: top-2k candidates
+// by cosine among the members, Eq. 8 against the global query gq (norm gnorm; have_g false: gamma = 0),
+// then the k best by the calibrated score.  PARALLEL / HIER callers pass semi = false: the k best by
+// cosine among the members.  Results (ascending ids) in sh->pick / sh->pick_score; returns the count.
+template <typename MemberFn>
+__device__ __noinline__ int rank_level(const double* scores, MemberFn member, int n, int k, bool semi, double lambda,
+                                       double delta, const float* keys, int C, const double* gq, double gnorm,
+                                       bool have_g, RankShared* sh) {
+  const int tid = threadIdx.x;
+  const ArrScore s1{scores};
+  if (!semi) return block_topk_set(s1, member, n, k, delta, sh->pick, sh->pick_score, &sh->sc);
+  const int n_cand = block_topk_set(s1, member, n, 2 * k, delta, sh->cand, sh->cand_score, &sh->sc);
+  // Eq. 8 for every candidate: one warp per candidate
+  const int lane = tid & 31, warp = tid >> 5;
+  for (int ci = warp; ci < n_cand; ci += kRankThreads / 32) {
+    const float* kr = keys + (long long)sh->cand[ci] * C;
+    double dot = 0.0, kk = 0.0;
+    for (int c = lane; c < C; c += 32) {
+      const double x = (double)kr[c];
+      dot = fma(x, gq[c], dot);
+      kk = fma(x, x, kk);
+    }
+    dot = warp_sum(dot);
+    kk = warp_sum(kk);
+    if (lane == 0) {
+      double gamma = 0.0;
+      if (have_g) {
+        double den = sqrt(kk) * gnorm;
+        den = den > 1e-12 ? den : 1e-12;
+        gamma = dot / den;
+      }
+      sh->s_new[ci] = (1.0 - lambda) * sh->cand_score[ci] + lambda * gamma;
+    }
+  }
+  __syncthreads();
+  const ArrScore new_score{sh->s_new};
+  const AllMembers always;
+  const int c = block_topk_set(new_score, always, n_cand, k, delta, sh->pick, sh->pick_score, &sh->sc);
+  // pick holds positions in the candidate list (ascending position = ascending block id)
+  for (int i = tid; i < c; i += kRankThreads) sh->pick[i] = sh->cand[sh->pick[i]];
+  __syncthreads();
+  return c;
+}
+
+__device__ __forceinline__ void rank_emit(int* idx, float* score, long long base, int k, int c, const RankShared* sh) {
+  for (int i = threadIdx.x; i < k; i += kRankThreads) {
+    idx[base + i] = i < c ? sh->pick[i] : -1;
+    if (score) score[base + i] = i < c ? (float)sh->pick_score[i] : 0.f;
+  }
+}
+
 __global__ void __launch_bounds__(kRankThreads) rank_kernel(const RankParams p, const QMeta meta) {
-  __shared__ RankScratch sc;
-  __shared__ int s_sel_seg[MUKV_MAX_TOPK];
-  __shared__ double s_sel_seg_score[MUKV_MAX_TOPK];
-  __shared__ int s_top[MUKV_MAX_TOPK];
-  __shared__ int s_cand[kMaxCand];
-  __shared__ double s_cand_score[kMaxCand];
-  __shared__ double s_new[kMaxCand];
-  __shared__ int s_pick[MUKV_MAX_TOPK];
-  __shared__ double s_pick_score[MUKV_MAX_TOPK];
+  __shared__ RankShared sh;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* gq = reinterpret_cast<double*>(smem_raw);               // [C] global query
-  __shared__ double s_gn;
 
   const int qi = blockIdx.x, tid = threadIdx.x;
   pdl_wait();                                                // the scores of the scan are complete
@@ -478,85 +554,78 @@ __global__ void __launch_bounds__(kRankThreads) rank_kernel(const RankParams p, 
     sf = st_f;
     ss = st_s;
   }
-  const ArrScore seg_score{ss}, frm_score{sf};
+  const ArrScore seg_score{ss};
   const AllMembers always;
+  const bool semi = p.mode == MUKV_RETR_SEMI;
 
-  // ---- segments: lambda = 0, final = stage-1 top-k
-  const int c_seg = block_topk_set(seg_score, always, n_seg, p.k_seg, p.delta, s_sel_seg, s_sel_seg_score, &sc);
-  for (int i = tid; i < p.k_seg; i += kRankThreads) {
-    p.seg_idx[(long long)qi * p.k_seg + i] = i < c_seg ? s_sel_seg[i] : -1;
-    if (p.seg_score) p.seg_score[(long long)qi * p.k_seg + i] = i < c_seg ? (float)s_sel_seg_score[i] : 0.f;
-  }
-  __syncthreads();
-
-  int c_frm = 0;
-  if (p.mode == MUKV_RETR_PARALLEL) {
-    c_frm = block_topk_set(frm_score, always, n_frm, p.k_frm, p.delta, s_pick, s_pick_score, &sc);
-  } else if (p.mode == MUKV_RETR_HIER) {
-    const int fseg = p.fseg;
-    auto inside = [&](int t) {
-      const int u = t / fseg;
-      for (int i = 0; i < c_seg; ++i)
-        if (s_sel_seg[i] == u) return true;
-      return false;
-    };
-    c_frm = block_topk_set(frm_score, inside, n_frm, p.k_frm, p.delta, s_pick, s_pick_score, &sc);
-  } else {
-    // stage 1: top-2k frame candidates
-    const int n_cand = block_topk_set(frm_score, always, n_frm, 2 * p.k_frm, p.delta, s_cand, s_cand_score, &sc);
-    // global query = mean of the top-N segment keys
+  // ---- global query = mean of the top-N segment keys (stage 1 order)
+  bool have_g = false;
+  double gnorm = 0.0;
+  if (semi) {
     const int N = p.top_n > 0 ? p.top_n : p.k_seg;
-    const int n_top = block_topk_set(seg_score, always, n_seg, N, p.delta, s_top, (double*)nullptr, &sc);
+    const int n_top = block_topk_set(seg_score, always, n_seg, N, p.delta, sh.top, (double*)nullptr, &sh.sc);
     double part = 0.0;
     for (int c = tid; c < C; c += kRankThreads) {
       double t = 0.0;
-      for (int i = 0; i < n_top; ++i) t += (double)p.seg_key[(long long)s_top[i] * C + c];
+      for (int i = 0; i < n_top; ++i) t += (double)p.seg_key[(long long)sh.top[i] * C + c];
       t = n_top > 0 ? t / (double)n_top : 0.0;
       gq[c] = t;
       part += t * t;
     }
-    if (tid == 0) s_gn = 0.0;
+    if (tid == 0) sh.gn = 0.0;
     __syncthreads();
     part = warp_sum(part);
-    if ((tid & 31) == 0) atomicAdd(&s_gn, part);
+    if ((tid & 31) == 0) atomicAdd(&sh.gn, part);
     __syncthreads();
-    const double gnorm = sqrt(s_gn);
-    // Eq. 8 for every candidate: one warp per candidate
-    const int lane = tid & 31, warp = tid >> 5;
-    for (int ci = warp; ci < n_cand; ci += kRankThreads / 32) {
-      const float* kr = p.frame_key + (long long)s_cand[ci] * C;
-      double dot = 0.0, kk = 0.0;
-      for (int c = lane; c < C; c += 32) {
-        const double x = (double)kr[c];
-        dot = fma(x, gq[c], dot);
-        kk = fma(x, x, kk);
-      }
-      dot = warp_sum(dot);
-      kk = warp_sum(kk);
-      if (lane == 0) {
-        double gamma = 0.0;
-        if (n_top > 0) {
-          double den = sqrt(kk) * gnorm;
-          den = den > 1e-12 ? den : 1e-12;
-          gamma = dot / den;
-        }
-        s_new[ci] = (1.0 - p.lambda) * s_cand_score[ci] + p.lambda * gamma;
+    gnorm = sqrt(sh.gn);
+    have_g = n_top > 0;
+  }
+
+  // ---- segments (the paper's lambda for them is 0: final = stage-1 top-k)
+  const int c_seg = rank_level(ss, always, n_seg, p.k_seg, semi && p.lam_seg > 0.0, p.lam_seg, p.delta, p.seg_key, C, gq,
+                               gnorm, have_g, &sh);
+  rank_emit(p.seg_idx, p.seg_score, (long long)qi * p.k_seg, p.k_seg, c_seg, &sh);
+  for (int i = tid; i < c_seg; i += kRankThreads) sh.sel_seg[i] = sh.pick[i];
+  __syncthreads();
+
+  // ---- frames
+  const int fseg = p.fseg;
+  auto in_sel_seg = [&](int t) {
+    const int u = t / fseg;
+    for (int i = 0; i < c_seg; ++i)
+      if (sh.sel_seg[i] == u) return true;
+    return false;
+  };
+  int c_frm;
+  if (p.mode == MUKV_RETR_HIER)
+    c_frm = rank_level(sf, in_sel_seg, n_frm, p.k_frm, false, 0.0, p.delta, p.frame_key, C, gq, gnorm, have_g, &sh);
+  else
+    c_frm = rank_level(sf, always, n_frm, p.k_frm, semi, p.lam_frm, p.delta, p.frame_key, C, gq, gnorm, have_g, &sh);
+  rank_emit(p.frm_idx, p.frm_score, (long long)qi * p.k_frm, p.k_frm, c_frm, &sh);
+  __syncthreads();
+
+  // ---- patch-level blocks: (frame, super patch) pairs that kept at least one token
+  int c_pat = 0;
+  if (p.k_pat > 0) {
+    const int S = p.S;
+    const int* cnt = p.patch_cnt;
+    const double* spat = p.s_pat + (long long)qi * p.pat_stride;
+    if (S > 0) {
+      if (p.mode == MUKV_RETR_HIER) {
+        auto member = [&](int b) { return cnt[b] > 0 && in_sel_seg(b / S); };
+        c_pat = rank_level(spat, member, n_frm * S, p.k_pat, false, 0.0, p.delta, p.patch_key, C, gq, gnorm, have_g, &sh);
+      } else {
+        auto member = [&](int b) { return cnt[b] > 0; };
+        c_pat = rank_level(spat, member, n_frm * S, p.k_pat, semi, p.lam_pat, p.delta, p.patch_key, C, gq, gnorm, have_g,
+                           &sh);
       }
     }
-    __syncthreads();
-    const ArrScore new_score{s_new};
-    c_frm = block_topk_set(new_score, always, n_cand, p.k_frm, p.delta, s_pick, s_pick_score, &sc);
-    // s_pick holds positions in the candidate list (ascending position = ascending frame id)
-    for (int i = tid; i < c_frm; i += kRankThreads) s_pick[i] = s_cand[s_pick[i]];
-    __syncthreads();
-  }
-  for (int i = tid; i < p.k_frm; i += kRankThreads) {
-    p.frm_idx[(long long)qi * p.k_frm + i] = i < c_frm ? s_pick[i] : -1;
-    if (p.frm_score) p.frm_score[(long long)qi * p.k_frm + i] = i < c_frm ? (float)s_pick_score[i] : 0.f;
+    rank_emit(p.pat_idx, p.pat_score, (long long)qi * p.k_pat, p.k_pat, c_pat, &sh);
   }
   if (tid == 0) {
-    p.counts[2 * qi] = c_seg;
-    p.counts[2 * qi + 1] = c_frm;
+    p.counts[p.counts_stride * qi] = c_seg;
+    p.counts[p.counts_stride * qi + 1] = c_frm;
+    if (p.counts_stride > 2) p.counts[p.counts_stride * qi + 2] = c_pat;
   }
 }
 
@@ -605,6 +674,101 @@ __global__ void __launch_bounds__(256) gather_kernel(const GatherParams p) {
         m[1] = p.kept_store[(long long)f * p.kappa + t];
       }
     }
+  }
+}
+
+// ------------------------------------------------------------------------------ Eq. 9, all granularities
+struct Gather3Params {
+  int nq, k_seg, k_frm, k_pat, L, kappa, C, P, S, grid_width, patch_split;
+  int tok_cap;                             // token slots per (layer, K|V) plane of a decode buffer
+  int esize;                               // bytes per element of the store dtype
+  const int* seg_idx; const int* frm_idx; const int* pat_idx; const int* counts;   // counts [nq][3]
+  const unsigned char* store; const long long* page_table; const int* kept_store;
+  const float* seg_entry;                  // [segments][L][2][C]
+  const int* patch_cnt;                    // [frames][S]
+  unsigned char* decode; long long decode_stride;
+  int* ntok; int* tok_meta;
+};
+
+__device__ __forceinline__ void copy_run16(unsigned char* dst, const unsigned char* src, long long bytes) {
+  const long long nvec = bytes >> 4;
+  for (long long v = threadIdx.x; v < nvec; v += blockDim.x) st_stream(dst + (v << 4), ld_stream(src + (v << 4)));
+}
+
+// Units, per question and (layer, K|V) plane: k_frm frame runs (one contiguous run of the page each),
+// then one unit for the summary tokens and the patch-level rows.  Token slots of a plane: summary
+// tokens of the selected segments, kept tokens of the selected frames, kept tokens of the selected
+// patch-level blocks.
+template <typename T>
+__global__ void __launch_bounds__(256) gather3_kernel(const Gather3Params p) {
+  __shared__ int s_off[MUKV_MAX_TOPK + 1];                 // first row of each selected patch block
+  const long long planes = (long long)p.L * 2;
+  const int upp = p.k_frm + 1;                             // units per (question, plane)
+  const long long n_units = (long long)p.nq * planes * upp;
+  const long long row_bytes = (long long)p.C * p.esize;
+  const long long run_bytes = (long long)p.kappa * row_bytes;
+  for (long long u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const int slot = (int)(u % upp);
+    const long long r = u / upp;
+    const int plane = (int)(r % planes);
+    const int qi = (int)(r / planes);
+    const int c_seg = p.counts[3 * qi], c_frm = p.counts[3 * qi + 1], c_pat = p.counts[3 * qi + 2];
+    unsigned char* dplane = p.decode + (long long)qi * p.decode_stride + (long long)plane * p.tok_cap * row_bytes;
+    int* meta = p.tok_meta ? p.tok_meta + (long long)qi * p.tok_cap * 2 : nullptr;
+    if (slot < p.k_frm) {
+      if (slot >= c_frm) continue;
+      const int f = p.frm_idx[(long long)qi * p.k_frm + slot];
+      const int row0 = c_seg + slot * p.kappa;
+      copy_run16(dplane + (long long)row0 * row_bytes, p.store + p.page_table[f] + (long long)plane * run_bytes, run_bytes);
+      if (plane == 0 && meta) {
+        for (int t = threadIdx.x; t < p.kappa; t += blockDim.x) {
+          meta[(row0 + t) * 2] = f;
+          meta[(row0 + t) * 2 + 1] = p.kept_store[(long long)f * p.kappa + t];
+        }
+      }
+      continue;
+    }
+    // ---- summary tokens: the segment's pooled entry of this plane, rounded to the store dtype
+    for (int i = 0; i < c_seg; ++i) {
+      const int useg = p.seg_idx[(long long)qi * p.k_seg + i];
+      const float* e = p.seg_entry + ((long long)useg * planes + plane) * p.C;
+      T* d = reinterpret_cast<T*>(dplane + (long long)i * row_bytes);
+      for (int c = threadIdx.x; c < p.C; c += blockDim.x) {
+        if constexpr (sizeof(T) == 2) d[c] = __float2bfloat16_rn(e[c]);
+        else d[c] = e[c];
+      }
+      if (plane == 0 && meta && threadIdx.x == 0) { meta[i * 2] = -1 - useg; meta[i * 2 + 1] = -1; }
+    }
+    // ---- patch-level rows: block b = frame * S + super patch holds the frame's kept rows inside it
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int off = c_seg + c_frm * p.kappa;
+      for (int i = 0; i < c_pat; ++i) {
+        s_off[i] = off;
+        off += p.patch_cnt[p.pat_idx[(long long)qi * p.k_pat + i]];
+      }
+      s_off[c_pat] = off;
+      if (plane == 0 && p.ntok) p.ntok[qi] = off;
+    }
+    __syncthreads();
+    // one warp per patch block: walk the frame's kept list, copy the rows of the super patch
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    for (int i = warp; i < c_pat; i += nwarp) {
+      const int b = p.pat_idx[(long long)qi * p.k_pat + i];
+      const int f = b / p.S, sp = b % p.S;
+      const unsigned char* page = p.store + p.page_table[f] + (long long)plane * run_bytes;
+      int row = s_off[i];
+      for (int t = 0; t < p.kappa; ++t) {
+        const int tok = p.kept_store[(long long)f * p.kappa + t];
+        if (super_patch_index(tok, p.P, p.grid_width, p.patch_split) != sp) continue;
+        const unsigned char* src = page + (long long)t * row_bytes;
+        unsigned char* dst = dplane + (long long)row * row_bytes;
+        for (long long v = lane; v < (row_bytes >> 4); v += 32) st_stream(dst + (v << 4), ld_stream(src + (v << 4)));
+        if (plane == 0 && meta && lane == 0) { meta[row * 2] = f; meta[row * 2 + 1] = tok; }
+        ++row;
+      }
+    }
+    __syncthreads();
   }
 }
 

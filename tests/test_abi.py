@@ -28,7 +28,7 @@ def good_config(**over):
 def test_exports_match_header(lib):
     text = open(os.path.join(ROOT, "include", "mukv.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    declared = sorted(set(re.findall(r"\b(mukv_[a-z_]+)\s*\(", text)))
+    declared = sorted(set(re.findall(r"\b(mukv_[a-z_0-9]+)\s*\(", text)))
     assert declared == sorted(B.EXPORTS)
     for name in declared:
         assert hasattr(lib, name), f"{name} is declared but not exported"
@@ -37,7 +37,8 @@ def test_exports_match_header(lib):
 
 
 def test_struct_sizes_match_header():
-    assert C.sizeof(B.MukvConfig) == 64 and C.sizeof(B.MukvStats) == 72 and C.sizeof(B.MukvStoreHeader) == 88
+    assert C.sizeof(B.MukvConfig) == 80 and C.sizeof(B.MukvStats) == 72 and C.sizeof(B.MukvStoreHeader) == 104
+    assert C.sizeof(B.MukvRetrParams) == 32
 
 
 def test_store_size_of_the_three_hour_stream(lib):
@@ -53,7 +54,8 @@ def test_store_size_of_the_three_hour_stream(lib):
 @pytest.mark.parametrize("over", [dict(head_dim=96), dict(n_q_heads=30), dict(tokens_per_frame=300),
                                   dict(keep_per_frame=0), dict(keep_per_frame=197), dict(alpha=1.5),
                                   dict(dtype=7), dict(max_frames=0), dict(n_kv_heads=3, n_q_heads=27),
-                                  dict(frames_per_segment=0)])
+                                  dict(frames_per_segment=0), dict(patch_split=5, grid_width=14),
+                                  dict(patch_split=2, grid_width=13), dict(patch_split=2, grid_width=0)])
 def test_bad_configs_are_rejected_on_the_host(lib, over):
     cfg = good_config(**over)
     assert lib.mukv_store_bytes(C.byref(cfg)) == 0

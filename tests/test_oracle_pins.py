@@ -425,3 +425,113 @@ def test_gather_layout_and_token_count():
                 assert meta[s * kap + r].tolist() == [t, int(j)]
     # the retrieved context has (blocks x kappa) tokens: 64 x 49 = 3,136 and 64 x 196 = 12,544
     assert 64 * O.keep_count(0.25, 196) == 3136 and 64 * O.keep_count(1.0, 196) == 12544
+
+
+# --------------------------------------------------------------------------- three granularities
+CFG3 = dict(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=8, tokens_per_frame=36, keep_per_frame=13,
+            frames_per_segment=3, alpha=0.7, patch_split=2, grid_width=6)
+
+
+def test_context_tokens_match_the_paper():
+    path = os.path.join(os.path.dirname(__file__), "golden", "paper_context_tokens.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    blocks = [(int(k), float(rho), int(n)) for name, k, rho, n in rows[:3]]
+    printed = float(rows[3][1])
+    with_floor = sum(k * O.keep_count(rho, n) for k, rho, n in blocks)
+    assert with_floor == 20 * 4 + 32 * 19 + 12 * 627
+    assert abs(with_floor / 1000.0 - printed) <= 0.1
+    assert abs(sum(k * rho * n for k, rho, n in blocks) / 1000.0 - printed) <= 0.05
+
+
+def test_super_patch_of_is_the_quadrant():
+    # 14 x 14 grid, 2 x 2 super patches of 7 x 7 = 49 tokens (the paper's S = 4, P = 196)
+    ids = np.arange(196)
+    sp = O.super_patch_of(ids, 196, 14, 2)
+    for j in ids:
+        assert sp[j] == (0 if j // 14 < 7 else 2) + (0 if j % 14 < 7 else 1)
+    assert np.bincount(sp).tolist() == [49, 49, 49, 49]
+    # a grid that does not divide evenly: 6 x 6 cut in 4 x 4 -> rectangles of 2 x 2, only 3 x 3 of them occupied
+    sp = O.super_patch_of(np.arange(36), 36, 6, 4)
+    assert sorted(set(sp.tolist())) == [0, 1, 2, 4, 5, 6, 8, 9, 10]
+
+
+def test_patch_blocks_partition_the_frame():
+    st, Q, K, V = make_store(5, CFG3)
+    S = st.n_patches()
+    assert S == 4
+    for t in range(5):
+        pos = np.concatenate([st.patch_tokens(t, sp) for sp in range(S)])
+        assert sorted(pos.tolist()) == list(range(CFG3["keep_per_frame"]))
+        # the count-weighted mean of the patch-level keys is the frame-level key (Eq. 5 both ways)
+        w = np.array([st.patch_count(t, sp) for sp in range(S)], dtype=np.float64)
+        keys = np.stack([st.patch_key(t, sp) for sp in range(S)]).astype(np.float64)
+        np.testing.assert_allclose((w[:, None] * keys).sum(0) / w.sum(), st.frame_key(t), rtol=1e-5, atol=1e-6)
+        for sp in range(S):
+            toks = st.kept[t][st.patch_tokens(t, sp)]
+            want = K[-1, t, toks].astype(np.float64).reshape(len(toks), -1).mean(0) if len(toks) else np.zeros(16)
+            np.testing.assert_allclose(st.patch_key(t, sp), want, rtol=1e-6, atol=1e-7)
+
+
+def test_retrieve3_reduces_to_retrieve_and_to_brute_force():
+    st, Q, K, V = make_store(11, CFG3, chunk=4)
+    S = st.n_patches()
+    Qq = rand(5, 4, 8)
+    for mode in (O.MODE_SEMI, O.MODE_PARALLEL, O.MODE_HIER):
+        for tl in (None, 7):
+            a = O.retrieve(st, Qq, 2, 3, 0, 0.3, mode, tl)
+            b = O.retrieve3(st, Qq, (4, 3, 2), (0.3, 0.3, 0.0), 0, mode, tl)
+            assert a["seg_idx"].tolist() == b["seg_idx"].tolist() and a["frm_idx"].tolist() == b["frm_idx"].tolist()
+            np.testing.assert_allclose(a["frm_score"], b["frm_score"], rtol=1e-12)
+    # patch level, stage 1 only: the k best existing blocks by cosine, by a plain sort
+    r = O.retrieve3(st, Qq, (5, 3, 2), (0.0, 0.0, 0.0), 0, O.MODE_PARALLEL)
+    q = O.pool_question(Qq, 2)
+    sc = []
+    for t in range(11):
+        for sp in range(S):
+            if st.patch_count(t, sp):
+                k = st.patch_key(t, sp).astype(np.float64)
+                sc.append((-(k @ q) / (np.linalg.norm(k) * np.linalg.norm(q)), t * S + sp))
+    want = sorted(b for _, b in sorted(sc)[:5])
+    assert r["patch_idx"].tolist() == want
+    # lambda = 0 makes the semi-hierarchical result equal the parallel one at every granularity
+    z = O.retrieve3(st, Qq, (5, 3, 2), (0.0, 0.0, 0.0), 0, O.MODE_SEMI)
+    assert z["patch_idx"].tolist() == want and z["frm_idx"].tolist() == r["frm_idx"].tolist()
+    # HIER: every frame and patch block lies inside a selected segment
+    h = O.retrieve3(st, Qq, (6, 4, 2), (0.3, 0.3, 0.0), 0, O.MODE_HIER)
+    inside = set(h["seg_idx"].tolist())
+    assert all(t // 3 in inside for t in h["frm_idx"]) and all((b // S) // 3 in inside for b in h["patch_idx"])
+    # a segment-level lambda > 0 picks among the 2k stage-1 candidates
+    s2 = O.retrieve3(st, Qq, (1, 1, 2), (0.3, 0.3, 0.5), 1, O.MODE_SEMI)
+    cand = O.topk_set(O.cosine(q, st.segment_keys().astype(np.float64)), 4)
+    assert set(s2["seg_idx"].tolist()) <= set(cand.tolist()) and len(s2["seg_idx"]) == 2
+
+
+def test_gather3_layout():
+    import torch
+    st, Q, K, V = make_store(7, CFG3, chunk=3)
+    S = st.n_patches()
+    seg, frm, pat = [0, 2], [1, 5], [2 * S + 1, 6 * S + 3]
+    dec, meta = O.gather3(st, seg, frm, pat)
+    kap = CFG3["keep_per_frame"]
+    n_pat = sum(st.patch_count(b // S, b % S) for b in pat)
+    assert dec.shape[2] == len(seg) + len(frm) * kap + n_pat == meta.shape[0]
+    # summary tokens: the segment entry in the storage type (float32 here: unchanged)
+    for i, u in enumerate(seg):
+        ek, ev = st.segment_entry(u)
+        assert dec[:, 0, i].reshape(2, -1).tobytes() == ek.tobytes() and dec[:, 1, i].reshape(2, -1).tobytes() == ev.tobytes()
+        assert meta[i].tolist() == [-1 - u, -1]
+    ref, ref_meta = O.gather(st, frm)
+    assert dec[:, :, len(seg):len(seg) + len(frm) * kap].tobytes() == ref.tobytes()
+    row = len(seg) + len(frm) * kap
+    for b in pat:
+        t, sp = b // S, b % S
+        for j in st.kept[t]:
+            if O.super_patch_of([j], 36, 6, 2)[0] == sp:
+                assert dec[1, 0, row].tobytes() == K[1, t, j].tobytes() and meta[row].tolist() == [t, int(j)]
+                row += 1
+    assert row == dec.shape[2]
+    # rounding to bfloat16 storage equals the library's round-to-nearest-even conversion
+    x = RNG.standard_normal(1000).astype(np.float32)
+    got = O.round_to_dtype(x, np.zeros(1, dtype=np.uint16))
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert got.tobytes() == want.tobytes()
