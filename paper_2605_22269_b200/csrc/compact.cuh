@@ -18,14 +18,14 @@
 // tie_eps + flag_margin is skipped here: the double-precision pass that follows decides it, and
 // segment_kernel then compacts it.
 //
-// tail_kernel<T, NC>: what has to wait for every frame of the chunk.  Normally that is only the
-// segment entries (Eq. 5 at segment level): blocks 0 .. 2L-1 refresh one (layer, K|V) plane each of
-// every segment entry the chunk touches (mean over the frames present), the other blocks leave at
-// once.  When frames were flagged (about one chunk in fifty on the synthetic streams) all blocks
-// first score those frames in double precision and select; once every block has finished that,
-// the flagged frames are compacted and then the segment entries written, one plane per block.
+// What has to wait for every frame of the chunk runs in two small launches behind compact_kernel.
+// segment_kernel: the segment entries (Eq. 5 at segment level) when no frame was flagged: one
+// (layer, K|V) plane per block, mean over the frames present.  tail_kernel<T, NC>: returns at once
+// unless frames were flagged (about one chunk in fifty on the synthetic streams); then all its
+// blocks first score those frames in double precision and select; once every block has finished
+// that, the flagged frames are compacted and then the segment entries written, one plane per block.
 // (Segment pooling by the compaction block that finishes a plane last was measured: the fence
-// every block then needs before it signs off costs more than this launch.)
+// every block then needs before it signs off costs more than a launch.)
 #pragma once
 #include "common.cuh"
 #include "score.cuh"
@@ -535,6 +535,19 @@ constexpr int kStatusTailWait = 6;   // tail_kernel: the wait for the double-pre
 // tail_kernel: see the head of this file.  sp is the scoring configuration of the double-precision
 // pass (its partial-sum buffers, refine = 1); the grid is a multiple of nothing in particular: blocks
 // stride over the work, and the host keeps the grid within what is resident at once.
+// segment_kernel: the common case of what has to wait for every frame of the chunk.  One block per
+// (layer, K|V) plane; when no frame was flagged it writes that plane of every segment entry the chunk
+// touches.  Otherwise it leaves everything to tail_kernel.  (It is a launch of its own because it
+// is light: no dynamic shared memory, 56 blocks.  One kernel for both cases was measured and cost
+// 2 us more per call.)
+__global__ void __launch_bounds__(kCompactThreads) segment_kernel(const CompactParams p) {
+  pdl_wait();
+  pdl_trigger();
+  if (*p.sp.n_flagged != 0) return;
+  for (int plane = blockIdx.x; plane < 2 * p.L; plane += gridDim.x)
+    compact_segment_plane(segment_args(p), plane >> 1, plane & 1);
+}
+
 template <typename T, int NC>
 __global__ void __launch_bounds__(kScoreThreads, 2) tail_kernel(const ScoreParams sp, const CompactParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -543,12 +556,7 @@ __global__ void __launch_bounds__(kScoreThreads, 2) tail_kernel(const ScoreParam
   const int tid = threadIdx.x;
   pdl_wait();
   const int n_fl = *sp.n_flagged;
-  if (n_fl == 0) {
-    // the common case: segment entries only
-    for (int plane = blockIdx.x; plane < 2 * p.L; plane += gridDim.x)
-      compact_segment_plane(segment_args(p), plane >> 1, plane & 1);
-    return;
-  }
+  if (n_fl == 0) return;                        // the common case: segment_kernel has done what was left
   // ---- scores of the flagged frames in double precision; the block that finishes a frame last selects
   const int units = sp.Hq * sp.row_split;
   for (int w = blockIdx.x; w < n_fl * units; w += gridDim.x) {

@@ -523,8 +523,15 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   }
   if (e != cudaSuccess) return broke_off(ctx, "compact kernel", e);
 
-  // What needs every frame of the chunk: the segment entries; before them, for frames too close to
-  // a tie boundary, scores and selection again in double precision and their compaction.
+  // What needs every frame of the chunk: the segment entries (segment_kernel, when no frame was
+  // flagged); otherwise, in tail_kernel, scores and selection of the flagged frames again in double
+  // precision, their compaction, and then the segment entries.
+  cp.sp.n_flagged = sp.n_flagged;
+  {
+    ProfScope ps(ctx, 3, st);
+    e = launch_k(segment_kernel, dim3(2 * L), kCompactThreads, 0, st, !ctx->prof_on, cp);
+  }
+  if (e != cudaSuccess) return broke_off(ctx, "segment kernel", e);
   sp.refine = 1;
   sp.row_split = kRefineSplit;
   sp.colsum_part = ctx->ws + ctx->wl.colsum_d;
@@ -538,7 +545,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   }
   if (e != cudaSuccess) return broke_off(ctx, "tail kernel", e);
 
-  ctx->launches += d_ext ? 2 : 3;
+  ctx->launches += d_ext ? 3 : 4;
   ctx->parity ^= 1;
   ctx->frames = t0 + n;
   return MUKV_OK;
