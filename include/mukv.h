@@ -35,7 +35,9 @@
  *     call except mukv_reset, mukv_get_stats and mukv_destroy.
  *
  * Tensor layouts are token-major; element type is mukv_config.dtype (bf16 or fp32):
- *     Q   [n_frames][P][Hq][D]        last-layer queries of the chunk's visual tokens
+ *     Q   [n_frames][P][Hq][D]        queries of the chunk's visual tokens in the scoring layer (the
+ *                                     last layer by default); [Ls][n_frames][P][Hq][D] when
+ *                                     n_score_layers = Ls > 1, ordered like the layers of K
  *     K,V [L][n_frames][P][Hkv][D]    keys / values of every layer
  * Query head h attends with key head h / (Hq / Hkv) (grouped-query attention).
  */
@@ -95,7 +97,13 @@ typedef struct {
                                     patch level; at most 4                               */
   int32_t grid_width;            /* tokens per row of the frame's token grid (only read
                                     when patch_split > 0; must divide P)                 */
-  int32_t reserved[3];           /* set to 0                                            */
+  int32_t n_score_layers;        /* Ls: Eq. 1-3 are averaged over Ls consecutive layers
+                                    (the layer-choice ablation's "last-5 fusion": 5);
+                                    0 counts as 1                                        */
+  int32_t score_layer_offset;    /* layers between the last scoring layer and the end of
+                                    the model: 0 = the last layer (paper default), 1 =
+                                    penultimate, L/2 = middle; offset + Ls <= L           */
+  int32_t reserved;              /* set to 0                                            */
   int64_t max_frames;            /* capacity of the store, in frames                    */
 } mukv_config;
 
@@ -148,7 +156,8 @@ typedef enum { MUKV_OPT_FLAG_MARGIN = 0, MUKV_OPT_SCORE_PATH = 1 } mukv_option;
 mukv_status mukv_set_option(mukv_ctx* ctx, int32_t option, double value);
 
 /* Sec. 3.3 + Eq. 5.  Compresses frames first_frame .. first_frame+n_frames-1.
- *   d_q [n_frames][P][Hq][D], d_k / d_v [L][n_frames][P][Hkv][D]: inputs, read only.
+ *   d_q [n_frames][P][Hq][D] ([Ls][n_frames][P][Hq][D] with Ls scoring layers), d_k / d_v
+ *   [L][n_frames][P][Hkv][D]: inputs, read only.
  *   first_frame must equal the number of frames already stored (timestamps are the
  *   absolute frame indices); 1 <= n_frames <= max_frames_per_chunk.
  *   d_kept_out  [n_frames][kappa] int32, ascending kept token ids per frame, or NULL.
@@ -306,8 +315,9 @@ mukv_status mukv_profile_read(mukv_ctx* ctx, double* ms, int64_t* launches);
  * cannot build the workspace a mukv_ctx needs, but it may still want to know which tokens of a
  * frame the method would keep.
  *
- *   cfg        shapes and method parameters; n_layers, frames_per_segment, max_frames and
- *              max_frames_per_chunk are ignored (whatever they hold).  Limits: n_frames <= MUKV_NOALLOC_MAX_FRAMES,
+ *   cfg        shapes and method parameters; n_layers, frames_per_segment, max_frames,
+ *              max_frames_per_chunk, the scoring-layer and the patch-level fields are ignored
+ *              (whatever they hold): the one layer the caller passes is scored.  Limits: n_frames <= MUKV_NOALLOC_MAX_FRAMES,
  *              n_q_heads <= MUKV_NOALLOC_MAX_Q_HEADS, n_kv_heads <= MUKV_NOALLOC_MAX_KV_HEADS,
  *              tokens_per_frame <= MUKV_MAX_TOKENS; larger requests return MUKV_E_CAPACITY.
  *   d_q        [n_frames][P][Hq][D] last-layer queries;  d_k_last [n_frames][P][Hkv][D] last-layer

@@ -167,10 +167,30 @@ def select_tokens(I, kappa: int, delta: float = TIE_EPS) -> np.ndarray:
 
 
 def score_frame(Q, K_last, alpha, causal=False, keep_low_freq=False):
-    """(I_att, I_fft, I) for one frame."""
-    ia = attention_importance(Q, K_last, causal)
-    ifr = frequency_importance(K_last)
+    """(I_att, I_fft, I) for one frame.
+
+    Q[P][Hq][D], K_last[P][Hkv][D]: one scoring layer (the paper's default: the last layer).
+    Q[Ls][P][Hq][D], K_last[Ls][P][Hkv][D]: several scoring layers (the layer-choice ablation's
+    "last-5 fusion"); both indicators are then the means of the per-layer indicators.
+    """
+    Q = np.asarray(Q)
+    K_last = np.asarray(K_last)
+    if Q.ndim == 4:
+        ia = np.mean([attention_importance(Q[l], K_last[l], causal) for l in range(Q.shape[0])], axis=0)
+        ifr = np.mean([frequency_importance(K_last[l]) for l in range(Q.shape[0])], axis=0)
+    else:
+        ia = attention_importance(Q, K_last, causal)
+        ifr = frequency_importance(K_last)
     return ia, ifr, fuse(ia, ifr, alpha, keep_low_freq)
+
+
+def score_layers(cfg: dict) -> range:
+    """Indices of the layers whose attention and keys give the indicators: n_score_layers layers
+    ending score_layer_offset layers before the end of the model (defaults: the last layer alone)."""
+    L = cfg["n_layers"]
+    Ls = max(int(cfg.get("n_score_layers", 1)), 1)
+    off = int(cfg.get("score_layer_offset", 0))
+    return range(L - off - Ls, L - off)
 
 
 def super_patch_of(token_ids, P: int, grid_width: int, split: int) -> np.ndarray:
@@ -283,7 +303,8 @@ class Store:
 
 
 def compress_chunk(store: Store, Q, K, V, select_scores=None) -> None:
-    """Append one chunk.  Q[n][P][Hq][D] (last layer), K,V[L][n][P][Hkv][D].
+    """Append one chunk.  Q[n][P][Hq][D] (queries of the scoring layer; [Ls][n][P][Hq][D] with
+    several scoring layers, see score_layers), K,V[L][n][P][Hkv][D].
 
     With select_scores[n][P] the tokens are ranked by those numbers instead of the dual signal:
     the "Rand(50%)" row of the paper's compression ablation (tokens dropped at random) is this
@@ -298,8 +319,14 @@ def compress_chunk(store: Store, Q, K, V, select_scores=None) -> None:
             I = np.asarray(select_scores, dtype=np.float64)[f]
             ia = ifr = np.zeros_like(I)
         else:
-            ia, ifr, I = score_frame(np.asarray(Q)[f], Kf[-1], cfg["alpha"],
-                                     cfg.get("attn_causal", False), cfg.get("keep_low_freq", False))
+            lay = score_layers(cfg)
+            Qa = np.asarray(Q)
+            if Qa.ndim == 5:
+                ia, ifr, I = score_frame(Qa[:, f], Kf[lay.start:lay.stop], cfg["alpha"],
+                                         cfg.get("attn_causal", False), cfg.get("keep_low_freq", False))
+            else:
+                ia, ifr, I = score_frame(Qa[f], Kf[lay.stop - 1], cfg["alpha"],
+                                         cfg.get("attn_causal", False), cfg.get("keep_low_freq", False))
         kept = select_tokens(I, cfg["keep_per_frame"], cfg.get("tie_eps", TIE_EPS))
         pk = compact_rows(Kf, kept)
         pv = compact_rows(Vf, kept)

@@ -97,7 +97,7 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
   const ScoreParams& sp = p.sp;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int NW = kCompactThreads / 32;
-  const int P = sp.P, Hkv = sp.Hkv, kappa = sp.kappa;
+  const int P = sp.P, Hkv = sp.Hkv * sp.Ls, kappa = sp.kappa;   // key heads of all scoring layers
   const bool valid = tid < P;
   float att = 0.f, fft = 0.f;
   if (valid) {
@@ -123,7 +123,7 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
     float a32 = x[0], f32 = y[0];
     for (int cc = c_first + 16; cc <= c_last; ++cc) a32 += __ldcg(cp + (long long)(cc + f) * P);
     for (int g = 8; g < Hkv; ++g) f32 += __ldcg(fp + (long long)g * P);
-    att = a32 * (1.f / (float)((long long)sp.Hq * P));
+    att = a32 * (1.f / (float)((long long)sp.Hq * sp.Ls * P));
     fft = f32 * (1.f / (float)((long long)Hkv * sp.D));
   }
   // ---- min / max of both signals over the frame (both are sums of non-negative terms)
@@ -558,7 +558,7 @@ __global__ void __launch_bounds__(kScoreThreads, 2) tail_kernel(const ScoreParam
   const int n_fl = *sp.n_flagged;
   if (n_fl == 0) return;                        // the common case: segment_kernel has done what was left
   // ---- scores of the flagged frames in double precision; the block that finishes a frame last selects
-  const int units = sp.Hq * sp.row_split;
+  const int units = sp.Ls * sp.Hq * sp.row_split;
   for (int w = blockIdx.x; w < n_fl * units; w += gridDim.x) {
     const int u = w % units;
     score_frame_block<T, double, NC>(sp, u / sp.row_split, u % sp.row_split, sp.flagged[w / units], smem_raw);

@@ -64,7 +64,7 @@ struct mukv_ctx {
   long long launches;
   int parity = 0;                        // which of the two flagged counters this chunk uses
   unsigned epoch = 0;                    // compress calls so far (tags the per-frame selection flags)
-  int C, G, esize, nc;
+  int C, G, esize, nc, Ls;
   float flag_margin, flat_ratio;
   bool force_fma = false;                // MUKV_OPT_SCORE_PATH 1: multiply-add scoring for every dtype
   bool failed = false;                   // a compress call broke off half way: only reset / stats / destroy
@@ -141,7 +141,11 @@ const char* check_config(const mukv_config* c) {
   if (c->patch_split < 0 || c->patch_split > MUKV_MAX_PATCH_SPLIT) return "patch_split out of range";
   if (c->patch_split > 0 && (c->grid_width < 1 || c->tokens_per_frame % c->grid_width != 0))
     return "grid_width must divide tokens_per_frame when patch_split > 0";
-  if (c->reserved[0] != 0 || c->reserved[1] != 0 || c->reserved[2] != 0) return "reserved fields must be 0";
+  if (c->reserved != 0) return "reserved fields must be 0";
+  if (c->n_score_layers < 0 || c->score_layer_offset < 0 ||
+      (c->n_score_layers > 1 ? c->n_score_layers : 1) + c->score_layer_offset > c->n_layers)
+    return "scoring layers must lie inside the model: n_score_layers + score_layer_offset <= n_layers";
+  if ((long long)(c->n_score_layers > 1 ? c->n_score_layers : 1) * c->n_q_heads > 4096) return "too many scoring layers";
   const long long esize = c->dtype == MUKV_BF16 ? 2 : 4;
   const long long row_vec = (long long)c->n_kv_heads * c->head_dim * esize / 16;
   if (!is_pow2(row_vec) || row_vec > 256) return "Hkv*D*sizeof(element)/16 must be a power of two <= 256";
@@ -207,11 +211,12 @@ WorkLayout work_layout(const mukv_config& c) {
   const size_t max_segs = (c.max_frames + c.frames_per_segment - 1) / c.frames_per_segment;
   size_t off = 0;
   const TcShape ts = tc_shape(c);
-  w.colsum_f = off;       off = align_up(off + F * (size_t)c.n_q_heads * P * sizeof(float));
+  const size_t Ls = c.n_score_layers > 1 ? c.n_score_layers : 1;
+  w.colsum_f = off;       off = align_up(off + F * Ls * (size_t)c.n_q_heads * P * sizeof(float));
   w.colsum_p = off;       off = align_up(off + (ts.ok ? (kPsMaxBlocks + F) * P * sizeof(float) : 0));
-  w.ifft_f = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(float));
-  w.colsum_d = off;       off = align_up(off + F * c.n_q_heads * kRefineSplit * P * sizeof(double));
-  w.ifft_d = off;         off = align_up(off + F * c.n_kv_heads * P * sizeof(double));
+  w.ifft_f = off;         off = align_up(off + F * Ls * c.n_kv_heads * P * sizeof(float));
+  w.colsum_d = off;       off = align_up(off + F * Ls * c.n_q_heads * kRefineSplit * P * sizeof(double));
+  w.ifft_d = off;         off = align_up(off + F * Ls * c.n_kv_heads * P * sizeof(double));
   w.zero_begin = off;
   w.frame_counter = off;  off = align_up(off + F * sizeof(int));
   w.flagged = off;        off = align_up(off + F * sizeof(int));
@@ -427,7 +432,7 @@ cudaError_t launch_score_ps(mukv_ctx* ctx, const ScoreParams& sp, const void* d_
   const TcShape& t = ctx->tcs;
   const int P = c.tokens_per_frame, D = c.head_dim;
   CUtensorMap qmap, kmap;
-  const long long rows = (long long)n * P;
+  const long long rows = (long long)ctx->Ls * n * P;
   if (!encode_map3(&qmap, d_q, D, c.n_q_heads, rows, ctx->G, t.tpt) ||
       !encode_map3(&kmap, k_last, D, c.n_kv_heads, rows, 1, t.npad)) {
     *why = "cuTensorMapEncodeTiled failed";
@@ -438,12 +443,12 @@ cudaError_t launch_score_ps(mukv_ctx* ctx, const ScoreParams& sp, const void* d_
   pp.sp = sp;
   pp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
   pp.tiles = t.tiles; pp.tpt = t.tpt; pp.npad = t.npad; pp.n_mt = t.n_mt; pp.n_stages = t.ps_stages;
-  pp.n_items = n * c.n_kv_heads * (t.n_mt + t.tiles);
+  pp.n_items = n * ctx->Ls * c.n_kv_heads * (t.n_mt + t.tiles);
   pp.exp2_scale = (float)(1.4426950408889634 / std::sqrt((double)D));
   pp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
   int blocks = ctx->n_sms < kPsMaxBlocks ? ctx->n_sms : kPsMaxBlocks;
   if (blocks > pp.n_items) blocks = pp.n_items;
-  *ps_grid = blocks; *ps_items = pp.n_items; *ps_ipf = c.n_kv_heads * (t.n_mt + t.tiles);
+  *ps_grid = blocks; *ps_items = pp.n_items; *ps_ipf = ctx->Ls * c.n_kv_heads * (t.n_mt + t.tiles);
   score_ps_kernel<<<blocks, kPsThreads, t.smem_ps, st>>>(pp, qmap, kmap, ctx->wmap);
   *why = "score_ps kernel";
   return cudaGetLastError();
@@ -461,7 +466,10 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   sp.alpha = c.alpha; sp.tie_eps = c.tie_eps; sp.flag_margin = ctx->flag_margin; sp.flat_ratio = ctx->flat_ratio;
   sp.first_frame = t0;
   sp.q = d_q;
-  sp.k_last = reinterpret_cast<const T*>(d_k) + (long long)(L - 1) * n * P * C;
+  sp.Ls = ctx->Ls;
+  sp.q_layer_stride = (long long)n * P * c.n_q_heads * c.head_dim;
+  sp.k_layer_stride = (long long)n * P * C;
+  sp.k_last = reinterpret_cast<const T*>(d_k) + (long long)(L - c.score_layer_offset - ctx->Ls) * n * P * C;
   sp.colsum_part = ctx->ws + ctx->wl.colsum_f;
   sp.ifft_part = ctx->ws + ctx->wl.ifft_f;
   sp.frame_counter = reinterpret_cast<int*>(ctx->ws + ctx->wl.frame_counter);
@@ -477,7 +485,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   sp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
   sp.refine = 0;
   sp.row_split = 1;
-  const dim3 grid(c.n_q_heads, n);
+  const dim3 grid(ctx->Ls * c.n_q_heads, n);
   cudaError_t e = cudaSuccess;
   const char* what = "score kernel";
   int ps_grid = 0, ps_items = 0, ps_ipf = 0;
@@ -538,7 +546,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   sp.ifft_part = ctx->ws + ctx->wl.ifft_d;
   {
     ProfScope ps(ctx, 1, st);
-    int grid_t = c.n_q_heads * kRefineSplit * (n < 2 ? n : 2);
+    int grid_t = ctx->Ls * c.n_q_heads * kRefineSplit * (n < 2 ? n : 2);
     if (grid_t < 2 * L + 1) grid_t = 2 * L + 1;
     if (grid_t > ctx->tail_capacity) grid_t = ctx->tail_capacity;
     e = launch_tail<T>(sp, cp, ctx->nc, grid_t, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
@@ -748,6 +756,7 @@ mukv_status create_impl(const mukv_config* cfg, void* d_store, size_t store_byte
   ctx->launches = 0;
   ctx->C = cfg->n_kv_heads * cfg->head_dim;
   ctx->G = cfg->n_q_heads / cfg->n_kv_heads;
+  ctx->Ls = cfg->n_score_layers > 1 ? cfg->n_score_layers : 1;
   ctx->esize = cfg->dtype == MUKV_BF16 ? 2 : 4;
   ctx->nc = pick_nc(cfg->tokens_per_frame);
   ctx->tcs = tc_shape(*cfg);
@@ -1130,6 +1139,7 @@ mukv_status noalloc_impl(const mukv_config& c, const void* d_q, const void* d_k_
   sp.P = P; sp.Hq = c.n_q_heads; sp.Hkv = c.n_kv_heads; sp.D = D; sp.G = c.n_q_heads / c.n_kv_heads;
   sp.kappa = c.keep_per_frame; sp.n_frames = n; sp.causal = c.attn_causal; sp.keep_low = c.keep_low_freq;
   sp.alpha = c.alpha; sp.tie_eps = c.tie_eps; sp.flag_margin = kFlagMargin; sp.flat_ratio = kFlatRatio;
+  sp.Ls = 1;                                             // one scoring layer: the one the caller passes
   sp.first_frame = 0;
   sp.q = d_q;
   sp.k_last = d_k_last;
@@ -1169,6 +1179,9 @@ extern "C" mukv_status mukv_score_frames_noalloc(const mukv_config* cfg, const v
     c.max_frames_per_chunk = 1;
     c.n_layers = 1;
     c.frames_per_segment = 1;
+    c.n_score_layers = 0;
+    c.score_layer_offset = 0;
+    c.patch_split = 0;
     if (const char* why = check_config(&c))
       return fail(nullptr, (c.dtype != MUKV_BF16 && c.dtype != MUKV_FP32) ? MUKV_E_DTYPE : MUKV_E_SHAPE, "%s", why);
     if (n_frames < 1) return fail(nullptr, MUKV_E_INVALID, "n_frames must be >= 1");

@@ -23,16 +23,19 @@ constexpr int kRowsPerStep = 4;
 
 struct ScoreParams {
   int P, Hq, Hkv, D, G, kappa;
+  int Ls;                       // scoring layers (Eq. 1-3 are averaged over them); >= 1
+  long long q_layer_stride;     // elements between the queries of two scoring layers (n * P * Hq * D)
+  long long k_layer_stride;     // elements between the keys of two layers (n * P * Hkv * D)
   int n_frames;                 // frames in this chunk
   int causal, keep_low;
   float alpha, tie_eps, flag_margin, flat_ratio;
   long long first_frame;
   // inputs
-  const void* q;                // [n][P][Hq][D]
-  const void* k_last;           // [n][P][Hkv][D]  (last layer of K)
+  const void* q;                // [Ls][n][P][Hq][D]
+  const void* k_last;           // [Ls][n][P][Hkv][D]  (the scoring layers of K; by default the last layer)
   // scratch
-  void* colsum_part;            // A [F][Hq * row_split][P]
-  void* ifft_part;              // A [F][Hkv][P]
+  void* colsum_part;            // A [F][Ls * Hq * row_split][P]
+  void* ifft_part;              // A [F][Ls * Hkv][P]
   int* frame_counter;           // [F], zero between launches
   int* flagged;                 // [F] frame slots needing the double pass
   int* n_flagged;               // count (written by the float pass, read by the double pass)
@@ -252,13 +255,15 @@ __device__ inline void select_frame(const ScoreParams& p, int f, const double (&
   }
 }
 
-// The work of one block: part q (of p.row_split) of the query rows of head h of frame f (a frame
-// slot of the chunk).
+// The work of one block: part q (of p.row_split) of the query rows of head hv of frame f (a frame
+// slot of the chunk); hv counts the query heads of all scoring layers, layer-major.
 template <typename T, typename A, int NC>
-__device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, int q, int f,
+__device__ __forceinline__ void score_frame_block(const ScoreParams& p, int hv, int q, int f,
                                                   unsigned char* smem_raw) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = p.P, D = p.D, Hq = p.Hq, Hkv = p.Hkv, G = p.G;
+  const int layer = hv / Hq, h = hv - layer * Hq;
+  const int HqV = p.Ls * Hq, HkvV = p.Ls * Hkv;
   const int g = h / G;
   constexpr int EPW = ElemTraits<T>::kPerWord;
   const int DS = score_row_stride<T>(D);
@@ -282,7 +287,7 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, i
   int* s_int = reinterpret_cast<int*>(smem_raw + off);
 
   // ---- stage K_g of this frame (rows padded so that 32 consecutive rows hit 32 banks)
-  const T* Kg = reinterpret_cast<const T*>(p.k_last) + ((long long)f * P * Hkv + g) * D;
+  const T* Kg = reinterpret_cast<const T*>(p.k_last) + layer * p.k_layer_stride + ((long long)f * P * Hkv + g) * D;
   {
     constexpr int VE = 16 / sizeof(T);             // elements per 16-byte vector
     const int vec_per_row = D / VE;
@@ -304,7 +309,7 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, i
   // ---- Eq. 1: column sums of the row softmax
   const uint32_t* Kw = reinterpret_cast<const uint32_t*>(Ks);
   uint32_t* Qw = reinterpret_cast<uint32_t*>(Qs) + (size_t)warp * kRowsPerStep * DW;
-  const T* Qh = reinterpret_cast<const T*>(p.q) + ((long long)f * P * Hq + h) * D;
+  const T* Qh = reinterpret_cast<const T*>(p.q) + layer * p.q_layer_stride + ((long long)f * P * Hq + h) * D;
   // 1/sqrt(D) as a two-term constant, so that single precision scales the logits without a
   // systematic relative error shared by every element
   const double scale_d = 1.0 / sqrt((double)D);
@@ -379,7 +384,7 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, i
   if (tid < P) {
     A t = (A)0;
     for (int w = 0; w < kScoreWarps; ++w) t += red[w * 256 + tid];
-    reinterpret_cast<A*>(p.colsum_part)[(((long long)f * Hq + h) * RS + q) * P + tid] = t;
+    reinterpret_cast<A*>(p.colsum_part)[(((long long)f * HqV + hv) * RS + q) * P + tid] = t;
   }
 
   // ---- Eq. 2-3: sum over the D bins of |DFT(k_j)| for this block's share of head g's tokens
@@ -410,7 +415,7 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, i
       total = warp_sum(total);
       alt = warp_sum(alt);
       if (lane == 0)
-        reinterpret_cast<A*>(p.ifft_part)[((long long)f * Hkv + g) * P + j] = total + (alt < (A)0 ? -alt : alt);
+        reinterpret_cast<A*>(p.ifft_part)[((long long)f * HkvV + layer * Hkv + g) * P + j] = total + (alt < (A)0 ? -alt : alt);
     }
   }
 
@@ -419,20 +424,20 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int h, i
   __syncthreads();
   if (tid == 0) {
     const int old = atomicAdd(p.frame_counter + f, 1);
-    s_int[63] = (old == Hq * RS - 1);
-    if (old == Hq * RS - 1) p.frame_counter[f] = 0;  // ready for the next launch
+    s_int[63] = (old == HqV * RS - 1);
+    if (old == HqV * RS - 1) p.frame_counter[f] = 0;  // ready for the next launch
   }
   __syncthreads();
   if (!s_int[63]) return;
   __threadfence();
   double att[1] = {0.0}, fft[1] = {0.0};
   if (tid < P) {
-    const A* cp = reinterpret_cast<const A*>(p.colsum_part) + (long long)f * Hq * RS * P + tid;
-    for (int hh = 0; hh < Hq * RS; ++hh) att[0] += (double)__ldcg(cp + (long long)hh * P);
-    att[0] = att[0] / (double)((long long)Hq * P);
-    const A* fp = reinterpret_cast<const A*>(p.ifft_part) + (long long)f * Hkv * P + tid;
-    for (int gg = 0; gg < Hkv; ++gg) fft[0] += (double)__ldcg(fp + (long long)gg * P);
-    fft[0] = fft[0] / (double)((long long)Hkv * D);
+    const A* cp = reinterpret_cast<const A*>(p.colsum_part) + (long long)f * HqV * RS * P + tid;
+    for (int hh = 0; hh < HqV * RS; ++hh) att[0] += (double)__ldcg(cp + (long long)hh * P);
+    att[0] = att[0] / (double)((long long)HqV * P);
+    const A* fp = reinterpret_cast<const A*>(p.ifft_part) + (long long)f * HkvV * P + tid;
+    for (int gg = 0; gg < HkvV; ++gg) fft[0] += (double)__ldcg(fp + (long long)gg * P);
+    fft[0] = fft[0] / (double)((long long)HkvV * D);
   }
   __syncthreads();
   select_frame<1>(p, f, att, fft, s_sc, s_int, s_misc);

@@ -1,7 +1,7 @@
 // Persistent, warp-specialised tensor-core scoring of a bf16 chunk (Sec. 3.3, Eq. 1-4).
 //
 // score_ps_kernel: one block of 640 threads per SM.  The chunk is a list of items, ordered by
-// (frame, key head): first the DFT row tiles of that head's keys (Eq. 2-3), then the attention
+// (frame, scoring layer, key head): first the DFT row tiles of that head's keys (Eq. 2-3), then the attention
 // row tiles (Eq. 1; the G query heads of the group are flattened with the tokens into rows: one
 // TMA box of tpt = 128/G tokens x G heads x 64 channels lands as up to 128 rows of a K-major,
 // 128-byte-swizzled operand).  Each block takes a contiguous share of the list.
@@ -55,7 +55,7 @@ struct ScorePsParams {
   ScoreParams sp;            // colsum_part: float [grid + n_frames][P] slots, ifft_part: float [F][Hkv][P]
   int tiles, tpt, npad, n_mt;
   int n_stages;              // operand stages in the ring (2 .. kPsMaxStages)
-  int n_items;               // n_frames * Hkv * (n_mt + tiles)
+  int n_items;               // n_frames * Ls * Hkv * (n_mt + tiles)
   float exp2_scale;          // log2(e) / sqrt(D)
   int* status;
 };
@@ -156,7 +156,12 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
   unsigned char* sm = smem_raw + (base - raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const ScoreParams& sp = p.sp;
-  const int P = sp.P, D = sp.D, G = sp.G, Hkv = sp.Hkv, KB = D >> 6;
+  const int P = sp.P, D = sp.D, G = sp.G, Hkv = sp.Hkv, KB = D >> 6, Ls = sp.Ls;
+  // a unit is (frame, scoring layer, key head), in that order; its rows in the K / Q maps (layer-major tensors)
+  auto unit_row = [&](int unit) {
+    const int fl = unit / Hkv;
+    return ((fl % Ls) * sp.n_frames + fl / Ls) * P;
+  };
   const int NS = p.n_stages;
   const int ipu = p.n_mt + p.tiles;                      // items per (frame, key head)
   const int n_cta = gridDim.x, cta = blockIdx.x;
@@ -211,16 +216,16 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
   bool pr_ok = true;
   if (tid == 0) {
     const int unit0 = i0 / ipu, x0 = i0 - unit0 * ipu;
-    const int f0 = unit0 / Hkv, g0 = unit0 - f0 * Hkv;
+    const int g0 = unit0 % Hkv, r0 = unit_row(unit0);
     tc::mbar_expect_tx(PS_BAR_KF(0), k_buf);
-    for (int kb = 0; kb < KB; ++kb) tc::tma_load_3d(sK + kb * k_kb, &kmap, kb * 64, g0, f0 * P, PS_BAR_KF(0));
+    for (int kb = 0; kb < KB; ++kb) tc::tma_load_3d(sK + kb * k_kb, &kmap, kb * 64, g0, r0, PS_BAR_KF(0));
     if (x0 < p.n_mt) {
       tc::mbar_expect_tx(PS_BAR_SF(0), (uint32_t)KB * (uint32_t)D * 128u);
       for (int kb = 0; kb < KB; ++kb) tc::tma_load_2d(sS + kb * st_kb, &wmap, kb * 64, 2 * D, PS_BAR_SF(0));
     } else {
       tc::mbar_expect_tx(PS_BAR_SF(0), (uint32_t)KB * (uint32_t)rows_q * 128u);
       for (int kb = 0; kb < KB; ++kb)
-        tc::tma_load_3d(sS + kb * st_kb, &qmap, kb * 64, g0 * G, f0 * P + (x0 - p.n_mt) * p.tpt, PS_BAR_SF(0));
+        tc::tma_load_3d(sS + kb * st_kb, &qmap, kb * 64, g0 * G, r0 + (x0 - p.n_mt) * p.tpt, PS_BAR_SF(0));
     }
     pr_nk = 1; pr_unit = unit0; pr_ns = 1; pr_t = 1;
     if (x0 >= p.n_mt) { pr_i = i0 + 1; pr_t = 0; }         // an attention item has this one operand load
@@ -228,14 +233,14 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
   auto produce = [&]() {
     while (pr_i < i1 && pr_ok) {
       const int unit = pr_i / ipu, x = pr_i % ipu;
-      const int f = unit / Hkv, g = unit % Hkv;
+      const int g = unit % Hkv, urow = unit_row(unit);
       if (unit != pr_unit) {
         const int kb_i = pr_nk & 1;
         pr_ok = tc::mbar_wait(PS_BAR_KE(kb_i), (uint32_t)(((pr_nk >> 1) & 1) ^ 1));
         if (!pr_ok) break;
         tc::mbar_expect_tx(PS_BAR_KF(kb_i), k_buf);
         for (int kb = 0; kb < KB; ++kb)
-          tc::tma_load_3d(sK + (uint32_t)kb_i * k_buf + kb * k_kb, &kmap, kb * 64, g, f * P, PS_BAR_KF(kb_i));
+          tc::tma_load_3d(sK + (uint32_t)kb_i * k_buf + kb * k_kb, &kmap, kb * 64, g, urow, PS_BAR_KF(kb_i));
         ++pr_nk;
         pr_unit = unit;
       }
@@ -252,7 +257,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
         } else {
           tc::mbar_expect_tx(PS_BAR_SF(s), (uint32_t)KB * (uint32_t)rows_q * 128u);
           for (int kb = 0; kb < KB; ++kb)
-            tc::tma_load_3d(dst + kb * st_kb, &qmap, kb * 64, g * G, f * P + (x - p.n_mt) * p.tpt, PS_BAR_SF(s));
+            tc::tma_load_3d(dst + kb * st_kb, &qmap, kb * 64, g * G, urow + (x - p.n_mt) * p.tpt, PS_BAR_SF(s));
         }
         ++pr_ns;
         ++pr_t;
@@ -364,7 +369,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
     for (int k = 0; k < kPsAccCols; ++k) acc[k] = 0.f;
     bool ok = true;
     int it = 0;
-    int x = i0 % ipu, g = (i0 / ipu) % Hkv, f = (i0 / ipu) / Hkv;
+    int x = i0 % ipu, g = (i0 / ipu) % Hkv, ly = ((i0 / ipu) / Hkv) % Ls, f = ((i0 / ipu) / Hkv) / Ls;
     for (int i = i0; i < i1; ++i, ++it) {
       const int b = it & 1;
       // A wait that runs out is recorded; the warp then goes on without waiting (every read
@@ -402,7 +407,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
           float t4 = 0.f;
 #pragma unroll
           for (int hh = 0; hh < kPsSplit; ++hh) t4 += xs[hh * 128 + row];
-          reinterpret_cast<float*>(sp.ifft_part)[((long long)f * Hkv + g) * P + token] = t4;
+          reinterpret_cast<float*>(sp.ifft_part)[(((long long)f * Ls + ly) * Hkv + g) * P + token] = t4;
         }
       } else {
         // ---- Eq. 1
@@ -458,7 +463,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(PS_BAR_AE(b));
 
-      const bool frame_ends = (i + 1 == i1) || (x == ipu - 1 && g == Hkv - 1);
+      const bool frame_ends = (i + 1 == i1) || (x == ipu - 1 && g == Hkv - 1 && ly == Ls - 1);
       if (frame_ends) {
         // ---- leaving frame f: this block's column sums go to its slot of the frame
 #pragma unroll
@@ -480,7 +485,10 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
       }
       if (++x == ipu) {
         x = 0;
-        if (++g == Hkv) { g = 0; ++f; }
+        if (++g == Hkv) {
+          g = 0;
+          if (++ly == Ls) { ly = 0; ++f; }
+        }
       }
     }
     if (!ok && lane == 0) atomicCAS(p.status, 0, 5);

@@ -535,3 +535,31 @@ def test_gather3_layout():
     got = O.round_to_dtype(x, np.zeros(1, dtype=np.uint16))
     want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert got.tobytes() == want.tobytes()
+
+
+# --------------------------------------------------------------------------- layer choice
+def test_scoring_layers():
+    # which layers: last (default), penultimate, middle, last-5 fusion of a 28-layer model
+    assert list(O.score_layers(dict(n_layers=28))) == [27]
+    assert list(O.score_layers(dict(n_layers=28, n_score_layers=1, score_layer_offset=1))) == [26]
+    assert list(O.score_layers(dict(n_layers=28, n_score_layers=1, score_layer_offset=14))) == [13]
+    assert list(O.score_layers(dict(n_layers=28, n_score_layers=5))) == [23, 24, 25, 26, 27]
+    # fusion = mean of the per-layer indicators; one layer given as a stack of one equals the plain call
+    Q, K = rand(3, 10, 4, 8), rand(3, 10, 2, 8)
+    ia, ifr, I = O.score_frame(Q, K, 0.7)
+    np.testing.assert_allclose(ia, np.mean([O.attention_importance(Q[l], K[l]) for l in range(3)], axis=0), rtol=1e-14)
+    np.testing.assert_allclose(ifr, np.mean([O.frequency_importance(K[l]) for l in range(3)], axis=0), rtol=1e-14)
+    assert abs(ia.sum() - 1.0) < 1e-12
+    a1 = O.score_frame(Q[:1], K[:1], 0.7)
+    a0 = O.score_frame(Q[0], K[0], 0.7)
+    for x, y in zip(a1, a0):
+        np.testing.assert_allclose(x, y, rtol=1e-14)
+    # through compress_chunk: a penultimate-layer configuration ranks by that layer's keys and queries
+    cfg = dict(CFG, n_score_layers=1, score_layer_offset=1)
+    st = O.Store(cfg)
+    L, Hq, Hkv, D, P = 3, 4, 2, 8, 12
+    Qc, Kc, Vc = rand(2, P, Hq, D), rand(L, 2, P, Hkv, D), rand(L, 2, P, Hkv, D)
+    O.compress_chunk(st, Qc, Kc, Vc)
+    for f in range(2):
+        want = O.topk_set(O.score_frame(Qc[f], Kc[1, f], 0.7)[2], 5)
+        assert st.kept[f].tolist() == want.tolist()

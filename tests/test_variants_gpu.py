@@ -80,3 +80,61 @@ def test_export_import_continues_the_stream():
     bad.magic = 1
     with pytest.raises(B.MukvError):
         B.MukvContext.from_copy(bad, b_ctx.store)
+
+
+def _layered_inputs(spec, n, Ls):
+    """Q for Ls scoring layers: layer l of the stack comes from the seeded stream of seed + 100 * l."""
+    import copy
+    qs = []
+    for l in range(Ls):
+        sp = copy.copy(spec)
+        sp.seed = spec.seed + 100 * l
+        qs.append(np.stack([sp.frame_q(t) for t in range(n)]))
+    q = np.stack(qs)                                            # [Ls][n][P][Hq][D]
+    kv = [spec.frame_kv(t) for t in range(n)]
+    k = np.stack([x[0] for x in kv], axis=1)                    # [L][n][P][Hkv][D]
+    v = np.stack([x[1] for x in kv], axis=1)
+    return q, k, v
+
+
+@pytest.mark.parametrize("name,Ls,off,opts", [("chunk7b", 5, 0, None), ("chunk7b", 1, 1, None), ("chunk7b", 1, 14, None),
+                                              ("chunk7b", 2, 3, {B.OPT_FLAG_MARGIN: 1.0}),
+                                              ("chunk7b", 3, 0, {B.OPT_SCORE_PATH: 1})])
+def test_scoring_layer_choice_bf16(name, Ls, off, opts):
+    # the layer-choice ablation: last-5 fusion, penultimate, middle; also through the double-precision
+    # pass (every frame flagged) and on the multiply-add kernel
+    n = 4
+    run = H.GpuRun(name, n_frames=n, n_score_layers=Ls, score_layer_offset=off, options=opts)
+    c = run.cfg
+    q, k, v = _layered_inputs(run.spec, n, Ls)
+    dq = H.to_device(q if Ls > 1 else q[0], True, run.device)
+    dk, dv = H.to_device(k, True, run.device), H.to_device(v, True, run.device)
+    kept = torch.full((n, c.keep_per_frame), -1, dtype=torch.int32, device=run.device)
+    sc = torch.zeros((3, n, c.tokens_per_frame), dtype=torch.float32, device=run.device)
+    run.ctx.mukv_compress_chunk(dq, dk, dv, n, 0, kept, sc)
+    torch.cuda.synchronize()
+    st = O.Store(H.oracle_cfg(c))
+    O.compress_chunk(st, q if Ls > 1 else q[0], k, v)
+    run.kept, run.scores = kept.cpu().numpy(), sc.cpu().numpy()
+    H.check_frames_against_oracle(run, st, range(n), full_layers=True)
+    stats = run.ctx.mukv_get_stats()
+    assert stats.device_status == 0
+    if opts and B.OPT_FLAG_MARGIN in opts:
+        assert stats.refined_frames == n
+
+
+def test_scoring_layer_choice_fp32():
+    spec = H.StreamSpec(seed=51, n_layers=4, n_q_heads=4, n_kv_heads=2, head_dim=64, tokens_per_frame=40, bf16=False,
+                        n_outlier=1, n_frames=3, scene_sigma=1.0, frame_sigma=0.5, scene_min=2, scene_max=3)
+    wl = dict(spec=spec, keep=11, fseg=2, chunk=3, alpha=0.7)
+    run = H.GpuRun(wl, n_score_layers=3, score_layer_offset=1)
+    q, k, v = _layered_inputs(spec, 3, 3)
+    dq, dk, dv = (H.to_device(x, False, run.device) for x in (q, k, v))
+    kept = torch.full((3, 11), -1, dtype=torch.int32, device=run.device)
+    sc = torch.zeros((3, 3, 40), dtype=torch.float32, device=run.device)
+    run.ctx.mukv_compress_chunk(dq, dk, dv, 3, 0, kept, sc)
+    torch.cuda.synchronize()
+    st = O.Store(H.oracle_cfg(run.cfg))
+    O.compress_chunk(st, q, k, v)
+    run.kept, run.scores = kept.cpu().numpy(), sc.cpu().numpy()
+    H.check_frames_against_oracle(run, st, range(3), full_layers=True)
