@@ -240,6 +240,9 @@ class Store:
     # Eq. 5 applied to every layer, K and V: float32 means over the kept tokens
     def frame_entry(self, t: int):
         kap = float(self.kept[t].shape[0])
+        if kap == 0.0:                      # segment-scope selection may leave a frame without tokens
+            z = np.zeros(self.sum_k[t].shape, dtype=np.float32)
+            return z, z.copy()
         return ((self.sum_k[t] / kap).astype(np.float32),
                 (self.sum_v[t] / kap).astype(np.float32))
 
@@ -312,6 +315,8 @@ def compress_chunk(store: Store, Q, K, V, select_scores=None) -> None:
     """
     cfg = store.cfg
     n = np.asarray(K).shape[1]
+    if int(cfg.get("keep_per_segment", 0)) > 0:
+        return _compress_chunk_segment_scope(store, Q, K, V)
     for f in range(n):
         Kf = np.asarray(K)[:, f]
         Vf = np.asarray(V)[:, f]
@@ -336,6 +341,54 @@ def compress_chunk(store: Store, Q, K, V, select_scores=None) -> None:
         store.sum_k.append(pool_rows(pk))
         store.sum_v.append(pool_rows(pv))
         store.scores.append((ia, ifr, I))
+
+
+def segment_keep_count(kappa_v: int, frames_present: int, frames_per_segment: int) -> int:
+    """Tokens kept in a segment of which only frames_present frames exist (the last one of a stream):
+    the budget kappa_v = floor(rho_v * O) of a full segment, scaled to the tokens present."""
+    return (int(kappa_v) * int(frames_present)) // int(frames_per_segment)
+
+
+def _compress_chunk_segment_scope(store: Store, Q, K, V) -> None:
+    """Segment-level DCP (Sec. 3.3: "similarly ... I_v in R^O", kappa_v = floor(rho_v * |v_t|)): the
+    indicators of every frame of a segment are computed as for a frame (attention inside the frame),
+    but the min-max normalisation of Eq. 4 and the top-kappa_v selection run over all O = F * P tokens
+    of the segment.  A frame then keeps a variable number of tokens.  The chunk must start on a
+    segment boundary and hold whole segments (the last segment of a stream may be short)."""
+    cfg = store.cfg
+    fs = cfg["frames_per_segment"]
+    P = cfg["tokens_per_frame"]
+    n = np.asarray(K).shape[1]
+    assert store.n_frames % fs == 0, "a chunk must start on a segment boundary"
+    lay = score_layers(cfg)
+    Qa = np.asarray(Q)
+    for s0 in range(0, n, fs):
+        m = min(fs, n - s0)
+        ia, ifr = [], []
+        for f in range(s0, s0 + m):
+            Kf = np.asarray(K)[:, f]
+            if Qa.ndim == 5:
+                a = np.mean([attention_importance(Qa[l, f], Kf[lay.start + l], cfg.get("attn_causal", False))
+                             for l in range(len(lay))], axis=0)
+                b = np.mean([frequency_importance(Kf[lay.start + l]) for l in range(len(lay))], axis=0)
+            else:
+                a = attention_importance(Qa[f], Kf[lay.stop - 1], cfg.get("attn_causal", False))
+                b = frequency_importance(Kf[lay.stop - 1])
+            ia.append(a)
+            ifr.append(b)
+        ia, ifr = np.concatenate(ia), np.concatenate(ifr)                  # [O]
+        I = fuse(ia, ifr, cfg["alpha"], cfg.get("keep_low_freq", False))
+        kept_all = select_tokens(I, segment_keep_count(cfg["keep_per_segment"], m, fs), cfg.get("tie_eps", TIE_EPS))
+        for i, f in enumerate(range(s0, s0 + m)):
+            kept = kept_all[(kept_all >= i * P) & (kept_all < (i + 1) * P)] - i * P
+            pk = compact_rows(np.asarray(K)[:, f], kept)
+            pv = compact_rows(np.asarray(V)[:, f], kept)
+            store.kept.append(kept)
+            store.page_k.append(pk)
+            store.page_v.append(pv)
+            store.sum_k.append(pool_rows(pk))
+            store.sum_v.append(pool_rows(pv))
+            store.scores.append((ia[i * P:(i + 1) * P], ifr[i * P:(i + 1) * P], I[i * P:(i + 1) * P]))
 
 
 # --------------------------------------------------------------------------

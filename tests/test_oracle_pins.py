@@ -563,3 +563,48 @@ def test_scoring_layers():
     for f in range(2):
         want = O.topk_set(O.score_frame(Qc[f], Kc[1, f], 0.7)[2], 5)
         assert st.kept[f].tolist() == want.tolist()
+
+
+# --------------------------------------------------------------------------- segment-level DCP
+def test_segment_scope_selection():
+    fs, P = 3, 12
+    cfg = dict(CFG, frames_per_segment=fs, keep_per_segment=O.keep_count(0.8, fs * P))
+    kv = cfg["keep_per_segment"]
+    assert kv == 28                                                     # floor(0.8 * 36)
+    L, Hq, Hkv, D = 3, 4, 2, 8
+    n = 8                                                               # two whole segments and one of two frames
+    Q, K, V = rand(n, P, Hq, D), rand(L, n, P, Hkv, D), rand(L, n, P, Hkv, D)
+    st = O.Store(cfg)
+    O.compress_chunk(st, Q[:6], K[:, :6], V[:, :6])
+    O.compress_chunk(st, Q[6:], K[:, 6:], V[:, 6:])
+    counts = [len(k) for k in st.kept]
+    assert sum(counts[0:3]) == kv and sum(counts[3:6]) == kv and sum(counts[6:8]) == (kv * 2) // 3
+    assert len(set(counts)) > 1                                         # the frames really keep different numbers
+    # by hand for the first segment: min-max over all O tokens, then the kappa_v best
+    ia = np.concatenate([O.attention_importance(Q[f], K[-1, f]) for f in range(3)])
+    ifr = np.concatenate([O.frequency_importance(K[-1, f]) for f in range(3)])
+    I = 0.7 * (ia - ia.min()) / (ia.max() - ia.min()) + 0.3 * (ifr - ifr.min()) / (ifr.max() - ifr.min())
+    want = np.sort(np.argsort(-I, kind="stable")[:kv])
+    got = np.concatenate([st.kept[f] + f * P for f in range(3)])
+    assert got.tolist() == want.tolist()
+    for f in range(3):
+        assert st.page_k[f].tobytes() == K[:, f][:, st.kept[f]].tobytes()
+    # the segment entry is the mean over all kept tokens of the segment
+    rows = np.concatenate([K[-1, f][st.kept[f]].astype(np.float64).reshape(len(st.kept[f]), -1) for f in range(3)])
+    np.testing.assert_allclose(st.segment_key(0), rows.mean(0), rtol=1e-6, atol=1e-7)
+    # rho = 1 keeps everything; identical frames keep the same token ids in each
+    st1 = O.Store(dict(cfg, keep_per_segment=fs * P))
+    O.compress_chunk(st1, Q[:3], K[:, :3], V[:, :3])
+    assert all(k.tolist() == list(range(P)) for k in st1.kept)
+    Qs, Ks = np.repeat(Q[:1], 3, axis=0), np.repeat(K[:, :1], 3, axis=1)
+    st2 = O.Store(dict(cfg, keep_per_segment=3 * 4))
+    O.compress_chunk(st2, Qs, Ks, Ks)
+    assert st2.kept[0].tolist() == st2.kept[1].tolist() == st2.kept[2].tolist() and len(st2.kept[0]) == 4
+    # a frame that keeps nothing has a zero entry and is still retrievable around
+    st3 = O.Store(dict(cfg, keep_per_segment=1))
+    O.compress_chunk(st3, Q[:3], K[:, :3], V[:, :3])
+    assert sorted(len(k) for k in st3.kept) == [0, 0, 1]
+    empty = [t for t in range(3) if len(st3.kept[t]) == 0][0]
+    assert not st3.frame_entry(empty)[0].any()
+    r = O.retrieve(st3, rand(2, Hq, D), 1, 2)
+    assert len(r["frm_idx"]) == 2
