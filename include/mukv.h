@@ -103,7 +103,11 @@ typedef struct {
   int32_t score_layer_offset;    /* layers between the last scoring layer and the end of
                                     the model: 0 = the last layer (paper default), 1 =
                                     penultimate, L/2 = middle; offset + Ls <= L           */
-  int32_t reserved;              /* set to 0                                            */
+  int32_t keep_per_segment;      /* 0: every frame keeps keep_per_frame tokens (frame-
+                                    level selection).  kappa_v > 0: segment-level selection
+                                    (Sec. 3.3, "I_v in R^O"): Eq. 4 and the top-kappa_v run
+                                    over all tokens of a segment, a frame keeps a variable
+                                    number; see mukv_compress_chunk                      */
   int64_t max_frames;            /* capacity of the store, in frames                    */
 } mukv_config;
 
@@ -168,6 +172,14 @@ mukv_status mukv_set_option(mukv_ctx* ctx, int32_t option, double value);
  * entry of every segment the chunk touches (mean over the frames present so far).
  * Frames whose selection lies too close to a tie boundary for single precision are
  * re-scored in double precision on the device before they are stored.
+ * With keep_per_segment = kappa_v > 0 the selection is made per segment: first_frame must be a
+ * multiple of frames_per_segment and the chunk must hold whole segments (a last, shorter one ends
+ * the stream and keeps kappa_v * frames / frames_per_segment tokens, rounded down); the min-max of
+ * Eq. 4 and the ranking run over all tokens of a segment in double precision; frame t keeps n_t
+ * tokens (region 10), its page is [L][2][n_t][Hkv][D], kept ids are stored and returned as
+ * [frames][P] int32 padded with -1 (d_kept_out must have that size), frames_per_segment * P <= 4096,
+ * no patch level.  Such a store is read with mukv_retrieve / mukv_retrieve3 and mukv_gather3
+ * (k_patch = 0); mukv_gather and mukv_compress_chunk_scored answer MUKV_E_UNSUPPORTED.
  * A frame whose fused scores are not all finite (Inf or NaN among its inputs) has no ranking:
  * its kappa lowest token ids are kept and device_status 7 is recorded.
  * Errors: INVALID, ALIGN, STATE (first_frame), CAPACITY (n_frames, store full), CUDA. */
@@ -269,6 +281,8 @@ mukv_status mukv_gather(mukv_ctx* ctx, const int32_t* d_frm_idx, const int32_t* 
  *        7 page table (int64 byte offsets from the store base) [max_frames]
  *        8 patch-level keys (float) [max_frames][S][C]     (patch_split > 0)
  *        9 patch-level token counts (int32) [max_frames][S]
+ *       10 tokens kept per frame (int32) [max_frames]       (keep_per_segment > 0; region 1 is then
+ *          [max_frames][P], padded with -1, and region 0 is packed pages of different lengths)
  * Returns NULL for an unknown region; *bytes (if not NULL) receives the region size. */
 void* mukv_store_region(const mukv_ctx* ctx, int32_t which, size_t* bytes);
 

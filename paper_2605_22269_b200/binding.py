@@ -44,7 +44,7 @@ class MukvConfig(C.Structure):
                 ("attn_causal", C.c_int32), ("keep_low_freq", C.c_int32),
                 ("alpha", C.c_float), ("tie_eps", C.c_float),
                 ("dtype", C.c_int32), ("patch_split", C.c_int32), ("grid_width", C.c_int32),
-                ("n_score_layers", C.c_int32), ("score_layer_offset", C.c_int32), ("reserved", C.c_int32),
+                ("n_score_layers", C.c_int32), ("score_layer_offset", C.c_int32), ("keep_per_segment", C.c_int32),
                 ("max_frames", C.c_int64)]
 
 
@@ -141,10 +141,10 @@ def _stream(stream) -> int:
 def make_config(*, n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, keep_per_frame,
                 frames_per_segment, max_frames_per_chunk, max_frames, dtype=BF16, alpha=0.7, tie_eps=1e-6,
                 attn_causal=0, keep_low_freq=0, patch_split=0, grid_width=0, n_score_layers=0,
-                score_layer_offset=0) -> MukvConfig:
+                score_layer_offset=0, keep_per_segment=0) -> MukvConfig:
     return MukvConfig(n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, keep_per_frame,
                       frames_per_segment, max_frames_per_chunk, attn_causal, keep_low_freq,
-                      alpha, tie_eps, dtype, patch_split, grid_width, n_score_layers, score_layer_offset, 0, max_frames)
+                      alpha, tie_eps, dtype, patch_split, grid_width, n_score_layers, score_layer_offset, keep_per_segment, max_frames)
 
 
 def mukv_score_frames_noalloc(cfg: MukvConfig, q, k_last, n_frames: int, kept_out=None, scores_out=None,
@@ -292,10 +292,14 @@ class MukvContext:
         c = self.cfg
         T = c.max_frames
         segs = (T + c.frames_per_segment - 1) // c.frames_per_segment
+        if which == 0 and c.keep_per_segment > 0:
+            return raw.view(self.torch_dtype)              # packed pages of different lengths: see the page table
         if which == 0:
             return raw.view(self.torch_dtype).view(T, c.n_layers, 2, c.keep_per_frame, c.n_kv_heads, c.head_dim)
         if which == 1:
-            return raw.view(torch.int32).view(T, c.keep_per_frame)
+            return raw.view(torch.int32).view(T, c.tokens_per_frame if c.keep_per_segment > 0 else c.keep_per_frame)
+        if which == 10:
+            return raw.view(torch.int32).view(T)
         if which == 2:
             return raw.view(torch.float32).view(T, c.n_layers, 2, self.C)
         if which == 3:

@@ -58,8 +58,11 @@ struct CompactParams {
   float* patch_key;               // [max_frames][S][C]
   int* patch_cnt;                 // [max_frames][S]
   int sel_mode;                   // 0: kept ids are in the store; 1: select here from the partial sums;
-                                  // 2: select here by the caller's scores
+                                  // 2: select here by the caller's scores; 3: ids and counts are in the store
+                                  // (segment-level selection)
   const float* ext_scores;        // [n_frames][P] (sel_mode 2)
+  const int* kept_count;          // [max_frames] (sel_mode 3: a frame's page holds that many tokens; ids in
+                                  // kept_store with a stride of P), else null
   int ps_grid, ps_items, ps_ipf;  // the scoring launch: blocks, items, items per frame
   unsigned* sel_flag;             // [F] (epoch << 1 | risky) once the plane-0 block has published its frame's ids
   unsigned epoch;                 // number of this call, never repeated
@@ -269,11 +272,13 @@ struct SegmentArgs {
   const double* frame_ksum;
   float* seg_entry;
   float* seg_key;
+  const int* kept_count;          // [max_frames] tokens kept per frame, or null: kappa in every frame
 };
 __device__ __forceinline__ SegmentArgs segment_args(const CompactParams& p) {
   SegmentArgs a;
   a.L = p.L; a.kappa = p.kappa; a.C = p.C; a.fseg = p.fseg; a.n_frames = p.n_frames; a.first_frame = p.first_frame;
   a.frame_entry = p.frame_entry; a.frame_ksum = p.frame_ksum; a.seg_entry = p.seg_entry; a.seg_key = p.seg_key;
+  a.kept_count = p.kept_count;
   return a;
 }
 
@@ -292,6 +297,27 @@ __device__ __noinline__ void compact_segment_plane(const SegmentArgs p, int l, i
     long long t1 = t0 + p.fseg;
     if (t1 > frames_total) t1 = frames_total;
     const int nf = (int)(t1 - t0);
+    if (p.kept_count) {
+      // frames keep different numbers of tokens (segment-level selection): the mean over all kept
+      // tokens of the segment is the count-weighted mean of the frame entries
+      long long n_tok = 0;
+      for (long long ff = t0; ff < t1; ++ff) n_tok += __ldcg(p.kept_count + ff);
+      for (int col = tid; col < C; col += kCompactThreads) {
+        if (exact) {
+          double t = 0.0;
+          for (long long ff = t0; ff < t1; ++ff) t += __ldcg(p.frame_ksum + ff * C + col);
+          const float m = n_tok ? (float)(t / (double)n_tok) : 0.f;
+          p.seg_key[u * C + col] = m;
+          p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = m;
+        } else {
+          float t = 0.f;
+          for (long long ff = t0; ff < t1; ++ff)
+            t += (float)__ldcg(p.kept_count + ff) * __ldcg(p.frame_entry + ((ff * p.L + l) * 2 + kv) * C + col);
+          p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = n_tok ? t / (float)n_tok : 0.f;
+        }
+      }
+      continue;
+    }
     if (exact) {
       for (int col = tid; col < C; col += kCompactThreads) {
         double t = 0.0;
@@ -336,20 +362,21 @@ struct CompactScratch {
   int kept[MUKV_MAX_TOKENS];
 };
 
-// Copies the kept rows (ids in sc->kept, ascending) of plane (l, kv) of chunk frame f to the
-// frame's page and writes the plane's frame entry (Eq. 5).  Run by a whole block.
+// Copies the kappa kept rows (ids in sc->kept, ascending) of plane (l, kv) of chunk frame f to the
+// frame's page (planes of kappa rows each, starting at `page`) and writes the plane's frame entry
+// (Eq. 5; zeros for a frame that keeps nothing).  Run by a whole block.
 // NV = 16-byte vectors per row; the block covers 256/NV rows per pass.
 template <typename T>
-__device__ inline void compact_plane(const CompactParams& p, int plane, int f, CompactScratch* sc) {
+__device__ inline void compact_plane(const CompactParams& p, int plane, int f, CompactScratch* sc, int kappa,
+                                     unsigned char* page) {
   constexpr int VE = 16 / sizeof(T);
   const int tid = threadIdx.x;
   const int l = plane >> 1, kv = plane & 1;
   const long long f_abs = p.first_frame + f;
-  const int kappa = p.kappa, C = p.C;
+  const int C = p.C;
   const int NV = C / VE;                        // vectors per row (power of two, <= 256)
   const int rows_per_pass = kCompactThreads / NV;
   const T* src_base = reinterpret_cast<const T*>(kv ? p.v : p.k) + ((long long)l * p.n_frames + f) * p.P * C;
-  unsigned char* page = p.store + p.sp.pages_off + f_abs * p.sp.page_bytes;
   T* dst_base = reinterpret_cast<T*>(page) + (long long)plane * kappa * C;
   const int c = tid % NV, r0 = tid / NV;
   const bool exact = (l == p.L - 1) && (kv == 0);
@@ -408,13 +435,13 @@ __device__ inline void compact_plane(const CompactParams& p, int plane, int f, C
       double t = 0.0;
       for (int g = 0; g < rows_per_pass; ++g) t += sc->red64[(g * NV + cv) * VE + ce];
       p.frame_ksum[f_abs * C + col] = t;
-      const float m = (float)(t / (double)kappa);
+      const float m = kappa ? (float)(t / (double)kappa) : 0.f;
       fe[col] = m;
       p.frame_key[f_abs * C + col] = m;
     } else {
       float t = 0.f;
       for (int g = 0; g < rows_per_pass; ++g) t += sc->red[(g * NV + cv) * VE + ce];
-      fe[col] = t / (float)kappa;
+      fe[col] = kappa ? t / (float)kappa : 0.f;
     }
   }
 }
@@ -466,6 +493,8 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(const Compa
   pdl_trigger();
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.n_flagged_next = 0;
   const long long f_abs = p.first_frame + f;
+  int kappa_f = p.kappa;
+  unsigned char* page = p.store + p.sp.pages_off + f_abs * p.sp.page_bytes;
   bool risky;
   if (p.sel_mode == 1) {
     // A block that starts after its frame's plane-0 block has published the ids (the blocks beyond
@@ -503,13 +532,20 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(const Compa
     if (bad && plane == 0 && tid == 0 && p.sp.status) atomicCAS(p.sp.status, 0, kStatusNonFinite);
     risky = false;
     __syncthreads();
+  } else if (p.sel_mode == 3) {
+    kappa_f = __ldcg(p.kept_count + f_abs);
+    kappa_f = kappa_f < 0 ? 0 : (kappa_f > p.P ? p.P : kappa_f);
+    page = p.store + __ldcg(p.sp.page_table + f_abs);
+    for (int r = tid; r < kappa_f; r += kCompactThreads) cs.kept[r] = token_id(__ldcg(p.sp.kept_store + f_abs * p.P + r), p.P);
+    risky = false;
+    __syncthreads();
   } else {
     risky = frame_is_flagged(p.sp.flagged, *p.sp.n_flagged, f);
     for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(p.sp.kept_store[f_abs * p.kappa + r], p.P);
     __syncthreads();
   }
   if (risky) return;
-  if (plane < 2 * p.L) compact_plane<T>(p, plane, f, &cs);
+  if (plane < 2 * p.L) compact_plane<T>(p, plane, f, &cs, kappa_f, page);
   else pool_patches<T>(p, f, &cs);                // the extra row of blocks when there is a patch level
 }
 
@@ -585,7 +621,7 @@ __global__ void __launch_bounds__(kScoreThreads, 2) tail_kernel(const ScoreParam
         __syncthreads();
         for (int r = tid; r < p.kappa; r += kCompactThreads) cs.kept[r] = token_id(__ldcg(sp.kept_store + f_abs * p.kappa + r), p.P);
         __syncthreads();
-        if (plane < 2 * p.L) compact_plane<T>(p, plane, f, &cs);
+        if (plane < 2 * p.L) compact_plane<T>(p, plane, f, &cs, p.kappa, p.store + sp.pages_off + f_abs * sp.page_bytes);
         else pool_patches<T>(p, f, &cs);
       }
       if (plane >= 2 * p.L) continue;

@@ -21,6 +21,7 @@
 #include "retrieve.cuh"
 #include "score.cuh"
 #include "score_ps.cuh"
+#include "segsel.cuh"
 
 using namespace mukv;
 
@@ -31,7 +32,8 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct StoreLayout {
   size_t pages, kept, frame_entry, seg_entry, frame_key, seg_key, frame_ts, page_table, frame_ksum, patch_key, patch_cnt,
-      total;
+      kept_count, total;
+  size_t pages_bytes, kept_stride;
   size_t page_bytes;
   long long max_segs;
 };
@@ -141,7 +143,13 @@ const char* check_config(const mukv_config* c) {
   if (c->patch_split < 0 || c->patch_split > MUKV_MAX_PATCH_SPLIT) return "patch_split out of range";
   if (c->patch_split > 0 && (c->grid_width < 1 || c->tokens_per_frame % c->grid_width != 0))
     return "grid_width must divide tokens_per_frame when patch_split > 0";
-  if (c->reserved != 0) return "reserved fields must be 0";
+  if (c->keep_per_segment < 0) return "keep_per_segment must be >= 0";
+  if (c->keep_per_segment > 0) {
+    if (c->patch_split != 0) return "segment-level selection has no patch level";
+    if ((long long)c->frames_per_segment * c->tokens_per_frame > kSegSelMaxTokens)
+      return "segment-level selection: frames_per_segment * tokens_per_frame must be <= 4096";
+    if (c->keep_per_segment > c->frames_per_segment * c->tokens_per_frame) return "keep_per_segment out of range";
+  }
   if (c->n_score_layers < 0 || c->score_layer_offset < 0 ||
       (c->n_score_layers > 1 ? c->n_score_layers : 1) + c->score_layer_offset > c->n_layers)
     return "scoring layers must lie inside the model: n_score_layers + score_layer_offset <= n_layers";
@@ -165,8 +173,12 @@ StoreLayout store_layout(const mukv_config& c) {
   s.max_segs = (c.max_frames + c.frames_per_segment - 1) / c.frames_per_segment;
   s.page_bytes = (size_t)c.n_layers * 2 * c.keep_per_frame * C * esize;
   size_t off = 0;
-  s.pages = off;        off = align_up(off + T * s.page_bytes);
-  s.kept = off;         off = align_up(off + T * c.keep_per_frame * sizeof(int));
+  // segment-level selection: a segment's pages share kappa_v token slots; kept ids are padded to P per frame
+  const bool seg_scope = c.keep_per_segment > 0;
+  s.pages_bytes = seg_scope ? (size_t)s.max_segs * c.keep_per_segment * c.n_layers * 2 * C * esize : T * s.page_bytes;
+  s.kept_stride = seg_scope ? (size_t)c.tokens_per_frame : (size_t)c.keep_per_frame;
+  s.pages = off;        off = align_up(off + s.pages_bytes);
+  s.kept = off;         off = align_up(off + T * s.kept_stride * sizeof(int));
   s.frame_entry = off;  off = align_up(off + T * c.n_layers * 2 * C * sizeof(float));
   s.seg_entry = off;    off = align_up(off + (size_t)s.max_segs * c.n_layers * 2 * C * sizeof(float));
   s.frame_key = off;    off = align_up(off + T * C * sizeof(float));
@@ -177,6 +189,7 @@ StoreLayout store_layout(const mukv_config& c) {
   const size_t S = (size_t)c.patch_split * c.patch_split;
   s.patch_key = off;    off = align_up(off + T * S * C * sizeof(float));
   s.patch_cnt = off;    off = align_up(off + T * S * sizeof(int));
+  s.kept_count = off;   off = align_up(off + (seg_scope ? T * sizeof(int) : 0));
   s.total = off;
   return s;
 }
@@ -339,6 +352,7 @@ cudaError_t raise_kernel_limits(int* n_sms) {
     if (e == cudaSuccess) e = raise_smem_limit(tail_fn<float>(ncs[i]), optin);
   }
   if (e == cudaSuccess) e = raise_smem_limit((const void*)rank_kernel, optin);
+  if (e == cudaSuccess) e = raise_smem_limit((const void*)segsel_kernel, optin);
   if (e == cudaSuccess) e = raise_smem_limit((const void*)score_ps_kernel, optin);
   if (e == cudaSuccess) g_limits_raised[dev] = true;
   return e;
@@ -459,6 +473,12 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
                           long long t0, int* d_kept_out, float* d_scores_out, cudaStream_t st) {
   const mukv_config& c = ctx->cfg;
   const int P = c.tokens_per_frame, L = c.n_layers, C = ctx->C;
+  const bool seg_scope = c.keep_per_segment > 0;
+  if (seg_scope) {
+    if (d_ext) return fail(ctx, MUKV_E_UNSUPPORTED, "caller-supplied scores are ranked per frame only");
+    if (t0 % c.frames_per_segment != 0)
+      return fail(ctx, MUKV_E_STATE, "segment-level selection: first_frame must be a multiple of frames_per_segment");
+  }
   ScoreParams sp;
   memset(&sp, 0, sizeof sp);
   sp.P = P; sp.Hq = c.n_q_heads; sp.Hkv = c.n_kv_heads; sp.D = c.head_dim; sp.G = ctx->G;
@@ -489,7 +509,33 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   cudaError_t e = cudaSuccess;
   const char* what = "score kernel";
   int ps_grid = 0, ps_items = 0, ps_ipf = 0;
-  if (!d_ext) {
+  if (seg_scope) {
+    // every frame's indicators in double precision (no per-frame selection), then one block per segment
+    ScoreParams sd = sp;
+    sd.no_select = 1;
+    sd.row_split = kRefineSplit;
+    sd.colsum_part = ctx->ws + ctx->wl.colsum_d;
+    sd.ifft_part = ctx->ws + ctx->wl.ifft_d;
+    {
+      ProfScope ps(ctx, 0, st);
+      e = launch_score<T, double>(sd, ctx->nc, dim3(ctx->Ls * c.n_q_heads * kRefineSplit, n),
+                                  score_smem_bytes<T, double>(P, c.head_dim), st);
+    }
+    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "score kernel: %s", cudaGetErrorString(e));
+    SegSelParams gp;
+    memset(&gp, 0, sizeof gp);
+    gp.sp = sd;
+    gp.fseg = c.frames_per_segment; gp.kappa_v = c.keep_per_segment;
+    gp.token_bytes = (long long)L * 2 * C * ctx->esize;
+    gp.kept_count = reinterpret_cast<int*>(ctx->store + ctx->sl.kept_count);
+    const int n_seg = (n + c.frames_per_segment - 1) / c.frames_per_segment;
+    const int seg_tokens = (n < c.frames_per_segment ? n : c.frames_per_segment) * P;
+    {
+      ProfScope ps(ctx, 1, st);
+      e = launch_k(segsel_kernel, dim3(n_seg), kSegSelThreads, segsel_smem_bytes(seg_tokens), st, false, gp);
+    }
+    if (e != cudaSuccess) return broke_off(ctx, "segment selection kernel", e);
+  } else if (!d_ext) {
     ProfScope ps(ctx, 0, st);
     if (ctx->tcs.ok && !ctx->force_fma)
       e = launch_score_ps(ctx, sp, d_q, sp.k_last, n, st, &what, &ps_grid, &ps_items, &ps_ipf);
@@ -519,7 +565,8 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   cp.patch_split = c.patch_split; cp.grid_width = c.grid_width;
   cp.patch_key = reinterpret_cast<float*>(ctx->store + ctx->sl.patch_key);
   cp.patch_cnt = reinterpret_cast<int*>(ctx->store + ctx->sl.patch_cnt);
-  cp.sel_mode = d_ext ? 2 : ps_grid > 0 ? 1 : 0;
+  cp.sel_mode = seg_scope ? 3 : d_ext ? 2 : ps_grid > 0 ? 1 : 0;
+  cp.kept_count = seg_scope ? reinterpret_cast<const int*>(ctx->store + ctx->sl.kept_count) : nullptr;
   cp.ext_scores = d_ext;
   cp.ps_grid = ps_grid; cp.ps_items = ps_items; cp.ps_ipf = ps_ipf;
   cp.sp = sp;
@@ -544,7 +591,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   sp.row_split = kRefineSplit;
   sp.colsum_part = ctx->ws + ctx->wl.colsum_d;
   sp.ifft_part = ctx->ws + ctx->wl.ifft_d;
-  {
+  if (!seg_scope) {                                      // (segment-level selection flags nothing)
     ProfScope ps(ctx, 1, st);
     int grid_t = ctx->Ls * c.n_q_heads * kRefineSplit * (n < 2 ? n : 2);
     if (grid_t < 2 * L + 1) grid_t = 2 * L + 1;
@@ -924,7 +971,10 @@ int64_t mukv_decode3_tokens(const mukv_ctx* ctx, int32_t k_seg, int32_t k_frm, i
     pmax = (long long)((rows + c.patch_split - 1) / c.patch_split) * ((c.grid_width + c.patch_split - 1) / c.patch_split);
     if (pmax > c.keep_per_frame) pmax = c.keep_per_frame;
   }
-  return (long long)k_seg + (long long)k_frm * c.keep_per_frame + (long long)k_patch * pmax;
+  long long per_frame = c.keep_per_frame;
+  if (c.keep_per_segment > 0)                            // a frame may hold up to a whole segment's budget
+    per_frame = c.keep_per_segment < c.tokens_per_frame ? c.keep_per_segment : c.tokens_per_frame;
+  return (long long)k_seg + (long long)k_frm * per_frame + (long long)k_patch * pmax;
 }
 
 mukv_status mukv_gather3(mukv_ctx* ctx, const int32_t* d_seg_idx, const int32_t* d_frm_idx, const int32_t* d_patch_idx,
@@ -961,6 +1011,8 @@ mukv_status mukv_gather3(mukv_ctx* ctx, const int32_t* d_seg_idx, const int32_t*
     gp.kept_store = reinterpret_cast<const int*>(ctx->store + ctx->sl.kept);
     gp.seg_entry = reinterpret_cast<const float*>(ctx->store + ctx->sl.seg_entry);
     gp.patch_cnt = reinterpret_cast<const int*>(ctx->store + ctx->sl.patch_cnt);
+    gp.kept_count = c.keep_per_segment > 0 ? reinterpret_cast<const int*>(ctx->store + ctx->sl.kept_count) : nullptr;
+    gp.kept_stride = (int)ctx->sl.kept_stride;
     gp.decode = static_cast<unsigned char*>(d_decode);
     gp.decode_stride = decode_stride_bytes;
     gp.ntok = d_ntok; gp.tok_meta = d_tok_meta;
@@ -989,6 +1041,8 @@ mukv_status mukv_gather(mukv_ctx* ctx, const int32_t* d_frm_idx, const int32_t* 
     if (!d_frm_idx || !d_counts || !d_decode) return fail(ctx, MUKV_E_INVALID, "null argument");
     if (!aligned4(d_frm_idx) || !aligned4(d_counts) || !aligned16(d_decode) || !aligned4(d_tok_meta))
       return fail(ctx, MUKV_E_ALIGN, "d_decode must be 16-byte aligned, index arrays 4-byte aligned");
+    if (ctx->cfg.keep_per_segment > 0)
+      return fail(ctx, MUKV_E_UNSUPPORTED, "pages have different lengths (segment-level selection): use mukv_gather3");
     if (nq < 1 || k_frm < 1) return fail(ctx, MUKV_E_INVALID, "nq and k_frm must be >= 1");
     if (nq > MUKV_MAX_QUESTIONS || k_frm > MUKV_MAX_TOPK)
       return fail(ctx, MUKV_E_CAPACITY, "nq or k_frm too large");
@@ -1031,8 +1085,9 @@ void* mukv_store_region(const mukv_ctx* ctx, int32_t which, size_t* bytes) {
   const size_t T = (size_t)c.max_frames, C = (size_t)ctx->C;
   size_t off = 0, sz = 0;
   switch (which) {
-    case 0: off = s.pages; sz = T * s.page_bytes; break;
-    case 1: off = s.kept; sz = T * c.keep_per_frame * sizeof(int); break;
+    case 0: off = s.pages; sz = s.pages_bytes; break;
+    case 1: off = s.kept; sz = T * s.kept_stride * sizeof(int); break;
+    case 10: if (c.keep_per_segment <= 0) return nullptr; off = s.kept_count; sz = T * sizeof(int); break;
     case 2: off = s.frame_entry; sz = T * c.n_layers * 2 * C * sizeof(float); break;
     case 3: off = s.seg_entry; sz = (size_t)s.max_segs * c.n_layers * 2 * C * sizeof(float); break;
     case 4: off = s.frame_key; sz = T * C * sizeof(float); break;
@@ -1064,6 +1119,12 @@ mukv_status mukv_get_stats(mukv_ctx* ctx, mukv_stats* out, mukv_stream stream) {
   out->kept_tokens = ctx->frames * c.keep_per_frame;
   out->page_bytes = (long long)ctx->sl.page_bytes;
   out->store_bytes_used = ctx->frames * (long long)ctx->sl.page_bytes;
+  if (c.keep_per_segment > 0) {
+    const long long fs = c.frames_per_segment, full = ctx->frames / fs, rest = ctx->frames % fs;
+    out->kept_tokens = full * c.keep_per_segment + (long long)c.keep_per_segment * rest / fs;
+    out->page_bytes = 0;                                 // pages have different lengths
+    out->store_bytes_used = out->kept_tokens * c.n_layers * 2 * ctx->C * ctx->esize;
+  }
   out->refined_frames = refined;
   out->kernel_launches = ctx->launches;
   out->device_status = dev_status;

@@ -686,6 +686,8 @@ struct Gather3Params {
   const unsigned char* store; const long long* page_table; const int* kept_store;
   const float* seg_entry;                  // [segments][L][2][C]
   const int* patch_cnt;                    // [frames][S]
+  const int* kept_count;                   // [frames] tokens in a frame's page, or null: kappa in every page
+  int kept_stride;                         // ints per frame in kept_store
   unsigned char* decode; long long decode_stride;
   int* ntok; int* tok_meta;
 };
@@ -702,6 +704,7 @@ __device__ __forceinline__ void copy_run16(unsigned char* dst, const unsigned ch
 template <typename T>
 __global__ void __launch_bounds__(256) gather3_kernel(const Gather3Params p) {
   __shared__ int s_off[MUKV_MAX_TOPK + 1];                 // first row of each selected patch block
+  __shared__ int s_row0;
   const long long planes = (long long)p.L * 2;
   const int upp = p.k_frm + 1;                             // units per (question, plane)
   const long long n_units = (long long)p.nq * planes * upp;
@@ -718,12 +721,25 @@ __global__ void __launch_bounds__(256) gather3_kernel(const Gather3Params p) {
     if (slot < p.k_frm) {
       if (slot >= c_frm) continue;
       const int f = p.frm_idx[(long long)qi * p.k_frm + slot];
-      const int row0 = c_seg + slot * p.kappa;
-      copy_run16(dplane + (long long)row0 * row_bytes, p.store + p.page_table[f] + (long long)plane * run_bytes, run_bytes);
+      int row0 = c_seg + slot * p.kappa, rows = p.kappa;
+      if (p.kept_count) {
+        // pages of different lengths: this frame's rows start behind those of the frames before it
+        __syncthreads();
+        if (threadIdx.x == 0) {
+          int off = c_seg;
+          for (int i = 0; i < slot; ++i) off += p.kept_count[p.frm_idx[(long long)qi * p.k_frm + i]];
+          s_row0 = off;
+        }
+        __syncthreads();
+        row0 = s_row0;
+        rows = p.kept_count[f];
+      }
+      const long long fbytes = (long long)rows * row_bytes;
+      copy_run16(dplane + (long long)row0 * row_bytes, p.store + p.page_table[f] + (long long)plane * fbytes, fbytes);
       if (plane == 0 && meta) {
-        for (int t = threadIdx.x; t < p.kappa; t += blockDim.x) {
+        for (int t = threadIdx.x; t < rows; t += blockDim.x) {
           meta[(row0 + t) * 2] = f;
-          meta[(row0 + t) * 2 + 1] = p.kept_store[(long long)f * p.kappa + t];
+          meta[(row0 + t) * 2 + 1] = p.kept_store[(long long)f * p.kept_stride + t];
         }
       }
       continue;
@@ -743,6 +759,10 @@ __global__ void __launch_bounds__(256) gather3_kernel(const Gather3Params p) {
     __syncthreads();
     if (threadIdx.x == 0) {
       int off = c_seg + c_frm * p.kappa;
+      if (p.kept_count) {
+        off = c_seg;
+        for (int i = 0; i < c_frm; ++i) off += p.kept_count[p.frm_idx[(long long)qi * p.k_frm + i]];
+      }
       for (int i = 0; i < c_pat; ++i) {
         s_off[i] = off;
         off += p.patch_cnt[p.pat_idx[(long long)qi * p.k_pat + i]];

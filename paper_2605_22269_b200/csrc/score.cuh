@@ -47,6 +47,7 @@ struct ScoreParams {
   long long* page_table;        // [max_frames]
   long long pages_off, page_bytes;
   int* status;                  // device event word (0 = nothing recorded); see mukv_stats.device_status
+  int no_select;                // 1: only the partial sums are wanted (the selection runs over a whole segment elsewhere)
   int refine;                   // 1: frames come from the flagged list, no further flagging
   int row_split;                // blocks that share a query head, each a range of query rows (>= 1)
 };
@@ -428,7 +429,7 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int hv, 
     if (old == HqV * RS - 1) p.frame_counter[f] = 0;  // ready for the next launch
   }
   __syncthreads();
-  if (!s_int[63]) return;
+  if (!s_int[63] || p.no_select) return;
   __threadfence();
   double att[1] = {0.0}, fft[1] = {0.0};
   if (tid < P) {
