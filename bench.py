@@ -25,8 +25,8 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch on a 16-frame chunk of this workload
-# (ncu capture summarised in profiles/score_ps_kernel_chunk16.md)
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture) of one launch of the
+# kernel on a 16-frame chunk of this workload; reported as `roofline.traffic`
 SCORE_TRAFFIC_BYTES = 25857792
 COMPACT_TRAFFIC_BYTES = 45182464 + 3919104
 
@@ -228,14 +228,15 @@ def main():
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_calls + 2)]
     step_no = [0]
 
-    def one_step():
+    def one_step(l2=None):
         """Returns (compress ms, retrieve ms, gather ms) of this step, device time."""
+        l2 = l2 or args.l2
         ctx.mukv_reset()
         for i, t0 in enumerate(range(0, T, chunk)):
             n = min(chunk, T - t0)
             q, k, v = bufs[n]
             gs.fill(t0, n, q, k, v)
-            if args.l2 == "flush":
+            if l2 == "flush":
                 flush.zero_()
             ev[i][0].record()
             ctx.mukv_compress_chunk(q, k, v, n, t0, kept[:n], None)
@@ -274,6 +275,10 @@ def main():
     fps = D.throughput(c_ms, T * args.steps, dev)
     rps = D.throughput(r_ms + g_ms, nq * args.steps, dev)
     step_ms, _ = D.combine((c_ms + r_ms + g_ms) / args.steps, 0, dev)
+
+    # ---- the other L2 mode, one extra step, so that both numbers stand side by side
+    other = "flush" if args.l2 == "inputs" else "inputs"
+    l2_modes = {args.l2: c_ms / args.steps, other: one_step(other)[0]}
 
     # ---- per-kernel durations, measured live with events around every launch (one extra step)
     ctx.mukv_profile_enable(True)
@@ -374,6 +379,7 @@ def main():
                               "larger than the 126 MB L2; the retrieval calls follow a 256 MiB memset")},
             "retrievals_per_s": rps,
             "retrieve_ms": r_ms / args.steps, "gather_ms": g_ms / args.steps, "compress_ms": c_ms / args.steps,
+            "compress_ms_by_l2_mode": l2_modes,
             "wall_s_per_step_with_generation": wall / args.steps,
             "path_algorithmic_gbs": {"compress": path_gbs, "compress_frac_of_peak": path_gbs / peaks["hbm_gbs"],
                                      "retrieve_gather": retr_gbs,

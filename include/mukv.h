@@ -313,8 +313,8 @@ mukv_status mukv_get_stats(mukv_ctx* ctx, mukv_stats* out, mukv_stream stream);
  * context is bracketed by a pair of CUDA events on the call's stream (host objects; no device
  * memory).  mukv_profile_read waits for the recorded events, adds up the elapsed milliseconds
  * and the launch counts per kernel kind since the last read, and forgets them.
- * Kinds: 0 score, 1 refine (double-precision score), 2 compact+pool, 3 segment pool,
- *        4 question pool, 5 index scan, 6 rank, 7 gather. */
+ * Kinds: 0 score, 1 tail (double-precision pass of flagged frames; segment-level selection),
+ *        2 compact+pool, 3 segment pool, 4 question pool, 5 index scan, 6 rank, 7 gather. */
 #define MUKV_PROF_KINDS 8
 mukv_status mukv_profile_enable(mukv_ctx* ctx, int32_t on);
 mukv_status mukv_profile_read(mukv_ctx* ctx, double* ms, int64_t* launches);

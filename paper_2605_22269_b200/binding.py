@@ -28,7 +28,7 @@ EXPORTS = ["mukv_store_bytes", "mukv_workspace_bytes", "mukv_create", "mukv_dest
            "mukv_compress_chunk", "mukv_compress_chunk_scored", "mukv_export_header", "mukv_import",
            "mukv_retrieve3", "mukv_gather3", "mukv_decode3_tokens", "mukv_retrieve", "mukv_gather", "mukv_store_region", "mukv_get_stats",
            "mukv_last_error", "mukv_profile_enable", "mukv_profile_read", "mukv_score_frames_noalloc"]
-PROF_KINDS = ["score", "refine", "compact", "segment", "qpool", "scan", "rank", "gather"]
+PROF_KINDS = ["score", "tail", "compact", "segment", "qpool", "scan", "rank", "gather"]
 
 
 class MukvError(RuntimeError):
