@@ -15,8 +15,7 @@
 // whole device, where a selection inside the scoring kernel left one block per frame working while
 // all others had finished.  After the other scoring kernels the ids are read from the store
 // (sel_mode 0).  Either way a frame whose lowest kept and highest dropped score are closer than
-// tie_eps + flag_margin is skipped here: the double-precision pass that follows decides it, and
-// segment_kernel then compacts it.
+// tie_eps + flag_margin is skipped here: tail_kernel decides it in double precision and compacts it.
 //
 // What has to wait for every frame of the chunk runs in two small launches behind compact_kernel.
 // segment_kernel: the segment entries (Eq. 5 at segment level) when no frame was flagged: one
