@@ -358,6 +358,28 @@ def main():
                "d2h_bytes_per_step": int(hkept.numel() * 4),
                "note": f"{n_e2e} chunks: pinned-host Q/K/V copied in, compressed, kept ids copied out; a step here "
                        f"is one chunk of {n} frames"}
+        # the retrieval half end to end: question tokens from pinned host memory, selected ids and counts back to
+        # the host, the gathered context stays on the device (it is the decoder's input)
+        hqtok = torch.empty(qtok.shape, dtype=qtok.dtype, pin_memory=True)
+        hqtok.copy_(qtok)
+        hfrm = torch.empty(frm_idx.shape, dtype=frm_idx.dtype, pin_memory=True)
+        hcnt = torch.empty(counts.shape, dtype=counts.dtype, pin_memory=True)
+        one_step()                                            # a full store again
+        torch.cuda.synchronize()
+        n_rep = 5
+        t0 = time.perf_counter()
+        for i in range(n_rep):
+            qtok.copy_(hqtok, non_blocking=True)
+            ctx.mukv_retrieve(qtok, offs, None, k_seg, k_frm, 0, lam, B.RETR_SEMI, seg_idx, frm_idx, seg_sc, frm_sc,
+                              counts)
+            ctx.mukv_gather(frm_idx, counts, nq, k_frm, decode[i % n_sets], stride, None)
+            hfrm.copy_(frm_idx, non_blocking=True)
+            hcnt.copy_(counts, non_blocking=True)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        e2e["retrievals_per_s"] = D.throughput(dt * 1e3, n_rep * nq, dev)
+        e2e["retrieval_h2d_bytes_per_step"] = int(hqtok.numel() * hqtok.element_size())
+        e2e["retrieval_d2h_bytes_per_step"] = int(hfrm.numel() * 4 + hcnt.numel() * 4)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
