@@ -50,27 +50,38 @@ def as_f64(x: np.ndarray) -> np.ndarray:
 # --------------------------------------------------------------------------
 # Sec. 3.3, Eq. 1: attention-based indicator
 # --------------------------------------------------------------------------
-def attention_importance(Q, K_last, causal: bool = False) -> np.ndarray:
+def attention_importance(Q, K_last, causal: bool = False, K_past=None) -> np.ndarray:
     """I_att[j] = 1/(H*P) * sum_h sum_i A_h[i, j]   (Eq. 1).
 
     A_h = row-softmax(Q_h K_g^T / sqrt(D)) over the P tokens of the frame,
     g = h // (Hq/Hkv).  With causal=True query i only sees keys j <= i.
+
+    K_past [n_past][Hkv][D] (Sec. 3.2: the prefill of a time step also sees the cached keys of the same
+    granularity): the softmax of every query then runs over the past keys and the frame's own tokens
+    (past keys are visible to every query, causal or not); the importance is still that of the
+    frame's own P tokens, so it sums to less than 1 by the attention mass the past takes.
     """
     Q = as_f64(Q)
     K = as_f64(K_last)
     P, Hq, D = Q.shape
     Hkv = K.shape[1]
     G = Hq // Hkv
+    n_past = 0
+    if K_past is not None and np.asarray(K_past).shape[0] > 0:
+        Kp = as_f64(K_past)
+        n_past = Kp.shape[0]
+        K = np.concatenate([Kp, K], axis=0)
     col = np.zeros(P, dtype=np.float64)
     for h in range(Hq):
         g = h // G
-        z = (Q[:, h, :] @ K[:, g, :].T) / np.sqrt(float(D))       # [i][j]
+        z = (Q[:, h, :] @ K[:, g, :].T) / np.sqrt(float(D))       # [i][past ++ own j]
         if causal:
-            z = np.where(np.tril(np.ones((P, P), dtype=bool)), z, -np.inf)
+            vis = np.concatenate([np.ones((P, n_past), dtype=bool), np.tril(np.ones((P, P), dtype=bool))], axis=1)
+            z = np.where(vis, z, -np.inf)
         m = z.max(axis=1, keepdims=True)
         e = np.exp(z - m)
         a = e / e.sum(axis=1, keepdims=True)
-        col += a.sum(axis=0)
+        col += a[:, n_past:].sum(axis=0)
     return col / float(Hq * P)
 
 
@@ -166,7 +177,7 @@ def select_tokens(I, kappa: int, delta: float = TIE_EPS) -> np.ndarray:
     return topk_set(I, kappa, delta)
 
 
-def score_frame(Q, K_last, alpha, causal=False, keep_low_freq=False):
+def score_frame(Q, K_last, alpha, causal=False, keep_low_freq=False, K_past=None):
     """(I_att, I_fft, I) for one frame.
 
     Q[P][Hq][D], K_last[P][Hkv][D]: one scoring layer (the paper's default: the last layer).
@@ -176,12 +187,25 @@ def score_frame(Q, K_last, alpha, causal=False, keep_low_freq=False):
     Q = np.asarray(Q)
     K_last = np.asarray(K_last)
     if Q.ndim == 4:
-        ia = np.mean([attention_importance(Q[l], K_last[l], causal) for l in range(Q.shape[0])], axis=0)
+        ia = np.mean([attention_importance(Q[l], K_last[l], causal, None if K_past is None else K_past[l])
+                      for l in range(Q.shape[0])], axis=0)
         ifr = np.mean([frequency_importance(K_last[l]) for l in range(Q.shape[0])], axis=0)
     else:
-        ia = attention_importance(Q, K_last, causal)
+        ia = attention_importance(Q, K_last, causal, K_past)
         ifr = frequency_importance(K_last)
     return ia, ifr, fuse(ia, ifr, alpha, keep_low_freq)
+
+
+def past_keys(store, t_chunk: int, cfg: dict):
+    """Cached keys the chunk's queries also attend to (past_frames = W > 0): the kept keys, in the
+    scoring layers, of the W most recent frames stored before the chunk (a chunk is one time step:
+    its frames do not see one another's cache).  [Ls][n_past][Hkv][D] in storage form, or None."""
+    W = int(cfg.get("past_frames", 0))
+    t0 = max(0, t_chunk - W)
+    if W <= 0 or t0 == t_chunk:
+        return None
+    lay = score_layers(cfg)
+    return np.stack([np.concatenate([store.page_k[t][l] for t in range(t0, t_chunk)], axis=0) for l in lay])
 
 
 def score_layers(cfg: dict) -> range:
@@ -317,6 +341,7 @@ def compress_chunk(store: Store, Q, K, V, select_scores=None) -> None:
     n = np.asarray(K).shape[1]
     if int(cfg.get("keep_per_segment", 0)) > 0:
         return _compress_chunk_segment_scope(store, Q, K, V)
+    t_chunk = store.n_frames                        # frames stored before this chunk
     for f in range(n):
         Kf = np.asarray(K)[:, f]
         Vf = np.asarray(V)[:, f]
@@ -326,12 +351,14 @@ def compress_chunk(store: Store, Q, K, V, select_scores=None) -> None:
         else:
             lay = score_layers(cfg)
             Qa = np.asarray(Q)
+            past = past_keys(store, t_chunk, cfg)
             if Qa.ndim == 5:
                 ia, ifr, I = score_frame(Qa[:, f], Kf[lay.start:lay.stop], cfg["alpha"],
-                                         cfg.get("attn_causal", False), cfg.get("keep_low_freq", False))
+                                         cfg.get("attn_causal", False), cfg.get("keep_low_freq", False), past)
             else:
                 ia, ifr, I = score_frame(Qa[f], Kf[lay.stop - 1], cfg["alpha"],
-                                         cfg.get("attn_causal", False), cfg.get("keep_low_freq", False))
+                                         cfg.get("attn_causal", False), cfg.get("keep_low_freq", False),
+                                         None if past is None else past[-1])
         kept = select_tokens(I, cfg["keep_per_frame"], cfg.get("tie_eps", TIE_EPS))
         pk = compact_rows(Kf, kept)
         pv = compact_rows(Vf, kept)

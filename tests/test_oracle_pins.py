@@ -608,3 +608,39 @@ def test_segment_scope_selection():
     assert not st3.frame_entry(empty)[0].any()
     r = O.retrieve(st3, rand(2, Hq, D), 1, 2)
     assert len(r["frm_idx"]) == 2
+
+
+# --------------------------------------------------------------------------- past keys in the softmax
+def test_attention_with_past_keys():
+    import torch
+    P, Hq, Hkv, D, n_past = 9, 4, 2, 8, 5
+    Q, K, Kp = rand(P, Hq, D), rand(P, Hkv, D), rand(n_past, Hkv, D)
+    for causal in (False, True):
+        got = O.attention_importance(Q, K, causal, Kp)
+        # library softmax over the concatenated keys, own columns summed
+        kk = torch.from_numpy(np.concatenate([Kp, K]).astype(np.float64)).repeat_interleave(Hq // Hkv, dim=1)
+        z = torch.einsum("ihd,jhd->hij", torch.from_numpy(Q.astype(np.float64)), kk) / np.sqrt(D)
+        if causal:
+            vis = torch.cat([torch.ones(P, n_past, dtype=torch.bool), torch.tril(torch.ones(P, P, dtype=torch.bool))], 1)
+            z = z.masked_fill(~vis, float("-inf"))
+        a = torch.softmax(z, dim=-1)
+        np.testing.assert_allclose(got, a[:, :, n_past:].sum(dim=(0, 1)).numpy() / (Hq * P), rtol=1e-12)
+        assert got.sum() < 1.0                                     # the past takes part of the attention mass
+    assert np.allclose(O.attention_importance(Q, K, False, Kp[:0]), O.attention_importance(Q, K))
+    # a past key far more similar to every query than any own key takes nearly all the mass
+    big = np.zeros((1, Hkv, D), dtype=np.float32)
+    Qc = np.ones((P, Hq, D), dtype=np.float32)
+    big[:] = 50.0
+    assert O.attention_importance(Qc, K, False, big).sum() < 1e-6
+    # through the store: the second chunk sees the kept keys of the last W frames before it, not its own frames
+    cfg = dict(CFG, past_frames=2)
+    st = O.Store(cfg)
+    L, P2 = 3, 12
+    Qs, Ks, Vs = rand(5, P2, 4, 8), rand(L, 5, P2, 2, 8), rand(L, 5, P2, 2, 8)
+    O.compress_chunk(st, Qs[:3], Ks[:, :3], Vs[:, :3])
+    O.compress_chunk(st, Qs[3:], Ks[:, 3:], Vs[:, 3:])
+    past = np.concatenate([st.page_k[1][-1], st.page_k[2][-1]], axis=0)
+    for f in (3, 4):
+        want = O.topk_set(O.score_frame(Qs[f], Ks[-1, f], 0.7, K_past=past)[2], 5)
+        assert st.kept[f].tolist() == want.tolist()
+    assert st.kept[0].tolist() == O.topk_set(O.score_frame(Qs[0], Ks[-1, 0], 0.7)[2], 5).tolist()
