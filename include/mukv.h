@@ -109,6 +109,12 @@ typedef struct {
                                     over all tokens of a segment, a frame keeps a variable
                                     number; see mukv_compress_chunk                      */
   int64_t max_frames;            /* capacity of the store, in frames                    */
+  int32_t past_frames;           /* W: the queries of a chunk also attend to the kept keys
+                                    of the W most recent frames stored before the chunk
+                                    (Sec. 3.2: past KV of the same granularity); P + W *
+                                    kappa <= 256; such a context scores on the multiply-add
+                                    kernels (every dtype); not with keep_per_segment; 0 = none */
+  int32_t reserved;              /* set to 0                                            */
 } mukv_config;
 
 typedef struct {

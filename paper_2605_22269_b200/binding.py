@@ -45,7 +45,7 @@ class MukvConfig(C.Structure):
                 ("alpha", C.c_float), ("tie_eps", C.c_float),
                 ("dtype", C.c_int32), ("patch_split", C.c_int32), ("grid_width", C.c_int32),
                 ("n_score_layers", C.c_int32), ("score_layer_offset", C.c_int32), ("keep_per_segment", C.c_int32),
-                ("max_frames", C.c_int64)]
+                ("max_frames", C.c_int64), ("past_frames", C.c_int32), ("reserved", C.c_int32)]
 
 
 class MukvRetrParams(C.Structure):
@@ -141,10 +141,10 @@ def _stream(stream) -> int:
 def make_config(*, n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, keep_per_frame,
                 frames_per_segment, max_frames_per_chunk, max_frames, dtype=BF16, alpha=0.7, tie_eps=1e-6,
                 attn_causal=0, keep_low_freq=0, patch_split=0, grid_width=0, n_score_layers=0,
-                score_layer_offset=0, keep_per_segment=0) -> MukvConfig:
+                score_layer_offset=0, keep_per_segment=0, past_frames=0) -> MukvConfig:
     return MukvConfig(n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, keep_per_frame,
                       frames_per_segment, max_frames_per_chunk, attn_causal, keep_low_freq,
-                      alpha, tie_eps, dtype, patch_split, grid_width, n_score_layers, score_layer_offset, keep_per_segment, max_frames)
+                      alpha, tie_eps, dtype, patch_split, grid_width, n_score_layers, score_layer_offset, keep_per_segment, max_frames, past_frames, 0)
 
 
 def mukv_score_frames_noalloc(cfg: MukvConfig, q, k_last, n_frames: int, kept_out=None, scores_out=None,

@@ -67,6 +67,7 @@ struct mukv_ctx {
   int parity = 0;                        // which of the two flagged counters this chunk uses
   unsigned epoch = 0;                    // compress calls so far (tags the per-frame selection flags)
   int C, G, esize, nc, Ls;
+  int key_rows;                          // key rows of the multiply-add scoring kernel: P + past_frames * kappa
   float flag_margin, flat_ratio;
   bool force_fma = false;                // MUKV_OPT_SCORE_PATH 1: multiply-add scoring for every dtype
   bool failed = false;                   // a compress call broke off half way: only reset / stats / destroy
@@ -143,6 +144,13 @@ const char* check_config(const mukv_config* c) {
   if (c->patch_split < 0 || c->patch_split > MUKV_MAX_PATCH_SPLIT) return "patch_split out of range";
   if (c->patch_split > 0 && (c->grid_width < 1 || c->tokens_per_frame % c->grid_width != 0))
     return "grid_width must divide tokens_per_frame when patch_split > 0";
+  if (c->reserved != 0) return "reserved fields must be 0";
+  if (c->past_frames < 0) return "past_frames must be >= 0";
+  if (c->past_frames > 0) {
+    if (c->keep_per_segment > 0) return "past keys are not combined with segment-level selection";
+    if ((long long)c->past_frames * c->keep_per_frame + c->tokens_per_frame > MUKV_MAX_TOKENS)
+      return "past_frames * keep_per_frame + tokens_per_frame must be <= 256";
+  }
   if (c->keep_per_segment < 0) return "keep_per_segment must be >= 0";
   if (c->keep_per_segment > 0) {
     if (c->patch_split != 0) return "segment-level selection has no patch level";
@@ -158,9 +166,9 @@ const char* check_config(const mukv_config* c) {
   const long long row_vec = (long long)c->n_kv_heads * c->head_dim * esize / 16;
   if (!is_pow2(row_vec) || row_vec > 256) return "Hkv*D*sizeof(element)/16 must be a power of two <= 256";
   // the scoring kernel keeps one key head of a frame in shared memory
-  const size_t smem = c->dtype == MUKV_BF16
-                          ? score_smem_bytes<__nv_bfloat16, double>(c->tokens_per_frame, c->head_dim)
-                          : score_smem_bytes<float, double>(c->tokens_per_frame, c->head_dim);
+  const int key_rows = c->tokens_per_frame + c->past_frames * c->keep_per_frame;
+  const size_t smem = c->dtype == MUKV_BF16 ? score_smem_bytes<__nv_bfloat16, double>(key_rows, c->head_dim)
+                                            : score_smem_bytes<float, double>(key_rows, c->head_dim);
   if (smem > 227 * 1024) return "tokens_per_frame * head_dim too large for shared memory";
   return nullptr;
 }
@@ -503,6 +511,10 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   sp.pages_off = (long long)ctx->sl.pages;
   sp.page_bytes = (long long)ctx->sl.page_bytes;
   sp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
+  sp.store = ctx->store;
+  sp.first_score_layer = L - c.score_layer_offset - ctx->Ls;
+  sp.past_first = t0 - c.past_frames > 0 ? t0 - c.past_frames : 0;
+  sp.n_past_frames = c.past_frames > 0 ? (int)(t0 - sp.past_first) : 0;
   sp.refine = 0;
   sp.row_split = 1;
   const dim3 grid(ctx->Ls * c.n_q_heads, n);
@@ -540,7 +552,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
     if (ctx->tcs.ok && !ctx->force_fma)
       e = launch_score_ps(ctx, sp, d_q, sp.k_last, n, st, &what, &ps_grid, &ps_items, &ps_ipf);
     else
-      e = launch_score<T, float>(sp, ctx->nc, grid, score_smem_bytes<T, float>(P, c.head_dim), st);
+      e = launch_score<T, float>(sp, ctx->nc, grid, score_smem_bytes<T, float>(ctx->key_rows, c.head_dim), st);
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "%s: %s", what, cudaGetErrorString(e));
 
@@ -596,7 +608,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
     int grid_t = ctx->Ls * c.n_q_heads * kRefineSplit * (n < 2 ? n : 2);
     if (grid_t < 2 * L + 1) grid_t = 2 * L + 1;
     if (grid_t > ctx->tail_capacity) grid_t = ctx->tail_capacity;
-    e = launch_tail<T>(sp, cp, ctx->nc, grid_t, score_smem_bytes<T, double>(P, c.head_dim), st, !ctx->prof_on);
+    e = launch_tail<T>(sp, cp, ctx->nc, grid_t, score_smem_bytes<T, double>(ctx->key_rows, c.head_dim), st, !ctx->prof_on);
   }
   if (e != cudaSuccess) return broke_off(ctx, "tail kernel", e);
 
@@ -805,7 +817,9 @@ mukv_status create_impl(const mukv_config* cfg, void* d_store, size_t store_byte
   ctx->G = cfg->n_q_heads / cfg->n_kv_heads;
   ctx->Ls = cfg->n_score_layers > 1 ? cfg->n_score_layers : 1;
   ctx->esize = cfg->dtype == MUKV_BF16 ? 2 : 4;
-  ctx->nc = pick_nc(cfg->tokens_per_frame);
+  ctx->key_rows = cfg->tokens_per_frame + cfg->past_frames * cfg->keep_per_frame;
+  ctx->nc = pick_nc(ctx->key_rows);
+  ctx->force_fma = cfg->past_frames > 0;       // the tensor-core kernel holds the frame's own keys only
   ctx->tcs = tc_shape(*cfg);
   ctx->n_sms = 1;
   ctx->flag_margin = kFlagMargin;
@@ -816,8 +830,8 @@ mukv_status create_impl(const mukv_config* cfg, void* d_store, size_t store_byte
     // the blocks of tail_kernel wait for one another: its grid must be resident as a whole
     int per_sm = 0;
     const bool bf = cfg->dtype == MUKV_BF16;
-    const size_t dyn = bf ? score_smem_bytes<__nv_bfloat16, double>(cfg->tokens_per_frame, D)
-                          : score_smem_bytes<float, double>(cfg->tokens_per_frame, D);
+    const size_t dyn = bf ? score_smem_bytes<__nv_bfloat16, double>(ctx->key_rows, D)
+                          : score_smem_bytes<float, double>(ctx->key_rows, D);
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bf ? tail_fn<__nv_bfloat16>(ctx->nc) : tail_fn<float>(ctx->nc),
                                                       kScoreThreads, dyn);
     if (e == cudaSuccess && per_sm < 1) e = cudaErrorInvalidConfiguration;
@@ -1243,6 +1257,9 @@ extern "C" mukv_status mukv_score_frames_noalloc(const mukv_config* cfg, const v
     c.n_score_layers = 0;
     c.score_layer_offset = 0;
     c.patch_split = 0;
+    c.keep_per_segment = 0;
+    c.past_frames = 0;
+    c.reserved = 0;
     if (const char* why = check_config(&c))
       return fail(nullptr, (c.dtype != MUKV_BF16 && c.dtype != MUKV_FP32) ? MUKV_E_DTYPE : MUKV_E_SHAPE, "%s", why);
     if (n_frames < 1) return fail(nullptr, MUKV_E_INVALID, "n_frames must be >= 1");

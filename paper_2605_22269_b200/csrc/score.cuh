@@ -47,6 +47,12 @@ struct ScoreParams {
   long long* page_table;        // [max_frames]
   long long pages_off, page_bytes;
   int* status;                  // device event word (0 = nothing recorded); see mukv_stats.device_status
+  // cached keys the queries also attend to (Sec. 3.2): the kept keys of the n_past_frames frames stored
+  // just before the chunk, kappa rows each, read from their pages; n_past_frames = 0: none
+  int n_past_frames;
+  long long past_first;         // absolute index of the first of those frames
+  int first_score_layer;        // layer of the model the first scoring layer is
+  const unsigned char* store;   // store base (page_table holds byte offsets from it)
   int no_select;                // 1: only the partial sums are wanted (the selection runs over a whole segment elsewhere)
   int refine;                   // 1: frames come from the flagged list, no further flagging
   int row_split;                // blocks that share a query head, each a range of query rows (>= 1)
@@ -55,6 +61,7 @@ struct ScoreParams {
 template <typename T>
 __host__ __device__ constexpr int score_row_stride(int D) { return D + ElemTraits<T>::kPad; }
 
+// P: key rows held in shared memory (the frame's tokens plus the past keys)
 template <typename T, typename A>
 __host__ inline size_t score_smem_bytes(int P, int D) {
   size_t ks = (size_t)P * score_row_stride<T>(D) * sizeof(T);
@@ -271,10 +278,13 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int hv, 
   const int WS = DS / EPW;                         // words per padded K row
   const int DW = D / EPW;                          // words per vector
 
+  // key rows: the past keys first, then the frame's own tokens
+  const int n_past = p.n_past_frames * p.kappa, Pk = n_past + P;
+
   // ---- shared memory carve-up
   size_t off = 0;
   T* Ks = reinterpret_cast<T*>(smem_raw);
-  off = (((size_t)P * DS * sizeof(T)) + 15) / 16 * 16;
+  off = (((size_t)Pk * DS * sizeof(T)) + 15) / 16 * 16;
   T* Qs = reinterpret_cast<T*>(smem_raw + off);
   off += (size_t)kScoreWarps * kRowsPerStep * D * sizeof(T);
   A* tw = reinterpret_cast<A*>(smem_raw + off);
@@ -292,10 +302,20 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int hv, 
   {
     constexpr int VE = 16 / sizeof(T);             // elements per 16-byte vector
     const int vec_per_row = D / VE;
+    for (int v = tid; v < n_past * vec_per_row; v += kScoreThreads) {
+      // row r of the past: kept row r % kappa of frame past_first + r / kappa, this layer's K plane of its page
+      const int r = v / vec_per_row, c = v % vec_per_row;
+      const long long t = p.past_first + r / p.kappa;
+      const T* page = reinterpret_cast<const T*>(p.store + p.page_table[t]);
+      const T* src = page + ((long long)(p.first_score_layer + layer) * 2 * p.kappa + r % p.kappa) * Hkv * D + g * D;
+      const uint4 x = *reinterpret_cast<const uint4*>(src + c * VE);
+      uint32_t* dst = reinterpret_cast<uint32_t*>(Ks + (size_t)r * DS + c * VE);
+      dst[0] = x.x; dst[1] = x.y; dst[2] = x.z; dst[3] = x.w;
+    }
     for (int v = tid; v < P * vec_per_row; v += kScoreThreads) {
       const int j = v / vec_per_row, c = v % vec_per_row;
       const uint4 x = *reinterpret_cast<const uint4*>(Kg + (long long)j * Hkv * D + c * VE);
-      uint32_t* dst = reinterpret_cast<uint32_t*>(Ks + (size_t)j * DS + c * VE);
+      uint32_t* dst = reinterpret_cast<uint32_t*>(Ks + (size_t)(n_past + j) * DS + c * VE);
       dst[0] = x.x; dst[1] = x.y; dst[2] = x.z; dst[3] = x.w;
     }
     for (int d = tid; d < D; d += kScoreThreads) {
@@ -321,7 +341,7 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int hv, 
   for (int c = 0; c < NC; ++c) csum[c] = (A)0;
   int jrow[NC];
 #pragma unroll
-  for (int c = 0; c < NC; ++c) jrow[c] = min(lane + 32 * c, P - 1) * WS;
+  for (int c = 0; c < NC; ++c) jrow[c] = min(lane + 32 * c, Pk - 1) * WS;
 
   const int RS = p.row_split;
   const int n_steps = (P + kRowsPerStep - 1) / kRowsPerStep;
@@ -360,8 +380,8 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int hv, 
       A m = neg_inf<A>();
 #pragma unroll
       for (int c = 0; c < NC; ++c) {
-        const int j = lane + 32 * c;
-        const bool ok = (j < P) && (!p.causal || j <= i);
+        const int j = lane + 32 * c;                     // past keys are visible to every query
+        const bool ok = (j < Pk) && (!p.causal || j - n_past <= i);
         z[c] = ok ? fma_acc(acc[r][c], scale, acc[r][c] * scale_lo) : neg_inf<A>();
         m = z[c] > m ? z[c] : m;
       }
@@ -382,9 +402,9 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int hv, 
 #pragma unroll
   for (int c = 0; c < NC; ++c) red[warp * 256 + lane + 32 * c] = csum[c];
   __syncthreads();
-  if (tid < P) {
+  if (tid < P) {                                       // the importance is that of the frame's own tokens
     A t = (A)0;
-    for (int w = 0; w < kScoreWarps; ++w) t += red[w * 256 + tid];
+    for (int w = 0; w < kScoreWarps; ++w) t += red[w * 256 + n_past + tid];
     reinterpret_cast<A*>(p.colsum_part)[(((long long)f * HqV + hv) * RS + q) * P + tid] = t;
   }
 
@@ -393,7 +413,7 @@ __device__ __forceinline__ void score_frame_block(const ScoreParams& p, int hv, 
     const int hg = (h % G) * RS + q;                 // the G * RS blocks that hold key head g share its tokens
     const int half = D / 2;
     for (int j = hg + warp * G * RS; j < P; j += kScoreWarps * G * RS) {
-      const T* kr = Ks + (size_t)j * DS;
+      const T* kr = Ks + (size_t)(n_past + j) * DS;
       A total = (A)0;
       // bins 1 .. D/2-1 (twice, by conjugate symmetry) and bin 0
       for (int b = lane; b < half; b += 32) {

@@ -32,7 +32,7 @@ def oracle_cfg(cfg: B.MukvConfig) -> dict:
                 attn_causal=bool(cfg.attn_causal), keep_low_freq=bool(cfg.keep_low_freq), tie_eps=float(cfg.tie_eps),
                 patch_split=int(cfg.patch_split), grid_width=int(cfg.grid_width),
                 n_score_layers=int(cfg.n_score_layers), score_layer_offset=int(cfg.score_layer_offset),
-                keep_per_segment=int(cfg.keep_per_segment))
+                keep_per_segment=int(cfg.keep_per_segment), past_frames=int(cfg.past_frames))
 
 
 def to_device(x: np.ndarray, bf16: bool, device="cuda:0") -> torch.Tensor:

@@ -37,7 +37,7 @@ def test_exports_match_header(lib):
 
 
 def test_struct_sizes_match_header():
-    assert C.sizeof(B.MukvConfig) == 80 and C.sizeof(B.MukvStats) == 72 and C.sizeof(B.MukvStoreHeader) == 104
+    assert C.sizeof(B.MukvConfig) == 88 and C.sizeof(B.MukvStats) == 72 and C.sizeof(B.MukvStoreHeader) == 112
     assert C.sizeof(B.MukvRetrParams) == 32
 
 
@@ -55,7 +55,8 @@ def test_store_size_of_the_three_hour_stream(lib):
                                   dict(keep_per_frame=0), dict(keep_per_frame=197), dict(alpha=1.5),
                                   dict(dtype=7), dict(max_frames=0), dict(n_kv_heads=3, n_q_heads=27),
                                   dict(frames_per_segment=0), dict(patch_split=5, grid_width=14),
-                                  dict(patch_split=2, grid_width=13), dict(patch_split=2, grid_width=0)])
+                                  dict(patch_split=2, grid_width=13), dict(patch_split=2, grid_width=0), dict(past_frames=2), dict(past_frames=-1),
+                                  dict(keep_per_segment=100000), dict(n_score_layers=20, score_layer_offset=9)])
 def test_bad_configs_are_rejected_on_the_host(lib, over):
     cfg = good_config(**over)
     assert lib.mukv_store_bytes(C.byref(cfg)) == 0

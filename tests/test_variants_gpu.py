@@ -138,3 +138,31 @@ def test_scoring_layer_choice_fp32():
     O.compress_chunk(st, q, k, v)
     run.kept, run.scores = kept.cpu().numpy(), sc.cpu().numpy()
     H.check_frames_against_oracle(run, st, range(3), full_layers=True)
+
+
+def _oracle_chunked(spec, ocfg, T, chunk):
+    st = O.Store(ocfg)
+    for t0 in range(0, T, chunk):
+        q, k, v = spec.chunk(t0, min(chunk, T - t0))
+        O.compress_chunk(st, q, k, v)
+    return st
+
+
+@pytest.mark.parametrize("name,T,chunk,W,over,opts", [
+    ("tiny", 8, 3, 3, dict(), None),
+    ("tiny", 8, 2, 2, dict(attn_causal=1), None),
+    ("chunk7b", 6, 2, 1, dict(), None),
+    ("chunk7b", 5, 2, 1, dict(attn_causal=1), {B.OPT_FLAG_MARGIN: 1.0}),
+])
+def test_past_keys_in_the_attention(name, T, chunk, W, over, opts):
+    # Sec. 3.2: the queries of a chunk also attend to the kept keys of the W frames stored before it
+    run = H.GpuRun(name, n_frames=T, past_frames=W, options=opts, **over)
+    run.compress(chunk)
+    st = _oracle_chunked(run.spec, H.oracle_cfg(run.cfg), T, chunk)
+    H.check_frames_against_oracle(run, st, range(T), full_layers=True)
+    # the past really takes attention mass away from the frame's own tokens (not in the first chunk)
+    assert abs(st.scores[0][0].sum() - 1.0) < 1e-9 and st.scores[T - 1][0].sum() < 0.999
+    stats = run.ctx.mukv_get_stats()
+    assert stats.device_status == 0
+    if opts:
+        assert stats.refined_frames == T
