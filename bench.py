@@ -27,8 +27,8 @@ if ROOT not in sys.path:
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture) of one launch of the
 # kernel on a 16-frame chunk of this workload; reported as `roofline.traffic`
-SCORE_TRAFFIC_BYTES = 25857792
-COMPACT_TRAFFIC_BYTES = 45182464 + 3919104
+SCORE_TRAFFIC_BYTES = 25858560
+COMPACT_TRAFFIC_BYTES = 45204224 + 3888640
 
 METRIC = "compressed_frames_per_s"
 UNIT = "frames/s"
