@@ -130,6 +130,8 @@ typedef struct {
                                     3, 4, 5  a bounded wait inside the tensor-core scoring kernel
                                              ran out (producer, MMA issuer, epilogue): the chunk's
                                              scores are not to be trusted;
+                                    6        the blocks of the double-precision pass waited in
+                                             vain for one another: flagged frames were not stored;
                                     7        a frame's scores were not finite (Inf/NaN inputs):
                                              its kappa lowest token ids were kept            */
   int32_t reserved;
