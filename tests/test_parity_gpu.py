@@ -167,6 +167,20 @@ def test_chunk7b_every_frame_through_the_double_pass():
     assert run.ctx.mukv_get_stats().refined_frames == 5
 
 
+@pytest.mark.parametrize("fseg,chunk,opts,over", [(4, 4, None, dict(patch_split=2, grid_width=14)),
+                                                  (2, 2, None, dict()),
+                                                  (16, 16, {B.OPT_FLAG_MARGIN: 1.0}, dict()),
+                                                  (4, 4, {B.OPT_FLAG_MARGIN: 2e-4}, dict())])
+def test_chunk_equal_to_a_segment(fseg, chunk, opts, over):
+    # chunks that are exactly one segment, with and without a patch level; flagged frames (all of them,
+    # or a few with the wider margin) leave the segment entries to the tail kernel
+    wl = dict(workload("chunk7b"))
+    wl["fseg"] = fseg
+    run = H.GpuRun(wl, n_frames=16 if fseg > 2 else 6, options=opts, **over)
+    full_compress_check(run, chunk=chunk)
+    assert run.ctx.mukv_get_stats().device_status == 0
+
+
 def test_chunk7b_cuda_core_scoring():
     # bf16 inputs scored by the plain multiply-add kernel (the one fp32 inputs always use)
     run = H.GpuRun("chunk7b", n_frames=3, options={B.OPT_SCORE_PATH: 1})
