@@ -280,6 +280,21 @@ def main():
     other = "flush" if args.l2 == "inputs" else "inputs"
     l2_modes = {args.l2: c_ms / args.steps, other: one_step(other)[0]}
 
+    # ---- latency of one question alone (retrieve + gather of the first question), L2 flushed before each
+    lat = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    q1 = qtok[:offs[1]]
+    for _ in range(13):
+        flush.zero_()
+        e0.record()
+        ctx.mukv_retrieve(q1, offs[:2], None, k_seg, k_frm, 0, lam, B.RETR_SEMI, seg_idx, frm_idx, seg_sc, frm_sc, counts)
+        ctx.mukv_gather(frm_idx, counts, 1, k_frm, decode[0], stride, None)
+        e1.record()
+        torch.cuda.synchronize()
+        lat.append(1e3 * e0.elapsed_time(e1))
+    lat = sorted(lat[3:])
+    single_q = {"median_us": lat[len(lat) // 2], "min_us": lat[0], "tokens": int(offs[1])}
+
     # ---- per-kernel durations, measured live with events around every launch (one extra step)
     ctx.mukv_profile_enable(True)
     one_step()
@@ -401,7 +416,7 @@ def main():
                               "larger than the 126 MB L2; the retrieval calls follow a 256 MiB memset")},
             "retrievals_per_s": rps,
             "retrieve_ms": r_ms / args.steps, "gather_ms": g_ms / args.steps, "compress_ms": c_ms / args.steps,
-            "compress_ms_by_l2_mode": l2_modes,
+            "compress_ms_by_l2_mode": l2_modes, "single_question_latency": single_q,
             "wall_s_per_step_with_generation": wall / args.steps,
             "path_algorithmic_gbs": {"compress": path_gbs, "compress_frac_of_peak": path_gbs / peaks["hbm_gbs"],
                                      "retrieve_gather": retr_gbs,
