@@ -447,28 +447,64 @@ __device__ inline void compact_plane(const CompactParams& p, int plane, int f, C
 
 // Patch-level block keys of chunk frame f (Eq. 5 on the kept tokens of each super patch): mean of
 // their last-layer keys, summed in double like the frame key; kept ids in sc->kept.  Run by a
-// whole block; thread t owns columns t, t + 256, ...  sc->red is used as scratch.
+// whole block; the kept rows are first grouped by super patch, then every thread sums its channels
+// of each group in ascending row order.  sc->red is used as scratch.
 template <typename T>
 __device__ inline void pool_patches(const CompactParams& p, int f, CompactScratch* sc) {
+  constexpr int EW = ElemTraits<T>::kPerWord;
   const int tid = threadIdx.x;
   const int S = p.patch_split * p.patch_split, C = p.C, kappa = p.kappa;
   const long long f_abs = p.first_frame + f;
-  int* sp_of = reinterpret_cast<int*>(sc->red);          // super patch of each kept row
+  int* order = reinterpret_cast<int*>(sc->red);          // kept ids grouped by super patch, ascending inside a group
+  int* start = order + MUKV_MAX_TOKENS;                  // [S + 1] first entry of every group
+  int* sp_of = start + 32;                               // [kappa] super patch of each kept row
+  static_assert(sizeof(sc->red) >= (2 * MUKV_MAX_TOKENS + 32) * sizeof(int), "scratch too small");
+  static_assert(MUKV_MAX_PATCH_SPLIT * MUKV_MAX_PATCH_SPLIT < 32, "group starts do not fit");
   __syncthreads();
   for (int r = tid; r < kappa; r += kCompactThreads) sp_of[r] = super_patch_index(sc->kept[r], p.P, p.grid_width, p.patch_split);
   __syncthreads();
-  const T* src = reinterpret_cast<const T*>(p.k) + ((long long)(p.L - 1) * p.n_frames + f) * p.P * C;
-  for (int sp = 0; sp < S; ++sp) {
-    int cnt = 0;
-    for (int r = 0; r < kappa; ++r) cnt += (sp_of[r] == sp);
-    for (int col = tid; col < C; col += kCompactThreads) {
-      double t = 0.0;
-      for (int r = 0; r < kappa; ++r)
-        if (sp_of[r] == sp) t += (double)elem_to_float<T>(src[(long long)sc->kept[r] * C + col]);
-      p.patch_key[((f_abs * S) + sp) * C + col] = cnt ? (float)(t / (double)cnt) : 0.f;
-    }
-    if (tid == 0) p.patch_cnt[f_abs * S + sp] = cnt;
+  if (tid <= S) {
+    int c = 0;
+    for (int r = 0; r < kappa; ++r) c += (sp_of[r] < tid);
+    start[tid] = c;
   }
+  __syncthreads();
+  for (int r = tid; r < kappa; r += kCompactThreads) {
+    const int s = sp_of[r];
+    int pos = start[s];
+    for (int q = 0; q < r; ++q) pos += (sp_of[q] == s);
+    order[pos] = sc->kept[r];
+  }
+  __syncthreads();
+  // a thread owns one 32-bit word of the row (one or two channels); eight rows are in flight at a time
+  const int wpr = C / EW;
+  const uint32_t* src = reinterpret_cast<const uint32_t*>(reinterpret_cast<const T*>(p.k) +
+                                                          ((long long)(p.L - 1) * p.n_frames + f) * p.P * C);
+  for (int w = tid; w < wpr; w += kCompactThreads) {
+    for (int sp = 0; sp < S; ++sp) {
+      const int b = start[sp], e = start[sp + 1];
+      double t0 = 0.0, t1 = 0.0;
+      for (int i = b; i < e; i += 8) {
+        uint32_t x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) x[u] = i + u < e ? __ldg(src + (long long)order[i + u] * wpr + w) : 0u;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {                      // (a zero word adds +0.0)
+          if (EW == 2) {
+            t0 += (double)bf16_lo(x[u]);
+            t1 += (double)bf16_hi(x[u]);
+          } else {
+            t0 += (double)__uint_as_float(x[u]);
+          }
+        }
+      }
+      const int cnt = e - b;
+      float* dst = p.patch_key + ((f_abs * S) + sp) * C + (long long)w * EW;
+      dst[0] = cnt ? (float)(t0 / (double)cnt) : 0.f;
+      if (EW == 2) dst[1] = cnt ? (float)(t1 / (double)cnt) : 0.f;
+    }
+  }
+  if (tid < S) p.patch_cnt[f_abs * S + tid] = start[tid + 1] - start[tid];
 }
 
 // is chunk frame f on the flagged list (of n entries)?

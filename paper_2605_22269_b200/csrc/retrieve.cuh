@@ -692,10 +692,24 @@ struct Gather3Params {
   int* ntok; int* tok_meta;
 };
 
+// one contiguous run, copied by a block of 256 threads with four 16-byte vectors in flight per thread
 __device__ __forceinline__ void copy_run16(unsigned char* dst, const unsigned char* src, long long bytes) {
   const long long nvec = bytes >> 4;
-  for (long long v = threadIdx.x; v < nvec; v += blockDim.x) st_stream(dst + (v << 4), ld_stream(src + (v << 4)));
+  long long v = threadIdx.x;
+  for (; v + 3 * 256 < nvec; v += 4 * 256) {
+    const uint4 x0 = ld_stream(src + (v << 4));
+    const uint4 x1 = ld_stream(src + ((v + 256) << 4));
+    const uint4 x2 = ld_stream(src + ((v + 512) << 4));
+    const uint4 x3 = ld_stream(src + ((v + 768) << 4));
+    st_stream(dst + (v << 4), x0);
+    st_stream(dst + ((v + 256) << 4), x1);
+    st_stream(dst + ((v + 512) << 4), x2);
+    st_stream(dst + ((v + 768) << 4), x3);
+  }
+  for (; v < nvec; v += 256) st_stream(dst + (v << 4), ld_stream(src + (v << 4)));
 }
+
+constexpr int kGatherListCap = 1024;       // rows of patch-level blocks listed at a time (>= MUKV_MAX_TOKENS)
 
 // Units, per question and (layer, K|V) plane: k_frm frame runs (one contiguous run of the page each),
 // then one unit for the summary tokens and the patch-level rows.  Token slots of a plane: summary
@@ -704,6 +718,7 @@ __device__ __forceinline__ void copy_run16(unsigned char* dst, const unsigned ch
 template <typename T>
 __global__ void __launch_bounds__(256) gather3_kernel(const Gather3Params p) {
   __shared__ int s_off[MUKV_MAX_TOPK + 1];                 // first row of each selected patch block
+  __shared__ long long s_src[kGatherListCap];              // byte offset in the store of each listed row
   __shared__ int s_row0;
   const long long planes = (long long)p.L * 2;
   const int upp = p.k_frm + 1;                             // units per (question, plane)
@@ -771,22 +786,56 @@ __global__ void __launch_bounds__(256) gather3_kernel(const Gather3Params p) {
       if (plane == 0 && p.ntok) p.ntok[qi] = off;
     }
     __syncthreads();
-    // one warp per patch block: walk the frame's kept list, copy the rows of the super patch
+    // Patch blocks in batches whose rows fit the list.  One warp per block walks the frame's kept
+    // list and notes where the rows of its super patch lie; then the whole block copies the rows.
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-    for (int i = warp; i < c_pat; i += nwarp) {
-      const int b = p.pat_idx[(long long)qi * p.k_pat + i];
-      const int f = b / p.S, sp = b % p.S;
-      const unsigned char* page = p.store + p.page_table[f] + (long long)plane * run_bytes;
-      int row = s_off[i];
-      for (int t = 0; t < p.kappa; ++t) {
-        const int tok = p.kept_store[(long long)f * p.kappa + t];
-        if (super_patch_index(tok, p.P, p.grid_width, p.patch_split) != sp) continue;
-        const unsigned char* src = page + (long long)t * row_bytes;
-        unsigned char* dst = dplane + (long long)row * row_bytes;
-        for (long long v = lane; v < (row_bytes >> 4); v += 32) st_stream(dst + (v << 4), ld_stream(src + (v << 4)));
-        if (plane == 0 && meta && lane == 0) { meta[row * 2] = f; meta[row * 2 + 1] = tok; }
-        ++row;
+    const int vpr = (int)(row_bytes >> 4);                 // 16-byte vectors per row
+    for (int b0 = 0; b0 < c_pat;) {
+      int b1 = b0 + 1;                                     // (one block has at most kappa <= list capacity rows)
+      while (b1 < c_pat && s_off[b1 + 1] - s_off[b0] <= kGatherListCap) ++b1;
+      for (int i = b0 + warp; i < b1; i += nwarp) {
+        const int b = p.pat_idx[(long long)qi * p.k_pat + i];
+        const int f = b / p.S, sp = b % p.S;
+        const long long page = p.page_table[f] + (long long)plane * run_bytes;
+        const int base = s_off[i] - s_off[b0], room = min(s_off[i + 1] - s_off[i], kGatherListCap - base);
+        int pos = 0;
+        for (int t0 = 0; t0 < p.kappa; t0 += 32) {
+          const int t = t0 + lane;
+          int tok = 0;
+          bool hit = false;
+          if (t < p.kappa) {
+            tok = p.kept_store[(long long)f * p.kappa + t];
+            hit = super_patch_index(tok, p.P, p.grid_width, p.patch_split) == sp;
+          }
+          const unsigned bal = __ballot_sync(kFull, hit);
+          const int at = pos + __popc(bal & ((1u << lane) - 1u));
+          if (hit && at < room) {
+            s_src[base + at] = page + (long long)t * row_bytes;
+            if (plane == 0 && meta) { meta[(s_off[i] + at) * 2] = f; meta[(s_off[i] + at) * 2 + 1] = tok; }
+          }
+          pos += __popc(bal);
+        }
+        // (a block with fewer rows than its count says, which a consistent store never has, repeats its first row)
+        for (int at = pos + lane; at < room; at += 32) s_src[base + at] = page;
       }
+      __syncthreads();
+      const int nvec = min(s_off[b1] - s_off[b0], kGatherListCap) * vpr;
+      unsigned char* dst = dplane + (long long)s_off[b0] * row_bytes;
+      int v = threadIdx.x;
+      for (; v + 3 * 256 < nvec; v += 4 * 256) {
+        uint4 x[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int vv = v + k * 256;
+          x[k] = ld_stream(p.store + s_src[vv / vpr] + ((long long)(vv % vpr) << 4));
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) st_stream(dst + ((long long)(v + k * 256) << 4), x[k]);
+      }
+      for (; v < nvec; v += 256)
+        st_stream(dst + ((long long)v << 4), ld_stream(p.store + s_src[v / vpr] + ((long long)(v % vpr) << 4)));
+      __syncthreads();                                     // the list is rewritten by the next batch
+      b0 = b1;
     }
     __syncthreads();
   }
