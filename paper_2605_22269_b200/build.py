@@ -1,6 +1,7 @@
 """In-tree build of the CUDA libraries (sm_100a only)."""
 from __future__ import annotations
 
+import glob
 import os
 import subprocess
 
@@ -12,7 +13,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
 
 TARGETS = {
     "libmukv.so": (os.path.join(HERE, "csrc", "mukv.cu"),
-                   [os.path.join(HERE, "csrc", n) for n in ("common.cuh", "score.cuh", "score_ps.cuh", "tc.cuh", "compact.cuh", "retrieve.cuh")]
+                   sorted(glob.glob(os.path.join(HERE, "csrc", "*.cuh")))
                    + [os.path.join(os.path.dirname(HERE), "include", "mukv.h")]),
     "libmukv_synth.so": (os.path.join(HERE, "synth", "synth.cu"), []),
 }

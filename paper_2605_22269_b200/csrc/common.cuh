@@ -135,6 +135,10 @@ __device__ __forceinline__ int super_patch_index(int j, int P, int grid_width, i
   return (j / grid_width) / rh * split + (j % grid_width) / cw;
 }
 
+// owner of item i when n items are split into contiguous shares [c*n/nb, (c+1)*n/nb) (the blocks of
+// the persistent scoring kernel take such shares of its item list)
+__device__ __forceinline__ int share_owner(unsigned i, unsigned n, unsigned nb) { return (int)(((i + 1u) * nb - 1u) / n); }
+
 // 16-byte streaming copies
 __device__ __forceinline__ uint4 ld_stream(const void* p) {
   uint4 v;

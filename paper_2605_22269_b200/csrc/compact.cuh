@@ -71,9 +71,6 @@ struct CompactParams {
 // a token id read back from memory, forced into the frame (row addresses are computed from it)
 __device__ __forceinline__ int token_id(int id, int P) { return (unsigned)id < (unsigned)P ? id : 0; }
 
-// owner of item i when n items are split into contiguous shares [c*n/nb, (c+1)*n/nb)
-__device__ __forceinline__ int share_owner(unsigned i, unsigned n, unsigned nb) { return (int)(((i + 1u) * nb - 1u) / n); }
-
 struct SelectScratch {
   unsigned mm[kCompactThreads / 32][4];   // per-warp min / max keys of the two signals
   int hist[256];
@@ -299,20 +296,37 @@ __device__ __noinline__ void compact_segment_plane(const SegmentArgs p, int l, i
     if (p.kept_count) {
       // frames keep different numbers of tokens (segment-level selection): the mean over all kept
       // tokens of the segment is the count-weighted mean of the frame entries
-      long long n_tok = 0;
-      for (long long ff = t0; ff < t1; ++ff) n_tok += __ldcg(p.kept_count + ff);
       for (int col = tid; col < C; col += kCompactThreads) {
+        long long n_tok = 0;
+        double td = 0.0;
+        float tf = 0.f;
+        for (long long ff = t0; ff < t1; ff += 16) {
+          int cn[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) cn[i] = ff + i < t1 ? __ldcg(p.kept_count + ff + i) : 0;
+          if (exact) {
+            double x[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) x[i] = ff + i < t1 ? __ldcg(p.frame_ksum + (ff + i) * C + col) : 0.0;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) td += x[i];
+          } else {
+            float x[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              x[i] = ff + i < t1 ? __ldcg(p.frame_entry + (((ff + i) * p.L + l) * 2 + kv) * C + col) : 0.f;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) tf += (float)cn[i] * x[i];
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i) n_tok += cn[i];
+        }
         if (exact) {
-          double t = 0.0;
-          for (long long ff = t0; ff < t1; ++ff) t += __ldcg(p.frame_ksum + ff * C + col);
-          const float m = n_tok ? (float)(t / (double)n_tok) : 0.f;
+          const float m = n_tok ? (float)(td / (double)n_tok) : 0.f;
           p.seg_key[u * C + col] = m;
           p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = m;
         } else {
-          float t = 0.f;
-          for (long long ff = t0; ff < t1; ++ff)
-            t += (float)__ldcg(p.kept_count + ff) * __ldcg(p.frame_entry + ((ff * p.L + l) * 2 + kv) * C + col);
-          p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = n_tok ? t / (float)n_tok : 0.f;
+          p.seg_entry[((u * p.L + l) * 2 + kv) * C + col] = n_tok ? tf / (float)n_tok : 0.f;
         }
       }
       continue;
@@ -523,7 +537,10 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(const Compa
   // frame is the fast block index: the blocks that start first cover the low planes of every frame,
   // the plane-0 blocks among them
   const int f = blockIdx.x;
-  const int plane = blockIdx.y;                 // l*2 + kv
+  // block row -> plane l*2 + kv; with a patch level its blocks (plane 2L) sit in row 1, so that they run
+  // in the first wave beside the copy blocks instead of alone at the end
+  const int row = blockIdx.y;
+  const int plane = p.patch_split > 0 && row >= 1 ? (row == 1 ? 2 * p.L : row - 1) : row;
   pdl_wait();
   pdl_trigger();
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.n_flagged_next = 0;
@@ -581,7 +598,7 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(const Compa
   }
   if (risky) return;
   if (plane < 2 * p.L) compact_plane<T>(p, plane, f, &cs, kappa_f, page);
-  else pool_patches<T>(p, f, &cs);                // the extra row of blocks when there is a patch level
+  else pool_patches<T>(p, f, &cs);
 }
 
 // Bounded wait until *ctr reaches `target` (other blocks of the same grid add to it; the grid is

@@ -40,7 +40,7 @@ struct StoreLayout {
 
 struct WorkLayout {
   size_t colsum_f, colsum_p, ifft_f, colsum_d, ifft_d, frame_counter, flagged, n_flagged, tail_ctr, sel_flag,
-      stat_refined, dev_status;
+      seg_flag, stat_refined, dev_status;
   size_t q64, qnorm, s_frm, s_seg, s_pat, wtab, total;
   size_t zero_begin, zero_end;          // region that must start as zeros
 };
@@ -244,6 +244,7 @@ WorkLayout work_layout(const mukv_config& c) {
   w.n_flagged = off;      off = align_up(off + 2 * sizeof(int));   // alternate between chunks
   w.tail_ctr = off;       off = align_up(off + 2 * sizeof(int));
   w.sel_flag = off;       off = align_up(off + F * sizeof(unsigned));
+  w.seg_flag = off;       off = align_up(off + F * sizeof(int));
   w.stat_refined = off;   off = align_up(off + sizeof(long long));
   w.dev_status = off;     off = align_up(off + sizeof(int));
   w.zero_end = off;
@@ -522,29 +523,64 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   const char* what = "score kernel";
   int ps_grid = 0, ps_items = 0, ps_ipf = 0;
   if (seg_scope) {
-    // every frame's indicators in double precision (no per-frame selection), then one block per segment
+    // One block per segment ranks all its tokens.  A bf16 chunk is first scored on the tensor cores and
+    // ranked from those single-precision sums; segments that are too close to call are scored and
+    // ranked again in double precision (both launches of that pass return at once for the others).
+    // Any other chunk goes through the double-precision pass as a whole.
+    const bool tc_first = ctx->tcs.ok && !ctx->force_fma;
+    const int n_seg = (n + c.frames_per_segment - 1) / c.frames_per_segment;
+    const int seg_tokens = (n < c.frames_per_segment ? n : c.frames_per_segment) * P;
+    const bool dep = !ctx->prof_on;
+    SegSelParams gp;
+    memset(&gp, 0, sizeof gp);
+    gp.fseg = c.frames_per_segment; gp.kappa_v = c.keep_per_segment;
+    gp.token_bytes = (long long)L * 2 * C * ctx->esize;
+    gp.kept_count = reinterpret_cast<int*>(ctx->store + ctx->sl.kept_count);
+    gp.seg_flag = reinterpret_cast<int*>(ctx->ws + ctx->wl.seg_flag);
+    gp.stat_refined = reinterpret_cast<unsigned long long*>(ctx->ws + ctx->wl.stat_refined);
+    if (tc_first) {
+      int ps_grid1 = 0, ps_items1 = 0, ps_ipf1 = 0;
+      {
+        ProfScope ps(ctx, 0, st);
+        e = launch_score_ps(ctx, sp, d_q, sp.k_last, n, st, &what, &ps_grid1, &ps_items1, &ps_ipf1);
+      }
+      if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "%s: %s", what, cudaGetErrorString(e));
+      gp.sp = sp;
+      gp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
+      gp.src32 = 1;
+      gp.ps_grid = ps_grid1; gp.ps_items = ps_items1; gp.ps_ipf = ps_ipf1;
+      {
+        ProfScope ps(ctx, 1, st);
+        e = launch_k(segsel_kernel, dim3(n_seg), kSegSelThreads, segsel_smem_bytes(seg_tokens), st, dep, gp);
+      }
+      if (e != cudaSuccess) return broke_off(ctx, "segment selection kernel", e);
+    }
     ScoreParams sd = sp;
     sd.no_select = 1;
     sd.row_split = kRefineSplit;
     sd.colsum_part = ctx->ws + ctx->wl.colsum_d;
     sd.ifft_part = ctx->ws + ctx->wl.ifft_d;
-    {
-      ProfScope ps(ctx, 0, st);
-      e = launch_score<T, double>(sd, ctx->nc, dim3(ctx->Ls * c.n_q_heads * kRefineSplit, n),
-                                  score_smem_bytes<T, double>(P, c.head_dim), st);
+    if (tc_first) {
+      sd.seg_gate = gp.seg_flag;
+      sd.gate_fseg = c.frames_per_segment;
     }
-    if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "score kernel: %s", cudaGetErrorString(e));
-    SegSelParams gp;
-    memset(&gp, 0, sizeof gp);
+    {
+      ProfScope ps(ctx, tc_first ? 1 : 0, st);
+      const int units = ctx->Ls * c.n_q_heads * kRefineSplit;
+      const dim3 grid_d = tc_first ? dim3(units < 2 * ctx->n_sms ? units : 2 * ctx->n_sms) : dim3(units, n);
+      e = launch_score<T, double>(sd, ctx->nc, grid_d,
+                                  score_smem_bytes<T, double>(P, c.head_dim), st, tc_first && dep);
+    }
+    if (e != cudaSuccess) {
+      if (tc_first) return broke_off(ctx, "score kernel", e);
+      return fail(ctx, MUKV_E_CUDA, "score kernel: %s", cudaGetErrorString(e));
+    }
     gp.sp = sd;
-    gp.fseg = c.frames_per_segment; gp.kappa_v = c.keep_per_segment;
-    gp.token_bytes = (long long)L * 2 * C * ctx->esize;
-    gp.kept_count = reinterpret_cast<int*>(ctx->store + ctx->sl.kept_count);
-    const int n_seg = (n + c.frames_per_segment - 1) / c.frames_per_segment;
-    const int seg_tokens = (n < c.frames_per_segment ? n : c.frames_per_segment) * P;
+    gp.src32 = 0;
+    gp.only_flagged = tc_first ? 1 : 0;
     {
       ProfScope ps(ctx, 1, st);
-      e = launch_k(segsel_kernel, dim3(n_seg), kSegSelThreads, segsel_smem_bytes(seg_tokens), st, false, gp);
+      e = launch_k(segsel_kernel, dim3(n_seg), kSegSelThreads, segsel_smem_bytes(seg_tokens), st, tc_first && dep, gp);
     }
     if (e != cudaSuccess) return broke_off(ctx, "segment selection kernel", e);
   } else if (!d_ext) {

@@ -56,6 +56,10 @@ struct ScoreParams {
   int no_select;                // 1: only the partial sums are wanted (the selection runs over a whole segment elsewhere)
   int refine;                   // 1: frames come from the flagged list, no further flagging
   int row_split;                // blocks that share a query head, each a range of query rows (>= 1)
+  // segment-level selection, double-precision pass: only the frames of segments whose word is non-zero
+  // are scored (segment of chunk frame f: f / gate_fseg); null: every frame
+  const int* seg_gate;
+  int gate_fseg;
 };
 
 template <typename T>
@@ -473,6 +477,18 @@ __global__ void __launch_bounds__(kScoreThreads) score_kernel(const ScoreParams 
   pdl_wait();
   pdl_trigger();
   if (!p.refine) {
+    if (p.seg_gate) {
+      // a small one-dimensional grid walks the frames and scores those of flagged segments (rarely any)
+      const int units = p.Ls * p.Hq * p.row_split;
+      for (int f = 0; f < p.n_frames; ++f) {
+        if (__ldcg(p.seg_gate + f / p.gate_fseg) == 0) continue;
+        for (int u = blockIdx.x; u < units; u += gridDim.x) {
+          score_frame_block<T, A, NC>(p, u / p.row_split, u % p.row_split, f, smem_raw);
+          __syncthreads();
+        }
+      }
+      return;
+    }
     score_frame_block<T, A, NC>(p, blockIdx.x / p.row_split, blockIdx.x % p.row_split, blockIdx.y, smem_raw);
     return;
   }

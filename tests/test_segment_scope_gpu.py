@@ -63,18 +63,25 @@ def check_store(run, st, kept, scores):
     assert stats.kept_tokens == sum(len(k) for k in st.kept) and stats.device_status == 0
 
 
-def test_segment_scope_bf16():
+@pytest.mark.parametrize("opts,refined", [(None, None), ({B.OPT_FLAG_MARGIN: 1.0}, 10), ({B.OPT_SCORE_PATH: 1}, 0)])
+def test_segment_scope_bf16(opts, refined):
     # the 7B layout, segments of 4 frames, rho_v = 0.25 over the 784 tokens of a segment; the stream
-    # ends with a segment of two frames
+    # ends with a segment of two frames.  Scored on the tensor cores and ranked in single precision
+    # where that is safe; with a margin nothing passes, every segment through the double-precision
+    # pass behind it; on the multiply-add path, double precision from the start
     wl = dict(workload("chunk7b"))
     wl["fseg"] = 4
     kv = O.keep_count(0.25, 4 * 196)
-    run = H.GpuRun(wl, n_frames=10, max_frames=12, keep_per_segment=kv)
+    run = H.GpuRun(wl, n_frames=10, max_frames=12, keep_per_segment=kv, options=opts)
     kept, scores = compress_segment_scope(run, 8)
     st = oracle_stream_chunked(run.spec, H.oracle_cfg(run.cfg), 10, 8)
     counts = [len(k) for k in st.kept]
     assert sum(counts[:4]) == kv and sum(counts[8:]) == kv // 2 and len(set(counts)) > 1
     check_store(run, st, kept, scores)
+    n_ref = run.ctx.mukv_get_stats().refined_frames
+    assert n_ref <= 4 if refined is None else n_ref == refined, n_ref
+    if opts:
+        return
     qtok, offs, _ = run.spec.questions(4, 3, 9)
     for mode in (B.RETR_SEMI, B.RETR_PARALLEL, B.RETR_HIER):
         retrieve3_check(run, st, qtok, offs, (0, 3, 2), (0.0, 0.3, 0.0), mode)
@@ -88,6 +95,40 @@ def test_segment_scope_bf16():
         q, k, v = run.gs.chunk(10, 1)
         run.ctx.mukv_compress_chunk(q, k, v, 1, 10)
     assert e.value.status == -6
+
+
+@pytest.mark.parametrize("over", [dict(), dict(alpha=0.0), dict(alpha=1.0), dict(keep_low_freq=1, attn_causal=1),
+                                  dict(n_score_layers=2, score_layer_offset=1)])
+def test_segment_scope_sixteen_frame_segments(over):
+    # segments of 16 frames (3,136 tokens ranked at once), two full segments and one of five frames,
+    # chunks of 16 frames; Eq. 4 variants and two scoring layers on the tensor-core path
+    wl = dict(workload("chunk7b"))
+    wl["fseg"] = 16
+    kv = O.keep_count(0.25, 16 * 196)
+    T = 37
+    run = H.GpuRun(wl, n_frames=T, max_frames=48, keep_per_segment=kv, **over)
+    c = run.cfg
+    Ls = max(1, c.n_score_layers)
+    P = c.tokens_per_frame
+    kept = torch.full((T, P), -7, dtype=torch.int32, device=run.device)
+    scores = torch.zeros((3, T, P), dtype=torch.float32, device=run.device)
+    st = O.Store(H.oracle_cfg(c))
+    for t0 in range(0, T, 16):
+        n = min(16, T - t0)
+        q, k, v = run.spec.chunk(t0, n)
+        if Ls > 1:                                            # a second scoring layer from another seeded stream
+            import copy
+            sp2 = copy.copy(run.spec)
+            sp2.seed = run.spec.seed + 100
+            q = np.stack([q, np.stack([sp2.frame_q(t) for t in range(t0, t0 + n)])])
+        O.compress_chunk(st, q, k, v)
+        dq, dk, dv = (H.to_device(x, True, run.device) for x in (q, k, v))
+        sc = torch.empty((3, n, P), dtype=torch.float32, device=run.device)
+        run.ctx.mukv_compress_chunk(dq, dk, dv, n, t0, kept[t0:t0 + n], sc)
+        scores[:, t0:t0 + n] = sc
+    torch.cuda.synchronize()
+    check_store(run, st, kept.cpu().numpy(), scores.cpu().numpy())
+    assert run.ctx.mukv_get_stats().refined_frames <= 16
 
 
 def oracle_stream_chunked(spec, ocfg, T, chunk):
