@@ -49,6 +49,7 @@ struct WorkLayout {
 struct TcShape {
   bool ok;                 // bf16 chunk scored on the tensor cores (every supported bf16 shape fits)
   int tpt, tiles, npad, n_mt, ps_stages;
+  int own_rows, past_pad;  // key-tile rows of the frame's own keys; rows reserved per cached past frame (0: none)
   size_t smem_ps;
 };
 
@@ -75,6 +76,7 @@ struct mukv_ctx {
   int n_sms;
   int tail_capacity = 1;                 // blocks of tail_kernel that are resident at once on this device
   CUtensorMap wmap;                      // DFT matrix terms [3*D][D] bf16
+  CUtensorMap pmap;                      // the page region as [frame][plane][kept row][key head][D] (past_frames > 0)
   std::string err;
   // optional per-kernel timing (host objects only)
   bool prof_on = false;
@@ -210,9 +212,18 @@ TcShape tc_shape(const mukv_config& c) {
   t.tpt = 128 / G;
   t.tiles = (c.tokens_per_frame + t.tpt - 1) / t.tpt;
   t.npad = (c.tokens_per_frame + 15) / 16 * 16;
+  t.own_rows = t.npad;
+  if (c.past_frames > 0) {
+    // the cached keys of a past frame start on a multiple of eight rows of the key tile (one swizzle
+    // atom), behind the frame's own keys
+    t.own_rows = (c.tokens_per_frame + 7) / 8 * 8;
+    t.past_pad = (c.keep_per_frame + 7) / 8 * 8;
+    t.npad = (t.own_rows + c.past_frames * t.past_pad + 15) / 16 * 16;
+    if (c.keep_per_segment > 0) return t;               // pages of different lengths are not one regular tensor
+  }
   t.n_mt = (c.tokens_per_frame + 127) / 128;
-  t.ps_stages = score_ps_stages(c.tokens_per_frame, c.head_dim, 227 * 1024);
-  t.smem_ps = score_ps_smem_bytes(c.tokens_per_frame, c.head_dim, t.ps_stages < 2 ? 2 : t.ps_stages);
+  t.ps_stages = score_ps_stages(t.npad, c.head_dim, 227 * 1024);
+  t.smem_ps = score_ps_smem_bytes(t.npad, c.head_dim, t.ps_stages < 2 ? 2 : t.ps_stages);
   t.ok = t.ps_stages >= 2 && t.npad <= kPsSplit * kPsAccCols;
   return t;
 }
@@ -362,7 +373,8 @@ cudaError_t raise_kernel_limits(int* n_sms) {
   }
   if (e == cudaSuccess) e = raise_smem_limit((const void*)rank_kernel, optin);
   if (e == cudaSuccess) e = raise_smem_limit((const void*)segsel_kernel, optin);
-  if (e == cudaSuccess) e = raise_smem_limit((const void*)score_ps_kernel, optin);
+  if (e == cudaSuccess) e = raise_smem_limit((const void*)score_ps_kernel<false>, optin);
+  if (e == cudaSuccess) e = raise_smem_limit((const void*)score_ps_kernel<true>, optin);
   if (e == cudaSuccess) g_limits_raised[dev] = true;
   return e;
 }
@@ -394,6 +406,22 @@ bool encode_map3(CUtensorMap* m, const void* base, int D, int mid, long long row
   const cuuint32_t box[3] = {64u, (cuuint32_t)box_mid, (cuuint32_t)box_rows};
   const cuuint32_t estr[3] = {1u, 1u, 1u};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The pages of a store with frame-level selection, bf16: [frames][2L planes][kappa rows][Hkv][D] as a
+// rank-5 map; the box is the kappa rows of one key head in one plane of one page, 64 channels wide.
+bool encode_map_pages(CUtensorMap* m, const void* pages, int D, int Hkv, int kappa, int planes, long long frames,
+                      long long page_bytes) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t row = (cuuint64_t)Hkv * D * 2;
+  const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)Hkv, (cuuint64_t)kappa, (cuuint64_t)planes, (cuuint64_t)frames};
+  const cuuint64_t strides[4] = {(cuuint64_t)D * 2, row, row * kappa, (cuuint64_t)page_bytes};
+  const cuuint32_t box[5] = {64u, 1u, (cuuint32_t)kappa, 1u, 1u};
+  const cuuint32_t estr[5] = {1u, 1u, 1u, 1u, 1u};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(pages), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -457,7 +485,7 @@ cudaError_t launch_score_ps(mukv_ctx* ctx, const ScoreParams& sp, const void* d_
   CUtensorMap qmap, kmap;
   const long long rows = (long long)ctx->Ls * n * P;
   if (!encode_map3(&qmap, d_q, D, c.n_q_heads, rows, ctx->G, t.tpt) ||
-      !encode_map3(&kmap, k_last, D, c.n_kv_heads, rows, 1, t.npad)) {
+      !encode_map3(&kmap, k_last, D, c.n_kv_heads, rows, 1, t.own_rows)) {
     *why = "cuTensorMapEncodeTiled failed";
     return cudaErrorInvalidValue;
   }
@@ -466,13 +494,18 @@ cudaError_t launch_score_ps(mukv_ctx* ctx, const ScoreParams& sp, const void* d_
   pp.sp = sp;
   pp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
   pp.tiles = t.tiles; pp.tpt = t.tpt; pp.npad = t.npad; pp.n_mt = t.n_mt; pp.n_stages = t.ps_stages;
+  pp.own_rows = t.own_rows; pp.n_past = sp.n_past_frames; pp.past_pad = t.past_pad; pp.kappa = c.keep_per_frame;
+  pp.past_plane0 = 2 * sp.first_score_layer; pp.past_first = sp.past_first;
   pp.n_items = n * ctx->Ls * c.n_kv_heads * (t.n_mt + t.tiles);
   pp.exp2_scale = (float)(1.4426950408889634 / std::sqrt((double)D));
   pp.status = reinterpret_cast<int*>(ctx->ws + ctx->wl.dev_status);
   int blocks = ctx->n_sms < kPsMaxBlocks ? ctx->n_sms : kPsMaxBlocks;
   if (blocks > pp.n_items) blocks = pp.n_items;
   *ps_grid = blocks; *ps_items = pp.n_items; *ps_ipf = ctx->Ls * c.n_kv_heads * (t.n_mt + t.tiles);
-  score_ps_kernel<<<blocks, kPsThreads, t.smem_ps, st>>>(pp, qmap, kmap, ctx->wmap);
+  if (sp.n_past_frames)
+    score_ps_kernel<true><<<blocks, kPsThreads, t.smem_ps, st>>>(pp, qmap, kmap, ctx->wmap, ctx->pmap);
+  else
+    score_ps_kernel<false><<<blocks, kPsThreads, t.smem_ps, st>>>(pp, qmap, kmap, ctx->wmap, kmap);
   *why = "score_ps kernel";
   return cudaGetLastError();
 }
@@ -855,7 +888,6 @@ mukv_status create_impl(const mukv_config* cfg, void* d_store, size_t store_byte
   ctx->esize = cfg->dtype == MUKV_BF16 ? 2 : 4;
   ctx->key_rows = cfg->tokens_per_frame + cfg->past_frames * cfg->keep_per_frame;
   ctx->nc = pick_nc(ctx->key_rows);
-  ctx->force_fma = cfg->past_frames > 0;       // the tensor-core kernel holds the frame's own keys only
   ctx->tcs = tc_shape(*cfg);
   ctx->n_sms = 1;
   ctx->flag_margin = kFlagMargin;
@@ -877,6 +909,10 @@ mukv_status create_impl(const mukv_config* cfg, void* d_store, size_t store_byte
     const std::vector<uint16_t> w = dft_terms(D);
     e = cudaMemcpy(ctx->ws + ctx->wl.wtab, w.data(), w.size() * 2, cudaMemcpyHostToDevice);
     if (e == cudaSuccess && !encode_map2(&ctx->wmap, ctx->ws + ctx->wl.wtab, D, 3LL * D, D)) e = cudaErrorInvalidValue;
+    if (e == cudaSuccess && cfg->past_frames > 0 &&
+        !encode_map_pages(&ctx->pmap, ctx->store + ctx->sl.pages, D, cfg->n_kv_heads, cfg->keep_per_frame, 2 * cfg->n_layers,
+                          cfg->max_frames, (long long)ctx->sl.page_bytes))
+      e = cudaErrorInvalidValue;
   }
   if (e == cudaSuccess)
     e = cudaMemset(ctx->ws + ctx->wl.zero_begin, 0, ctx->wl.zero_end - ctx->wl.zero_begin);

@@ -53,7 +53,13 @@ typedef NamedGroup<5, kPsEpiThreads, kPsEpiOff> PsEpiGroup;
 
 struct ScorePsParams {
   ScoreParams sp;            // colsum_part: float [grid + n_frames][P] slots, ifft_part: float [F][Hkv][P]
-  int tiles, tpt, npad, n_mt;
+  int tiles, tpt, npad, n_mt;  // npad: rows of a key tile = columns of an attention product
+  // cached keys the queries also attend to (Sec. 3.2): rows own_rows + w * past_pad .. + kappa of the key
+  // tile hold the kept keys of frame past_first + w (w < n_past), read from that frame's page
+  int own_rows;              // rows the box of the frame's own keys covers (P rounded up to 8 with cached keys, else npad)
+  int n_past, past_pad, kappa;
+  int past_plane0;           // plane (layer * 2) of the first scoring layer's keys in a page
+  long long past_first;
   int n_stages;              // operand stages in the ring (2 .. kPsMaxStages)
   int n_items;               // n_frames * Ls * Hkv * (n_mt + tiles)
   float exp2_scale;          // log2(e) / sqrt(D)
@@ -62,13 +68,13 @@ struct ScorePsParams {
 
 constexpr int kPsMaxStages = 6;
 // two key buffers + n_stages operand stages + scratch (+ slack to align the tiles to 1024 bytes)
-__host__ inline size_t score_ps_smem_bytes(int P, int D, int n_stages) {
-  const size_t KB = D / 64, npad = (P + 15) / 16 * 16;
-  return 2 * KB * npad * 128 + (size_t)n_stages * KB * 128 * 128 + kPsMiscBytes + 1024;
+__host__ inline size_t score_ps_smem_bytes(int npad, int D, int n_stages) {
+  const size_t KB = D / 64;
+  return 2 * KB * (size_t)npad * 128 + (size_t)n_stages * KB * 128 * 128 + kPsMiscBytes + 1024;
 }
-__host__ inline int score_ps_stages(int P, int D, size_t limit) {
+__host__ inline int score_ps_stages(int npad, int D, size_t limit) {
   int n = kPsMaxStages;
-  while (n >= 2 && score_ps_smem_bytes(P, D, n) > limit) --n;
+  while (n >= 2 && score_ps_smem_bytes(npad, D, n) > limit) --n;
   return n;                  // < 2: the kernel does not fit
 }
 
@@ -100,8 +106,13 @@ __device__ __forceinline__ float sqrt_approx(float x) {
   return y;
 }
 
-__device__ __forceinline__ float ps_chunk_max(const uint32_t (&r)[16], int col0, int P, bool causal, int i_tok) {
-  if (!causal && col0 + 16 <= P) {
+// vm: bit k set when column col0 + k of the key tile holds a key (an own token or a cached past key);
+// with a causal mask an own token j (j < P) also needs j <= i_tok
+// (PAST = false: the tile holds the frame's own keys only and vm is not looked at: column j holds a key when j < P)
+template <bool PAST>
+__device__ __forceinline__ float ps_chunk_max(const uint32_t (&r)[16], int col0, int P, uint32_t vm, bool causal,
+                                              int i_tok) {
+  if (!causal && (PAST ? vm == 0xffffu : col0 + 16 <= P)) {
     const float a = tc::fmax3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
     const float b = tc::fmax3(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
     const float c = tc::fmax3(__uint_as_float(r[6]), __uint_as_float(r[7]), __uint_as_float(r[8]));
@@ -113,17 +124,18 @@ __device__ __forceinline__ float ps_chunk_max(const uint32_t (&r)[16], int col0,
 #pragma unroll
   for (int k = 0; k < 16; ++k) {
     const int j = col0 + k;
-    const bool ok = (j < P) && (!causal || j <= i_tok);
+    const bool ok = PAST ? ((vm >> k) & 1u) && (!causal || j >= P || j <= i_tok) : (j < P) && (!causal || j <= i_tok);
     m = ok ? fmaxf(m, __uint_as_float(r[k])) : m;
   }
   return m;
 }
 
 // r <- exp2(r * c - mc) (0 where masked); returns the sum
-__device__ __forceinline__ float ps_chunk_exp(uint32_t (&r)[16], float c, float mc, int col0, int P, bool causal,
-                                              int i_tok) {
+template <bool PAST>
+__device__ __forceinline__ float ps_chunk_exp(uint32_t (&r)[16], float c, float mc, int col0, int P, uint32_t vm,
+                                              bool causal, int i_tok) {
   float l0 = 0.f, l1 = 0.f;
-  if (!causal && col0 + 16 <= P) {
+  if (!causal && (PAST ? vm == 0xffffu : col0 + 16 <= P)) {
 #pragma unroll
     for (int k = 0; k < 16; k += 2) {
       const float e0 = ex2_approx(fmaf(__uint_as_float(r[k]), c, -mc));
@@ -137,7 +149,7 @@ __device__ __forceinline__ float ps_chunk_exp(uint32_t (&r)[16], float c, float 
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
       const int j = col0 + k;
-      const bool ok = (j < P) && (!causal || j <= i_tok);
+      const bool ok = PAST ? ((vm >> k) & 1u) && (!causal || j >= P || j <= i_tok) : (j < P) && (!causal || j <= i_tok);
       const float e = ok ? ex2_approx(fmaf(__uint_as_float(r[k]), c, -mc)) : 0.f;
       l0 += e;
       r[k] = __float_as_uint(e);
@@ -146,10 +158,14 @@ __device__ __forceinline__ float ps_chunk_exp(uint32_t (&r)[16], float c, float 
   return l0 + l1;
 }
 
+// PAST: the key tile also holds cached keys of past frames (a second instantiation, so that the common
+// case keeps its shorter inner loop: the epilogue is bound by instruction issue)
+template <bool PAST>
 __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
                                                  const __grid_constant__ CUtensorMap qmap,
                                                  const __grid_constant__ CUtensorMap kmap,
-                                                 const __grid_constant__ CUtensorMap wmap) {
+                                                 const __grid_constant__ CUtensorMap wmap,
+                                                 const __grid_constant__ CUtensorMap pmap) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = tc::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -207,6 +223,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
     tc::prefetch_tmap(&qmap);
     tc::prefetch_tmap(&kmap);
     tc::prefetch_tmap(&wmap);
+    if (PAST) tc::prefetch_tmap(&pmap);
   }
   // ---- TMA producer (thread 0).  The key tile of the block's first (frame, head) and its first
   // operand stage are requested here, before the block-wide barrier and with as little code in
@@ -214,11 +231,25 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
   // that they are on their way while tensor memory is being allocated; produce() issues the rest.
   int pr_i = i0, pr_t = 0, pr_nk = 0, pr_ns = 0, pr_unit = -1;
   bool pr_ok = true;
+  // the key tile of a unit into key buffer kb_i: the frame's own keys, then the cached keys of the past frames
+  const uint32_t k_tx = (uint32_t)KB * 128u * (uint32_t)(p.own_rows + (PAST ? p.n_past * p.kappa : 0));
+  auto load_keys = [&](int unit, int kb_i) {
+    const uint32_t dst = sK + (uint32_t)kb_i * k_buf, bar = PS_BAR_KF(kb_i);
+    const int g = unit % Hkv;
+    tc::mbar_expect_tx(bar, k_tx);
+    for (int kb = 0; kb < KB; ++kb) tc::tma_load_3d(dst + kb * k_kb, &kmap, kb * 64, g, unit_row(unit), bar);
+    if constexpr (PAST) {
+      const int plane = p.past_plane0 + 2 * ((unit / Hkv) % Ls);
+      for (int w = 0; w < p.n_past; ++w)
+        for (int kb = 0; kb < KB; ++kb)
+          tc::tma_load_5d(dst + kb * k_kb + (uint32_t)(p.own_rows + w * p.past_pad) * 128u, &pmap, kb * 64, g, 0, plane,
+                          (int)(p.past_first + w), bar);
+    }
+  };
   if (tid == 0) {
     const int unit0 = i0 / ipu, x0 = i0 - unit0 * ipu;
     const int g0 = unit0 % Hkv, r0 = unit_row(unit0);
-    tc::mbar_expect_tx(PS_BAR_KF(0), k_buf);
-    for (int kb = 0; kb < KB; ++kb) tc::tma_load_3d(sK + kb * k_kb, &kmap, kb * 64, g0, r0, PS_BAR_KF(0));
+    load_keys(unit0, 0);
     if (x0 < p.n_mt) {
       tc::mbar_expect_tx(PS_BAR_SF(0), (uint32_t)KB * (uint32_t)D * 128u);
       for (int kb = 0; kb < KB; ++kb) tc::tma_load_2d(sS + kb * st_kb, &wmap, kb * 64, 2 * D, PS_BAR_SF(0));
@@ -238,9 +269,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
         const int kb_i = pr_nk & 1;
         pr_ok = tc::mbar_wait(PS_BAR_KE(kb_i), (uint32_t)(((pr_nk >> 1) & 1) ^ 1));
         if (!pr_ok) break;
-        tc::mbar_expect_tx(PS_BAR_KF(kb_i), k_buf);
-        for (int kb = 0; kb < KB; ++kb)
-          tc::tma_load_3d(sK + (uint32_t)kb_i * k_buf + kb * k_kb, &kmap, kb * 64, g, urow, PS_BAR_KF(kb_i));
+        load_keys(unit, kb_i);
         ++pr_nk;
         pr_unit = unit;
       }
@@ -359,11 +388,29 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
     const int row_tok = row / G;                         // token of this row inside its tile
     const uint32_t tlane = (uint32_t)(q * 32) << 16;
     // the columns of a row go to its four warps in chunks of 16
-    const int nch16 = (P + 15) >> 4, ch_base = nch16 / kPsSplit, ch_rem = nch16 % kPsSplit;
+    const int nch16 = p.npad >> 4, ch_base = nch16 / kPsSplit, ch_rem = nch16 % kPsSplit;
     const int my_c0 = h * ch_base + (h < ch_rem ? h : ch_rem), my_nch = ch_base + (h < ch_rem ? 1 : 0);
     const bool causal = sp.causal != 0;
     const float c = p.exp2_scale;
     constexpr int kMaxCh = kPsAccCols / 16;
+    // which of the 16 columns from col0 on hold a key: the frame's own tokens, and behind them the
+    // kappa cached keys at the front of every past frame's share of the tile
+    const int past_end = p.own_rows + p.n_past * p.past_pad;
+    auto chunk_mask = [&](int col0) -> uint32_t {
+      const int nv = P - col0;
+      uint32_t vm = nv >= 16 ? 0xffffu : (nv <= 0 ? 0u : (1u << nv) - 1u);
+      if (col0 + 16 > p.own_rows && col0 < past_end) {
+        int r = col0 - p.own_rows, rem = r >= 0 ? r % p.past_pad : 0;
+#pragma unroll
+        for (int k = 0; k < 16; ++k, ++r) {
+          if (r >= 0 && r < past_end - p.own_rows) {
+            if (rem < p.kappa) vm |= 1u << k;
+            rem = rem + 1 == p.past_pad ? 0 : rem + 1;
+          }
+        }
+      }
+      return vm;
+    };
     float acc[kPsAccCols];                               // column sums of this thread's row, over tiles
 #pragma unroll
     for (int k = 0; k < kPsAccCols; ++k) acc[k] = 0.f;
@@ -423,9 +470,10 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
           uint32_t ra[16];
           tc::tmem_ld16(tb + col, ra);
           tc::tmem_wait_ld16(ra);
-          const float m_new = fmaxf(m_run, ps_chunk_max(ra, col, P, causal, i_tok));
+          const uint32_t vm = PAST ? chunk_mask(col) : 0u;
+          const float m_new = fmaxf(m_run, ps_chunk_max<PAST>(ra, col, P, vm, causal, i_tok));
           const float resc = (m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * c);
-          l = l * resc + ps_chunk_exp(ra, c, m_new * c, col, P, causal, i_tok);
+          l = l * resc + ps_chunk_exp<PAST>(ra, c, m_new * c, col, P, vm, causal, i_tok);
           tc::tmem_st16(tb + col, ra);
           s_mref[ch * kPsEpiThreads + et] = m_new;
           m_run = m_new;

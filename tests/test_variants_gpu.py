@@ -140,6 +140,39 @@ def test_scoring_layer_choice_fp32():
     H.check_frames_against_oracle(run, st, range(3), full_layers=True)
 
 
+def _small_bf16_spec(T):
+    return H.StreamSpec(seed=71, n_layers=3, n_q_heads=8, n_kv_heads=2, head_dim=64, tokens_per_frame=100, bf16=True,
+                        n_outlier=1, n_frames=T, scene_sigma=1.0, frame_sigma=0.5, scene_min=2, scene_max=4)
+
+
+def test_past_keys_with_two_scoring_layers_bf16():
+    # cached keys of the matching layer for each scoring layer (planes of the stored pages)
+    import copy
+    T, chunk, W = 7, 2, 3
+    spec = _small_bf16_spec(T)
+    run = H.GpuRun(dict(spec=spec, keep=25, fseg=2, chunk=chunk, alpha=0.7), past_frames=W, n_score_layers=2,
+                   score_layer_offset=0)
+    c = run.cfg
+    sp2 = copy.copy(spec)
+    sp2.seed = spec.seed + 100
+    st = O.Store(H.oracle_cfg(c))
+    kept = torch.full((T, c.keep_per_frame), -1, dtype=torch.int32, device=run.device)
+    scores = torch.zeros((3, T, c.tokens_per_frame), dtype=torch.float32, device=run.device)
+    for t0 in range(0, T, chunk):
+        n = min(chunk, T - t0)
+        q, k, v = spec.chunk(t0, n)
+        q = np.stack([q, np.stack([sp2.frame_q(t) for t in range(t0, t0 + n)])])
+        O.compress_chunk(st, q, k, v)
+        dq, dk, dv = (H.to_device(x, True, run.device) for x in (q, k, v))
+        sc = torch.empty((3, n, c.tokens_per_frame), dtype=torch.float32, device=run.device)
+        run.ctx.mukv_compress_chunk(dq, dk, dv, n, t0, kept[t0:t0 + n], sc)
+        scores[:, t0:t0 + n] = sc
+    torch.cuda.synchronize()
+    run.kept, run.scores = kept.cpu().numpy(), scores.cpu().numpy()
+    H.check_frames_against_oracle(run, st, range(T), full_layers=True)
+    assert st.scores[T - 1][0].sum() < 0.999 and run.ctx.mukv_get_stats().device_status == 0
+
+
 def _oracle_chunked(spec, ocfg, T, chunk):
     st = O.Store(ocfg)
     for t0 in range(0, T, chunk):
@@ -153,9 +186,16 @@ def _oracle_chunked(spec, ocfg, T, chunk):
     ("tiny", 8, 2, 2, dict(attn_causal=1), None),
     ("chunk7b", 6, 2, 1, dict(), None),
     ("chunk7b", 5, 2, 1, dict(attn_causal=1), {B.OPT_FLAG_MARGIN: 1.0}),
+    ("chunk7b", 4, 2, 1, dict(), {B.OPT_SCORE_PATH: 1}),
+    ("small_bf16", 9, 2, 3, dict(), None),
+    ("small_bf16", 7, 3, 2, dict(attn_causal=1, keep_low_freq=1), None),
 ])
 def test_past_keys_in_the_attention(name, T, chunk, W, over, opts):
-    # Sec. 3.2: the queries of a chunk also attend to the kept keys of the W frames stored before it
+    # Sec. 3.2: the queries of a chunk also attend to the kept keys of the W frames stored before it.
+    # bf16 chunks go through the tensor-core kernel (the cached keys are rows of its key tile) unless
+    # the multiply-add path is asked for; "small_bf16" has room for three past frames in the tile
+    if name == "small_bf16":
+        name = dict(spec=_small_bf16_spec(T), keep=25, fseg=2, chunk=chunk, alpha=0.7)
     run = H.GpuRun(name, n_frames=T, past_frames=W, options=opts, **over)
     run.compress(chunk)
     st = _oracle_chunked(run.spec, H.oracle_cfg(run.cfg), T, chunk)
@@ -164,5 +204,5 @@ def test_past_keys_in_the_attention(name, T, chunk, W, over, opts):
     assert abs(st.scores[0][0].sum() - 1.0) < 1e-9 and st.scores[T - 1][0].sum() < 0.999
     stats = run.ctx.mukv_get_stats()
     assert stats.device_status == 0
-    if opts:
+    if opts and B.OPT_FLAG_MARGIN in opts:
         assert stats.refined_frames == T
