@@ -116,6 +116,99 @@ def algorithmic_bytes(cfg, k_frm: int) -> dict:
                 gather_per_question=gather_q, index_row=C * 4)
 
 
+def next_rows(B, GpuStream, wl, dev, peaks, frames: int) -> dict:
+    """The variants of the path beyond the headline configuration, timed at the shape of the workload on a
+    shorter stream (`frames` frames): other scoring layers, cached past keys in the attention, segment-level
+    selection, a patch level with retrieval over three granularities.  Device time, CUDA events around the
+    library calls, the chunk generator excluded; every chunk is generated right before its call."""
+    import statistics as st
+    import torch
+    spec, chunk = wl["spec"], wl["chunk"]
+    T = frames - frames % chunk
+    gs = GpuStream(spec, dev)
+    q, k, v = gs.alloc(chunk)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    n_calls = T // chunk
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_calls)]
+
+    def compress(**over):
+        Ls = max(1, over.get("n_score_layers", 0))
+        qs = torch.empty((Ls,) + tuple(q.shape), dtype=q.dtype, device=dev) if Ls > 1 else None
+        kw = dict(n_layers=spec.n_layers, n_q_heads=spec.n_q_heads, n_kv_heads=spec.n_kv_heads,
+                  head_dim=spec.head_dim, tokens_per_frame=spec.tokens_per_frame, keep_per_frame=wl["keep"],
+                  frames_per_segment=wl["fseg"], max_frames_per_chunk=chunk, max_frames=T, alpha=wl["alpha"])
+        kw.update(over)
+        cfg = B.make_config(**kw)
+        ctx = B.MukvContext(cfg, dev)
+        for _ in range(3):
+            ctx.mukv_reset()
+            for i in range(n_calls):
+                gs.fill(i * chunk, chunk, q, k, v)
+                if qs is not None:                            # the same queries stand in for every scoring layer
+                    for layer in range(Ls):
+                        qs[layer].copy_(q)
+                ev[i][0].record()
+                ctx.mukv_compress_chunk(q if qs is None else qs, k, v, chunk, i * chunk)
+                ev[i][1].record()
+            torch.cuda.synchronize()
+        us = st.median(1e3 * a.elapsed_time(b) for a, b in ev[1:])
+        stats = ctx.mukv_get_stats()
+        ab = algorithmic_bytes(cfg, wl["k_frm"])
+        fps = chunk / us * 1e6
+        return ctx, cfg, {"us_per_chunk": us, "frames_per_s": fps, "refined_frames": int(stats.refined_frames),
+                          "frac_of_hbm_peak": ab["per_frame"] * fps / 1e9 / peaks["hbm_gbs"],
+                          "device_status": int(stats.device_status)}
+
+    P = spec.tokens_per_frame
+    width = int(round(P ** 0.5))
+    if width * width != P:
+        width = P
+    out = {"frames": T, "chunk_frames": chunk}
+    for name, over in (("scoring_layers_last5", dict(n_score_layers=5)),
+                       ("scoring_layer_penultimate", dict(n_score_layers=1, score_layer_offset=1)),
+                       ("past_frames_1", dict(past_frames=1)),
+                       ("segment_level_selection", dict(keep_per_segment=wl["keep"] * wl["fseg"]))):
+        ctx, _, out[name] = compress(**over)
+        del ctx
+    ctx, cfg, out["patch_level_2x2"] = compress(patch_split=2, grid_width=width)
+    # retrieval over three granularities with the paper's k_g = {20, 32, 12}, lambda_g = {0.3, 0.3, 0}
+    nq = wl["n_questions"]
+    qtok_np, offs, _ = spec.questions(nq, *wl["q_len"])
+    qtok = torch.from_numpy(qtok_np).view(torch.int16).to(dev).view(torch.bfloat16)
+    kp, kf, ks = 20, 32, 12
+    i32, f32 = torch.int32, torch.float32
+    seg, frm, pat = (torch.empty((nq, n), dtype=i32, device=dev) for n in (ks, kf, kp))
+    ssc, fsc, psc = (torch.empty((nq, n), dtype=f32, device=dev) for n in (ks, kf, kp))
+    counts = torch.empty((nq, 3), dtype=i32, device=dev)
+    cap = ctx.mukv_decode3_tokens(ks, kf, kp)
+    row_bytes = cfg.n_kv_heads * cfg.head_dim * 2
+    stride = cfg.n_layers * 2 * cap * row_bytes
+    dec = torch.empty((nq, stride), dtype=torch.uint8, device=dev)
+    ntok = torch.empty((nq,), dtype=i32, device=dev)
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    out["retrieve3"] = {"k_patch": kp, "k_frm": kf, "k_seg": ks, "questions": nq}
+    for mode, mname in ((B.RETR_SEMI, "semi"), (B.RETR_HIER, "hier"), (B.RETR_PARALLEL, "parallel")):
+        prm = B.MukvRetrParams(kp, kf, ks, 0.3, 0.3, 0.0, 0, mode)
+        tr, tg = [], []
+        for _ in range(7):
+            flush.zero_()
+            e[0].record()
+            ctx.mukv_retrieve3(qtok, offs, None, prm, seg, frm, pat, ssc, fsc, psc, counts)
+            e[1].record()
+            ctx.mukv_gather3(seg, frm, pat, counts, nq, ks, kf, kp, dec, stride, ntok, None)
+            e[2].record()
+            torch.cuda.synchronize()
+            tr.append(e[0].elapsed_time(e[1]))
+            tg.append(e[1].elapsed_time(e[2]))
+        tokens = float(ntok.sum().item())
+        g_ms = st.median(tg[2:])
+        gbs = 2.0 * tokens * cfg.n_layers * 2 * row_bytes / (g_ms * 1e-3) / 1e9
+        out["retrieve3"][mname] = {"retrieve_us": 1e3 * st.median(tr[2:]), "gather_us": 1e3 * g_ms,
+                                   "tokens_per_question": tokens / nq, "gather_gbs": gbs,
+                                   "gather_frac_of_hbm_peak": gbs / peaks["hbm_gbs"]}
+    return out
+
+
 def oracle_sample(n_frames: int, n_questions: int):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload.  Returns
     (frames/s, retrievals/s, threads, description)."""
@@ -178,6 +271,8 @@ def main():
     ap.add_argument("--oracle-frames", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-next-rows", action="store_true", help="skip the timing of the variants beyond the headline path")
+    ap.add_argument("--next-frames", type=int, default=1600, help="frames of the stream the variants are timed on")
     ap.add_argument("--l2", default="inputs", choices=["inputs", "flush"],
                     help="inputs: every call reads a freshly generated 202 MB chunk (larger than L2); "
                          "flush: additionally overwrite L2 with a 256 MiB memset before every timed call")
@@ -402,6 +497,14 @@ def main():
         cpu = {"value": o_fps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
                "retrievals_per_s": o_rps}
 
+    nxt = None
+    if rank == 0 and world == 1 and not args.no_next_rows and cfg.dtype == 0:
+        decode.clear()
+        try:
+            nxt = next_rows(B, GpuStream, wl, dev, peaks, min(args.next_frames, T))
+        except Exception as ex:                               # the headline figures stand without them
+            nxt = {"error": f"{type(ex).__name__}: {ex}"}
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -425,6 +528,7 @@ def main():
             "roofline": roofline, "kernels": kernels,
             "refined_frames": int(stats.refined_frames),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "cpu_baseline": cpu,
+            "next_rows": nxt,
         }
         print(json.dumps(line))
     if world > 1:

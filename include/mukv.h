@@ -112,8 +112,11 @@ typedef struct {
   int32_t past_frames;           /* W: the queries of a chunk also attend to the kept keys
                                     of the W most recent frames stored before the chunk
                                     (Sec. 3.2: past KV of the same granularity); P + W *
-                                    kappa <= 256; such a context scores on the multiply-add
-                                    kernels (every dtype); not with keep_per_segment; 0 = none */
+                                    kappa <= 256; not with keep_per_segment; 0 = none.  A
+                                    bf16 context stays on the tensor-core kernel while
+                                    ceil8(P) + W * ceil8(kappa) <= 256 (the cached keys are
+                                    rows of its key tile), else it scores on the multiply-
+                                    add kernels, as every fp32 context does                */
   int32_t reserved;              /* set to 0                                            */
 } mukv_config;
 
