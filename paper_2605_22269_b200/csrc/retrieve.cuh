@@ -589,18 +589,21 @@ __global__ void __launch_bounds__(kRankThreads) rank_kernel(const RankParams p, 
   __syncthreads();
 
   // ---- frames
+  // HIER: only what lies inside the selected segments is a candidate.  Those are few, so the ranking
+  // runs over positions in the list "selected segments (ascending) x their frames" and maps the
+  // winners back (ascending position = ascending frame).
   const int fseg = p.fseg;
-  auto in_sel_seg = [&](int t) {
-    const int u = t / fseg;
-    for (int i = 0; i < c_seg; ++i)
-      if (sh.sel_seg[i] == u) return true;
-    return false;
-  };
   int c_frm;
-  if (p.mode == MUKV_RETR_HIER)
-    c_frm = rank_level(sf, in_sel_seg, n_frm, p.k_frm, false, 0.0, p.delta, p.frame_key, C, gq, gnorm, have_g, &sh);
-  else
+  if (p.mode == MUKV_RETR_HIER) {
+    auto frame_of = [&](int i) { return sh.sel_seg[i / fseg] * fseg + i % fseg; };
+    auto score_h = [&](int i) { return sf[frame_of(i)]; };
+    auto member_h = [&](int i) { return frame_of(i) < n_frm; };
+    c_frm = block_topk_set(score_h, member_h, c_seg * fseg, p.k_frm, p.delta, sh.pick, sh.pick_score, &sh.sc);
+    for (int i = tid; i < c_frm; i += kRankThreads) sh.pick[i] = frame_of(sh.pick[i]);
+    __syncthreads();
+  } else {
     c_frm = rank_level(sf, always, n_frm, p.k_frm, semi, p.lam_frm, p.delta, p.frame_key, C, gq, gnorm, have_g, &sh);
+  }
   rank_emit(p.frm_idx, p.frm_score, (long long)qi * p.k_frm, p.k_frm, c_frm, &sh);
   __syncthreads();
 
@@ -612,8 +615,16 @@ __global__ void __launch_bounds__(kRankThreads) rank_kernel(const RankParams p, 
     const double* spat = p.s_pat + (long long)qi * p.pat_stride;
     if (S > 0) {
       if (p.mode == MUKV_RETR_HIER) {
-        auto member = [&](int b) { return cnt[b] > 0 && in_sel_seg(b / S); };
-        c_pat = rank_level(spat, member, n_frm * S, p.k_pat, false, 0.0, p.delta, p.patch_key, C, gq, gnorm, have_g, &sh);
+        const int per_seg = fseg * S;
+        auto block_of = [&](int i) { return sh.sel_seg[i / per_seg] * per_seg + i % per_seg; };
+        auto score_h = [&](int i) { return spat[block_of(i)]; };
+        auto member_h = [&](int i) {
+          const int b = block_of(i);
+          return b < n_frm * S && cnt[b] > 0;
+        };
+        c_pat = block_topk_set(score_h, member_h, c_seg * per_seg, p.k_pat, p.delta, sh.pick, sh.pick_score, &sh.sc);
+        for (int i = tid; i < c_pat; i += kRankThreads) sh.pick[i] = block_of(sh.pick[i]);
+        __syncthreads();
       } else {
         auto member = [&](int b) { return cnt[b] > 0; };
         c_pat = rank_level(spat, member, n_frm * S, p.k_pat, semi, p.lam_pat, p.delta, p.patch_key, C, gq, gnorm, have_g,
