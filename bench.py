@@ -27,8 +27,8 @@ if ROOT not in sys.path:
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture) of one launch of the
 # kernel on a 16-frame chunk of this workload; reported as `roofline.traffic`
-SCORE_TRAFFIC_BYTES = 25858560
-COMPACT_TRAFFIC_BYTES = 45204224 + 3888640
+SCORE_TRAFFIC_BYTES = 25858304
+COMPACT_TRAFFIC_BYTES = 45205248 + 3958784
 
 METRIC = "compressed_frames_per_s"
 UNIT = "frames/s"
@@ -273,6 +273,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-next-rows", action="store_true", help="skip the timing of the variants beyond the headline path")
     ap.add_argument("--next-frames", type=int, default=1600, help="frames of the stream the variants are timed on")
+    ap.add_argument("--only-next-rows", action="store_true",
+                    help="time the variants only and print {\"next_rows\": ...} (profiling)")
     ap.add_argument("--l2", default="inputs", choices=["inputs", "flush"],
                     help="inputs: every call reads a freshly generated 202 MB chunk (larger than L2); "
                          "flush: additionally overwrite L2 with a 256 MiB memset before every timed call")
@@ -297,6 +299,10 @@ def main():
     dev = f"cuda:{local}"
     wl = workload(WORKLOAD)
     spec = wl["spec"]
+    if args.only_next_rows:
+        if rank == 0:
+            print(json.dumps({"next_rows": next_rows(B, GpuStream, wl, dev, load_peaks(), args.next_frames)}))
+        return
     spec.seed = spec.seed + 1000 * rank                      # every replica compresses its own stream
     T = args.frames or spec.n_frames
     chunk = wl["chunk"]
