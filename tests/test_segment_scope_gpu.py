@@ -127,8 +127,12 @@ def test_segment_scope_sixteen_frame_segments(over):
         run.ctx.mukv_compress_chunk(dq, dk, dv, n, t0, kept[t0:t0 + n], sc)
         scores[:, t0:t0 + n] = sc
     torch.cuda.synchronize()
-    check_store(run, st, kept.cpu().numpy(), scores.cpu().numpy())
+    sc_np = scores.cpu().numpy()
+    check_store(run, st, kept.cpu().numpy(), sc_np)
     assert run.ctx.mukv_get_stats().refined_frames <= 16
+    # the headroom the single-precision ranking rests on: fused scores within half the safety margin
+    worst = max(float(np.max(np.abs(sc_np[2, t] - st.scores[t][2]))) for t in range(T))
+    assert worst < H.FLAG_MARGIN / 2, worst
 
 
 def oracle_stream_chunked(spec, ocfg, T, chunk):
