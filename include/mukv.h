@@ -180,13 +180,19 @@ mukv_status mukv_set_option(mukv_ctx* ctx, int32_t option, double value);
  * Per frame the call scores every token, keeps the kappa best (ties within tie_eps go to
  * the lowest index), copies their K/V rows of all layers into the frame's page, writes the
  * frame-level entry (float mean of the kept rows per layer, K and V) and refreshes the
- * entry of every segment the chunk touches (mean over the frames present so far).
+ * entry of every segment the chunk touches (mean over the frames present so far).  With
+ * frame-level selection that last step is owed to the store until it is next needed: the
+ * next compress call, mukv_retrieve / mukv_retrieve3, mukv_gather3, mukv_store_region or
+ * mukv_export_header pools the entries before anything reads them (the library's own kernel,
+ * on the stream of the call that needs them).
  * Frames whose selection lies too close to a tie boundary for single precision are
  * re-scored in double precision on the device before they are stored.
  * With keep_per_segment = kappa_v > 0 the selection is made per segment: first_frame must be a
  * multiple of frames_per_segment and the chunk must hold whole segments (a last, shorter one ends
  * the stream and keeps kappa_v * frames / frames_per_segment tokens, rounded down); the min-max of
- * Eq. 4 and the ranking run over all tokens of a segment in double precision; frame t keeps n_t
+ * Eq. 4 and the ranking run over all tokens of a segment (bf16 chunks: scored on the tensor cores
+ * and ranked in single precision where the margin of mukv_set_option allows, else, like fp32
+ * chunks, in double precision); frame t keeps n_t
  * tokens (region 10), its page is [L][2][n_t][Hkv][D], kept ids are stored and returned as
  * [frames][P] int32 padded with -1 (d_kept_out must have that size), frames_per_segment * P <= 4096,
  * no patch level.  Such a store is read with mukv_retrieve / mukv_retrieve3 and mukv_gather3
@@ -294,14 +300,20 @@ mukv_status mukv_gather(mukv_ctx* ctx, const int32_t* d_frm_idx, const int32_t* 
  *        9 patch-level token counts (int32) [max_frames][S]
  *       10 tokens kept per frame (int32) [max_frames]       (keep_per_segment > 0; region 1 is then
  *          [max_frames][P], padded with -1, and region 0 is packed pages of different lengths)
- * Returns NULL for an unknown region; *bytes (if not NULL) receives the region size. */
+ * Returns NULL for an unknown region; *bytes (if not NULL) receives the region size.
+ * Segment entries and keys (regions 3, 5) of the chunk of the last compress call are pooled lazily
+ * (by the next compress call, or by whatever reads them first): this call, like
+ * mukv_export_header, launches that pooling on the stream of that compress call if it is still
+ * owed and waits for that stream, so what the pointer shows is complete; NULL also if that fails. */
 void* mukv_store_region(const mukv_ctx* ctx, int32_t which, size_t* bytes);
 
 /* Moving a store (the paper's "offline memory" outlives the questions; it prints no format).
  * The store buffer is position independent: every reference inside it is an offset from its
  * base.  mukv_export_header fills a small plain header (configuration, frames stored); the caller
  * copies the store's bytes wherever it likes (cudaMemcpy to another buffer, another device, the
- * host) once the stream has finished.  mukv_import builds a context over such a copy: like
+ * host) once the stream has finished (mukv_export_header itself waits for the stream of the last
+ * compress call when that call's segment entries were still to be pooled: see mukv_store_region;
+ * it returns MUKV_E_CUDA if that fails).  mukv_import builds a context over such a copy: like
  * mukv_create, but the store's contents are kept and the stream continues at header->frames.
  * Errors of mukv_import: INVALID (null, bad magic / version), SHAPE/DTYPE, ALIGN, CAPACITY
  * (store_bytes below header->store_bytes, workspace too small). */

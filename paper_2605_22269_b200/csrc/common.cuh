@@ -139,6 +139,20 @@ __device__ __forceinline__ int super_patch_index(int j, int P, int grid_width, i
 // the persistent scoring kernel take such shares of its item list)
 __device__ __forceinline__ int share_owner(unsigned i, unsigned n, unsigned nb) { return (int)(((i + 1u) * nb - 1u) / n); }
 
+// ---------------------------------------------------------------- segment entries (Eq. 5 at segment level)
+// What the pooling of segment entries needs, small enough to travel in registers (compact_segment_plane
+// is kept out of line so that its 32 loads in flight do not set the register count of the kernels that
+// call it; a reference to a kernel's parameter block would force a per-thread copy of the block instead).
+struct SegmentArgs {
+  int L, kappa, C, fseg, n_frames;
+  long long first_frame;
+  const float* frame_entry;
+  const double* frame_ksum;
+  float* seg_entry;
+  float* seg_key;
+  const int* kept_count;          // [max_frames] tokens kept per frame, or null: kappa in every frame
+};
+
 // 16-byte streaming copies
 __device__ __forceinline__ uint4 ld_stream(const void* p) {
   uint4 v;

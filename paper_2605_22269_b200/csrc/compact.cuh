@@ -56,6 +56,10 @@ struct CompactParams {
   int patch_split, grid_width;    // 0: no patch level
   float* patch_key;               // [max_frames][S][C]
   int* patch_cnt;                 // [max_frames][S]
+  int pool_always;                // segment_kernel: pool whatever the flagged count says (the entries of an earlier call)
+  // compact_kernel: with prev.n_frames > 0 the grid has one more row of blocks (the second one), which pools
+  // the segment entries the previous call left to this one
+  SegmentArgs prev;
   int sel_mode;                   // 0: kept ids are in the store; 1: select here from the partial sums;
                                   // 2: select here by the caller's scores; 3: ids and counts are in the store
                                   // (segment-level selection)
@@ -258,18 +262,6 @@ __device__ inline bool select_from_partials(const CompactParams& p, int f, bool 
   return risky;
 }
 
-// What compact_segment_plane needs, small enough to travel in registers (the function is kept out
-// of line so that its 32 loads in flight do not set the register count of the kernels that call it;
-// a reference to the kernel's parameter block would force a per-thread copy of the block instead).
-struct SegmentArgs {
-  int L, kappa, C, fseg, n_frames;
-  long long first_frame;
-  const float* frame_entry;
-  const double* frame_ksum;
-  float* seg_entry;
-  float* seg_key;
-  const int* kept_count;          // [max_frames] tokens kept per frame, or null: kappa in every frame
-};
 __device__ __forceinline__ SegmentArgs segment_args(const CompactParams& p) {
   SegmentArgs a;
   a.L = p.L; a.kappa = p.kappa; a.C = p.C; a.fseg = p.fseg; a.n_frames = p.n_frames; a.first_frame = p.first_frame;
@@ -539,7 +531,15 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(const Compa
   const int f = blockIdx.x;
   // block row -> plane l*2 + kv; with a patch level its blocks (plane 2L) sit in row 1, so that they run
   // in the first wave beside the copy blocks instead of alone at the end
-  const int row = blockIdx.y;
+  int row = blockIdx.y;
+  if (p.prev.n_frames > 0) {
+    if (row == 1) {
+      // nothing of this call is needed for the entries of the previous one: no wait for the scoring kernel
+      for (int pl = blockIdx.x; pl < 2 * p.prev.L; pl += gridDim.x) compact_segment_plane(p.prev, pl >> 1, pl & 1);
+      return;
+    }
+    if (row > 1) --row;
+  }
   const int plane = p.patch_split > 0 && row >= 1 ? (row == 1 ? 2 * p.L : row - 1) : row;
   pdl_wait();
   pdl_trigger();
@@ -631,7 +631,7 @@ constexpr int kStatusTailWait = 6;   // tail_kernel: the wait for the double-pre
 __global__ void __launch_bounds__(kCompactThreads) segment_kernel(const CompactParams p) {
   pdl_wait();
   pdl_trigger();
-  if (*p.sp.n_flagged != 0) return;
+  if (!p.pool_always && *p.sp.n_flagged != 0) return;
   for (int plane = blockIdx.x; plane < 2 * p.L; plane += gridDim.x)
     compact_segment_plane(segment_args(p), plane >> 1, plane & 1);
 }
@@ -644,7 +644,7 @@ __global__ void __launch_bounds__(kScoreThreads, 2) tail_kernel(const ScoreParam
   const int tid = threadIdx.x;
   pdl_wait();
   const int n_fl = *sp.n_flagged;
-  if (n_fl == 0) return;                        // the common case: segment_kernel has done what was left
+  if (n_fl == 0) return;                        // the common case: the next call pools this chunk's segment entries
   // ---- scores of the flagged frames in double precision; the block that finishes a frame last selects
   const int units = sp.Ls * sp.Hq * sp.row_split;
   for (int w = blockIdx.x; w < n_fl * units; w += gridDim.x) {

@@ -77,6 +77,12 @@ struct mukv_ctx {
   int tail_capacity = 1;                 // blocks of tail_kernel that are resident at once on this device
   CUtensorMap wmap;                      // DFT matrix terms [3*D][D] bf16
   CUtensorMap pmap;                      // the page region as [frame][plane][kept row][key head][D] (past_frames > 0)
+  // Segment entries a compress call left to whoever comes next (see flush_segments): the frames whose
+  // segments still have to be pooled, and the stream that call ran on
+  mutable bool seg_pending = false;
+  mutable long long seg_first = 0;
+  mutable int seg_n = 0;
+  mutable cudaStream_t seg_stream = nullptr;
   std::string err;
   // optional per-kernel timing (host objects only)
   bool prof_on = false;
@@ -475,6 +481,39 @@ std::vector<uint16_t> dft_terms(int D) {
   return w;
 }
 
+// The pooling of segment entries (Eq. 5 at segment level) for frames first .. first + n - 1.
+SegmentArgs segment_args_of(const mukv_ctx* ctx, long long first, int n) {
+  const mukv_config& c = ctx->cfg;
+  SegmentArgs a;
+  memset(&a, 0, sizeof a);
+  a.L = c.n_layers; a.kappa = c.keep_per_frame; a.C = ctx->C; a.fseg = c.frames_per_segment;
+  a.n_frames = n; a.first_frame = first;
+  a.frame_entry = reinterpret_cast<const float*>(ctx->store + ctx->sl.frame_entry);
+  a.frame_ksum = reinterpret_cast<const double*>(ctx->store + ctx->sl.frame_ksum);
+  a.seg_entry = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_entry);
+  a.seg_key = reinterpret_cast<float*>(ctx->store + ctx->sl.seg_key);
+  if (c.keep_per_segment > 0) a.kept_count = reinterpret_cast<const int*>(ctx->store + ctx->sl.kept_count);
+  return a;
+}
+
+// With frame-level selection a compress call does not pool the segment entries of its chunk itself (unless
+// frames were flagged: tail_kernel then does): the next compress call does it with one more row of blocks in its compaction
+// kernel, which do not wait for that call's scoring kernel.  Whoever else needs the entries first
+// (retrieval, a gather with summary tokens, a view of the store, an export) pools them with one launch here.
+cudaError_t flush_segments(const mukv_ctx* ctx, cudaStream_t st) {
+  if (!ctx->seg_pending) return cudaSuccess;
+  CompactParams cp;
+  memset(&cp, 0, sizeof cp);
+  const SegmentArgs a = segment_args_of(ctx, ctx->seg_first, ctx->seg_n);
+  cp.L = a.L; cp.kappa = a.kappa; cp.C = a.C; cp.fseg = a.fseg; cp.n_frames = a.n_frames; cp.first_frame = a.first_frame;
+  cp.frame_entry = const_cast<float*>(a.frame_entry); cp.frame_ksum = const_cast<double*>(a.frame_ksum);
+  cp.seg_entry = a.seg_entry; cp.seg_key = a.seg_key; cp.kept_count = a.kept_count;
+  cp.pool_always = 1;
+  const cudaError_t e = launch_k(segment_kernel, dim3(2 * a.L), kCompactThreads, 0, st, false, cp);
+  if (e == cudaSuccess) ctx->seg_pending = false;
+  return e;
+}
+
 // Scores a bf16 chunk on the tensor cores (Eq. 1-3; Eq. 4 and the selection follow in compact_kernel).
 cudaError_t launch_score_ps(mukv_ctx* ctx, const ScoreParams& sp, const void* d_q, const void* k_last, int n,
                             cudaStream_t st, const char** why, int* ps_grid, int* ps_items, int* ps_ipf) {
@@ -555,6 +594,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   cudaError_t e = cudaSuccess;
   const char* what = "score kernel";
   int ps_grid = 0, ps_items = 0, ps_ipf = 0;
+  int n_launch = 0;
   if (seg_scope) {
     // One block per segment ranks all its tokens.  A bf16 chunk is first scored on the tensor cores and
     // ranked from those single-precision sums; segments that are too close to call are scored and
@@ -578,6 +618,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
         e = launch_score_ps(ctx, sp, d_q, sp.k_last, n, st, &what, &ps_grid1, &ps_items1, &ps_ipf1);
       }
       if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "%s: %s", what, cudaGetErrorString(e));
+      n_launch += 2;
       gp.sp = sp;
       gp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
       gp.src32 = 1;
@@ -616,12 +657,14 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
       e = launch_k(segsel_kernel, dim3(n_seg), kSegSelThreads, segsel_smem_bytes(seg_tokens), st, tc_first && dep, gp);
     }
     if (e != cudaSuccess) return broke_off(ctx, "segment selection kernel", e);
+    n_launch += 2;
   } else if (!d_ext) {
     ProfScope ps(ctx, 0, st);
     if (ctx->tcs.ok && !ctx->force_fma)
       e = launch_score_ps(ctx, sp, d_q, sp.k_last, n, st, &what, &ps_grid, &ps_items, &ps_ipf);
     else
       e = launch_score<T, float>(sp, ctx->nc, grid, score_smem_bytes<T, float>(ctx->key_rows, c.head_dim), st);
+    ++n_launch;
   }
   if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "%s: %s", what, cudaGetErrorString(e));
 
@@ -652,20 +695,31 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   cp.ps_grid = ps_grid; cp.ps_items = ps_items; cp.ps_ipf = ps_ipf;
   cp.sp = sp;
   if (ps_grid > 0) cp.sp.colsum_part = ctx->ws + ctx->wl.colsum_p;
+  // segment entries the previous call left behind: one more row of blocks (with per-kernel timing on,
+  // a launch of their own, so that each kernel is timed doing its own work only)
+  if (ctx->seg_pending && ctx->prof_on) {
+    ProfScope ps(ctx, 3, st);
+    e = flush_segments(ctx, st);
+    if (e != cudaSuccess) return broke_off(ctx, "segment kernel", e);
+    ++n_launch;
+  }
+  if (ctx->seg_pending) cp.prev = segment_args_of(ctx, ctx->seg_first, ctx->seg_n);
   {
     ProfScope ps(ctx, 2, st);
-    e = launch_k(compact_kernel<T>, dim3(n, L * 2 + (c.patch_split > 0 ? 1 : 0)), kCompactThreads, 0, st, !ctx->prof_on,
-                 cp);
+    e = launch_k(compact_kernel<T>, dim3(n, L * 2 + (c.patch_split > 0 ? 1 : 0) + (ctx->seg_pending ? 1 : 0)),
+                 kCompactThreads, 0, st, !ctx->prof_on, cp);
   }
   if (e != cudaSuccess) return broke_off(ctx, "compact kernel", e);
+  ctx->seg_pending = false;
 
-  // What needs every frame of the chunk: the segment entries (segment_kernel, when no frame was
-  // flagged); otherwise, in tail_kernel, scores and selection of the flagged frames again in double
-  // precision, their compaction, and then the segment entries.
+  // The segment entries need every frame of the chunk.  With frame-level selection they are left to the
+  // next call (flush_segments); when frames were flagged, tail_kernel pools them after it has redone those
+  // frames.  With segment-level selection (count-weighted entries, no tail_kernel) they are pooled here.
   cp.sp.n_flagged = sp.n_flagged;
-  {
+  if (seg_scope) {
     ProfScope ps(ctx, 3, st);
     e = launch_k(segment_kernel, dim3(2 * L), kCompactThreads, 0, st, !ctx->prof_on, cp);
+    ++n_launch;
   }
   if (e != cudaSuccess) return broke_off(ctx, "segment kernel", e);
   sp.refine = 1;
@@ -678,10 +732,15 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
     if (grid_t < 2 * L + 1) grid_t = 2 * L + 1;
     if (grid_t > ctx->tail_capacity) grid_t = ctx->tail_capacity;
     e = launch_tail<T>(sp, cp, ctx->nc, grid_t, score_smem_bytes<T, double>(ctx->key_rows, c.head_dim), st, !ctx->prof_on);
+    ++n_launch;
   }
   if (e != cudaSuccess) return broke_off(ctx, "tail kernel", e);
+  ctx->seg_pending = !seg_scope;
+  ctx->seg_first = t0;
+  ctx->seg_n = n;
+  ctx->seg_stream = st;
 
-  ctx->launches += d_ext ? 3 : 4;
+  ctx->launches += n_launch + 1;                          // + compact_kernel
   ctx->parity ^= 1;
   ctx->frames = t0 + n;
   return MUKV_OK;
@@ -716,6 +775,11 @@ mukv_status retrieve_impl(mukv_ctx* ctx, const void* d_qtok, const int32_t* h_q_
     for (float lam : {prm.lambda_patch, prm.lambda_frm, prm.lambda_seg})
       if (!(lam >= 0.f && lam <= 1.f)) return fail(ctx, MUKV_E_INVALID, "every lambda must lie in [0, 1]");
     if (ctx->frames < 1) return fail(ctx, MUKV_E_STATE, "the store is empty");
+    if (ctx->seg_pending) {                                // the last chunk's segment entries are read below
+      const cudaError_t ef = flush_segments(ctx, static_cast<cudaStream_t>(stream));
+      if (ef != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "segment kernel: %s", cudaGetErrorString(ef));
+      ctx->launches += 1;
+    }
     QMeta meta;
     if (h_q_offsets[0] != 0) return fail(ctx, MUKV_E_INVALID, "q_offsets[0] must be 0");
     for (int i = 0; i < nq; ++i) {
@@ -830,8 +894,19 @@ mukv_status mukv_create(const mukv_config* cfg, void* d_store, size_t store_byte
   return create_impl(cfg, d_store, store_bytes, d_workspace, workspace_bytes, 0, out);
 }
 
+// Host readers of the store (a view of a region, an export): segment entries still owed by the last
+// compress call are pooled on that call's stream, and the stream is waited for.
+static cudaError_t settle_store(const mukv_ctx* ctx) {
+  if (!ctx->seg_pending) return cudaSuccess;
+  const cudaStream_t st = ctx->seg_stream;
+  cudaError_t e = flush_segments(ctx, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  return e;
+}
+
 mukv_status mukv_export_header(const mukv_ctx* ctx, mukv_store_header* out) {
   if (!ctx || !out) return MUKV_E_INVALID;
+  if (settle_store(ctx) != cudaSuccess) return MUKV_E_CUDA;
   memset(out, 0, sizeof *out);
   out->magic = MUKV_STORE_MAGIC;
   out->version = MUKV_STORE_VERSION;
@@ -966,6 +1041,7 @@ mukv_status mukv_reset(mukv_ctx* ctx, mukv_stream stream) {
   ctx->frames = 0;
   ctx->parity = 0;
   ctx->failed = false;
+  ctx->seg_pending = false;
   return MUKV_OK;
 }
 
@@ -1086,6 +1162,11 @@ mukv_status mukv_gather3(mukv_ctx* ctx, const int32_t* d_seg_idx, const int32_t*
       return fail(ctx, MUKV_E_CAPACITY, "decode_stride_bytes %lld < %lld needed per question",
                   (long long)decode_stride_bytes, need);
     if (decode_stride_bytes % 16 != 0) return fail(ctx, MUKV_E_ALIGN, "decode_stride_bytes must be a multiple of 16");
+    if (ctx->seg_pending) {                                // the summary tokens are segment entries
+      const cudaError_t ef = flush_segments(ctx, static_cast<cudaStream_t>(stream));
+      if (ef != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "segment kernel: %s", cudaGetErrorString(ef));
+      ctx->launches += 1;
+    }
     Gather3Params gp;
     memset(&gp, 0, sizeof gp);
     gp.nq = nq; gp.k_seg = k_seg; gp.k_frm = k_frm; gp.k_pat = k_patch; gp.L = c.n_layers; gp.kappa = c.keep_per_frame;
@@ -1166,6 +1247,7 @@ mukv_status mukv_gather(mukv_ctx* ctx, const int32_t* d_frm_idx, const int32_t* 
 
 void* mukv_store_region(const mukv_ctx* ctx, int32_t which, size_t* bytes) {
   if (!ctx) return nullptr;
+  if (settle_store(ctx) != cudaSuccess) return nullptr;
   const mukv_config& c = ctx->cfg;
   const StoreLayout& s = ctx->sl;
   const size_t T = (size_t)c.max_frames, C = (size_t)ctx->C;
