@@ -411,6 +411,11 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
       }
       return vm;
     };
+    // (the masks of this thread's chunks, 16 bits each, worked out once)
+    unsigned long long vmask = 0ull;
+    if constexpr (PAST) {
+      for (int ch = 0; ch < my_nch; ++ch) vmask |= (unsigned long long)chunk_mask((my_c0 + ch) * 16) << (16 * ch);
+    }
     float acc[kPsAccCols];                               // column sums of this thread's row, over tiles
 #pragma unroll
     for (int k = 0; k < kPsAccCols; ++k) acc[k] = 0.f;
@@ -470,7 +475,7 @@ __global__ void __maxnreg__(96) score_ps_kernel(const ScorePsParams p,
           uint32_t ra[16];
           tc::tmem_ld16(tb + col, ra);
           tc::tmem_wait_ld16(ra);
-          const uint32_t vm = PAST ? chunk_mask(col) : 0u;
+          const uint32_t vm = PAST ? (uint32_t)(vmask >> (16 * ch)) & 0xffffu : 0u;
           const float m_new = fmaxf(m_run, ps_chunk_max<PAST>(ra, col, P, vm, causal, i_tok));
           const float resc = (m_new == m_run) ? 1.f : ex2_approx((m_run - m_new) * c);
           l = l * resc + ps_chunk_exp<PAST>(ra, c, m_new * c, col, P, vm, causal, i_tok);
