@@ -496,9 +496,10 @@ SegmentArgs segment_args_of(const mukv_ctx* ctx, long long first, int n) {
   return a;
 }
 
-// With frame-level selection a compress call does not pool the segment entries of its chunk itself (unless
-// frames were flagged: tail_kernel then does): the next compress call does it with one more row of blocks in its compaction
-// kernel, which do not wait for that call's scoring kernel.  Whoever else needs the entries first
+// A compress call does not pool the segment entries of its chunk itself (unless frames were flagged:
+// tail_kernel then does): the next compress call does it with blocks that do not wait for that call's
+// scoring kernel (one more row in its compaction kernel; with segment-level selection, extra blocks of its
+// first segsel_kernel launch).  Whoever else needs the entries first
 // (retrieval, a gather with summary tokens, a view of the store, an export) pools them with one launch here.
 cudaError_t flush_segments(const mukv_ctx* ctx, cudaStream_t st) {
   if (!ctx->seg_pending) return cudaSuccess;
@@ -610,6 +611,20 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
     gp.token_bytes = (long long)L * 2 * C * ctx->esize;
     gp.kept_count = reinterpret_cast<int*>(ctx->store + ctx->sl.kept_count);
     gp.seg_flag = reinterpret_cast<int*>(ctx->ws + ctx->wl.seg_flag);
+    gp.n_seg = n_seg;
+    // Segment entries the previous call left behind: pooled by extra blocks of the first segsel_kernel launch
+    // (that kernel uses one SM per segment); with per-kernel timing on, by a launch of their own
+    if (ctx->seg_pending && ctx->prof_on) {
+      ProfScope ps(ctx, 3, st);
+      e = flush_segments(ctx, st);
+      if (e != cudaSuccess) return fail(ctx, MUKV_E_CUDA, "segment kernel: %s", cudaGetErrorString(e));
+      ++n_launch;
+    }
+    int extra = 0;
+    if (ctx->seg_pending) {
+      gp.prev = segment_args_of(ctx, ctx->seg_first, ctx->seg_n);
+      extra = 2 * L;
+    }
     gp.stat_refined = reinterpret_cast<unsigned long long*>(ctx->ws + ctx->wl.stat_refined);
     if (tc_first) {
       int ps_grid1 = 0, ps_items1 = 0, ps_ipf1 = 0;
@@ -625,9 +640,12 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
       gp.ps_grid = ps_grid1; gp.ps_items = ps_items1; gp.ps_ipf = ps_ipf1;
       {
         ProfScope ps(ctx, 1, st);
-        e = launch_k(segsel_kernel, dim3(n_seg), kSegSelThreads, segsel_smem_bytes(seg_tokens), st, dep, gp);
+        e = launch_k(segsel_kernel, dim3(n_seg + extra), kSegSelThreads, segsel_smem_bytes(seg_tokens), st, dep, gp);
       }
       if (e != cudaSuccess) return broke_off(ctx, "segment selection kernel", e);
+      ctx->seg_pending = false;
+      extra = 0;
+      memset(&gp.prev, 0, sizeof gp.prev);
     }
     ScoreParams sd = sp;
     sd.no_select = 1;
@@ -654,9 +672,11 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
     gp.only_flagged = tc_first ? 1 : 0;
     {
       ProfScope ps(ctx, 1, st);
-      e = launch_k(segsel_kernel, dim3(n_seg), kSegSelThreads, segsel_smem_bytes(seg_tokens), st, tc_first && dep, gp);
+      e = launch_k(segsel_kernel, dim3(n_seg + extra), kSegSelThreads, segsel_smem_bytes(seg_tokens), st, tc_first && dep,
+                   gp);
     }
     if (e != cudaSuccess) return broke_off(ctx, "segment selection kernel", e);
+    ctx->seg_pending = false;
     n_launch += 2;
   } else if (!d_ext) {
     ProfScope ps(ctx, 0, st);
@@ -712,16 +732,9 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
   if (e != cudaSuccess) return broke_off(ctx, "compact kernel", e);
   ctx->seg_pending = false;
 
-  // The segment entries need every frame of the chunk.  With frame-level selection they are left to the
-  // next call (flush_segments); when frames were flagged, tail_kernel pools them after it has redone those
-  // frames.  With segment-level selection (count-weighted entries, no tail_kernel) they are pooled here.
+  // The segment entries need every frame of the chunk.  They are left to the next call (flush_segments);
+  // when frames were flagged, tail_kernel pools them after it has redone those frames.
   cp.sp.n_flagged = sp.n_flagged;
-  if (seg_scope) {
-    ProfScope ps(ctx, 3, st);
-    e = launch_k(segment_kernel, dim3(2 * L), kCompactThreads, 0, st, !ctx->prof_on, cp);
-    ++n_launch;
-  }
-  if (e != cudaSuccess) return broke_off(ctx, "segment kernel", e);
   sp.refine = 1;
   sp.row_split = kRefineSplit;
   sp.colsum_part = ctx->ws + ctx->wl.colsum_d;
@@ -735,7 +748,7 @@ mukv_status compress_impl(mukv_ctx* ctx, const void* d_q, const float* d_ext, co
     ++n_launch;
   }
   if (e != cudaSuccess) return broke_off(ctx, "tail kernel", e);
-  ctx->seg_pending = !seg_scope;
+  ctx->seg_pending = true;
   ctx->seg_first = t0;
   ctx->seg_n = n;
   ctx->seg_stream = st;

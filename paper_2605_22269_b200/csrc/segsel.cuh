@@ -41,6 +41,10 @@ struct SegSelParams {
   int* seg_flag;                // [segments of the chunk]; written with src32 = 1, read with only_flagged
   int ps_grid, ps_items, ps_ipf;  // the persistent scoring launch: blocks, items, items per frame (src32 = 1)
   unsigned long long* stat_refined;  // frames ranked by the gated double-precision pass are added here
+  // Blocks n_seg, n_seg + 1, ... of the grid (one per (layer, K|V) plane, present when prev.n_frames > 0)
+  // pool the segment entries the previous call left to this one, on SMs this kernel leaves idle
+  int n_seg;
+  SegmentArgs prev;
 };
 
 __host__ inline size_t segsel_smem_bytes(int tokens) {
@@ -260,7 +264,64 @@ __device__ inline int segment_select32(const SegSelParams& p, int f0, int O, int
   return risky ? -1 : n_kept;                              // (the same decision in every thread)
 }
 
+// Segment entries (Eq. 5 at segment level) of one (layer, K|V) plane for every segment that frames
+// a.first_frame .. a.first_frame + a.n_frames - 1 touch: the same sums in the same frame order as
+// compact_segment_plane, one channel per thread at a time, eight loads in flight.
+__device__ inline void pool_plane_entries(const SegmentArgs& a, int plane) {
+  const int C = a.C, l = plane >> 1, kv = plane & 1;
+  const bool exact = (l == a.L - 1) && (kv == 0);
+  const long long frames_total = a.first_frame + a.n_frames;
+  const long long first_seg = a.first_frame / a.fseg, last_seg = (frames_total - 1) / a.fseg;
+  const long long fstride = 2LL * a.L * C;                  // floats between the entries of two frames
+  for (long long u = first_seg; u <= last_seg; ++u) {
+    const long long t0 = u * a.fseg;
+    const long long t1 = t0 + a.fseg < frames_total ? t0 + a.fseg : frames_total;
+    const int nf = (int)(t1 - t0);
+    for (int col = threadIdx.x; col < C; col += blockDim.x) {
+      float* dst = a.seg_entry + ((u * a.L + l) * 2 + kv) * C + col;
+      const float* src = a.frame_entry + ((t0 * a.L + l) * 2 + kv) * C + col;
+      const double* srck = a.frame_ksum + t0 * C + col;
+      double td = 0.0;
+      float tf = 0.f;
+      long long n_tok = 0;
+      for (int i0 = 0; i0 < nf; i0 += 8) {
+        int cn[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cn[i] = (a.kept_count && i0 + i < nf) ? __ldcg(a.kept_count + t0 + i0 + i) : 0;
+        if (exact) {
+          double x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[i] = i0 + i < nf ? __ldcg(srck + (long long)(i0 + i) * C) : 0.0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) td += x[i];
+        } else {
+          float x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[i] = i0 + i < nf ? __ldcg(src + (i0 + i) * fstride) : 0.f;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) tf += a.kept_count ? (float)cn[i] * x[i] : x[i];
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) n_tok += cn[i];
+      }
+      float m;
+      if (a.kept_count)                                       // frames keep different numbers of tokens: count-weighted
+        m = exact ? (n_tok ? (float)(td / (double)n_tok) : 0.f) : (n_tok ? tf / (float)n_tok : 0.f);
+      else
+        m = exact ? (float)(td / ((double)nf * (double)a.kappa)) : tf / (float)nf;
+      if (exact) a.seg_key[u * C + col] = m;
+      *dst = m;
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kSegSelThreads) segsel_kernel(const SegSelParams p) {
+  if (p.prev.n_frames > 0 && (int)blockIdx.x >= p.n_seg) {
+    // nothing of this call is needed for the previous call's entries: no wait for the scoring kernel
+    for (int plane = (int)blockIdx.x - p.n_seg; plane < 2 * p.prev.L; plane += (int)gridDim.x - p.n_seg)
+      pool_plane_entries(p.prev, plane);
+    return;
+  }
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ RankScratch sc;
   __shared__ SegSel32Scratch sc32;
