@@ -95,6 +95,43 @@ def test_tiny_chunking_and_partial_segment():
     retrieval_check(run, st, qtok, offs, 50, 50, 0.5, B.RETR_SEMI)          # k larger than what exists
 
 
+@pytest.mark.parametrize("name,T,chunk", [("tiny", 7, 3), ("chunk7b", 6, 4)])
+def test_segment_entries_owed_by_a_call_reach_every_reader(name, T, chunk):
+    # A compress call leaves the segment entries of its chunk to whoever comes next.  Here: calls on a side
+    # stream and a view of the store right behind the last call, with no synchronisation by the caller;
+    # the same after a reset in the middle of a segment; and a retrieval as the first reader.
+    wl = dict(workload(name))
+    run = H.GpuRun(wl, n_frames=T)
+    side = torch.cuda.Stream()
+
+    def compress(frames):
+        with torch.cuda.stream(side):
+            for t0 in range(0, frames, chunk):
+                n = min(chunk, frames - t0)
+                q, k, v = run.gs.chunk(t0, n)
+                run.ctx.mukv_compress_chunk(q, k, v, n, t0, stream=side)
+
+    def check_segments(st):
+        seg = run.ctx.region(3).cpu().numpy()                  # pools what is owed and waits for `side`
+        key = run.ctx.region(5).cpu().numpy()
+        for u in range(st.n_segments):
+            sk, sv = st.segment_entry(u)
+            H.close(seg[u][:, 0], sk, f"segment entry K {u}")
+            H.close(seg[u][:, 1], sv, f"segment entry V {u}")
+            assert key[u].tobytes() == st.segment_key(u).tobytes(), f"segment key {u}"
+
+    compress(T)
+    check_segments(H.oracle_stream(run.spec, H.oracle_cfg(run.cfg), range(T), last_only=False, workers=1))
+    with torch.cuda.stream(side):
+        run.ctx.mukv_reset(stream=side)
+    compress(T - 1)                                            # what the dropped call owed must not come back
+    st = H.oracle_stream(run.spec, H.oracle_cfg(run.cfg), range(T - 1), last_only=False, workers=1)
+    torch.cuda.synchronize()
+    qtok, offs, _ = run.spec.questions(3, 1, 9)
+    retrieval_check(run, st, qtok, offs, 2, 3, 0.3, B.RETR_SEMI)   # the retrieval is the first reader
+    check_segments(st)
+
+
 @pytest.mark.parametrize("over", [dict(attn_causal=1), dict(keep_low_freq=1), dict(alpha=0.0), dict(alpha=1.0),
                                   dict(alpha=0.5), dict(keep_per_frame=1), dict(keep_per_frame=64)])
 def test_tiny_variants(over):
