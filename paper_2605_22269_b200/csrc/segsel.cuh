@@ -90,7 +90,46 @@ __device__ inline int segment_select32(const SegSelParams& p, int f0, int O, int
   const float na = 1.f / (float)((long long)sp.Ls * sp.Hq * P), nf = 1.f / (float)((long long)HkvV * sp.D);
   unsigned k0 = 0xffffffffu, k1 = 0u, k2 = 0xffffffffu, k3 = 0u;
   bool bad = false;
-  for (int i = tid; i < O; i += kSegSelThreads) {
+  // (with P a multiple of four a thread takes four neighbouring tokens of a frame with 16-byte loads, so that
+  // one trip covers a 16-frame segment: the loads of this one block are what the kernel spends most time on)
+  const bool vec4 = (P & 3) == 0;
+  for (int i = tid * 4; vec4 && i < O; i += 4 * kSegSelThreads) {
+    const int f = f0 + i / P, j = i % P;
+    const int c_first = share_owner((unsigned)(f * p.ps_ipf), (unsigned)p.ps_items, (unsigned)p.ps_grid);
+    const int c_last = share_owner((unsigned)((f + 1) * p.ps_ipf - 1), (unsigned)p.ps_items, (unsigned)p.ps_grid);
+    const float* cp = reinterpret_cast<const float*>(sp.colsum_part) + j;
+    const float* fp = reinterpret_cast<const float*>(sp.ifft_part) + (long long)f * HkvV * P + j;
+    float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f), f4 = a4;
+    for (int c0 = c_first; c0 <= c_last; c0 += 8) {
+      float4 x[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        x[u] = c0 + u <= c_last ? __ldcg(reinterpret_cast<const float4*>(cp + (long long)(c0 + u + f) * P))
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { a4.x += x[u].x; a4.y += x[u].y; a4.z += x[u].z; a4.w += x[u].w; }
+    }
+    for (int g0 = 0; g0 < HkvV; g0 += 8) {
+      float4 y[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        y[u] = g0 + u < HkvV ? __ldcg(reinterpret_cast<const float4*>(fp + (long long)(g0 + u) * P))
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { f4.x += y[u].x; f4.y += y[u].y; f4.z += y[u].z; f4.w += y[u].w; }
+    }
+    const float av[4] = {a4.x * na, a4.y * na, a4.z * na, a4.w * na};
+    const float bv[4] = {f4.x * nf, f4.y * nf, f4.z * nf, f4.w * nf};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      att[i + e] = av[e];
+      fft[i + e] = bv[e];
+      bad |= !(isfinite(av[e]) && isfinite(bv[e]));
+      const unsigned ka = __float_as_uint(av[e]), kf = __float_as_uint(bv[e]);
+      k0 = min(k0, ka); k1 = max(k1, ka); k2 = min(k2, kf); k3 = max(k3, kf);
+    }
+  }
+  for (int i = tid; !vec4 && i < O; i += kSegSelThreads) {
     const int f = f0 + i / P, j = i % P;
     const int c_first = share_owner((unsigned)(f * p.ps_ipf), (unsigned)p.ps_items, (unsigned)p.ps_grid);
     const int c_last = share_owner((unsigned)((f + 1) * p.ps_ipf - 1), (unsigned)p.ps_items, (unsigned)p.ps_grid);

@@ -135,6 +135,19 @@ def test_segment_scope_sixteen_frame_segments(over):
     assert worst < H.FLAG_MARGIN / 2, worst
 
 
+def test_segment_scope_bf16_odd_token_count():
+    # P = 77 (not a multiple of four: the scalar loads of the single-precision ranking), G = 3, D = 64,
+    # segments of four frames in chunks of eight, a last segment of three frames
+    spec = StreamSpec(seed=13, n_layers=3, n_q_heads=6, n_kv_heads=2, head_dim=64, tokens_per_frame=77, bf16=True,
+                      n_outlier=2, n_frames=11, scene_sigma=1.0, frame_sigma=0.5, scene_min=3, scene_max=5)
+    wl = dict(spec=spec, keep=19, fseg=4, chunk=8, alpha=0.7)
+    run = H.GpuRun(wl, keep_per_segment=O.keep_count(0.3, 4 * 77))
+    kept, scores = compress_segment_scope(run, 8)
+    st = oracle_stream_chunked(spec, H.oracle_cfg(run.cfg), 11, 8)
+    check_store(run, st, kept, scores)
+    assert run.ctx.mukv_get_stats().refined_frames <= 4
+
+
 def oracle_stream_chunked(spec, ocfg, T, chunk):
     st = O.Store(ocfg)
     for t0 in range(0, T, chunk):
