@@ -17,14 +17,17 @@
 // (sel_mode 0).  Either way a frame whose lowest kept and highest dropped score are closer than
 // tie_eps + flag_margin is skipped here: tail_kernel decides it in double precision and compacts it.
 //
-// What has to wait for every frame of the chunk runs in two small launches behind compact_kernel.
-// segment_kernel: the segment entries (Eq. 5 at segment level) when no frame was flagged: one
-// (layer, K|V) plane per block, mean over the frames present.  tail_kernel<T, NC>: returns at once
-// unless frames were flagged (about one chunk in fifty on the synthetic streams); then all its
-// blocks first score those frames in double precision and select; once every block has finished
-// that, the flagged frames are compacted and then the segment entries written, one plane per block.
-// (Segment pooling by the compaction block that finishes a plane last was measured: the fence
-// every block then needs before it signs off costs more than a launch.)
+// What has to wait for every frame of the chunk:
+// tail_kernel<T, NC>, launched behind compact_kernel: returns at once unless frames were flagged (about
+// one chunk in fifty on the synthetic streams); then all its blocks first score those frames in double
+// precision and select; once every block has finished that, the flagged frames are compacted and then
+// the segment entries written, one plane per block.
+// The segment entries (Eq. 5 at segment level; one (layer, K|V) plane per block, mean over the frames
+// present) of the common case are not written by the call itself.  The next call pools them with a row
+// of compact_kernel blocks that does not wait for its scoring kernel (CompactParams::prev), or the first
+// reader launches segment_kernel for them.  (As the last launch of every call that kernel cost 6 us;
+// pooling by the compaction block that finishes a plane last was measured too: the fence every block
+// then needs before it signs off costs more than a launch.)
 #pragma once
 #include "common.cuh"
 #include "score.cuh"
@@ -623,11 +626,10 @@ constexpr int kStatusTailWait = 6;   // tail_kernel: the wait for the double-pre
 // tail_kernel: see the head of this file.  sp is the scoring configuration of the double-precision
 // pass (its partial-sum buffers, refine = 1); the grid is a multiple of nothing in particular: blocks
 // stride over the work, and the host keeps the grid within what is resident at once.
-// segment_kernel: the common case of what has to wait for every frame of the chunk.  One block per
-// (layer, K|V) plane; when no frame was flagged it writes that plane of every segment entry the chunk
-// touches.  Otherwise it leaves everything to tail_kernel.  (It is a launch of its own because it
-// is light: no dynamic shared memory, 56 blocks.  One kernel for both cases was measured and cost
-// 2 us more per call.)
+// segment_kernel: one block per (layer, K|V) plane writes that plane of every segment entry the frames
+// first_frame .. first_frame + n_frames - 1 touch.  Launched for the chunk of an earlier call when
+// something is about to read its segment entries (pool_always = 1); without pool_always it leaves
+// everything to tail_kernel when frames were flagged.
 __global__ void __launch_bounds__(kCompactThreads) segment_kernel(const CompactParams p) {
   pdl_wait();
   pdl_trigger();
