@@ -87,3 +87,45 @@ def test_retrieval_stress(stream3h):
         for s, t in enumerate(frm[i]):
             got = dec[i][:, :, s * kap:(s + 1) * kap]
             assert bool((got.reshape(-1) == pages[int(t)].reshape(-1)).all())
+
+
+def test_stream_3h_segment_level_selection(stream3h):
+    # The same stream with segment-level selection (kappa_v = 16 * 49 over the 3,136 tokens of a segment), in
+    # the launch configuration of the benchmark's variant: kept ids and per-frame counts of all 675 segments.
+    # The indicators of a frame do not depend on the scope of the selection, so the oracle's frame-level run
+    # above supplies them; Eq. 4 over the segment and the ranking are the oracle's functions.
+    import torch
+    run0, st = stream3h
+    wl = dict(run0.wl)
+    fseg, chunk = wl["fseg"], wl["chunk"]
+    kv = wl["keep"] * fseg
+    run = H.GpuRun(wl, keep_per_segment=kv, want_scores=False)
+    c, T = run.cfg, run.n_frames
+    P = c.tokens_per_frame
+    kept = torch.full((T, P), -7, dtype=torch.int32, device=run.device)
+    q, k, v = run.gs.alloc(chunk)
+    for t0 in range(0, T, chunk):
+        run.gs.fill(t0, chunk, q, k, v)
+        run.ctx.mukv_compress_chunk(q, k, v, chunk, t0, kept[t0:t0 + chunk])
+    torch.cuda.synchronize()
+    kept = kept.cpu().numpy()
+    cnt = run.ctx.region(10).cpu().numpy()
+    ocfg = H.oracle_cfg(c)
+    uneven = 0
+    for u in range(T // fseg):
+        frames = range(u * fseg, (u + 1) * fseg)
+        ia = np.concatenate([st.scores[t][0] for t in frames])
+        ifr = np.concatenate([st.scores[t][1] for t in frames])
+        fused = O.fuse(ia, ifr, ocfg["alpha"], False)
+        sel = O.select_tokens(fused, O.segment_keep_count(kv, fseg, fseg), ocfg["tie_eps"])
+        assert len(sel) == kv
+        for i, t in enumerate(frames):
+            ref = sel[(sel >= i * P) & (sel < (i + 1) * P)] - i * P
+            assert cnt[t] == len(ref), f"frame {t}: {cnt[t]} tokens kept, oracle {len(ref)}"
+            assert kept[t, :len(ref)].tolist() == ref.tolist() and np.all(kept[t, len(ref):] == -1), f"frame {t}"
+            uneven += int(len(ref) != wl["keep"])
+    stats = run.ctx.mukv_get_stats()
+    print(f"segment-level selection: {uneven} of {T} frames keep another number of tokens than 49; "
+          f"{stats.refined_frames} frames went through the double-precision pass")
+    assert uneven > T // 2 and stats.device_status == 0 and stats.kept_tokens == (T // fseg) * kv
+    assert stats.refined_frames <= T // 25
