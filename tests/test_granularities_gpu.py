@@ -107,6 +107,21 @@ def test_three_granularities_bf16():
     retrieve3_check(run, st, qtok, offs, (0, 4, 2), (0.0, 0.3, 0.0), B.RETR_SEMI)          # no patch level asked for
 
 
+def test_many_patch_rows_and_k_beyond_the_store():
+    # one super patch per frame with 98 kept tokens: a question's patch-level rows (12 blocks x 98 rows) do not
+    # fit the gather kernel's row list at once; k beyond what exists in the two modes that rank without rerank
+    wl = dict(workload("chunk7b"))
+    wl["fseg"] = 4
+    run = H.GpuRun(wl, n_frames=12, keep_per_frame=98, patch_split=1, grid_width=14).compress(chunk=5)
+    st = H.oracle_stream(run.spec, H.oracle_cfg(run.cfg), range(12), last_only=False, workers=1)
+    H.check_frames_against_oracle(run, st, range(12), full_layers=True)
+    check_patch_level(run, st, 12)
+    qtok, offs, _ = run.spec.questions(3, 3, 9)
+    retrieve3_check(run, st, qtok, offs, (12, 3, 2), (0.3, 0.3, 0.0), B.RETR_SEMI)
+    for mode in (B.RETR_HIER, B.RETR_PARALLEL):
+        retrieve3_check(run, st, qtok, offs, (200, 30, 9), (0.3, 0.3, 0.0), mode)
+
+
 def test_three_granularities_fp32_every_frame_flagged():
     # small fp32 stream; the flagged frames' patch-level keys are written by the tail kernel
     spec = StreamSpec(seed=41, n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, tokens_per_frame=36, bf16=False,
